@@ -1,0 +1,185 @@
+/*
+ * tq.h -- C ABI of the TurboQuant hot path for NVIDIA B200 (sm_100a).
+ *
+ * TurboQuant (arxiv 2504.19874) quantises a vector x in R^d in two ways:
+ *   TurboQuant_mse  (Algorithm 1): y = Pi x with a random rotation Pi, then the index of the
+ *                   nearest centroid of a precomputed scalar codebook for every coordinate.
+ *   TurboQuant_prod (Algorithm 2): the same at b-1 bits, plus the sign bits of S r for the
+ *                   residual r = x - DeQuant_mse(idx) (the QJL map of Definition 1) and ||r||.
+ * This library computes those maps, their inverses, and the inner-product estimator of
+ * Section 3.2 evaluated directly on the packed codes (dense scores or top-k).
+ *
+ * Notation used below: n vectors, d dimensions, b total bits per coordinate, b_m = bits of
+ * the MSE stage (b for TQ_MSE, b-1 for TQ_PROD), nu = ||x||, u = x/nu, gamma = ||r||.
+ * Following Section 1.3 the stored norm nu is kept in floating point, the unit vector u is
+ * what gets quantised, and every reconstruction / estimate is rescaled by nu.
+ *
+ * Conventions for every entry point
+ *   - returns 0 (TQ_OK) or a TQ_ERR_* code; tq_last_error() gives a thread-local message.
+ *     No exception crosses the boundary.  Invalid arguments are rejected on the host before
+ *     anything is launched.
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are CUDA global memory of the
+ *     current device, owned by the caller, 16-byte aligned, never retained after the call.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).  Device work
+ *     is only enqueued; the calls do not synchronise and allocate nothing (callers pass
+ *     scratch sized by tq_workspace_bytes).  tq_plan_create/destroy are the exceptions.
+ *   - n = 0 (or nq = 0) is a no-op that returns TQ_OK.
+ *
+ * Packed layouts (the paper says only "b-bit integers"; this layout is the library's)
+ *   idx row : little-endian bit stream, coordinate j in bits [j*b_m, (j+1)*b_m); bit p of the
+ *             row is bit (p & 7) of byte (p >> 3); value k names the k-th centroid in
+ *             ascending order (0-based).  Row stride tq_idx_row_bytes(d, b_m); pad bits are 0.
+ *   qjl row : bit j = 1 iff (S r)_j >= 0 (sign(0) = +1).  Row stride tq_qjl_row_bytes(d).
+ *   gamma, norms : float32 arrays of length n.
+ */
+#ifndef TQ_H_
+#define TQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  TQ_OK = 0,
+  TQ_ERR_INVALID_ARG = 1,   /* NULL pointer, negative size, inconsistent arguments           */
+  TQ_ERR_UNSUPPORTED = 2,   /* d, bits, k or dtype outside the supported range               */
+  TQ_ERR_ALIGNMENT = 3,     /* a device pointer or leading dimension is not aligned          */
+  TQ_ERR_CUDA = 4,          /* a CUDA runtime call failed (message has the CUDA error)       */
+  TQ_ERR_NOT_CONVERGED = 5, /* Lloyd-Max iteration did not converge                          */
+  TQ_ERR_TIMEOUT = 6,       /* a bounded device-side wait ran out                            */
+  TQ_ERR_WORKSPACE = 7      /* scratch / workspace smaller than tq_workspace_bytes says      */
+};
+enum { TQ_MSE = 0, TQ_PROD = 1 };              /* plan mode                                   */
+enum { TQ_F32 = 0, TQ_BF16 = 1 };              /* element type of X / Q                       */
+enum { TQ_ORTHOGONAL = 0, TQ_GAUSSIAN = 1 };   /* tq_rotation kind                            */
+enum { TQ_OP_QUANTIZE = 0, TQ_OP_SCORE = 1, TQ_OP_TOPK = 2, TQ_OP_WSUM = 3, TQ_OP_DEQUANTIZE = 4 };
+
+#define TQ_MAX_D 8192
+#define TQ_MAX_K 1024
+
+typedef struct tq_plan tq_plan;
+
+/* Message of the last error raised on the calling thread ("" if none). Never NULL. */
+const char* tq_last_error(void);
+
+/*
+ * Lloyd-Max codebook of Eq. (4): the 2^bits centroids c_1 <= ... <= c_{2^bits} in [-1,1] that
+ * minimise the scalar k-means cost for the coordinate density of Lemma 1,
+ * f_X(x) = Gamma(d/2) / (sqrt(pi) Gamma((d-1)/2)) (1 - x^2)^((d-3)/2)  (exact for this d, not its
+ * Gaussian limit).  Host only, fp64 inside, results rounded to float32.
+ *   d          2..TQ_MAX_D;   bits 0..4 (bits = 0 gives the single centroid 0)
+ *   centroids  host, 2^bits floats, ascending, exactly antisymmetric (c_i = -c_{2^bits-1-i})
+ *   boundaries host, 2^bits - 1 floats or NULL: fl32(0.5f * (c_i + c_{i+1})), the decision
+ *              thresholds of the nearest-centroid rule of Algorithm 1 (step idx_j)
+ */
+int tq_codebook(int d, int bits, float* centroids, float* boundaries);
+
+/*
+ * Seeded d x d matrix, host, row-major float32.
+ *   TQ_GAUSSIAN   i.i.d. N(0,1) entries: the matrix S of Definition 1 / Algorithm 2.  Entry
+ *                 e = r*d + c is sqrt(-2 ln u1) cos(2 pi u2) with u1 = ((h(2e) >> 11) + 0.5) 2^-53,
+ *                 u2 = (h(2e+1) >> 11) 2^-53, h(t) = mix(mix(seed + G) + t*G), mix = SplitMix64
+ *                 finaliser, G = 0x9E3779B97F4A7C15 (64-bit wrap-around arithmetic).
+ *   TQ_ORTHOGONAL the rotation Pi of Section 3.1: Q of the QR decomposition of that Gaussian
+ *                 matrix, columns signed so that R has a positive diagonal.  fp64 Householder.
+ */
+int tq_rotation(int d, uint64_t seed, int kind, float* out);
+
+/* Row strides in bytes.  ceil(d*bits/8) rounded up to a multiple of 16; rows shorter than
+ * 16 bytes are rounded up to a power of two (at least 4) instead.  bits = 0 gives 0. */
+size_t tq_idx_row_bytes(int d, int bits);
+size_t tq_qjl_row_bytes(int d);
+
+/*
+ * Builds the per-(d, b, mode) state ("global parameters" of Algorithms 1 and 2) on the current
+ * device: copies Pi, S and the codebook, forms S' = S Pi^T (fp64 on the device, rounded to
+ * fp32), the decision boundaries and the operand splits the kernels use.
+ *   d         2..TQ_MAX_D
+ *   bits      total bits b per coordinate: TQ_MSE 1..4; TQ_PROD 1..5 (b_m = b-1, so b = 1 has a
+ *             0-bit MSE stage: idx arrays are then unused and may be NULL)
+ *   Pi        host, d*d floats, row-major: y = Pi x
+ *   S         host, d*d floats, row-major (TQ_PROD); ignored / may be NULL for TQ_MSE
+ *   centroids host, 2^b_m floats, ascending
+ *   out       receives the plan; free with tq_plan_destroy.  The plan owns device memory only.
+ * Allocates device memory and synchronises the device.
+ */
+int tq_plan_create(int d, int bits, int mode, const float* Pi, const float* S,
+                   const float* centroids, tq_plan** out);
+int tq_plan_destroy(tq_plan* plan);
+
+/* Bytes of device scratch the given operation needs (0 if none).  For TQ_OP_TOPK and
+ * TQ_OP_SCORE any size >= the returned minimum is accepted; larger buffers let the scan work
+ * on bigger blocks of vectors.   op = TQ_OP_*;  nq, k ignored where they do not apply. */
+size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int nq, int k);
+
+/*
+ * Quant_mse of Algorithm 1 for n vectors (plan mode TQ_MSE).
+ *   X        device, n rows of d elements (x_dtype), row stride ldx elements (ldx >= d)
+ *   idx      device out, n rows of tq_idx_row_bytes(d, b) bytes
+ *   norms    device out, n floats: nu = ||x||.  NULL: rows are taken as already unit-norm and
+ *            quantised as they are.  A zero row gives nu = 0 and the codes of y = 0.
+ * Nearest centroid = number of boundaries strictly below y_j (a coordinate exactly on a
+ * boundary takes the lower index).
+ */
+int tq_quantize_mse(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t ldx,
+                    uint8_t* idx, float* norms, void* scratch, size_t scratch_bytes, void* stream);
+
+/*
+ * Quant_prod of Algorithm 2 for n vectors (plan mode TQ_PROD): idx at b-1 bits, qjl = sign(S r)
+ * and gamma = ||r|| for r = u - DeQuant_mse(idx).  Uses r = Pi^T (Pi u - c[idx]), so that
+ * ||r|| = ||Pi u - c[idx]|| and S r = S' (Pi u - c[idx]) -- two d x d products instead of three.
+ *   idx, norms as above;  qjl device out, n rows of tq_qjl_row_bytes(d);  gamma device out, n floats
+ *   scratch  device, scratch_bytes >= tq_workspace_bytes(plan, TQ_OP_QUANTIZE, n, 0, 0)
+ * A zero row gives gamma = 0 and all qjl bits 1.
+ */
+int tq_quantize_prod(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t ldx,
+                     uint8_t* idx, uint8_t* qjl, float* gamma, float* norms,
+                     void* scratch, size_t scratch_bytes, void* stream);
+
+/*
+ * DeQuant_mse / DeQuant_prod: Xhat = nu * (Pi^T c[idx] + sqrt(pi/2)/d * gamma * S^T qjl).
+ *   qjl, gamma  used for TQ_PROD plans only;  norms NULL means nu = 1
+ *   Xhat        device out, n rows of d floats, row stride ldxh
+ */
+int tq_dequantize(const tq_plan* plan, int64_t n, const uint8_t* idx, const uint8_t* qjl,
+                  const float* gamma, const float* norms, float* Xhat, int64_t ldxh, void* stream);
+
+/*
+ * Inner-product estimator of Section 3.2 for every (query, vector) pair, evaluated on the codes:
+ *   est = nu * ( sum_j (Pi q)_j c[idx_j]  +  sqrt(pi/2)/d * gamma * sum_i (S q)_i z_i ),  z_i = +-1
+ * which equals <q, DeQuant(code)> because Pi is orthogonal.
+ *   Q       device, nq rows of d elements (q_dtype), row stride ldq
+ *   scores  device out, nq rows of n floats, row stride lds
+ *   workspace  >= tq_workspace_bytes(plan, TQ_OP_SCORE, n, nq, 0)
+ */
+int tq_score(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, int64_t n,
+             const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms,
+             float* scores, int64_t lds, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The k vectors with the largest estimate per query (nearest-neighbour search by estimated
+ * inner product, Section 4.4), sorted by descending score, equal scores by ascending id.
+ * The nq x n score matrix is never formed.
+ *   k 1..min(n, TQ_MAX_K);  top_scores device out [nq, k] floats;  top_ids device out [nq, k] int32
+ */
+int tq_topk(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, int64_t n,
+            const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms, int k,
+            float* top_scores, int32_t* top_ids, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Weighted sum of dequantised vectors (the value side of attention over a compressed cache):
+ *   out[w, :] = sum_t W[w, t] * Xhat_t,   Xhat_t as in tq_dequantize.
+ *   W    device, nw rows of n floats (e.g. softmax weights), row stride ldw
+ *   out  device out, nw rows of d floats, row stride ldo
+ */
+int tq_wsum(const tq_plan* plan, const float* W, int nw, int64_t ldw, int64_t n,
+            const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms,
+            float* out, int64_t ldo, void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TQ_H_ */

@@ -1,0 +1,197 @@
+"""ctypes binding of include/tq.h.  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+TQ_MSE, TQ_PROD = 0, 1
+TQ_F32, TQ_BF16 = 0, 1
+TQ_ORTHOGONAL, TQ_GAUSSIAN = 0, 1
+TQ_OP_QUANTIZE, TQ_OP_SCORE, TQ_OP_TOPK, TQ_OP_WSUM, TQ_OP_DEQUANTIZE = 0, 1, 2, 3, 4
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libtq.so")
+_lib = None
+
+c_void_p, c_int, c_int64, c_size_t, c_u64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t, ctypes.c_uint64
+_F = ctypes.POINTER(ctypes.c_float)
+
+_SIGNATURES = {
+    "tq_last_error": (ctypes.c_char_p, []),
+    "tq_codebook": (c_int, [c_int, c_int, _F, _F]),
+    "tq_rotation": (c_int, [c_int, c_u64, c_int, _F]),
+    "tq_idx_row_bytes": (c_size_t, [c_int, c_int]),
+    "tq_qjl_row_bytes": (c_size_t, [c_int]),
+    "tq_plan_create": (c_int, [c_int, c_int, c_int, _F, _F, _F, ctypes.POINTER(c_void_p)]),
+    "tq_plan_destroy": (c_int, [c_void_p]),
+    "tq_workspace_bytes": (c_size_t, [c_void_p, c_int, c_int64, c_int, c_int]),
+    "tq_quantize_mse": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "tq_quantize_prod": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
+                                 c_void_p, c_size_t, c_void_p]),
+    "tq_dequantize": (c_int, [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p]),
+    "tq_score": (c_int, [c_void_p, c_void_p, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
+                         c_void_p, c_int64, c_void_p, c_size_t, c_void_p]),
+    "tq_topk": (c_int, [c_void_p, c_void_p, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
+                        c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "tq_wsum": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
+                        c_void_p, c_int64, c_void_p, c_size_t, c_void_p]),
+}
+
+
+class TqError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"tq error {code}: {message}")
+        self.code = code
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libtq.so (built in-tree by paper_2504_19874_b200/build.py).  Raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: run `python -m paper_2504_19874_b200.build` first "
+                               "(there is no fallback path)")
+        handle = ctypes.CDLL(_LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def _check(code: int):
+    if code != 0:
+        raise TqError(code, lib().tq_last_error().decode())
+
+
+def _fptr(a: np.ndarray):
+    return a.ctypes.data_as(_F)
+
+
+def _dev(t):
+    """Device pointer of a CUDA tensor (None -> NULL)."""
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor (this library has no CPU path)")
+    return t.data_ptr()
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return TQ_F32
+    if t.dtype == torch.bfloat16:
+        return TQ_BF16
+    raise ValueError(f"unsupported dtype {t.dtype}")
+
+
+def _rows(t: torch.Tensor):
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError("expected a 2-D tensor with unit inner stride")
+    return t.shape[0], t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def tq_idx_row_bytes(d: int, bits: int) -> int:
+    return lib().tq_idx_row_bytes(d, bits)
+
+
+def tq_qjl_row_bytes(d: int) -> int:
+    return lib().tq_qjl_row_bytes(d)
+
+
+def tq_codebook(d: int, bits: int):
+    """(centroids, boundaries) as float32 numpy arrays."""
+    levels = 1 << min(max(bits, 0), 8)        # the library rejects bits outside 0..4
+    c = np.zeros(levels, dtype=np.float32)
+    t = np.zeros(max(levels - 1, 1), dtype=np.float32)
+    _check(lib().tq_codebook(d, bits, _fptr(c), _fptr(t)))
+    return c, t[:levels - 1]
+
+
+def tq_rotation(d: int, seed: int, kind: int = TQ_ORTHOGONAL) -> np.ndarray:
+    out = np.zeros((d, d), dtype=np.float32)
+    _check(lib().tq_rotation(d, seed, kind, _fptr(out)))
+    return out
+
+
+class Plan:
+    """Owner of a tq_plan handle (device copies of Pi, S', codebook for one (d, b, mode))."""
+
+    def __init__(self, d: int, bits: int, mode: int, Pi, S, centroids):
+        Pi = np.ascontiguousarray(Pi, dtype=np.float32)
+        cent = np.ascontiguousarray(centroids, dtype=np.float32)
+        Sp = None if S is None else np.ascontiguousarray(S, dtype=np.float32)
+        if Pi.shape != (d, d) or (Sp is not None and Sp.shape != (d, d)):
+            raise ValueError("Pi and S must be d x d")
+        self.d, self.bits, self.mode = d, bits, mode
+        self.mse_bits = bits - 1 if mode == TQ_PROD else bits
+        if cent.size != (1 << max(self.mse_bits, 0)):
+            raise ValueError("centroids must hold 2^b_m values")
+        self.idx_row_bytes = tq_idx_row_bytes(d, self.mse_bits)
+        self.qjl_row_bytes = tq_qjl_row_bytes(d)
+        h = c_void_p()
+        _check(lib().tq_plan_create(d, bits, mode, _fptr(Pi), None if Sp is None else _fptr(Sp), _fptr(cent),
+                                    ctypes.byref(h)))
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().tq_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def tq_workspace_bytes(plan: Plan, op: int, n: int, nq: int = 0, k: int = 0) -> int:
+    return lib().tq_workspace_bytes(plan.handle, op, n, nq, k)
+
+
+def _scratch_args(t):
+    return (_dev(t), 0 if t is None else t.numel() * t.element_size())
+
+
+def tq_quantize_mse(plan: Plan, X, idx, norms=None, scratch=None):
+    n, ldx = _rows(X)
+    _check(lib().tq_quantize_mse(plan.handle, _dev(X), _dtype_code(X), n, ldx, _dev(idx), _dev(norms),
+                                 *_scratch_args(scratch), _stream()))
+
+
+def tq_quantize_prod(plan: Plan, X, idx, qjl, gamma, norms=None, scratch=None):
+    n, ldx = _rows(X)
+    _check(lib().tq_quantize_prod(plan.handle, _dev(X), _dtype_code(X), n, ldx, _dev(idx), _dev(qjl), _dev(gamma),
+                                  _dev(norms), *_scratch_args(scratch), _stream()))
+
+
+def tq_dequantize(plan: Plan, n: int, idx, qjl, gamma, norms, Xhat):
+    _, ld = _rows(Xhat)
+    _check(lib().tq_dequantize(plan.handle, n, _dev(idx), _dev(qjl), _dev(gamma), _dev(norms), _dev(Xhat), ld, _stream()))
+
+
+def tq_score(plan: Plan, Q, n: int, idx, qjl, gamma, norms, scores, workspace):
+    nq, ldq = _rows(Q)
+    _, lds = _rows(scores)
+    _check(lib().tq_score(plan.handle, _dev(Q), _dtype_code(Q), nq, ldq, n, _dev(idx), _dev(qjl), _dev(gamma),
+                          _dev(norms), _dev(scores), lds, *_scratch_args(workspace), _stream()))
+
+
+def tq_topk(plan: Plan, Q, n: int, idx, qjl, gamma, norms, k: int, top_scores, top_ids, workspace):
+    nq, ldq = _rows(Q)
+    _check(lib().tq_topk(plan.handle, _dev(Q), _dtype_code(Q), nq, ldq, n, _dev(idx), _dev(qjl), _dev(gamma),
+                         _dev(norms), k, _dev(top_scores), _dev(top_ids), *_scratch_args(workspace), _stream()))
+
+
+def tq_wsum(plan: Plan, W, n: int, idx, qjl, gamma, norms, out, workspace):
+    nw, ldw = _rows(W)
+    _, ldo = _rows(out)
+    _check(lib().tq_wsum(plan.handle, _dev(W), nw, ldw, n, _dev(idx), _dev(qjl), _dev(gamma), _dev(norms),
+                         _dev(out), ldo, *_scratch_args(workspace), _stream()))

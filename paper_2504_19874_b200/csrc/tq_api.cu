@@ -1,0 +1,503 @@
+// C ABI of libtq: argument checking, plan set-up and kernel dispatch.
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "tq_gemm_simt.cuh"
+#include "tq_internal.h"
+#include "tq_scan_simt.cuh"
+
+using namespace tq;
+
+namespace {
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// S' = S Pi^T in fp64 (set-up, once per plan): out[i][j] = sum_k S[i][k] Pi[j][k].
+__global__ void sprime_kernel(const float* __restrict__ S, const float* __restrict__ Pi, float* __restrict__ out, int d) {
+  __shared__ double sa[16][17], sb[16][17];
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  const int i = blockIdx.y * 16 + ty, j = blockIdx.x * 16 + tx;
+  double acc = 0.0;
+  for (int k0 = 0; k0 < d; k0 += 16) {
+    const int ia = blockIdx.y * 16 + ty, jb = blockIdx.x * 16 + ty;
+    sa[ty][tx] = (ia < d && k0 + tx < d) ? (double)S[(size_t)ia * d + k0 + tx] : 0.0;
+    sb[ty][tx] = (jb < d && k0 + tx < d) ? (double)Pi[(size_t)jb * d + k0 + tx] : 0.0;
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 16; ++k) acc += sa[ty][k] * sb[tx][k];
+    __syncthreads();
+  }
+  if (i < d && j < d) out[(size_t)i * d + j] = (float)acc;
+}
+
+int check_plan(const tq_plan* plan, const char* who) {
+  TQ_REQUIRE(plan != nullptr, TQ_ERR_INVALID_ARG, "%s: plan is NULL", who);
+  int dev = -1;
+  TQ_CHECK_CUDA(cudaGetDevice(&dev), who);
+  TQ_REQUIRE(dev == plan->device, TQ_ERR_INVALID_ARG, "%s: plan was created on device %d, current device is %d", who,
+             plan->device, dev);
+  return TQ_OK;
+}
+
+int check_rows(const char* who, const char* name, const void* p, int dtype, int64_t rows, int64_t ld, int d) {
+  TQ_REQUIRE(dtype == TQ_F32 || dtype == TQ_BF16, TQ_ERR_UNSUPPORTED, "%s: unknown dtype %d for %s", who, dtype, name);
+  TQ_REQUIRE(p != nullptr, TQ_ERR_INVALID_ARG, "%s: %s is NULL", who, name);
+  TQ_REQUIRE(ld >= d, TQ_ERR_INVALID_ARG, "%s: row stride of %s (%lld) is smaller than d (%d)", who, name, (long long)ld, d);
+  TQ_REQUIRE(aligned(p, 16), TQ_ERR_ALIGNMENT, "%s: %s is not 16-byte aligned", who, name);
+  (void)rows;
+  return TQ_OK;
+}
+
+int check_codes(const tq_plan* plan, const char* who, const uint8_t* idx, const uint8_t* qjl, const float* gamma) {
+  if (plan->mse_bits > 0) {
+    TQ_REQUIRE(idx != nullptr, TQ_ERR_INVALID_ARG, "%s: idx is NULL", who);
+    TQ_REQUIRE(aligned(idx, 16), TQ_ERR_ALIGNMENT, "%s: idx is not 16-byte aligned", who);
+  }
+  if (plan->mode == TQ_PROD) {
+    TQ_REQUIRE(qjl != nullptr && gamma != nullptr, TQ_ERR_INVALID_ARG, "%s: qjl / gamma is NULL for a TQ_PROD plan", who);
+    TQ_REQUIRE(aligned(qjl, 16) && aligned(gamma, 4), TQ_ERR_ALIGNMENT, "%s: qjl / gamma is misaligned", who);
+  }
+  return TQ_OK;
+}
+
+simt::Codes make_codes(const tq_plan* plan, int64_t n, const uint8_t* idx, const uint8_t* qjl, const float* gamma) {
+  simt::Codes c;
+  c.idx = idx;
+  c.idx_rb = plan->idx_row_bytes;
+  c.qjl = (plan->mode == TQ_PROD) ? qjl : nullptr;
+  c.qjl_rb = plan->qjl_row_bytes;
+  c.gamma = gamma;
+  c.cb = plan->cb;
+  c.d = plan->d;
+  c.dpad = plan->dpad;
+  c.coef = plan->coef;
+  c.rows = n;
+  return c;
+}
+
+size_t qcat_bytes(const tq_plan* plan, int nq) {
+  return align_up((size_t)nq * plan->ncat * plan->dpad * sizeof(float), 256);
+}
+
+constexpr int64_t kResidualChunk = 16384;  // rows of E kept in flight by tq_quantize_prod (L2-sized)
+constexpr int64_t kTopkBlockMin = 4096, kTopkBlockPref = 65536;
+constexpr int kFewQueries = 16;  // up to this many queries the code scan is bandwidth-bound
+
+template <typename T>
+cudaError_t launch_row_norm(const T* X, int64_t ld, int64_t n, int d, float* out, cudaStream_t st) {
+  if (n <= 0) return cudaSuccess;
+  const int64_t blocks = std::min<int64_t>((n + 7) / 8, 148 * 16);
+  scan::row_norm_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(X, ld, n, d, out);
+  return cudaGetLastError();
+}
+
+// Stage-1 GEMM of both quantisers: Y = X Pi^T with the nearest-centroid epilogue.
+template <int BITS, int MODE>
+cudaError_t launch_rotate_quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t ldx,
+                                   const float* nu, uint8_t* idx, float* E, int64_t ldE, cudaStream_t st) {
+  simt::EpQuantize<BITS, MODE> ep;
+  ep.cb = plan->cb;
+  ep.nu = nu;
+  ep.out = idx;
+  ep.out_rb = plan->idx_row_bytes;
+  ep.E = E;
+  ep.ldE = ldE;
+  ep.d = plan->d;
+  simt::RowsF32 B{plan->dPi, plan->d, plan->d, plan->d};
+  if (x_dtype == TQ_F32) {
+    simt::RowsF32 A{static_cast<const float*>(X), ldx, n, plan->d};
+    return simt::launch_gemm(A, B, ep, n, (int64_t)plan->d, plan->d, st);
+  }
+  simt::RowsBF16 A{static_cast<const __nv_bfloat16*>(X), ldx, n, plan->d};
+  return simt::launch_gemm(A, B, ep, n, (int64_t)plan->d, plan->d, st);
+}
+
+template <int MODE>
+cudaError_t dispatch_rotate_quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t ldx,
+                                     const float* nu, uint8_t* idx, float* E, int64_t ldE, cudaStream_t st) {
+  switch (plan->mse_bits) {
+    case 0: return launch_rotate_quantize<0, MODE>(plan, X, x_dtype, n, ldx, nu, idx, E, ldE, st);
+    case 1: return launch_rotate_quantize<1, MODE>(plan, X, x_dtype, n, ldx, nu, idx, E, ldE, st);
+    case 2: return launch_rotate_quantize<2, MODE>(plan, X, x_dtype, n, ldx, nu, idx, E, ldE, st);
+    case 3: return launch_rotate_quantize<3, MODE>(plan, X, x_dtype, n, ldx, nu, idx, E, ldE, st);
+    default: return launch_rotate_quantize<4, MODE>(plan, X, x_dtype, n, ldx, nu, idx, E, ldE, st);
+  }
+}
+
+cudaError_t compute_norms(const void* X, int x_dtype, int64_t n, int64_t ldx, int d, float* norms, cudaStream_t st) {
+  if (x_dtype == TQ_F32) return launch_row_norm(static_cast<const float*>(X), ldx, n, d, norms, st);
+  return launch_row_norm(static_cast<const __nv_bfloat16*>(X), ldx, n, d, norms, st);
+}
+
+// True when the packed rows have bytes that no 32-coordinate group writes.
+bool has_pad_words(int d, int bits, size_t row_bytes) {
+  return bits > 0 && (size_t)((d + 31) / 32) * bits * 4 < row_bytes;
+}
+
+// Q' = Q Pi^T and Q'' = Q S^T side by side: Qcat[nq, ncat*dpad].
+cudaError_t prepare_queries(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, float* Qcat,
+                            cudaStream_t st) {
+  const int ncols = plan->ncat * plan->dpad;
+  simt::RowsF32 B{plan->dRotCat, plan->d, ncols, plan->d};
+  simt::EpStore ep{Qcat, ncols, nullptr, nullptr};
+  if (q_dtype == TQ_F32) {
+    simt::RowsF32 A{static_cast<const float*>(Q), ldq, nq, plan->d};
+    return simt::launch_gemm(A, B, ep, (int64_t)nq, (int64_t)ncols, plan->d, st);
+  }
+  simt::RowsBF16 A{static_cast<const __nv_bfloat16*>(Q), ldq, nq, plan->d};
+  return simt::launch_gemm(A, B, ep, (int64_t)nq, (int64_t)ncols, plan->d, st);
+}
+
+template <int BITS, bool PROD>
+cudaError_t launch_scan_few(const scan::ScanArgs& base, int nq, cudaStream_t st) {
+  const size_t per_query = (size_t)(PROD ? 2 : 1) * 32 * base.groups * sizeof(float);
+  int tile = 8;
+  while (tile > 1 && per_query * tile > 200 * 1024) tile >>= 1;
+  if (per_query * tile > 220 * 1024) return cudaErrorInvalidConfiguration;
+  const int64_t blocks = std::min<int64_t>((base.n + 255) / 256, 148 * 2);
+  for (int q0 = 0; q0 < nq; q0 += tile) {
+    scan::ScanArgs a = base;
+    a.q0 = q0;
+    a.nq_tile = std::min(tile, nq - q0);
+    cudaError_t e = cudaSuccess;
+    const size_t smem = per_query * tile;
+#define TQ_SCAN_LAUNCH(NQ)                                                                                  \
+  e = cudaFuncSetAttribute(scan::scan_few_kernel<BITS, NQ, PROD>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                           (int)smem);                                                                      \
+  if (e == cudaSuccess) scan::scan_few_kernel<BITS, NQ, PROD><<<(unsigned)blocks, 256, smem, st>>>(a);
+    switch (tile) {
+      case 8: TQ_SCAN_LAUNCH(8) break;
+      case 4: TQ_SCAN_LAUNCH(4) break;
+      case 2: TQ_SCAN_LAUNCH(2) break;
+      default: TQ_SCAN_LAUNCH(1) break;
+    }
+#undef TQ_SCAN_LAUNCH
+    if (e != cudaSuccess) return e;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+// Scores of queries (already prepared in Qcat) against vectors [v0, v0 + cn).
+cudaError_t score_block(const tq_plan* plan, const float* Qcat, int nq, int64_t v0, int64_t cn, const uint8_t* idx,
+                        const uint8_t* qjl, const float* gamma, const float* norms, float* scores, int64_t lds,
+                        cudaStream_t st) {
+  const uint8_t* idx_b = idx ? idx + (size_t)v0 * plan->idx_row_bytes : nullptr;
+  const uint8_t* qjl_b = qjl ? qjl + (size_t)v0 * plan->qjl_row_bytes : nullptr;
+  const float* gamma_b = gamma ? gamma + v0 : nullptr;
+  const float* norms_b = norms ? norms + v0 : nullptr;
+  const int ncols = plan->ncat * plan->dpad;
+  if (nq <= kFewQueries) {
+    scan::ScanArgs a;
+    a.idx = idx_b;
+    a.idx_rb = plan->idx_row_bytes;
+    a.qjl = (plan->mode == TQ_PROD) ? qjl_b : nullptr;
+    a.qjl_rb = plan->qjl_row_bytes;
+    a.gamma = gamma_b;
+    a.norms = norms_b;
+    a.cb = plan->cb;
+    a.d = plan->d;
+    a.groups = (plan->d + 31) / 32;
+    a.coef = plan->coef;
+    a.n = cn;
+    a.Qcat = Qcat;
+    a.ldq = ncols;
+    a.dpad = plan->dpad;
+    a.q0 = 0;
+    a.nq_tile = 0;
+    a.scores = scores;
+    a.lds = lds;
+    const bool prod = plan->mode == TQ_PROD;
+    switch (plan->mse_bits) {
+      case 0: return launch_scan_few<0, true>(a, nq, st);
+      case 1: return prod ? launch_scan_few<1, true>(a, nq, st) : launch_scan_few<1, false>(a, nq, st);
+      case 2: return prod ? launch_scan_few<2, true>(a, nq, st) : launch_scan_few<2, false>(a, nq, st);
+      case 3: return prod ? launch_scan_few<3, true>(a, nq, st) : launch_scan_few<3, false>(a, nq, st);
+      default: return prod ? launch_scan_few<4, true>(a, nq, st) : launch_scan_few<4, false>(a, nq, st);
+    }
+  }
+  simt::RowsF32 A{Qcat, ncols, nq, ncols};
+  simt::Codes B = make_codes(plan, cn, idx_b, qjl_b, gamma_b);
+  simt::EpStore ep{scores, lds, nullptr, norms_b};
+  return simt::launch_gemm(A, B, ep, (int64_t)nq, cn, ncols, st);
+}
+
+}  // namespace
+
+// ======================================================================================
+extern "C" int tq_plan_create(int d, int bits, int mode, const float* Pi, const float* S, const float* centroids,
+                              tq_plan** out) {
+  const char* who = "tq_plan_create";
+  TQ_REQUIRE(out != nullptr, TQ_ERR_INVALID_ARG, "%s: out is NULL", who);
+  *out = nullptr;
+  TQ_REQUIRE(mode == TQ_MSE || mode == TQ_PROD, TQ_ERR_INVALID_ARG, "%s: unknown mode %d", who, mode);
+  TQ_REQUIRE(d >= 2 && d <= TQ_MAX_D, TQ_ERR_UNSUPPORTED, "%s: d=%d outside 2..%d", who, d, TQ_MAX_D);
+  const int mse_bits = (mode == TQ_PROD) ? bits - 1 : bits;
+  TQ_REQUIRE(bits >= 1 && mse_bits <= 4, TQ_ERR_UNSUPPORTED, "%s: bits=%d unsupported for this mode", who, bits);
+  TQ_REQUIRE(Pi != nullptr && centroids != nullptr, TQ_ERR_INVALID_ARG, "%s: Pi / centroids is NULL", who);
+  TQ_REQUIRE(mode == TQ_MSE || S != nullptr, TQ_ERR_INVALID_ARG, "%s: S is NULL for a TQ_PROD plan", who);
+  const int levels = 1 << mse_bits;
+  for (int i = 0; i < levels; ++i) {
+    TQ_REQUIRE(std::isfinite(centroids[i]), TQ_ERR_INVALID_ARG, "%s: centroid %d is not finite", who, i);
+    TQ_REQUIRE(i == 0 || centroids[i] > centroids[i - 1], TQ_ERR_INVALID_ARG, "%s: centroids must be strictly ascending", who);
+  }
+
+  tq_plan* p = new (std::nothrow) tq_plan();
+  TQ_REQUIRE(p != nullptr, TQ_ERR_INVALID_ARG, "%s: out of host memory", who);
+  std::memset(p, 0, sizeof(*p));
+  p->d = d;
+  p->dpad = round_up(d, 8);
+  p->bits = bits;
+  p->mode = mode;
+  p->mse_bits = mse_bits;
+  p->ncat = (mode == TQ_PROD) ? 2 : 1;
+  p->coef = (float)(std::sqrt(M_PI / 2.0) / d);
+  p->idx_row_bytes = tq_idx_row_bytes(d, mse_bits);
+  p->qjl_row_bytes = tq_qjl_row_bytes(d);
+  p->cb.bits = mse_bits;
+  for (int i = 0; i < 16; ++i) p->cb.c[i] = (i < levels) ? centroids[i] : 0.f;
+  for (int i = 0; i < 15; ++i) p->cb.t[i] = (i + 1 < levels) ? 0.5f * (centroids[i] + centroids[i + 1]) : INFINITY;
+
+  const size_t dd = (size_t)d * d;
+  const int ncols = p->ncat * p->dpad;
+  auto fail = [&](int code) {
+    tq_plan_destroy(p);
+    return code;
+  };
+#define PLAN_CUDA(call, what)                                        \
+  do {                                                               \
+    cudaError_t e_ = (call);                                         \
+    if (e_ != cudaSuccess) {                                         \
+      set_error("%s: %s: %s", who, what, cudaGetErrorString(e_));    \
+      return fail(TQ_ERR_CUDA);                                      \
+    }                                                                \
+  } while (0)
+  PLAN_CUDA(cudaGetDevice(&p->device), "cudaGetDevice");
+  PLAN_CUDA(cudaMalloc(&p->dPi, dd * sizeof(float)), "cudaMalloc Pi");
+  PLAN_CUDA(cudaMemcpy(p->dPi, Pi, dd * sizeof(float), cudaMemcpyHostToDevice), "copy Pi");
+  std::vector<float> rot((size_t)ncols * d, 0.f), back((size_t)d * ncols, 0.f);
+  for (int i = 0; i < d; ++i) {
+    std::memcpy(&rot[(size_t)i * d], Pi + (size_t)i * d, d * sizeof(float));
+    for (int j = 0; j < d; ++j) back[(size_t)j * ncols + i] = Pi[(size_t)i * d + j];
+  }
+  float* dS = nullptr;
+  if (mode == TQ_PROD) {
+    for (int i = 0; i < d; ++i) {
+      std::memcpy(&rot[(size_t)(p->dpad + i) * d], S + (size_t)i * d, d * sizeof(float));
+      for (int j = 0; j < d; ++j) back[(size_t)j * ncols + p->dpad + i] = S[(size_t)i * d + j];
+    }
+    PLAN_CUDA(cudaMalloc(&dS, dd * sizeof(float)), "cudaMalloc S");
+    cudaError_t e = cudaMemcpy(dS, S, dd * sizeof(float), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMalloc(&p->dSp, dd * sizeof(float));
+    if (e == cudaSuccess) {
+      dim3 grid((d + 15) / 16, (d + 15) / 16), block(16, 16);
+      sprime_kernel<<<grid, block>>>(dS, p->dPi, p->dSp, d);
+      e = cudaGetLastError();
+      if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    }
+    cudaFree(dS);
+    PLAN_CUDA(e, "S' = S Pi^T");
+  }
+  PLAN_CUDA(cudaMalloc(&p->dRotCat, rot.size() * sizeof(float)), "cudaMalloc RotCat");
+  PLAN_CUDA(cudaMemcpy(p->dRotCat, rot.data(), rot.size() * sizeof(float), cudaMemcpyHostToDevice), "copy RotCat");
+  PLAN_CUDA(cudaMalloc(&p->dBackT, back.size() * sizeof(float)), "cudaMalloc BackT");
+  PLAN_CUDA(cudaMemcpy(p->dBackT, back.data(), back.size() * sizeof(float), cudaMemcpyHostToDevice), "copy BackT");
+  PLAN_CUDA(cudaDeviceSynchronize(), "synchronize");
+#undef PLAN_CUDA
+  *out = p;
+  return TQ_OK;
+}
+
+extern "C" int tq_plan_destroy(tq_plan* plan) {
+  if (!plan) return TQ_OK;
+  cudaFree(plan->dPi);
+  cudaFree(plan->dSp);
+  cudaFree(plan->dRotCat);
+  cudaFree(plan->dBackT);
+  delete plan;
+  return TQ_OK;
+}
+
+extern "C" size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int nq, int k) {
+  if (!plan || n < 0 || nq < 0) return 0;
+  (void)k;
+  switch (op) {
+    case TQ_OP_QUANTIZE:
+      if (plan->mode != TQ_PROD || n == 0) return 0;
+      return align_up((size_t)std::min<int64_t>(n, kResidualChunk) * plan->dpad * sizeof(float), 256);
+    case TQ_OP_SCORE:
+      return qcat_bytes(plan, nq);
+    case TQ_OP_TOPK:
+      return qcat_bytes(plan, nq) + align_up((size_t)nq * std::min<int64_t>(n, kTopkBlockPref) * sizeof(float), 256);
+    case TQ_OP_WSUM:
+      return align_up((size_t)nq * plan->ncat * plan->dpad * sizeof(float), 256);
+    default:
+      return 0;
+  }
+}
+
+extern "C" int tq_quantize_mse(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t ldx, uint8_t* idx,
+                               float* norms, void* scratch, size_t scratch_bytes, void* stream) {
+  const char* who = "tq_quantize_mse";
+  (void)scratch;
+  (void)scratch_bytes;
+  int rc = check_plan(plan, who);
+  if (rc) return rc;
+  TQ_REQUIRE(plan->mode == TQ_MSE, TQ_ERR_INVALID_ARG, "%s: plan was created for TQ_PROD", who);
+  TQ_REQUIRE(n >= 0, TQ_ERR_INVALID_ARG, "%s: n is negative", who);
+  if (n == 0) return TQ_OK;
+  if ((rc = check_rows(who, "X", X, x_dtype, n, ldx, plan->d))) return rc;
+  TQ_REQUIRE(idx != nullptr, TQ_ERR_INVALID_ARG, "%s: idx is NULL", who);
+  TQ_REQUIRE(aligned(idx, 16) && aligned(norms, 4), TQ_ERR_ALIGNMENT, "%s: idx / norms is misaligned", who);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (norms) TQ_CHECK_CUDA(compute_norms(X, x_dtype, n, ldx, plan->d, norms, st), who);
+  if (has_pad_words(plan->d, plan->mse_bits, plan->idx_row_bytes))
+    TQ_CHECK_CUDA(cudaMemsetAsync(idx, 0, (size_t)n * plan->idx_row_bytes, st), who);
+  TQ_CHECK_CUDA(dispatch_rotate_quantize<0>(plan, X, x_dtype, n, ldx, norms, idx, nullptr, 0, st), who);
+  return TQ_OK;
+}
+
+extern "C" int tq_quantize_prod(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t ldx, uint8_t* idx,
+                                uint8_t* qjl, float* gamma, float* norms, void* scratch, size_t scratch_bytes,
+                                void* stream) {
+  const char* who = "tq_quantize_prod";
+  int rc = check_plan(plan, who);
+  if (rc) return rc;
+  TQ_REQUIRE(plan->mode == TQ_PROD, TQ_ERR_INVALID_ARG, "%s: plan was created for TQ_MSE", who);
+  TQ_REQUIRE(n >= 0, TQ_ERR_INVALID_ARG, "%s: n is negative", who);
+  if (n == 0) return TQ_OK;
+  if ((rc = check_rows(who, "X", X, x_dtype, n, ldx, plan->d))) return rc;
+  if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
+  TQ_REQUIRE(aligned(norms, 4), TQ_ERR_ALIGNMENT, "%s: norms is misaligned", who);
+  const size_t need = tq_workspace_bytes(plan, TQ_OP_QUANTIZE, n, 0, 0);
+  TQ_REQUIRE(scratch != nullptr && scratch_bytes >= need, TQ_ERR_WORKSPACE, "%s: scratch of %zu bytes, %zu needed", who,
+             scratch_bytes, need);
+  TQ_REQUIRE(aligned(scratch, 16), TQ_ERR_ALIGNMENT, "%s: scratch is not 16-byte aligned", who);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int d = plan->d;
+  const int64_t ldE = plan->dpad;
+  float* E = static_cast<float*>(scratch);
+  int64_t chunk = (int64_t)(scratch_bytes / ((size_t)ldE * sizeof(float)));
+  if (chunk < n) chunk = chunk / simt::BM * simt::BM;
+  chunk = std::min(chunk, n);
+  TQ_REQUIRE(chunk > 0, TQ_ERR_WORKSPACE, "%s: scratch too small for one block of rows", who);
+
+  if (norms) TQ_CHECK_CUDA(compute_norms(X, x_dtype, n, ldx, d, norms, st), who);
+  if (has_pad_words(d, plan->mse_bits, plan->idx_row_bytes))
+    TQ_CHECK_CUDA(cudaMemsetAsync(idx, 0, (size_t)n * plan->idx_row_bytes, st), who);
+  if (has_pad_words(d, 1, plan->qjl_row_bytes))
+    TQ_CHECK_CUDA(cudaMemsetAsync(qjl, 0, (size_t)n * plan->qjl_row_bytes, st), who);
+  const size_t xsz = (x_dtype == TQ_F32) ? 4 : 2;
+  for (int64_t r0 = 0; r0 < n; r0 += chunk) {
+    const int64_t rows = std::min(chunk, n - r0);
+    const void* Xc = static_cast<const char*>(X) + (size_t)r0 * ldx * xsz;
+    uint8_t* idx_c = idx ? idx + (size_t)r0 * plan->idx_row_bytes : nullptr;
+    // Stage 1: y = Pi x, idx, rotated residual e = y/nu - c[idx]   (Algorithm 2, steps idx and r)
+    TQ_CHECK_CUDA(dispatch_rotate_quantize<1>(plan, Xc, x_dtype, rows, ldx, norms ? norms + r0 : nullptr, idx_c, E, ldE, st), who);
+    // gamma = ||r|| = ||e||
+    TQ_CHECK_CUDA(launch_row_norm(E, ldE, rows, d, gamma + r0, st), who);
+    // Stage 2: qjl = sign(S r) = sign(S' e)
+    simt::EpQuantize<1, 2> ep;
+    ep.cb = plan->cb;
+    ep.nu = nullptr;
+    ep.out = qjl + (size_t)r0 * plan->qjl_row_bytes;
+    ep.out_rb = plan->qjl_row_bytes;
+    ep.E = nullptr;
+    ep.ldE = 0;
+    ep.d = d;
+    simt::RowsF32 A{E, ldE, rows, d};
+    simt::RowsF32 B{plan->dSp, d, d, d};
+    TQ_CHECK_CUDA(simt::launch_gemm(A, B, ep, rows, (int64_t)d, d, st), who);
+  }
+  return TQ_OK;
+}
+
+extern "C" int tq_dequantize(const tq_plan* plan, int64_t n, const uint8_t* idx, const uint8_t* qjl, const float* gamma,
+                             const float* norms, float* Xhat, int64_t ldxh, void* stream) {
+  const char* who = "tq_dequantize";
+  int rc = check_plan(plan, who);
+  if (rc) return rc;
+  TQ_REQUIRE(n >= 0, TQ_ERR_INVALID_ARG, "%s: n is negative", who);
+  if (n == 0) return TQ_OK;
+  if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
+  TQ_REQUIRE(Xhat != nullptr, TQ_ERR_INVALID_ARG, "%s: Xhat is NULL", who);
+  TQ_REQUIRE(ldxh >= plan->d, TQ_ERR_INVALID_ARG, "%s: ldxh < d", who);
+  TQ_REQUIRE(aligned(Xhat, 16), TQ_ERR_ALIGNMENT, "%s: Xhat is not 16-byte aligned", who);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int ncols = plan->ncat * plan->dpad;
+  simt::Codes A = make_codes(plan, n, idx, qjl, gamma);
+  simt::RowsF32 B{plan->dBackT, ncols, plan->d, ncols};
+  simt::EpStore ep{Xhat, ldxh, norms, nullptr};
+  TQ_CHECK_CUDA(simt::launch_gemm(A, B, ep, n, (int64_t)plan->d, ncols, st), who);
+  return TQ_OK;
+}
+
+extern "C" int tq_score(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, int64_t n,
+                        const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms, float* scores,
+                        int64_t lds, void* workspace, size_t workspace_bytes, void* stream) {
+  const char* who = "tq_score";
+  int rc = check_plan(plan, who);
+  if (rc) return rc;
+  TQ_REQUIRE(n >= 0 && nq >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
+  if (n == 0 || nq == 0) return TQ_OK;
+  if ((rc = check_rows(who, "Q", Q, q_dtype, nq, ldq, plan->d))) return rc;
+  if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
+  TQ_REQUIRE(scores != nullptr && lds >= n, TQ_ERR_INVALID_ARG, "%s: scores is NULL or lds < n", who);
+  TQ_REQUIRE(aligned(scores, 16), TQ_ERR_ALIGNMENT, "%s: scores is not 16-byte aligned", who);
+  const size_t need = tq_workspace_bytes(plan, TQ_OP_SCORE, n, nq, 0);
+  TQ_REQUIRE(workspace != nullptr && workspace_bytes >= need, TQ_ERR_WORKSPACE, "%s: workspace of %zu bytes, %zu needed",
+             who, workspace_bytes, need);
+  TQ_REQUIRE(aligned(workspace, 16), TQ_ERR_ALIGNMENT, "%s: workspace is not 16-byte aligned", who);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* Qcat = static_cast<float*>(workspace);
+  TQ_CHECK_CUDA(prepare_queries(plan, Q, q_dtype, nq, ldq, Qcat, st), who);
+  TQ_CHECK_CUDA(score_block(plan, Qcat, nq, 0, n, idx, qjl, gamma, norms, scores, lds, st), who);
+  return TQ_OK;
+}
+
+extern "C" int tq_topk(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, int64_t n,
+                       const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms, int k,
+                       float* top_scores, int32_t* top_ids, void* workspace, size_t workspace_bytes, void* stream) {
+  const char* who = "tq_topk";
+  int rc = check_plan(plan, who);
+  if (rc) return rc;
+  TQ_REQUIRE(n >= 0 && nq >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
+  if (nq == 0) return TQ_OK;
+  TQ_REQUIRE(n <= 0x7fffffffLL, TQ_ERR_UNSUPPORTED, "%s: ids are int32, n too large", who);
+  TQ_REQUIRE(k >= 1 && k <= TQ_MAX_K && k <= n, TQ_ERR_UNSUPPORTED, "%s: k=%d outside 1..min(n, %d)", who, k, TQ_MAX_K);
+  if ((rc = check_rows(who, "Q", Q, q_dtype, nq, ldq, plan->d))) return rc;
+  if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
+  TQ_REQUIRE(top_scores != nullptr && top_ids != nullptr, TQ_ERR_INVALID_ARG, "%s: output is NULL", who);
+  const size_t qb = qcat_bytes(plan, nq);
+  const size_t need = qb + align_up((size_t)nq * std::min<int64_t>(n, kTopkBlockMin) * sizeof(float), 256);
+  TQ_REQUIRE(workspace != nullptr && workspace_bytes >= need, TQ_ERR_WORKSPACE, "%s: workspace of %zu bytes, %zu needed",
+             who, workspace_bytes, need);
+  TQ_REQUIRE(aligned(workspace, 16), TQ_ERR_ALIGNMENT, "%s: workspace is not 16-byte aligned", who);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* Qcat = static_cast<float*>(workspace);
+  float* blockbuf = reinterpret_cast<float*>(static_cast<char*>(workspace) + qb);
+  int64_t block = (int64_t)((workspace_bytes - qb) / ((size_t)nq * sizeof(float)));
+  block = std::min(block, n);
+  if (block < n) block = block / 256 * 256;
+  TQ_CHECK_CUDA(prepare_queries(plan, Q, q_dtype, nq, ldq, Qcat, st), who);
+  for (int64_t v0 = 0; v0 < n; v0 += block) {
+    const int64_t cn = std::min(block, n - v0);
+    TQ_CHECK_CUDA(score_block(plan, Qcat, nq, v0, cn, idx, qjl, gamma, norms, blockbuf, block, st), who);
+    scan::topk_merge_kernel<<<nq, 256, 0, st>>>(blockbuf, block, v0, cn, k, v0 == 0 ? 1 : 0, top_scores, top_ids);
+    TQ_CHECK_CUDA(cudaGetLastError(), who);
+  }
+  return TQ_OK;
+}
+
+extern "C" int tq_wsum(const tq_plan* plan, const float* W, int nw, int64_t ldw, int64_t n, const uint8_t* idx,
+                       const uint8_t* qjl, const float* gamma, const float* norms, float* out, int64_t ldo,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+  (void)plan; (void)W; (void)nw; (void)ldw; (void)n; (void)idx; (void)qjl; (void)gamma; (void)norms;
+  (void)out; (void)ldo; (void)workspace; (void)workspace_bytes; (void)stream;
+  set_error("tq_wsum: not implemented yet");
+  return TQ_ERR_UNSUPPORTED;
+}

@@ -1,0 +1,63 @@
+// Internal declarations shared by the translation units of libtq (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+
+#include <cstdarg>
+#include <cstdint>
+#include <cstdio>
+
+#include "tq.h"
+
+namespace tq {
+
+void set_error(const char* fmt, ...);
+int lloyd_max(int d, int bits, double* c_out);
+
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+inline int64_t round_up64(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
+
+// Codebook and thresholds by value, so kernels get them through the parameter space.
+struct Codebook {
+  float c[16];   // centroids, ascending
+  float t[15];   // boundaries fl32(0.5f * (c_i + c_{i+1}))
+  int bits;      // b_m
+};
+
+}  // namespace tq
+
+// Per-(d, b, mode) device state: the "global parameters" of Algorithms 1 and 2.
+struct tq_plan {
+  int d;          // dimension
+  int dpad;       // d rounded up to a multiple of 8 (virtual K extent of one code half)
+  int bits;       // total bits b
+  int mode;       // TQ_MSE / TQ_PROD
+  int mse_bits;   // b_m
+  int device;
+  float coef;     // sqrt(pi/2) / d
+  size_t idx_row_bytes, qjl_row_bytes;
+  tq::Codebook cb;
+  float* dPi;      // [d, d]            y = Pi x            (rows of Pi)
+  float* dSp;      // [d, d]            S' = S Pi^T         (TQ_PROD)
+  float* dRotCat;  // [ncat*dpad, d]    rows: Pi (padded to dpad rows) then S     (query preparation)
+  float* dBackT;   // [d, ncat*dpad]    row j: [ Pi[:, j] | S[:, j] ]             (dequantisation)
+  int ncat;        // 1 (mse) or 2 (prod): halves of the virtual K axis [ c[idx] | coef*gamma*z ]
+};
+
+#define TQ_CHECK_CUDA(call, what)                                                        \
+  do {                                                                                   \
+    cudaError_t e_ = (call);                                                             \
+    if (e_ != cudaSuccess) {                                                             \
+      tq::set_error("%s: %s", what, cudaGetErrorString(e_));                             \
+      return TQ_ERR_CUDA;                                                                \
+    }                                                                                    \
+  } while (0)
+
+#define TQ_REQUIRE(cond, code, ...)                                                      \
+  do {                                                                                   \
+    if (!(cond)) {                                                                       \
+      tq::set_error(__VA_ARGS__);                                                        \
+      return code;                                                                       \
+    }                                                                                    \
+  } while (0)
