@@ -1,0 +1,367 @@
+"""Benchmark of the TurboQuant hot path on B200.
+
+One "step" = one pass of the whole hot path over one batch of synthetic vectors:
+  Quant_prod (rotate, nearest centroid, pack, residual, QJL signs, norms) of n vectors, then the
+  packed-code inner-product scan of nq rotated queries against those codes with top-k selection.
+Workload at N = 1: d = 1536, b = 4 (3-bit MSE stage + 1-bit QJL), n = 1,000,000 embedding-like
+vectors, nq = 8 queries, k = 100 (the configuration the headline metric is quoted on).
+
+  python bench.py --gpus N --steps K --warmup W          (N > 1: launched by torch.distributed.run)
+  python bench.py --impl reference ...                   (times the CPU oracle on a bounded sample)
+
+Prints ONE JSON line.  `value` is vectors/s through the whole step with inputs resident in HBM;
+`e2e` is the same with the inputs starting in pinned host memory and the codes and top-k
+returned to the host.  Vectors shard across GPUs with no exchange in the quantise phase; the
+top-k lists of the shards are all-gathered (nq*k*8 bytes per rank) and merged.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "quantize+scan throughput at d=1536, b=4 (TurboQuant_prod), n=1M, nq=8, top-100"
+UNIT = "vectors/s"
+WORKLOAD = {"name": "c4", "bits": 4, "mode": "prod", "n": 1_000_000, "nq": 8, "k": 100}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--n", type=int, default=WORKLOAD["n"], help="vectors per GPU (smaller only for profiling runs)")
+    ap.add_argument("--nq", type=int, default=WORKLOAD["nq"])
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [v for v in sm if v > 0.5 * max(sm)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------
+def cpu_oracle_sample(d, bits, nq, k, sample_n, Pi=None, S=None):
+    """Times the oracle (as it stands) on `sample_n` vectors of the workload: Quant_prod, then
+    DeQuant_prod + inner products + top-k for nq queries.  Returns (seconds, threads)."""
+    import numpy as np
+    import threadpoolctl
+
+    import tq_workloads as wl
+    from oracle import turboquant_oracle as orc
+    cfg = wl.CONFIGS[WORKLOAD["name"]]
+    X = wl.database(cfg, sample_n).numpy()
+    Q = wl.queries(cfg, nq).numpy()
+    Pi = orc.rotation(d, cfg.pi_seed).astype(np.float32) if Pi is None else Pi
+    S = orc.projection(d, cfg.s_seed).astype(np.float32) if S is None else S
+    c = orc.codebook(d, bits - 1).astype(np.float32)
+    threads = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info() if p.get("user_api") == "blas"] or [1])
+    t0 = time.perf_counter()
+    idx, z, gamma, nu = orc.quant_prod(X, Pi, S, c)
+    Xh = orc.dequant_prod(idx, z, gamma, nu, Pi, S, c)
+    orc.topk(orc.score(Q, Xh), min(k, sample_n))
+    return time.perf_counter() - t0, threads, (Pi, S)
+
+
+def run_reference(args):
+    """The reference arm is the CPU oracle: each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import tq_workloads as wl
+    d = wl.CONFIGS[WORKLOAD["name"]].d
+    sample = 8192
+    mats = None
+    times = []
+    for it in range(args.warmup + args.steps):
+        dt, threads, mats = cpu_oracle_sample(d, WORKLOAD["bits"], args.nq, WORKLOAD["k"], sample, *(mats or (None, None)))
+        if it >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = sample * len(times) / total
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"c4 d={d} prod b=4, sample of {sample} vectors per step, nq={args.nq}, k=100"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": f"{sample} vectors x {args.nq} queries per step"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------
+def run_b200(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import paper_2504_19874_b200 as tq
+    import tq_workloads as wl
+    from paper_2504_19874_b200 import build as tq_build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    tq_build.build()
+    tq.lib()
+
+    cfg = wl.CONFIGS[WORKLOAD["name"]]
+    d, bits, n, nq, k = cfg.d, WORKLOAD["bits"], args.n, args.nq, WORKLOAD["k"]
+    Pi = tq.tq_rotation(d, cfg.pi_seed)
+    S = tq.tq_rotation(d, cfg.s_seed, tq.TQ_GAUSSIAN)
+    cent, _ = tq.tq_codebook(d, bits - 1)
+    plan = tq.Plan(d, bits, tq.TQ_PROD, Pi, S, cent)
+
+    # Synthetic inputs, resident in HBM before the timed region (each rank draws its own shard).
+    X = wl.make_vectors(cfg, n, cfg.data_seed + 1000 * rank, dev)
+    Q = wl.queries(cfg, nq, dev)
+    idx = torch.empty((n, plan.idx_row_bytes), dtype=torch.uint8, device=dev)
+    qjl = torch.empty((n, plan.qjl_row_bytes), dtype=torch.uint8, device=dev)
+    gamma = torch.empty(n, dtype=torch.float32, device=dev)
+    norms = torch.empty(n, dtype=torch.float32, device=dev)
+    scratch = torch.empty(max(tq.tq_workspace_bytes(plan, tq.TQ_OP_QUANTIZE, n), 16), dtype=torch.uint8, device=dev)
+    ws = torch.empty(max(tq.tq_workspace_bytes(plan, tq.TQ_OP_TOPK, n, nq, k), 16), dtype=torch.uint8, device=dev)
+    top_s = torch.empty((nq, k), dtype=torch.float32, device=dev)
+    top_i = torch.empty((nq, k), dtype=torch.int32, device=dev)
+    gathered_s = torch.empty((world, nq, k), dtype=torch.float32, device=dev) if world > 1 else None
+    gathered_i = torch.empty((world, nq, k), dtype=torch.int32, device=dev) if world > 1 else None
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    phase_ms = {"quantize": [], "scan": []}
+
+    def step(record: bool):
+        e0, e1, e2 = ev(), ev(), ev()
+        e0.record()
+        tq.tq_quantize_prod(plan, X, idx, qjl, gamma, norms, scratch)
+        e1.record()
+        tq.tq_topk(plan, Q, n, idx, qjl, gamma, norms, k, top_s, top_i, ws)
+        if world > 1:
+            dist.all_gather_into_tensor(gathered_s, top_s)
+            dist.all_gather_into_tensor(gathered_i, top_i + rank * n)
+            allc = gathered_s.permute(1, 0, 2).reshape(nq, world * k)
+            best = torch.topk(allc, k, dim=1)       # merge of world*k candidates per query
+            _ = best
+        e2.record()
+        if record:
+            return e0, e1, e2
+        return None
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step(False)
+    barrier()
+    launches0 = tq.tq_launch_count()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    t_start = ev()
+    t_end = ev()
+    t_start.record()
+    evs = [step(True) for _ in range(args.steps)]
+    t_end.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    launches = tq.tq_launch_count() - launches0
+    total_ms = t_start.elapsed_time(t_end)
+    for e0, e1, e2 in evs:
+        phase_ms["quantize"].append(e0.elapsed_time(e1))
+        phase_ms["scan"].append(e1.elapsed_time(e2))
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = t.item()
+    ms_per_step = total_ms / args.steps
+    value = world * n / (ms_per_step * 1e-3)
+
+    # ---- end to end: inputs start in pinned host memory, codes and top-k go back to the host ----
+    e2e = None
+    if not args.no_e2e:
+        chunk = 65536
+        hX = torch.empty((n, d), dtype=torch.float32).pin_memory()
+        hX.copy_(X)
+        h_idx = torch.empty((n, plan.idx_row_bytes), dtype=torch.uint8).pin_memory()
+        h_qjl = torch.empty((n, plan.qjl_row_bytes), dtype=torch.uint8).pin_memory()
+        h_gamma = torch.empty(n, dtype=torch.float32).pin_memory()
+        h_norms = torch.empty(n, dtype=torch.float32).pin_memory()
+        h_ts = torch.empty((nq, k), dtype=torch.float32).pin_memory()
+        h_ti = torch.empty((nq, k), dtype=torch.int32).pin_memory()
+        hQ = Q.cpu().pin_memory()
+        copy_stream = torch.cuda.Stream(device=dev)
+        out_stream = torch.cuda.Stream(device=dev)
+        stage = [torch.empty((chunk, d), dtype=torch.float32, device=dev) for _ in range(2)]
+        dQ = torch.empty_like(Q)
+
+        def e2e_step():
+            main = torch.cuda.current_stream()
+            ready = [None, None]
+            freed = [None, None]
+            done_evs = []
+            for ci, r0 in enumerate(range(0, n, chunk)):
+                rows = min(chunk, n - r0)
+                b = ci & 1
+                with torch.cuda.stream(copy_stream):
+                    if freed[b] is not None:
+                        copy_stream.wait_event(freed[b])
+                    stage[b][:rows].copy_(hX[r0:r0 + rows], non_blocking=True)
+                    ready[b] = torch.cuda.Event()
+                    ready[b].record(copy_stream)
+                main.wait_event(ready[b])
+                tq.tq_quantize_prod(plan, stage[b][:rows], idx[r0:r0 + rows], qjl[r0:r0 + rows], gamma[r0:r0 + rows],
+                                    norms[r0:r0 + rows], scratch)
+                freed[b] = torch.cuda.Event()
+                freed[b].record(main)
+                with torch.cuda.stream(out_stream):
+                    out_stream.wait_event(freed[b])
+                    h_idx[r0:r0 + rows].copy_(idx[r0:r0 + rows], non_blocking=True)
+                    h_qjl[r0:r0 + rows].copy_(qjl[r0:r0 + rows], non_blocking=True)
+                    h_gamma[r0:r0 + rows].copy_(gamma[r0:r0 + rows], non_blocking=True)
+                    h_norms[r0:r0 + rows].copy_(norms[r0:r0 + rows], non_blocking=True)
+            dQ.copy_(hQ, non_blocking=True)
+            tq.tq_topk(plan, dQ, n, idx, qjl, gamma, norms, k, top_s, top_i, ws)
+            h_ts.copy_(top_s, non_blocking=True)
+            h_ti.copy_(top_i, non_blocking=True)
+            done = torch.cuda.Event()
+            done.record(out_stream)
+            main.wait_event(done)
+
+        e2e_step()
+        barrier()
+        a, b_ = ev(), ev()
+        a.record()
+        reps = max(1, min(args.steps, 3))
+        for _ in range(reps):
+            e2e_step()
+        b_.record()
+        barrier()
+        e2e_ms = a.elapsed_time(b_) / reps
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = t.item()
+        h2d = n * d * 4 + nq * d * 4
+        d2h = n * (plan.idx_row_bytes + plan.qjl_row_bytes + 8) + nq * k * 8
+        e2e = {"value": world * n / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        del hX, stage
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    q_ms = statistics.mean(phase_ms["quantize"])
+    s_ms = statistics.mean(phase_ms["scan"])
+    code_bytes = n * (plan.idx_row_bytes + plan.qjl_row_bytes + 8)
+    passes = math.ceil(nq / 8)                     # the few-query scan streams the codes once per 8 queries
+    scan_gbs = code_bytes * passes / (s_ms * 1e-3) / 1e9
+    # Dominant kernels: the two d x d contractions of Quant_prod (4 n d^2 flops in all).
+    gemm_flops = 4.0 * n * d * d
+    achieved_tf = gemm_flops / (q_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "rotate+quantize GEMMs (Y = X Pi^T, Z = E S'^T)",
+                "achieved": achieved_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": achieved_tf / peaks["bf16_tflops_sustained"], "traffic": None,
+                "peak_source": f"bf16 sustained, of {peaks['source']}",
+                "note": "algorithmic flops (one pass); duration = quantize phase of the step (CUDA events)"}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"c4: d={d}, TurboQuant_prod b={bits}, n={n} per GPU, nq={nq}, top-{k}",
+                       "l2": "inputs (6.1 GB of vectors, 0.78 GB of codes) are larger than L2; no flush needed"},
+            "quantize_vectors_per_s": n / (q_ms * 1e-3), "quantize_ms": q_ms,
+            "scan_ms": s_ms, "scan_codes_gbs": scan_gbs, "scan_frac_hbm": scan_gbs / peaks["hbm_gbs"],
+            "scan_queries_per_s": nq / (s_ms * 1e-3),
+            "roofline": roofline, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches)}
+    if not args.no_cpu_baseline:
+        sample = 32768
+        dt, threads, _ = cpu_oracle_sample(d, bits, nq, k, sample)
+        line["cpu_baseline"] = {"value": sample / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": f"{sample} vectors x {nq} queries, {dt:.1f} s"}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_b200(a)

@@ -65,6 +65,10 @@ typedef struct tq_plan tq_plan;
 /* Message of the last error raised on the calling thread ("" if none). Never NULL. */
 const char* tq_last_error(void);
 
+/* Number of kernels this library has enqueued so far in this process (all threads, all
+ * devices).  Diagnostic only: lets a harness verify that the CUDA path did the work. */
+uint64_t tq_launch_count(void);
+
 /*
  * Lloyd-Max codebook of Eq. (4): the 2^bits centroids c_1 <= ... <= c_{2^bits} in [-1,1] that
  * minimise the scalar k-means cost for the coordinate density of Lemma 1,

@@ -20,6 +20,7 @@ _F = ctypes.POINTER(ctypes.c_float)
 
 _SIGNATURES = {
     "tq_last_error": (ctypes.c_char_p, []),
+    "tq_launch_count": (c_u64, []),
     "tq_codebook": (c_int, [c_int, c_int, _F, _F]),
     "tq_rotation": (c_int, [c_int, c_u64, c_int, _F]),
     "tq_idx_row_bytes": (c_size_t, [c_int, c_int]),
@@ -95,6 +96,10 @@ def _rows(t: torch.Tensor):
 
 def _stream():
     return torch.cuda.current_stream().cuda_stream
+
+
+def tq_launch_count() -> int:
+    return lib().tq_launch_count()
 
 
 def tq_idx_row_bytes(d: int, bits: int) -> int:

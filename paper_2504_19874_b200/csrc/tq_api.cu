@@ -91,6 +91,7 @@ cudaError_t launch_row_norm(const T* X, int64_t ld, int64_t n, int d, float* out
   if (n <= 0) return cudaSuccess;
   const int64_t blocks = std::min<int64_t>((n + 7) / 8, 148 * 16);
   scan::row_norm_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(X, ld, n, d, out);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -176,6 +177,7 @@ cudaError_t launch_scan_few(const scan::ScanArgs& base, int nq, cudaStream_t st)
     }
 #undef TQ_SCAN_LAUNCH
     if (e != cudaSuccess) return e;
+    count_launches(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
@@ -488,6 +490,7 @@ extern "C" int tq_topk(const tq_plan* plan, const void* Q, int q_dtype, int nq, 
     const int64_t cn = std::min(block, n - v0);
     TQ_CHECK_CUDA(score_block(plan, Qcat, nq, v0, cn, idx, qjl, gamma, norms, blockbuf, block, st), who);
     scan::topk_merge_kernel<<<nq, 256, 0, st>>>(blockbuf, block, v0, cn, k, v0 == 0 ? 1 : 0, top_scores, top_ids);
+    count_launches(1);
     TQ_CHECK_CUDA(cudaGetLastError(), who);
   }
   return TQ_OK;

@@ -290,6 +290,7 @@ inline cudaError_t launch_gemm(const AL& A, const BL& B, const EP& ep, int64_t M
   const int64_t blocks = tiles_n * tiles_m;
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
   gemm_tn_kernel<AL, BL, EP><<<(unsigned)blocks, NT, 0, st>>>(A, B, ep, M, N, K, tiles_n);
+  count_launches(1);
   return cudaGetLastError();
 }
 

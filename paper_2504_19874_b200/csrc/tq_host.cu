@@ -4,6 +4,7 @@
 #include "tq_internal.h"
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <vector>
@@ -11,6 +12,9 @@
 namespace tq {
 
 static thread_local char g_err[512] = "";
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launches(int k) { g_launches.fetch_add((unsigned long long)k, std::memory_order_relaxed); }
 
 void set_error(const char* fmt, ...) {
   va_list ap;
@@ -206,6 +210,8 @@ static void householder_q(int d, std::vector<double>& a /* d*d, column j at a[j*
 using namespace tq;
 
 extern "C" const char* tq_last_error(void) { return g_err; }
+
+extern "C" uint64_t tq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 extern "C" size_t tq_idx_row_bytes(int d, int bits) {
   if (d <= 0 || bits <= 0) return 0;

@@ -13,6 +13,7 @@
 namespace tq {
 
 void set_error(const char* fmt, ...);
+void count_launches(int k);   // kernels enqueued by this library (diagnostic counter)
 int lloyd_max(int d, int bits, double* c_out);
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
