@@ -114,9 +114,17 @@ int tq_plan_create(int d, int bits, int mode, const float* Pi, const float* S,
                    const float* centroids, tq_plan** out);
 int tq_plan_destroy(tq_plan* plan);
 
-/* Bytes of device scratch the given operation needs (0 if none).  For TQ_OP_TOPK and
- * TQ_OP_SCORE any size >= the returned minimum is accepted; larger buffers let the scan work
- * on bigger blocks of vectors.   op = TQ_OP_*;  nq, k ignored where they do not apply. */
+/* Synchronises the device and reports whether any kernel launched for this plan since the
+ * last call gave up one of its bounded device-side waits (TQ_ERR_TIMEOUT; the outputs of that
+ * call are then invalid).  Every producer/consumer wait inside the tensor-core kernels has a
+ * time limit so that a stalled pipeline ends as this status instead of a hung GPU. */
+int tq_plan_status(tq_plan* plan);
+
+/* Bytes of device scratch the given operation asks for (0 if none).  For TQ_OP_QUANTIZE and
+ * TQ_OP_TOPK this is the preferred size: any buffer that holds at least one block of rows is
+ * accepted (the value returned for n = 128 resp. the SCORE size plus nq*4096 floats), larger
+ * buffers mean fewer, bigger launches.   op = TQ_OP_*;  nq, k ignored where they do not apply.
+ * Scratch must be 256-byte aligned. */
 size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int nq, int k);
 
 /*
@@ -130,6 +138,8 @@ size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int nq, int k)
  */
 int tq_quantize_mse(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t ldx,
                     uint8_t* idx, float* norms, void* scratch, size_t scratch_bytes, void* stream);
+/*   scratch  device, sized by tq_workspace_bytes(plan, TQ_OP_QUANTIZE, n, 0, 0): holds the bf16
+ *            operand splits of a block of rows (d >= 128); may be NULL when that size is 0. */
 
 /*
  * Quant_prod of Algorithm 2 for n vectors (plan mode TQ_PROD): idx at b-1 bits, qjl = sign(S r)

@@ -27,6 +27,7 @@ _SIGNATURES = {
     "tq_qjl_row_bytes": (c_size_t, [c_int]),
     "tq_plan_create": (c_int, [c_int, c_int, c_int, _F, _F, _F, ctypes.POINTER(c_void_p)]),
     "tq_plan_destroy": (c_int, [c_void_p]),
+    "tq_plan_status": (c_int, [c_void_p]),
     "tq_workspace_bytes": (c_size_t, [c_void_p, c_int, c_int64, c_int, c_int]),
     "tq_quantize_mse": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "tq_quantize_prod": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -155,6 +156,11 @@ class Plan:
             self.close()
         except Exception:
             pass
+
+
+def tq_plan_status(plan: Plan) -> None:
+    """Synchronises and raises TqError(6) if a kernel of this plan gave up a bounded wait."""
+    _check(lib().tq_plan_status(plan.handle))
 
 
 def tq_workspace_bytes(plan: Plan, op: int, n: int, nq: int = 0, k: int = 0) -> int:

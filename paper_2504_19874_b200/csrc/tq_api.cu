@@ -6,6 +6,7 @@
 
 #include "tq_gemm_simt.cuh"
 #include "tq_internal.h"
+#include "tq_quantize_tc.h"
 #include "tq_scan_simt.cuh"
 
 using namespace tq;
@@ -82,6 +83,7 @@ size_t qcat_bytes(const tq_plan* plan, int nq) {
   return align_up((size_t)nq * plan->ncat * plan->dpad * sizeof(float), 256);
 }
 
+constexpr int64_t kTensorChunk = 65536;    // rows per launch the tensor-core quantiser asks scratch for
 constexpr int64_t kResidualChunk = 16384;  // rows of E kept in flight by tq_quantize_prod (L2-sized)
 constexpr int64_t kTopkBlockMin = 4096, kTopkBlockPref = 65536;
 constexpr int kFewQueries = 16;  // up to this many queries the code scan is bandwidth-bound
@@ -308,6 +310,15 @@ extern "C" int tq_plan_create(int d, int bits, int mode, const float* Pi, const 
   PLAN_CUDA(cudaMemcpy(p->dRotCat, rot.data(), rot.size() * sizeof(float), cudaMemcpyHostToDevice), "copy RotCat");
   PLAN_CUDA(cudaMalloc(&p->dBackT, back.size() * sizeof(float)), "cudaMalloc BackT");
   PLAN_CUDA(cudaMemcpy(p->dBackT, back.data(), back.size() * sizeof(float), cudaMemcpyHostToDevice), "copy BackT");
+  PLAN_CUDA(cudaMalloc(&p->d_status, sizeof(int)), "cudaMalloc status");
+  PLAN_CUDA(cudaMemset(p->d_status, 0, sizeof(int)), "clear status");
+  if (tc::supported(d)) {
+    p->tc_bn = tc::pick_bn(d);
+    PLAN_CUDA(tc::build_matrix_limbs(p->dPi, d, d, p->dpad, p->tc_bn, &p->pi_limbs), "bf16 limbs of Pi");
+    if (mode == TQ_PROD)
+      PLAN_CUDA(tc::build_matrix_limbs(p->dSp, d, d, p->dpad, p->tc_bn, &p->sp_limbs), "bf16 limbs of S'");
+    p->tc_ok = 1;
+  }
   PLAN_CUDA(cudaDeviceSynchronize(), "synchronize");
 #undef PLAN_CUDA
   *out = p;
@@ -320,7 +331,24 @@ extern "C" int tq_plan_destroy(tq_plan* plan) {
   cudaFree(plan->dSp);
   cudaFree(plan->dRotCat);
   cudaFree(plan->dBackT);
+  cudaFree(plan->d_status);
+  tc::free_matrix_limbs(&plan->pi_limbs);
+  tc::free_matrix_limbs(&plan->sp_limbs);
   delete plan;
+  return TQ_OK;
+}
+
+extern "C" int tq_plan_status(tq_plan* plan) {
+  const char* who = "tq_plan_status";
+  TQ_REQUIRE(plan != nullptr, TQ_ERR_INVALID_ARG, "%s: plan is NULL", who);
+  TQ_CHECK_CUDA(cudaDeviceSynchronize(), who);
+  int st = 0;
+  TQ_CHECK_CUDA(cudaMemcpy(&st, plan->d_status, sizeof(int), cudaMemcpyDeviceToHost), who);
+  if (st != 0) {
+    cudaMemset(plan->d_status, 0, sizeof(int));
+    set_error("%s: a kernel gave up a bounded wait (pipeline stall); results of that call are invalid", who);
+    return TQ_ERR_TIMEOUT;
+  }
   return TQ_OK;
 }
 
@@ -329,7 +357,10 @@ extern "C" size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int
   (void)k;
   switch (op) {
     case TQ_OP_QUANTIZE:
-      if (plan->mode != TQ_PROD || n == 0) return 0;
+      if (n == 0) return 0;
+      if (plan->tc_ok)
+        return align_up((size_t)std::min<int64_t>(round_up64(n, 128), kTensorChunk) * tc::scratch_bytes_per_row(plan), 256);
+      if (plan->mode != TQ_PROD) return 0;
       return align_up((size_t)std::min<int64_t>(n, kResidualChunk) * plan->dpad * sizeof(float), 256);
     case TQ_OP_SCORE:
       return qcat_bytes(plan, nq);
@@ -345,8 +376,6 @@ extern "C" size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int
 extern "C" int tq_quantize_mse(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t ldx, uint8_t* idx,
                                float* norms, void* scratch, size_t scratch_bytes, void* stream) {
   const char* who = "tq_quantize_mse";
-  (void)scratch;
-  (void)scratch_bytes;
   int rc = check_plan(plan, who);
   if (rc) return rc;
   TQ_REQUIRE(plan->mode == TQ_MSE, TQ_ERR_INVALID_ARG, "%s: plan was created for TQ_PROD", who);
@@ -356,6 +385,13 @@ extern "C" int tq_quantize_mse(const tq_plan* plan, const void* X, int x_dtype, 
   TQ_REQUIRE(idx != nullptr, TQ_ERR_INVALID_ARG, "%s: idx is NULL", who);
   TQ_REQUIRE(aligned(idx, 16) && aligned(norms, 4), TQ_ERR_ALIGNMENT, "%s: idx / norms is misaligned", who);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (plan->tc_ok) {
+    const size_t need = tq_workspace_bytes(plan, TQ_OP_QUANTIZE, std::min<int64_t>(n, 128), 0, 0);
+    TQ_REQUIRE(scratch != nullptr && scratch_bytes >= need, TQ_ERR_WORKSPACE, "%s: scratch of %zu bytes, at least %zu needed",
+               who, scratch_bytes, need);
+    TQ_REQUIRE(aligned(scratch, 256), TQ_ERR_ALIGNMENT, "%s: scratch is not 256-byte aligned", who);
+    return tc::quantize(plan, X, x_dtype, n, ldx, idx, nullptr, nullptr, norms, scratch, scratch_bytes, st, who);
+  }
   if (norms) TQ_CHECK_CUDA(compute_norms(X, x_dtype, n, ldx, plan->d, norms, st), who);
   if (has_pad_words(plan->d, plan->mse_bits, plan->idx_row_bytes))
     TQ_CHECK_CUDA(cudaMemsetAsync(idx, 0, (size_t)n * plan->idx_row_bytes, st), who);
@@ -375,11 +411,18 @@ extern "C" int tq_quantize_prod(const tq_plan* plan, const void* X, int x_dtype,
   if ((rc = check_rows(who, "X", X, x_dtype, n, ldx, plan->d))) return rc;
   if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
   TQ_REQUIRE(aligned(norms, 4), TQ_ERR_ALIGNMENT, "%s: norms is misaligned", who);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (plan->tc_ok) {
+    const size_t least = tq_workspace_bytes(plan, TQ_OP_QUANTIZE, std::min<int64_t>(n, 128), 0, 0);
+    TQ_REQUIRE(scratch != nullptr && scratch_bytes >= least, TQ_ERR_WORKSPACE,
+               "%s: scratch of %zu bytes, at least %zu needed", who, scratch_bytes, least);
+    TQ_REQUIRE(aligned(scratch, 256), TQ_ERR_ALIGNMENT, "%s: scratch is not 256-byte aligned", who);
+    return tc::quantize(plan, X, x_dtype, n, ldx, idx, qjl, gamma, norms, scratch, scratch_bytes, st, who);
+  }
   const size_t need = tq_workspace_bytes(plan, TQ_OP_QUANTIZE, n, 0, 0);
   TQ_REQUIRE(scratch != nullptr && scratch_bytes >= need, TQ_ERR_WORKSPACE, "%s: scratch of %zu bytes, %zu needed", who,
              scratch_bytes, need);
   TQ_REQUIRE(aligned(scratch, 16), TQ_ERR_ALIGNMENT, "%s: scratch is not 16-byte aligned", who);
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int d = plan->d;
   const int64_t ldE = plan->dpad;
   float* E = static_cast<float*>(scratch);

@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of libtq (not part of the ABI).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 
@@ -26,6 +27,15 @@ struct Codebook {
   int bits;      // b_m
 };
 
+// A d x d fp32 matrix split into two bf16 limbs (M = hi + lo + O(2^-17)), rows padded to dpad,
+// with the TMA descriptors the tensor-core GEMM uses for it as the B operand.
+struct MatrixLimbs {
+  __nv_bfloat16* hi;
+  __nv_bfloat16* lo;
+  alignas(64) CUtensorMap map_hi;
+  alignas(64) CUtensorMap map_lo;
+};
+
 }  // namespace tq
 
 // Per-(d, b, mode) device state: the "global parameters" of Algorithms 1 and 2.
@@ -44,6 +54,12 @@ struct tq_plan {
   float* dRotCat;  // [ncat*dpad, d]    rows: Pi (padded to dpad rows) then S     (query preparation)
   float* dBackT;   // [d, ncat*dpad]    row j: [ Pi[:, j] | S[:, j] ]             (dequantisation)
   int ncat;        // 1 (mse) or 2 (prod): halves of the virtual K axis [ c[idx] | coef*gamma*z ]
+  // tensor-core quantisation path (d >= 128)
+  int tc_ok;       // 1 when the limbs / TMA descriptors below are built
+  int tc_bn;       // N extent of its MMA tile
+  tq::MatrixLimbs pi_limbs;   // Pi
+  tq::MatrixLimbs sp_limbs;   // S' (TQ_PROD)
+  int* d_status;   // device word: set to TQ_ERR_TIMEOUT by a kernel whose bounded wait ran out
 };
 
 #define TQ_CHECK_CUDA(call, what)                                                        \

@@ -1,0 +1,539 @@
+// Tensor-core quantisation path (sm_100a): the rotation y = Pi u and the QJL projection
+// z = S' e as tcgen05 GEMMs fed by TMA, with the nearest-centroid search, bit packing,
+// residual and sign extraction fused into the epilogue that reads the accumulators from TMEM.
+//
+// fp32 fidelity on bf16 tensor cores: every fp32 operand is split into two bf16 limbs
+// (v = hi + lo + O(2^-17 |v|)), and each product is formed as hi*hi + hi*lo + lo*hi with fp32
+// accumulation (3 MMA passes).  The dropped terms are ~2^-17 relative per product, i.e.
+// ~1e-7 on a rotated coordinate of a unit vector at d = 1536 -- far inside the 1e-5 window in
+// which a nearest-centroid decision may legitimately differ from exact arithmetic.
+#include <algorithm>
+#include <mutex>
+
+#include "tq_quantize_tc.h"
+#include "tq_tc.cuh"
+
+namespace tq {
+namespace tc {
+
+namespace {
+
+constexpr int BM = 128;          // rows of X per tile = TMEM lanes
+constexpr int BK = 64;           // bf16 elements per 128-byte swizzled row
+constexpr int UMMA_K = 16;
+constexpr int NTHREADS = 192;    // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+
+template <int BN>
+struct Cfg {
+  static constexpr int kStageBytes = 2 * BM * BK * 2 + 2 * BN * BK * 2;   // A hi/lo + B hi/lo
+  static constexpr int kStages = (BN == 256) ? 2 : (BN == 128 ? 3 : 4);
+  static constexpr int kTmemCols = 2 * BN;                                  // two accumulators
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+struct GemmArgs {
+  int64_t M;             // valid rows
+  int N, K;              // = d, d
+  int tiles_m, tiles_n;
+  Codebook cb;
+  uint8_t* out;          // packed idx (MODE 0/1) or qjl (MODE 2) rows
+  size_t out_rb;
+  __nv_bfloat16* E1;     // MODE 1: residual limbs, pitch ldE
+  __nv_bfloat16* E2;
+  int64_t ldE;
+  float* gpart;          // MODE 1: [tiles_n][Mpad] partial sums of e^2
+  int64_t Mpad;
+  const float* nu;       // MODE 1: per-row norm (row with nu == 0 has residual 0); nullable
+  int* status;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// MODE 0: idx.  MODE 1: idx + residual limbs + partial ||e||^2.  MODE 2: sign bits.
+template <int BN, int MODE, int BITS>
+__global__ void __launch_bounds__(NTHREADS, 1)
+quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2,
+                     const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmArgs a) {
+  using C = Cfg<BN>;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kStages * C::kStageBytes);
+  uint64_t* full = bars;                    // [kStages]  TMA -> MMA
+  uint64_t* empty = bars + C::kStages;      // [kStages]  MMA -> TMA
+  uint64_t* tfull = bars + 2 * C::kStages;  // [2]        MMA -> epilogue
+  uint64_t* tempty = tfull + 2;             // [2]        epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_kb = (a.K + BK - 1) / BK;
+  const int64_t num_tiles = (int64_t)a.tiles_m * a.tiles_n;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&tfull[i], 1);
+      mbar_init(&tempty[i], 4);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(&tmA1);
+    tma_prefetch_desc(&tmA2);
+    tma_prefetch_desc(&tmB1);
+    tma_prefetch_desc(&tmB2);
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, C::kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        const int m0 = (int)(t / a.tiles_n) * BM, n0 = (int)(t % a.tiles_n) * BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!(ok = mbar_wait(&empty[stage], phase ^ 1u, abort_flag, a.status))) break;
+          unsigned char* sa = smem + stage * C::kStageBytes;
+          mbar_arrive_expect_tx(&full[stage], C::kStageBytes);
+          tma_load_2d(sa, &tmA1, &full[stage], kb * BK, m0);
+          tma_load_2d(sa + BM * BK * 2, &tmA2, &full[stage], kb * BK, m0);
+          tma_load_2d(sa + 2 * BM * BK * 2, &tmB1, &full[stage], kb * BK, n0);
+          tma_load_2d(sa + 2 * BM * BK * 2 + BN * BK * 2, &tmB2, &full[stage], kb * BK, n0);
+          if (++stage == C::kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+      if (!ok) {
+        // let copies already in flight land before the CTA's shared memory is given up
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc_bf16(BM, BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      int64_t it = 0;
+      for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+        const uint32_t acc = (uint32_t)(it & 1), acc_phase = (uint32_t)((it >> 1) & 1);
+        if (!(ok = mbar_wait(&tempty[acc], acc_phase ^ 1u, abort_flag, a.status))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!(ok = mbar_wait(&full[stage], phase, abort_flag, a.status))) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + stage * C::kStageBytes);
+          const uint64_t a1 = smem_desc_sw128(sa), a2 = smem_desc_sw128(sa + BM * BK * 2);
+          const uint64_t b1 = smem_desc_sw128(sa + 2 * BM * BK * 2);
+          const uint64_t b2 = smem_desc_sw128(sa + 2 * BM * BK * 2 + BN * BK * 2);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t off = (uint64_t)((k * UMMA_K * 2) >> 4);   // 32 bytes per K step
+            umma_bf16(d_tmem, a1 + off, b2 + off, idesc, (kb | k) != 0 ? 1u : 0u);   // hi * lo
+            umma_bf16(d_tmem, a2 + off, b1 + off, idesc, 1u);                        // lo * hi
+            umma_bf16(d_tmem, a1 + off, b1 + off, idesc, 1u);                        // hi * hi
+          }
+          umma_commit(&empty[stage]);   // frees the stage once these MMAs have read it
+          if (++stage == C::kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        if (ok) umma_commit(&tfull[acc]);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------ epilogue (4 warps, 128 TMEM lanes)
+    const int lg = warp & 3;   // TMEM lane group this warp may read
+    bool ok = true;
+    int64_t it = 0;
+    for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+      const uint32_t acc = (uint32_t)(it & 1), acc_phase = (uint32_t)((it >> 1) & 1);
+      const int tm = (int)(t / a.tiles_n), tn = (int)(t % a.tiles_n);
+      const int64_t row = (int64_t)tm * BM + lg * 32 + lane;
+      const int n0 = tn * BN;
+      if (!(ok = mbar_wait(&tfull[acc], acc_phase, abort_flag, a.status))) break;
+      tc_fence_after();
+      const bool row_ok = row < a.M;
+      bool zero_row = false;
+      if (MODE == 1 && a.nu != nullptr && row_ok) zero_row = (__ldg(a.nu + row) == 0.f);
+      float gsum = 0.f;
+      uint32_t* out_row = reinterpret_cast<uint32_t*>(a.out + (size_t)(row_ok ? row : 0) * a.out_rb);
+      const size_t row_words = a.out_rb / 4;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        const int col0 = n0 + c * 32;
+        if (col0 >= a.N) break;   // uniform across the CTA: nothing but zero padding beyond
+        uint32_t v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(lg * 32) << 16) + acc * BN + c * 32, v);
+        tmem_ld_wait();
+        if (MODE == 2) {
+          uint32_t word = 0;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const bool bit = (__uint_as_float(v[i]) >= 0.f) && (col0 + i < a.N);
+            word |= (bit ? 1u : 0u) << i;
+          }
+          const size_t w = (size_t)(col0 >> 5);
+          if (row_ok && w < row_words) out_row[w] = word;
+        } else {
+          constexpr int NB = (1 << BITS) - 1;
+          unsigned long long bitbuf = 0;
+          int nb = 0, nw = 0;
+          uint32_t words[BITS > 0 ? BITS : 1];
+          uint32_t e1[16], e2[16];
+#pragma unroll
+          for (int i2 = 0; i2 < 16; ++i2) {
+            float ehi[2] = {0.f, 0.f}, elo[2] = {0.f, 0.f};
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              const int i = 2 * i2 + q;
+              const float y = __uint_as_float(v[i]);
+              const bool col_ok = (col0 + i < a.N);
+              int code = 0;
+#pragma unroll
+              for (int tix = 0; tix < NB; ++tix) code += (y > a.cb.t[tix]) ? 1 : 0;
+              if (!col_ok) code = 0;
+              if (BITS > 0) {
+                bitbuf |= (unsigned long long)code << nb;
+                nb += BITS;
+                if (nb >= 32) {
+                  words[nw++] = (uint32_t)bitbuf;
+                  bitbuf >>= 32;
+                  nb -= 32;
+                }
+              }
+              if (MODE == 1) {
+                const float e = (col_ok && !zero_row) ? (y - a.cb.c[code]) : 0.f;
+                gsum = fmaf(e, e, gsum);
+                ehi[q] = __bfloat162float(__float2bfloat16_rn(e));
+                elo[q] = e - ehi[q];
+              }
+            }
+            if (MODE == 1) {
+              e1[i2] = pack_bf16x2(ehi[0], ehi[1]);
+              e2[i2] = pack_bf16x2(elo[0], elo[1]);
+            }
+          }
+          if (BITS > 0 && row_ok) {
+            const size_t w0 = (size_t)(col0 >> 5) * BITS;
+#pragma unroll
+            for (int q = 0; q < BITS; ++q)
+              if (w0 + q < row_words) out_row[w0 + q] = words[q];
+          }
+          if (MODE == 1 && row_ok) {
+            uint4* d1 = reinterpret_cast<uint4*>(a.E1 + row * a.ldE + col0);
+            uint4* d2 = reinterpret_cast<uint4*>(a.E2 + row * a.ldE + col0);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              if (col0 + q * 8 + 8 <= a.ldE) {
+                d1[q] = make_uint4(e1[4 * q], e1[4 * q + 1], e1[4 * q + 2], e1[4 * q + 3]);
+                d2[q] = make_uint4(e2[4 * q], e2[4 * q + 1], e2[4 * q + 2], e2[4 * q + 3]);
+              }
+            }
+          }
+        }
+      }
+      // accumulator fully read: hand the TMEM buffer back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[acc]);
+      if (MODE == 1 && row_ok) a.gpart[(int64_t)tn * a.Mpad + row] = gsum;
+      // pad words past the last tile's columns (rows whose stride exceeds the tiles' coverage)
+      if (tn == a.tiles_n - 1 && row_ok) {
+        constexpr int kBitsPerCoord = (MODE == 2) ? 1 : BITS;
+        if (kBitsPerCoord > 0) {
+          const size_t covered = (size_t)((a.N + 31) >> 5) * kBitsPerCoord;
+          for (size_t w = covered; w < row_words; ++w) out_row[w] = 0u;
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------- operand splitting
+// One warp per row: nu = ||x|| (optional), u = x / nu, u = hi + lo in bf16.
+template <typename T, bool NORMALIZE>
+__global__ void __launch_bounds__(256) split_rows_kernel(const T* __restrict__ X, int64_t ldx, int64_t n, int d, int dpad,
+                                                         __nv_bfloat16* __restrict__ L1, __nv_bfloat16* __restrict__ L2,
+                                                         float* __restrict__ norms) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  for (int64_t r = warp; r < n; r += nwarps) {
+    const T* row = X + r * ldx;
+    float inv = 1.f;
+    if (NORMALIZE) {
+      float s = 0.f;
+      for (int j = lane; j < d; j += 32) {
+        float v;
+        if constexpr (sizeof(T) == 4) v = row[j]; else v = __bfloat162float(row[j]);
+        s = fmaf(v, v, s);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      const float nu = sqrtf(s);
+      inv = (nu > 0.f) ? 1.f / nu : 0.f;
+      if (lane == 0 && norms != nullptr) norms[r] = nu;
+    }
+    for (int j0 = lane * 8; j0 < dpad; j0 += 256) {
+      uint32_t h[4], l[4];
+#pragma unroll
+      for (int p = 0; p < 4; ++p) {
+        float u[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int j = j0 + 2 * p + q;
+          float v = 0.f;
+          if (j < d) {
+            if constexpr (sizeof(T) == 4) v = row[j]; else v = __bfloat162float(row[j]);
+          }
+          u[q] = v * inv;
+        }
+        const float h0 = __bfloat162float(__float2bfloat16_rn(u[0]));
+        const float h1 = __bfloat162float(__float2bfloat16_rn(u[1]));
+        h[p] = pack_bf16x2(h0, h1);
+        l[p] = pack_bf16x2(u[0] - h0, u[1] - h1);
+      }
+      *reinterpret_cast<uint4*>(L1 + r * dpad + j0) = make_uint4(h[0], h[1], h[2], h[3]);
+      *reinterpret_cast<uint4*>(L2 + r * dpad + j0) = make_uint4(l[0], l[1], l[2], l[3]);
+    }
+  }
+}
+
+// gamma = sqrt(sum over column tiles of the partial sums), in tile order (deterministic).
+__global__ void gamma_finish_kernel(const float* __restrict__ gpart, int64_t Mpad, int tiles_n, int64_t rows,
+                                    float* __restrict__ gamma) {
+  const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= rows) return;
+  float s = 0.f;
+  for (int t = 0; t < tiles_n; ++t) s += gpart[(int64_t)t * Mpad + r];
+  gamma[r] = sqrtf(s);
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// bf16 matrix [rows, cols] with row pitch `pitch` elements; box = 64 columns x box_rows, 128B swizzle.
+bool make_map(CUtensorMap* map, const __nv_bfloat16* base, int64_t rows, int cols, int64_t pitch, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)pitch * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  }
+  return sms;
+}
+
+template <int BN, int MODE, int BITS>
+cudaError_t launch_gemm_t(const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b1, const CUtensorMap& b2,
+                          const GemmArgs& args, cudaStream_t st) {
+  auto kern = quantize_gemm_kernel<BN, MODE, BITS>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int64_t tiles = (int64_t)args.tiles_m * args.tiles_n;
+  const int grid = (int)std::min<int64_t>(tiles, sm_count());
+  kern<<<grid, NTHREADS, Cfg<BN>::kSmemBytes, st>>>(a1, a2, b1, b2, args);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+template <int BN, int MODE>
+cudaError_t launch_gemm_bits(int bits, const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b1,
+                             const CUtensorMap& b2, const GemmArgs& args, cudaStream_t st) {
+  if constexpr (MODE == 2) {
+    return launch_gemm_t<BN, 2, 1>(a1, a2, b1, b2, args, st);
+  } else {
+    switch (bits) {
+      case 0: return launch_gemm_t<BN, MODE, 0>(a1, a2, b1, b2, args, st);
+      case 1: return launch_gemm_t<BN, MODE, 1>(a1, a2, b1, b2, args, st);
+      case 2: return launch_gemm_t<BN, MODE, 2>(a1, a2, b1, b2, args, st);
+      case 3: return launch_gemm_t<BN, MODE, 3>(a1, a2, b1, b2, args, st);
+      default: return launch_gemm_t<BN, MODE, 4>(a1, a2, b1, b2, args, st);
+    }
+  }
+}
+
+template <int MODE>
+cudaError_t launch_gemm(int bn, int bits, const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b1,
+                        const CUtensorMap& b2, const GemmArgs& args, cudaStream_t st) {
+  if (bn == 256) return launch_gemm_bits<256, MODE>(bits, a1, a2, b1, b2, args, st);
+  return launch_gemm_bits<128, MODE>(bits, a1, a2, b1, b2, args, st);
+}
+
+}  // namespace
+
+int pick_bn(int d) { return d > 128 ? 256 : 128; }
+
+bool supported(int d) { return d >= 128 && encode_fn() != nullptr; }
+
+cudaError_t build_matrix_limbs(const float* dM, int rows, int d, int dpad, int bn, MatrixLimbs* out) {
+  out->hi = out->lo = nullptr;
+  const size_t bytes = (size_t)rows * dpad * sizeof(__nv_bfloat16);
+  cudaError_t e = cudaMalloc(&out->hi, bytes);
+  if (e != cudaSuccess) return e;
+  e = cudaMalloc(&out->lo, bytes);
+  if (e != cudaSuccess) return e;
+  const int blocks = std::min((rows + 7) / 8, 148 * 8);
+  split_rows_kernel<float, false><<<blocks, 256>>>(dM, d, rows, d, dpad, out->hi, out->lo, nullptr);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (!make_map(&out->map_hi, out->hi, rows, d, dpad, bn) || !make_map(&out->map_lo, out->lo, rows, d, dpad, bn))
+    return cudaErrorInvalidValue;
+  return cudaSuccess;
+}
+
+void free_matrix_limbs(MatrixLimbs* m) {
+  cudaFree(m->hi);
+  cudaFree(m->lo);
+  m->hi = m->lo = nullptr;
+}
+
+size_t scratch_bytes_per_row(const tq_plan* plan) {
+  const int tiles_n = (plan->d + plan->tc_bn - 1) / plan->tc_bn;
+  size_t per = (size_t)plan->dpad * 2 * 2 + sizeof(float);                            // X limbs + nu
+  if (plan->mode == TQ_PROD) per += (size_t)plan->dpad * 2 * 2 + (size_t)tiles_n * 4;  // E limbs + partial sums
+  return per;
+}
+
+int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t ldx, uint8_t* idx, uint8_t* qjl,
+             float* gamma, float* norms, void* scratch, size_t scratch_bytes, cudaStream_t st, const char* who) {
+  const int d = plan->d, dpad = plan->dpad, bn = plan->tc_bn;
+  const int tiles_n = (d + bn - 1) / bn;
+  const bool prod = plan->mode == TQ_PROD;
+  const size_t per_row = scratch_bytes_per_row(plan);
+  int64_t R = (int64_t)(scratch_bytes / per_row) / BM * BM;
+  R = std::min<int64_t>(R, round_up64(n, BM));
+  TQ_REQUIRE(R >= BM, TQ_ERR_WORKSPACE, "%s: scratch of %zu bytes cannot hold one block of %d rows", who, scratch_bytes, BM);
+  // carve the scratch (every part is a multiple of 256 bytes because R is a multiple of 128)
+  char* p = static_cast<char*>(scratch);
+  __nv_bfloat16* XL1 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
+  __nv_bfloat16* XL2 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
+  __nv_bfloat16 *EL1 = nullptr, *EL2 = nullptr;
+  float* gpart = nullptr;
+  if (prod) {
+    EL1 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
+    EL2 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
+    gpart = reinterpret_cast<float*>(p); p += (size_t)R * tiles_n * 4;
+  }
+  float* nu_scratch = reinterpret_cast<float*>(p);
+  const size_t xsz = (x_dtype == TQ_F32) ? 4 : 2;
+
+  for (int64_t r0 = 0; r0 < n; r0 += R) {
+    const int64_t rows = std::min(R, n - r0);
+    const void* Xc = static_cast<const char*>(X) + (size_t)r0 * ldx * xsz;
+    float* nu_out = norms ? norms + r0 : nullptr;
+    const int blocks = (int)std::min<int64_t>((rows + 7) / 8, (int64_t)sm_count() * 8);
+    // 1. nu, u = x / nu, bf16 limbs of u
+    if (norms) {
+      if (x_dtype == TQ_F32)
+        split_rows_kernel<float, true><<<blocks, 256, 0, st>>>(static_cast<const float*>(Xc), ldx, rows, d, dpad, XL1, XL2, nu_out);
+      else
+        split_rows_kernel<__nv_bfloat16, true><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(Xc), ldx, rows, d, dpad, XL1, XL2, nu_out);
+    } else {
+      if (x_dtype == TQ_F32)
+        split_rows_kernel<float, false><<<blocks, 256, 0, st>>>(static_cast<const float*>(Xc), ldx, rows, d, dpad, XL1, XL2, nullptr);
+      else
+        split_rows_kernel<__nv_bfloat16, false><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(Xc), ldx, rows, d, dpad, XL1, XL2, nullptr);
+    }
+    count_launches(1);
+    TQ_CHECK_CUDA(cudaGetLastError(), who);
+    (void)nu_scratch;
+
+    CUtensorMap mA1, mA2;
+    TQ_REQUIRE(make_map(&mA1, XL1, rows, d, dpad, BM) && make_map(&mA2, XL2, rows, d, dpad, BM), TQ_ERR_CUDA,
+               "%s: cuTensorMapEncodeTiled failed", who);
+    GemmArgs g;
+    g.M = rows;
+    g.N = d;
+    g.K = d;
+    g.tiles_m = (int)((rows + BM - 1) / BM);
+    g.tiles_n = tiles_n;
+    g.cb = plan->cb;
+    g.out = idx ? idx + (size_t)r0 * plan->idx_row_bytes : nullptr;
+    g.out_rb = plan->idx_row_bytes;
+    g.E1 = EL1;
+    g.E2 = EL2;
+    g.ldE = dpad;
+    g.gpart = gpart;
+    g.Mpad = R;
+    g.nu = nu_out;
+    g.status = plan->d_status;
+    // 2. y = Pi u, idx (+ residual limbs and partial norms)
+    if (!prod) {
+      TQ_CHECK_CUDA(launch_gemm<0>(bn, plan->mse_bits, mA1, mA2, plan->pi_limbs.map_hi, plan->pi_limbs.map_lo, g, st), who);
+      continue;
+    }
+    TQ_CHECK_CUDA(launch_gemm<1>(bn, plan->mse_bits, mA1, mA2, plan->pi_limbs.map_hi, plan->pi_limbs.map_lo, g, st), who);
+    // 3. gamma = ||e||
+    gamma_finish_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(gpart, R, tiles_n, rows, gamma + r0);
+    count_launches(1);
+    TQ_CHECK_CUDA(cudaGetLastError(), who);
+    // 4. qjl = sign(S' e)
+    CUtensorMap mE1, mE2;
+    TQ_REQUIRE(make_map(&mE1, EL1, rows, d, dpad, BM) && make_map(&mE2, EL2, rows, d, dpad, BM), TQ_ERR_CUDA,
+               "%s: cuTensorMapEncodeTiled failed", who);
+    g.out = qjl + (size_t)r0 * plan->qjl_row_bytes;
+    g.out_rb = plan->qjl_row_bytes;
+    TQ_CHECK_CUDA(launch_gemm<2>(bn, 1, mE1, mE2, plan->sp_limbs.map_hi, plan->sp_limbs.map_lo, g, st), who);
+  }
+  return TQ_OK;
+}
+
+}  // namespace tc
+}  // namespace tq

@@ -39,21 +39,21 @@ class Setup:
         self.qjl_rb = tq.tq_qjl_row_bytes(d)
 
     # ---- GPU calls ---------------------------------------------------------------------
-    def quantize(self, X: torch.Tensor, with_norms=True):
+    def quantize(self, X: torch.Tensor, with_norms=True, scratch_bytes=None):
         n = X.shape[0]
         dev = X.device
         idx = torch.full((n, max(self.idx_rb, 1)), 0xAB, dtype=torch.uint8, device=dev)
         norms = torch.full((n,), -7.0, dtype=torch.float32, device=dev) if with_norms else None
+        ws = scratch_bytes if scratch_bytes is not None else tq.tq_workspace_bytes(self.plan, tq.TQ_OP_QUANTIZE, n)
+        scratch = torch.empty(max(ws, 16), dtype=torch.uint8, device=dev)
         if self.mode == tq.TQ_MSE:
-            tq.tq_quantize_mse(self.plan, X, idx, norms)
+            tq.tq_quantize_mse(self.plan, X, idx, norms, scratch)
             qjl = gamma = None
         else:
             qjl = torch.full((n, self.qjl_rb), 0xCD, dtype=torch.uint8, device=dev)
             gamma = torch.full((n,), -7.0, dtype=torch.float32, device=dev)
-            ws = tq.tq_workspace_bytes(self.plan, tq.TQ_OP_QUANTIZE, n)
-            scratch = torch.empty(max(ws, 16), dtype=torch.uint8, device=dev)
             tq.tq_quantize_prod(self.plan, X, idx, qjl, gamma, norms, scratch)
-        torch.cuda.synchronize()
+        tq.tq_plan_status(self.plan)
         return idx, qjl, gamma, norms
 
     def dequantize(self, n, idx, qjl, gamma, norms):

@@ -80,8 +80,22 @@ def test_embedding_configs_subset(name, bits, mode, n):
     assert stats["idx_mismatch"] == 0
 
 
-def test_bf16_inputs_and_unit_norm_mode():
-    d = 64
+def test_small_scratch_forces_several_blocks_of_rows():
+    cfg = wl.CONFIGS["c2"]
+    for bits, mode in ((3, tq.TQ_PROD), (2, tq.TQ_MSE)):
+        su = P.Setup(cfg.d, bits, mode, cfg.pi_seed, cfg.s_seed)
+        X = wl.database(cfg, 1000, device=DEV)
+        full = su.quantize(X)
+        small = tq.tq_workspace_bytes(su.plan, tq.TQ_OP_QUANTIZE, 256)
+        assert small < tq.tq_workspace_bytes(su.plan, tq.TQ_OP_QUANTIZE, 1000)
+        part = su.quantize(X, scratch_bytes=small)
+        for u, v in zip(full, part):
+            assert (u is None and v is None) or torch.equal(u, v)
+        P.check_quantize(su, X, *part)
+
+
+@pytest.mark.parametrize("d", [64, 256])
+def test_bf16_inputs_and_unit_norm_mode(d):
     su = P.Setup(d, 3, tq.TQ_PROD)
     g = torch.Generator(device="cpu").manual_seed(9)
     X = torch.randn((900, d), generator=g).to(torch.bfloat16).to(DEV)
@@ -169,6 +183,7 @@ def test_library_codebook_and_rotation_drive_the_same_path():
     X = wl.database(wl.CONFIGS["c1"], 512, device=DEV)
     i1 = torch.empty((512, su.idx_rb), dtype=torch.uint8, device=DEV)
     n1 = torch.empty(512, device=DEV)
-    tq.tq_quantize_mse(plan, X, i1, n1)
+    sc = torch.empty(tq.tq_workspace_bytes(plan, tq.TQ_OP_QUANTIZE, 512), dtype=torch.uint8, device=DEV)
+    tq.tq_quantize_mse(plan, X, i1, n1, sc)
     i2, _, _, n2 = su.quantize(X)
     assert (i1 != i2).float().mean().item() < 1e-3       # Pi differs by float32 rounding only
