@@ -174,6 +174,35 @@ int tq_score(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ld
              float* scores, int64_t lds, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * tq_score without caller-provided workspace and without any allocation (the paper has no
+ * counterpart: this is a packaging variant of tq_score, same arithmetic, same kernels).
+ *
+ * Who needs it: callers that are not allowed to obtain device memory at the time they score --
+ * an inference server that gave the whole GPU to its own memory pool at start-up, a plug-in whose
+ * host forbids driver allocations after initialisation, a latency-critical loop that cannot afford
+ * the device-wide synchronisation cudaMalloc / cudaFree imply.  Such a caller has nowhere to take
+ * the rotated-query workspace from, so the library keeps it: a fixed array of
+ * TQ_STATIC_SCRATCH_BYTES that lives in the library's device image.  Every GPU that loads the
+ * library holds that array until the process exits, whether or not this function is ever called.
+ *
+ *   arguments   as tq_score, minus workspace / workspace_bytes
+ *   limit       nq * ncat * dpad * 4 <= TQ_STATIC_SCRATCH_BYTES, ncat = 1 (TQ_MSE) or 2 (TQ_PROD),
+ *               dpad = d rounded up to a multiple of 8; larger requests return TQ_ERR_WORKSPACE
+ *               and launch nothing (largest accepted nq: 85 at d = 1536 TQ_PROD, 256 at d = 512 TQ_PROD).
+ *   first call  the first call on each device looks up the array's device address (with that
+ *               device current) and remembers it; make that first call outside any stream capture.
+ *   sharing     all calls on a device use the same array and it keeps whatever the previous call
+ *               left there.  Nothing in it needs to start at zero: each call overwrites the part
+ *               it reads before reading it.  Two calls whose kernels may overlap on the GPU
+ *               (different streams, no dependency between them) race on the array; serialise them.
+ * Calls no cudaMalloc / cudaFree and no allocating library routine.
+ */
+#define TQ_STATIC_SCRATCH_BYTES (1u << 20)
+int tq_score_static(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, int64_t n,
+                    const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms,
+                    float* scores, int64_t lds, void* stream);
+
+/*
  * The k vectors with the largest estimate per query (nearest-neighbour search by estimated
  * inner product, Section 4.4), sorted by descending score, equal scores by ascending id.
  * The nq x n score matrix is never formed.

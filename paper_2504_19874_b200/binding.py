@@ -11,6 +11,7 @@ TQ_MSE, TQ_PROD = 0, 1
 TQ_F32, TQ_BF16 = 0, 1
 TQ_ORTHOGONAL, TQ_GAUSSIAN = 0, 1
 TQ_OP_QUANTIZE, TQ_OP_SCORE, TQ_OP_TOPK, TQ_OP_WSUM, TQ_OP_DEQUANTIZE = 0, 1, 2, 3, 4
+TQ_STATIC_SCRATCH_BYTES = 1 << 20
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libtq.so")
 _lib = None
@@ -35,6 +36,8 @@ _SIGNATURES = {
     "tq_dequantize": (c_int, [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p]),
     "tq_score": (c_int, [c_void_p, c_void_p, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                          c_void_p, c_int64, c_void_p, c_size_t, c_void_p]),
+    "tq_score_static": (c_int, [c_void_p, c_void_p, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
+                                c_void_p, c_int64, c_void_p]),
     "tq_topk": (c_int, [c_void_p, c_void_p, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                         c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "tq_wsum": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -193,6 +196,15 @@ def tq_score(plan: Plan, Q, n: int, idx, qjl, gamma, norms, scores, workspace):
     _, lds = _rows(scores)
     _check(lib().tq_score(plan.handle, _dev(Q), _dtype_code(Q), nq, ldq, n, _dev(idx), _dev(qjl), _dev(gamma),
                           _dev(norms), _dev(scores), lds, *_scratch_args(workspace), _stream()))
+
+
+def tq_score_static(plan: Plan, Q, n: int, idx, qjl, gamma, norms, scores):
+    """tq_score for callers that cannot allocate device memory: the rotated-query workspace is an
+    array built into the library (TQ_STATIC_SCRATCH_BYTES), shared by every call on the device."""
+    nq, ldq = _rows(Q)
+    _, lds = _rows(scores)
+    _check(lib().tq_score_static(plan.handle, _dev(Q), _dtype_code(Q), nq, ldq, n, _dev(idx), _dev(qjl), _dev(gamma),
+                                 _dev(norms), _dev(scores), lds, _stream()))
 
 
 def tq_topk(plan: Plan, Q, n: int, idx, qjl, gamma, norms, k: int, top_scores, top_ids, workspace):

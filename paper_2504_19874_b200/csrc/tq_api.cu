@@ -1,6 +1,7 @@
 // C ABI of libtq: argument checking, plan set-up and kernel dispatch.
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -546,4 +547,61 @@ extern "C" int tq_wsum(const tq_plan* plan, const float* W, int nw, int64_t ldw,
   (void)out; (void)ldo; (void)workspace; (void)workspace_bytes; (void)stream;
   set_error("tq_wsum: not implemented yet");
   return TQ_ERR_UNSUPPORTED;
+}
+
+// ======================================================================================
+// tq_score_static: tq_score for callers that cannot allocate.  The rotated-query workspace is
+// this file-scope device array instead of a caller buffer.  In host code the array's name is
+// only a handle for the runtime, not a device address, so the address is looked up once per
+// device with cudaGetSymbolAddress and that pointer is what the kernels get.
+namespace {
+
+static __device__ __align__(256) unsigned char g_static_scratch[TQ_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device ordinal
+
+// Device address of the static scratch on the current device (looked up on first use).
+int static_scratch(const char* who, int device, void** out) {
+  TQ_REQUIRE(device >= 0 && device < kMaxDevices, TQ_ERR_UNSUPPORTED, "%s: device ordinal %d not supported", who, device);
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_ptr[device] == nullptr) {
+    void* p = nullptr;
+    TQ_CHECK_CUDA(cudaGetSymbolAddress(&p, g_static_scratch), who);
+    TQ_REQUIRE(p != nullptr && aligned(p, 256), TQ_ERR_CUDA, "%s: static scratch has no usable device address", who);
+    g_static_ptr[device] = p;
+  }
+  *out = g_static_ptr[device];
+  return TQ_OK;
+}
+
+}  // namespace
+
+extern "C" int tq_score_static(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, int64_t n,
+                               const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms,
+                               float* scores, int64_t lds, void* stream) {
+  const char* who = "tq_score_static";
+  int rc = check_plan(plan, who);   // also makes sure the plan's device is the current one
+  if (rc) return rc;
+  TQ_REQUIRE(n >= 0 && nq >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
+  if (n == 0 || nq == 0) return TQ_OK;
+  if ((rc = check_rows(who, "Q", Q, q_dtype, nq, ldq, plan->d))) return rc;
+  if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
+  TQ_REQUIRE(scores != nullptr && lds >= n, TQ_ERR_INVALID_ARG, "%s: scores is NULL or lds < n", who);
+  TQ_REQUIRE(aligned(scores, 16), TQ_ERR_ALIGNMENT, "%s: scores is not 16-byte aligned", who);
+  const size_t need = qcat_bytes(plan, nq);
+  TQ_REQUIRE(need <= (size_t)TQ_STATIC_SCRATCH_BYTES, TQ_ERR_WORKSPACE,
+             "%s: %d queries at d=%d need %zu bytes of rotated-query scratch, the built-in array holds %u; "
+             "use tq_score with a caller workspace or fewer queries per call",
+             who, nq, plan->d, need, (unsigned)TQ_STATIC_SCRATCH_BYTES);
+  void* ws = nullptr;
+  if ((rc = static_scratch(who, plan->device, &ws))) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* Qcat = static_cast<float*>(ws);
+  // Every element of Qcat[nq, ncat*dpad] is written by prepare_queries before score_block reads
+  // it, so the previous call's leftovers never show.
+  TQ_CHECK_CUDA(prepare_queries(plan, Q, q_dtype, nq, ldq, Qcat, st), who);
+  TQ_CHECK_CUDA(score_block(plan, Qcat, nq, 0, n, idx, qjl, gamma, norms, scores, lds, st), who);
+  return TQ_OK;
 }
