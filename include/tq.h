@@ -121,10 +121,10 @@ int tq_plan_destroy(tq_plan* plan);
 int tq_plan_status(tq_plan* plan);
 
 /* Bytes of device scratch the given operation asks for (0 if none).  For TQ_OP_QUANTIZE and
- * TQ_OP_TOPK this is the preferred size: any buffer that holds at least one block of rows is
- * accepted (the value returned for n = 128 resp. the SCORE size plus nq*4096 floats), larger
- * buffers mean fewer, bigger launches.   op = TQ_OP_*;  nq, k ignored where they do not apply.
- * Scratch must be 256-byte aligned. */
+ * TQ_OP_TOPK this is the preferred size; a smaller buffer is accepted down to the value returned
+ * for n = 128 (QUANTIZE) resp. n = 4096 (TOPK) and means more, smaller launches (for TOPK also the
+ * slower block-by-block selection instead of the thresholded single pass).
+ * op = TQ_OP_*;  nq, k ignored where they do not apply.  Scratch must be 256-byte aligned. */
 size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int nq, int k);
 
 /*

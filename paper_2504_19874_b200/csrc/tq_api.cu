@@ -8,6 +8,7 @@
 #include "tq_gemm_simt.cuh"
 #include "tq_internal.h"
 #include "tq_quantize_tc.h"
+#include "tq_scan_mma.h"
 #include "tq_scan_simt.cuh"
 
 using namespace tq;
@@ -88,6 +89,16 @@ constexpr int64_t kTensorChunk = 65536;    // rows per launch the tensor-core qu
 constexpr int64_t kResidualChunk = 16384;  // rows of E kept in flight by tq_quantize_prod (L2-sized)
 constexpr int64_t kTopkBlockMin = 4096, kTopkBlockPref = 65536;
 constexpr int kFewQueries = 16;  // up to this many queries the code scan is bandwidth-bound
+// top-k on the tensor-path scan: candidate pairs kept per query, queries per pass, dense-buffer rows
+constexpr int kCandCap = 32768;
+constexpr int kPassQueries = 4;
+constexpr int64_t kFilterMinN = 65536;
+constexpr int64_t kDenseRowsPref = 1 << 20, kDenseRowsMin = 4096;
+
+size_t ms_score_fixed(const tq_plan* plan, int nq) { return qcat_bytes(plan, nq) + mscan::workspace_bytes(plan); }
+size_t ms_topk_fixed(const tq_plan* plan, int nq) {
+  return ms_score_fixed(plan, nq) + 256 /* tau, count, overflow */ + (size_t)kPassQueries * kCandCap * 8;
+}
 
 template <typename T>
 cudaError_t launch_row_norm(const T* X, int64_t ld, int64_t n, int d, float* out, cudaStream_t st) {
@@ -141,10 +152,76 @@ bool has_pad_words(int d, int bits, size_t row_bytes) {
   return bits > 0 && (size_t)((d + 31) / 32) * bits * 4 < row_bytes;
 }
 
+// Few queries: one warp per output column j forms <Rot[j, :], q> for up to 8 queries at a time, with
+// the queries staged in shared memory (the matrix is read once per 8 queries); each lane sums its
+// d/32 products in fp32 and the 32 partial sums are added in fp64.
+constexpr int kRotQ = 8, kRotChunk = 1024;
+
+template <typename T>
+__global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __restrict__ Rot, int nrows, int d,
+                                                             const T* __restrict__ Q, int64_t ldq, int nq,
+                                                             float* __restrict__ Qcat, int64_t ldo) {
+  __shared__ __align__(16) float qs[kRotQ][kRotChunk];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int j = blockIdx.x * 8 + warp;
+  const float* row = Rot + (size_t)min(j, nrows - 1) * d;
+  for (int q0 = 0; q0 < nq; q0 += kRotQ) {
+    float acc[kRotQ];
+#pragma unroll
+    for (int qq = 0; qq < kRotQ; ++qq) acc[qq] = 0.f;
+    for (int c0 = 0; c0 < d; c0 += kRotChunk) {
+      const int len = min(kRotChunk, d - c0);
+      __syncthreads();
+      for (int e = threadIdx.x; e < kRotQ * kRotChunk; e += blockDim.x) {
+        const int qq = e / kRotChunk, c = e % kRotChunk;
+        float v = 0.f;
+        if (q0 + qq < nq && c < len) v = scan::to_f32<T>(Q[(int64_t)(q0 + qq) * ldq + c0 + c]);
+        qs[qq][c] = v;
+      }
+      __syncthreads();
+      if ((d & 3) == 0) {   // rows are 16-byte aligned: 128-bit loads, four in flight per lane
+        const float4* row4 = reinterpret_cast<const float4*>(row + c0);
+        const int len4 = len >> 2;
+#pragma unroll 4
+        for (int c4 = lane; c4 < len4; c4 += 32) {
+          const float4 r = __ldg(row4 + c4);
+#pragma unroll
+          for (int qq = 0; qq < kRotQ; ++qq) {
+            const float4 v = *reinterpret_cast<const float4*>(&qs[qq][4 * c4]);
+            acc[qq] = fmaf(r.x, v.x, fmaf(r.y, v.y, fmaf(r.z, v.z, fmaf(r.w, v.w, acc[qq]))));
+          }
+        }
+      } else {
+        for (int c = lane; c < len; c += 32) {
+          const float r = __ldg(row + c0 + c);
+#pragma unroll
+          for (int qq = 0; qq < kRotQ; ++qq) acc[qq] = fmaf(r, qs[qq][c], acc[qq]);
+        }
+      }
+    }
+#pragma unroll
+    for (int qq = 0; qq < kRotQ; ++qq) {
+      double v = (double)acc[qq];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0 && j < nrows && q0 + qq < nq) Qcat[(int64_t)(q0 + qq) * ldo + j] = (float)v;
+    }
+  }
+}
+
 // Q' = Q Pi^T and Q'' = Q S^T side by side: Qcat[nq, ncat*dpad].
 cudaError_t prepare_queries(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, float* Qcat,
                             cudaStream_t st) {
   const int ncols = plan->ncat * plan->dpad;
+  if (nq <= 64) {
+    const unsigned blocks = (unsigned)((ncols + 7) / 8);
+    if (q_dtype == TQ_F32)
+      rotate_queries_kernel<float><<<blocks, 256, 0, st>>>(plan->dRotCat, ncols, plan->d, static_cast<const float*>(Q), ldq, nq, Qcat, ncols);
+    else
+      rotate_queries_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(plan->dRotCat, ncols, plan->d, static_cast<const __nv_bfloat16*>(Q), ldq, nq, Qcat, ncols);
+    count_launches(1);
+    return cudaGetLastError();
+  }
   simt::RowsF32 B{plan->dRotCat, plan->d, ncols, plan->d};
   simt::EpStore ep{Qcat, ncols, nullptr, nullptr};
   if (q_dtype == TQ_F32) {
@@ -320,6 +397,7 @@ extern "C" int tq_plan_create(int d, int bits, int mode, const float* Pi, const 
       PLAN_CUDA(tc::build_matrix_limbs(p->dSp, d, d, p->dpad, p->tc_bn, &p->sp_limbs), "bf16 limbs of S'");
     p->tc_ok = 1;
   }
+  mscan::plan_init(p);
   PLAN_CUDA(cudaDeviceSynchronize(), "synchronize");
 #undef PLAN_CUDA
   *out = p;
@@ -364,8 +442,11 @@ extern "C" size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int
       if (plan->mode != TQ_PROD) return 0;
       return align_up((size_t)std::min<int64_t>(n, kResidualChunk) * plan->dpad * sizeof(float), 256);
     case TQ_OP_SCORE:
-      return qcat_bytes(plan, nq);
+      return plan->ms.ok ? ms_score_fixed(plan, nq) : qcat_bytes(plan, nq);
     case TQ_OP_TOPK:
+      if (plan->ms.ok)
+        return ms_topk_fixed(plan, nq) +
+               align_up((size_t)kPassQueries * std::max<int64_t>(std::min<int64_t>(n, kDenseRowsPref), kDenseRowsMin) * sizeof(float), 256);
       return qcat_bytes(plan, nq) + align_up((size_t)nq * std::min<int64_t>(n, kTopkBlockPref) * sizeof(float), 256);
     case TQ_OP_WSUM:
       return align_up((size_t)nq * plan->ncat * plan->dpad * sizeof(float), 256);
@@ -501,7 +582,76 @@ extern "C" int tq_score(const tq_plan* plan, const void* Q, int q_dtype, int nq,
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   float* Qcat = static_cast<float*>(workspace);
   TQ_CHECK_CUDA(prepare_queries(plan, Q, q_dtype, nq, ldq, Qcat, st), who);
+  if (plan->ms.ok) {
+    void* msw = static_cast<char*>(workspace) + qcat_bytes(plan, nq);
+    const int ncols = plan->ncat * plan->dpad;
+    const int qpp = mscan::queries_per_pass(plan, nq);
+    for (int q0 = 0; q0 < nq; q0 += qpp) {
+      const int nqp = std::min(qpp, nq - q0);
+      if ((rc = mscan::prepare(plan, Qcat + (size_t)q0 * ncols, nqp, msw, st, who))) return rc;
+      if ((rc = mscan::run(plan, nqp, n, idx, qjl, gamma, norms, scores + (int64_t)q0 * lds, lds, nullptr, nullptr, msw, st, who)))
+        return rc;
+    }
+    return TQ_OK;
+  }
   TQ_CHECK_CUDA(score_block(plan, Qcat, nq, 0, n, idx, qjl, gamma, norms, scores, lds, st), who);
+  return TQ_OK;
+}
+
+// Top-k through the tensor-path scan.  Large n: a pilot pass over the first rows gives, per query,
+// the k-th best score among them -- a lower bound on the final k-th score -- and the full pass
+// keeps only (score, id) pairs at or above it; a final selection sorts the survivors.  Should a
+// candidate list overflow (massive ties, adversarial order) a device-side flag switches on a
+// dense block-by-block rescue pass that is otherwise launched as a no-op.
+static int topk_ms(const tq_plan* plan, const float* Qcat, int nq, int64_t n, const uint8_t* idx, const uint8_t* qjl,
+                   const float* gamma, const float* norms, int k, float* top_scores, int32_t* top_ids, char* ws,
+                   size_t ws_bytes, cudaStream_t st, const char* who) {
+  int rc;
+  void* msw = ws;
+  char* p = ws + mscan::workspace_bytes(plan);
+  float* tau = reinterpret_cast<float*>(p);
+  int* count = reinterpret_cast<int*>(p + 64);
+  int* overflow = reinterpret_cast<int*>(p + 128);
+  p += 256;
+  float* cand_s = reinterpret_cast<float*>(p);
+  int* cand_i = reinterpret_cast<int*>(p + (size_t)kPassQueries * kCandCap * 4);
+  p += (size_t)kPassQueries * kCandCap * 8;
+  float* dense = reinterpret_cast<float*>(p);
+  const int64_t dense_floats = (int64_t)((ws + ws_bytes - p) / sizeof(float));
+  const int ncols = plan->ncat * plan->dpad;
+  const int qpp = mscan::queries_per_pass(plan, nq);
+  const size_t xrb = plan->idx_row_bytes, qrb = plan->qjl_row_bytes;
+  for (int q0 = 0; q0 < nq; q0 += qpp) {
+    const int nqp = std::min(qpp, nq - q0);
+    float* ts = top_scores + (size_t)q0 * k;
+    int32_t* ti = top_ids + (size_t)q0 * k;
+    if ((rc = mscan::prepare(plan, Qcat + (size_t)q0 * ncols, nqp, msw, st, who))) return rc;
+    const int64_t dense_rows = dense_floats / nqp;
+    const bool use_filter = n >= kFilterMinN && dense_rows >= std::min<int64_t>(n, kDenseRowsPref);
+    const int* guard = nullptr;
+    if (use_filter) {
+      int64_t m = std::max<int64_t>(round_up64(n / 64, 256), round_up64(std::max(k, 4096), 256));
+      m = std::min<int64_t>(m, std::min<int64_t>(dense_rows / 256 * 256, n));
+      if ((rc = mscan::run(plan, nqp, m, idx, qjl, gamma, norms, dense, m, nullptr, nullptr, msw, st, who))) return rc;
+      TQ_CHECK_CUDA(mscan::select_topk(dense, nullptr, nullptr, (int)m, (int)m, 0, nqp, k, 0, ts, ti, tau, nullptr, nullptr, st), who);
+      TQ_CHECK_CUDA(cudaMemsetAsync(count, 0, 128, st), who);   // counters and the overflow flag
+      mscan::Filter f{tau, count, cand_s, cand_i, kCandCap};
+      if ((rc = mscan::run(plan, nqp, n, idx, qjl, gamma, norms, nullptr, 0, &f, nullptr, msw, st, who))) return rc;
+      TQ_CHECK_CUDA(mscan::select_topk(cand_s, cand_i, count, kCandCap, 0, 0, nqp, k, 0, ts, ti, nullptr, overflow, nullptr, st), who);
+      guard = overflow;
+    }
+    // dense block flow: the whole job for small n, the guarded rescue otherwise
+    int64_t block = std::min<int64_t>(dense_rows, n);
+    if (block < n) block = block / 256 * 256;
+    for (int64_t v0 = 0; v0 < n; v0 += block) {
+      const int64_t cn = std::min(block, n - v0);
+      if ((rc = mscan::run(plan, nqp, cn, idx ? idx + (size_t)v0 * xrb : nullptr, qjl ? qjl + (size_t)v0 * qrb : nullptr,
+                           gamma ? gamma + v0 : nullptr, norms ? norms + v0 : nullptr, dense, block, nullptr, guard, msw, st, who)))
+        return rc;
+      TQ_CHECK_CUDA(mscan::select_topk(dense, nullptr, nullptr, (int)block, (int)cn, (int)v0, nqp, k, v0 > 0 ? 1 : 0, ts, ti,
+                                       nullptr, nullptr, guard, st), who);
+    }
+  }
   return TQ_OK;
 }
 
@@ -519,12 +669,18 @@ extern "C" int tq_topk(const tq_plan* plan, const void* Q, int q_dtype, int nq, 
   if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
   TQ_REQUIRE(top_scores != nullptr && top_ids != nullptr, TQ_ERR_INVALID_ARG, "%s: output is NULL", who);
   const size_t qb = qcat_bytes(plan, nq);
-  const size_t need = qb + align_up((size_t)nq * std::min<int64_t>(n, kTopkBlockMin) * sizeof(float), 256);
+  const size_t need = plan->ms.ok ? ms_topk_fixed(plan, nq) + (size_t)kPassQueries * kDenseRowsMin * sizeof(float)
+                                  : qb + align_up((size_t)nq * std::min<int64_t>(n, kTopkBlockMin) * sizeof(float), 256);
   TQ_REQUIRE(workspace != nullptr && workspace_bytes >= need, TQ_ERR_WORKSPACE, "%s: workspace of %zu bytes, %zu needed",
              who, workspace_bytes, need);
-  TQ_REQUIRE(aligned(workspace, 16), TQ_ERR_ALIGNMENT, "%s: workspace is not 16-byte aligned", who);
+  TQ_REQUIRE(aligned(workspace, 256), TQ_ERR_ALIGNMENT, "%s: workspace is not 256-byte aligned", who);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   float* Qcat = static_cast<float*>(workspace);
+  if (plan->ms.ok) {
+    TQ_CHECK_CUDA(prepare_queries(plan, Q, q_dtype, nq, ldq, Qcat, st), who);
+    return topk_ms(plan, Qcat, nq, n, idx, qjl, gamma, norms, k, top_scores, top_ids, static_cast<char*>(workspace) + qb,
+                   workspace_bytes - qb, st, who);
+  }
   float* blockbuf = reinterpret_cast<float*>(static_cast<char*>(workspace) + qb);
   int64_t block = (int64_t)((workspace_bytes - qb) / ((size_t)nq * sizeof(float)));
   block = std::min(block, n);

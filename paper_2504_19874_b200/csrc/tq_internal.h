@@ -59,6 +59,14 @@ struct tq_plan {
   int tc_bn;       // N extent of its MMA tile
   tq::MatrixLimbs pi_limbs;   // Pi
   tq::MatrixLimbs sp_limbs;   // S' (TQ_PROD)
+  // bit-plane scan on the integer tensor path (d >= 128, antisymmetric codebook)
+  struct {
+    int ok;            // 1 when this plan can use it
+    int R;             // ranges of 512 coordinates per row
+    double alpha[8];   // odd Walsh coefficients of the codebook: index bits 0..3, then the 3-bit parities
+    double amax;       // max |alpha|
+    double csum;       // mean term minus the sum of alpha: constant part of sum_j q'_j c[idx_j]
+  } ms;
   int* d_status;   // device word: set to TQ_ERR_TIMEOUT by a kernel whose bounded wait ran out
 };
 

@@ -62,7 +62,8 @@ def test_many_query_path_and_topk_blocks():
     tol = P.score_tolerance(su, Q, norms, n)
     ts, ti = su.topk(Q, n, idx, qjl, gamma, norms, k)
     P.check_topk(ref, tol, ts, ti, k)
-    small = tq.tq_workspace_bytes(su.plan, tq.TQ_OP_SCORE, n, nq) + nq * 4096 * 4
+    small = tq.tq_workspace_bytes(su.plan, tq.TQ_OP_TOPK, 4096, nq, k)      # the documented minimum
+    assert small < tq.tq_workspace_bytes(su.plan, tq.TQ_OP_TOPK, n, nq, k)
     ts2, ti2 = su.topk(Q, n, idx, qjl, gamma, norms, k, workspace_bytes=small)
     assert torch.equal(ts, ts2) and torch.equal(ti, ti2)
     # few-query path gives the same answers

@@ -1,0 +1,117 @@
+"""The packed-code scan on the integer tensor path (d >= 128) against the oracle: every bit width of
+both variants, ragged sizes, each query-count configuration, and the three top-k flows (dense
+blocks, pilot threshold + filter, overflow rescue)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2504_19874_b200 as tq
+import tq_workloads as wl
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _data(d, n, nq, seed):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    X = (torch.randn((n, d), generator=g) * torch.rand((n, 1), generator=g).mul(2).add(0.3)).to(DEV)
+    Q = (torch.randn((nq, d), generator=g) * torch.rand((nq, 1), generator=g).mul(4).add(0.1)).to(DEV)
+    return X, Q
+
+
+@pytest.mark.parametrize("d", [128, 200, 520, 1536])
+@pytest.mark.parametrize("bits,mode", [(1, tq.TQ_MSE), (2, tq.TQ_MSE), (3, tq.TQ_MSE), (4, tq.TQ_MSE), (1, tq.TQ_PROD),
+                                       (2, tq.TQ_PROD), (3, tq.TQ_PROD), (4, tq.TQ_PROD), (5, tq.TQ_PROD)])
+def test_scores_every_bit_width(d, bits, mode):
+    su = P.Setup(d, bits, mode)
+    n = 300 if d == 1536 else 777
+    X, Q = _data(d, n, 5, 1000 * d + 10 * bits + mode)
+    codes = su.quantize(X)
+    sc = su.score(Q, n, *codes)
+    P.check_scores(su, sc, Q, *codes)
+
+
+@pytest.mark.parametrize("nq", [1, 2, 3, 4, 7])
+def test_scores_every_pass_shape_and_determinism(nq):
+    d = 264
+    su = P.Setup(d, 4, tq.TQ_PROD)
+    n = 1000
+    X, Q = _data(d, n, nq, 77 + nq)
+    codes = su.quantize(X)
+    sc = su.score(Q, n, *codes)
+    ref = P.check_scores(su, sc, Q, *codes)
+    assert torch.equal(sc, su.score(Q, n, *codes))
+    # a query's estimate does not depend on which other queries share its pass
+    one = su.score(Q[nq - 1:nq].contiguous(), n, *codes)
+    assert torch.equal(one[0], sc[nq - 1])
+    ts, ti = su.topk(Q, n, *codes, 37)
+    P.check_topk(ref, P.score_tolerance(su, Q, codes[3], n), ts, ti, 37)
+
+
+def test_zero_and_huge_queries_and_unit_norm_codes():
+    d = 200
+    su = P.Setup(d, 3, tq.TQ_PROD)
+    n = 500
+    X, Q = _data(d, n, 4, 5)
+    Q[1].zero_()
+    Q[2] *= 1e6
+    Q[3] *= 1e-6
+    idx, qjl, gamma, _ = su.quantize(torch.nn.functional.normalize(X, dim=1), with_norms=False)
+    sc = su.score(Q, n, idx, qjl, gamma, None)
+    P.check_scores(su, sc, Q, idx, qjl, gamma, None)
+    assert bool((sc[1] == 0).all())
+
+
+def test_topk_threshold_filter_flow_matches_oracle():
+    cfg = wl.CONFIGS["c2"]
+    su = P.Setup(cfg.d, 3, tq.TQ_PROD, cfg.pi_seed, cfg.s_seed)
+    n, nq, k = 70001, 6, 100
+    X, Q = wl.database(cfg, n, device=DEV), wl.queries(cfg, nq, device=DEV)
+    codes = su.quantize(X)
+    sc = su.score(Q, n, *codes)
+    ref = P.check_scores(su, sc, Q, *codes)
+    tol = P.score_tolerance(su, Q, codes[3], n)
+    ts, ti = su.topk(Q, n, *codes, k)
+    P.check_topk(ref, tol, ts, ti, k)
+    # exactly the library's own dense scores, sorted (score desc, id asc)
+    for q in range(nq):
+        order = np.lexsort((np.arange(n), -sc[q].cpu().numpy().astype(np.float64)))[:k]
+        assert np.array_equal(ti[q].cpu().numpy(), order)
+        assert torch.equal(ts[q], sc[q][torch.from_numpy(order).to(DEV)])
+    # the minimum workspace takes the dense block flow and must agree bit for bit
+    small = tq.tq_workspace_bytes(su.plan, tq.TQ_OP_TOPK, 4096, nq, k)
+    ts2, ti2 = su.topk(Q, n, *codes, k, workspace_bytes=small)
+    assert torch.equal(ts, ts2) and torch.equal(ti, ti2)
+
+
+def test_topk_overflow_rescue_on_massive_ties():
+    """All vectors identical: every score ties, the candidate list overflows, the rescue pass must
+    return the k smallest ids."""
+    d = 128
+    su = P.Setup(d, 2, tq.TQ_MSE)
+    n, k = 66000, 50
+    row = torch.randn((1, d), generator=torch.Generator().manual_seed(3))
+    X = row.expand(n, d).contiguous().to(DEV)
+    Q = torch.randn((2, d), generator=torch.Generator().manual_seed(4)).to(DEV)
+    codes = su.quantize(X)
+    ts, ti = su.topk(Q, n, *codes, k)
+    assert torch.equal(ti, torch.arange(k, dtype=torch.int32, device=DEV).expand(2, k))
+    sc = su.score(Q, n, *codes)
+    assert torch.equal(ts, sc[:, :k])
+
+
+def test_topk_adversarial_order_descending_scores():
+    """Best vectors last: the pilot threshold is weak, the filter admits many candidates."""
+    cfg = wl.CONFIGS["c2"]
+    su = P.Setup(cfg.d, 3, tq.TQ_PROD, cfg.pi_seed, cfg.s_seed)
+    n, k = 66049, 64
+    X = wl.database(cfg, n, device=DEV)
+    Q = wl.queries(cfg, 1, device=DEV)
+    order = torch.argsort(X @ Q[0])            # ascending true inner product
+    X = X[order].contiguous()
+    codes = su.quantize(X)
+    sc = su.score(Q, n, *codes)
+    ts, ti = su.topk(Q, n, *codes, k)
+    want = np.lexsort((np.arange(n), -sc[0].cpu().numpy().astype(np.float64)))[:k]
+    assert np.array_equal(ti[0].cpu().numpy(), want)
