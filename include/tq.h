@@ -213,14 +213,28 @@ int tq_topk(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq
             float* top_scores, int32_t* top_ids, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * Weighted sum of dequantised vectors (the value side of attention over a compressed cache):
- *   out[w, :] = sum_t W[w, t] * Xhat_t,   Xhat_t as in tq_dequantize.
+ * Weighted sum of dequantised vectors (the value side of attention over a compressed cache,
+ * Section 4.3):   out[w, :] = sum_t W[w, t] * Xhat_t,   Xhat_t as in tq_dequantize.
+ * Formed in the code domain -- sum_t W nu c[idx_t] and coef * sum_t W nu gamma z_t per coordinate,
+ * then one product with Pi (and S) per output row -- so no token is dequantised.
  *   W    device, nw rows of n floats (e.g. softmax weights), row stride ldw
- *   out  device out, nw rows of d floats, row stride ldo
+ *   out  device out, nw rows of d floats, row stride ldo;  n = 0 gives zeros
+ *   workspace  >= tq_workspace_bytes(plan, TQ_OP_WSUM, n, nw, 0)
+ * Partial sums are combined in a fixed order: results are deterministic.
  */
 int tq_wsum(const tq_plan* plan, const float* W, int nw, int64_t ldw, int64_t n,
             const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms,
             float* out, int64_t ldo, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Attention weights from estimated scores: W[w, t] = softmax over t of scale * (s1[w, t] + s2[w, t]).
+ * Two score arrays are accepted because a head whose channels are split into two separately
+ * quantised groups (the outlier / regular split of Section 4.3) has its score as the sum of the two
+ * groups' estimates; s2 may be NULL.
+ *   s1, s2  device, nw rows of n floats, row stride lds;   W device out, row stride ldw (may alias s1)
+ */
+int tq_softmax(const float* s1, const float* s2, int nw, int64_t n, int64_t lds, float scale,
+               float* W, int64_t ldw, void* stream);
 
 #ifdef __cplusplus
 }

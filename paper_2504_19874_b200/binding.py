@@ -40,6 +40,7 @@ _SIGNATURES = {
                                 c_void_p, c_int64, c_void_p]),
     "tq_topk": (c_int, [c_void_p, c_void_p, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                         c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "tq_softmax": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, ctypes.c_float, c_void_p, c_int64, c_void_p]),
     "tq_wsum": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                         c_void_p, c_int64, c_void_p, c_size_t, c_void_p]),
 }
@@ -214,7 +215,16 @@ def tq_topk(plan: Plan, Q, n: int, idx, qjl, gamma, norms, k: int, top_scores, t
 
 
 def tq_wsum(plan: Plan, W, n: int, idx, qjl, gamma, norms, out, workspace):
-    nw, ldw = _rows(W)
-    _, ldo = _rows(out)
+    nw, ldo = _rows(out)
+    ldw = _rows(W)[1] if W is not None else n
     _check(lib().tq_wsum(plan.handle, _dev(W), nw, ldw, n, _dev(idx), _dev(qjl), _dev(gamma), _dev(norms),
                          _dev(out), ldo, *_scratch_args(workspace), _stream()))
+
+
+def tq_softmax(s1, s2, scale: float, W):
+    nw, lds = _rows(s1)
+    _, ldw = _rows(W)
+    n = s1.shape[1]
+    if s2 is not None and (_rows(s2)[1] != lds or s2.shape != s1.shape):
+        raise ValueError("s2 must have the shape and row stride of s1")
+    _check(lib().tq_softmax(_dev(s1), _dev(s2), nw, n, lds, scale, _dev(W), ldw, _stream()))

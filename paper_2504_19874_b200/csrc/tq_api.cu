@@ -5,6 +5,7 @@
 #include <new>
 #include <vector>
 
+#include "tq_attend_simt.cuh"
 #include "tq_gemm_simt.cuh"
 #include "tq_internal.h"
 #include "tq_quantize_tc.h"
@@ -448,8 +449,12 @@ extern "C" size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int
         return ms_topk_fixed(plan, nq) +
                align_up((size_t)kPassQueries * std::max<int64_t>(std::min<int64_t>(n, kDenseRowsPref), kDenseRowsMin) * sizeof(float), 256);
       return qcat_bytes(plan, nq) + align_up((size_t)nq * std::min<int64_t>(n, kTopkBlockPref) * sizeof(float), 256);
-    case TQ_OP_WSUM:
-      return align_up((size_t)nq * plan->ncat * plan->dpad * sizeof(float), 256);
+    case TQ_OP_WSUM: {
+      const size_t ncols = (size_t)plan->ncat * plan->dpad;
+      const size_t chunks = (size_t)((n + attend::WS_TOK - 1) / attend::WS_TOK);
+      return align_up((size_t)nq * ncols * sizeof(float), 256) +
+             align_up(chunks * std::min(nq, attend::WS_NW) * ncols * sizeof(float), 256);
+    }
     default:
       return 0;
   }
@@ -696,13 +701,93 @@ extern "C" int tq_topk(const tq_plan* plan, const void* Q, int q_dtype, int nq, 
   return TQ_OK;
 }
 
+template <int BITS>
+static cudaError_t launch_wsum_partial(const tq_plan* plan, const attend::WsumArgs& a, dim3 grid, cudaStream_t st) {
+  if (plan->mode == TQ_PROD) attend::wsum_partial_kernel<BITS, true><<<grid, 128, 0, st>>>(a);
+  else attend::wsum_partial_kernel<BITS, false><<<grid, 128, 0, st>>>(a);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
 extern "C" int tq_wsum(const tq_plan* plan, const float* W, int nw, int64_t ldw, int64_t n, const uint8_t* idx,
                        const uint8_t* qjl, const float* gamma, const float* norms, float* out, int64_t ldo,
                        void* workspace, size_t workspace_bytes, void* stream) {
-  (void)plan; (void)W; (void)nw; (void)ldw; (void)n; (void)idx; (void)qjl; (void)gamma; (void)norms;
-  (void)out; (void)ldo; (void)workspace; (void)workspace_bytes; (void)stream;
-  set_error("tq_wsum: not implemented yet");
-  return TQ_ERR_UNSUPPORTED;
+  const char* who = "tq_wsum";
+  int rc = check_plan(plan, who);
+  if (rc) return rc;
+  TQ_REQUIRE(n >= 0 && nw >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
+  if (nw == 0) return TQ_OK;
+  TQ_REQUIRE(out != nullptr && ldo >= plan->d, TQ_ERR_INVALID_ARG, "%s: out is NULL or ldo < d", who);
+  TQ_REQUIRE(aligned(out, 16), TQ_ERR_ALIGNMENT, "%s: out is not 16-byte aligned", who);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (n == 0) {
+    TQ_CHECK_CUDA(cudaMemset2DAsync(out, (size_t)ldo * sizeof(float), 0, (size_t)plan->d * sizeof(float), nw, st), who);
+    return TQ_OK;
+  }
+  TQ_REQUIRE(W != nullptr && ldw >= n, TQ_ERR_INVALID_ARG, "%s: W is NULL or ldw < n", who);
+  if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
+  const size_t need = tq_workspace_bytes(plan, TQ_OP_WSUM, n, nw, 0);
+  TQ_REQUIRE(workspace != nullptr && workspace_bytes >= need, TQ_ERR_WORKSPACE, "%s: workspace of %zu bytes, %zu needed",
+             who, workspace_bytes, need);
+  TQ_REQUIRE(aligned(workspace, 16), TQ_ERR_ALIGNMENT, "%s: workspace is not 16-byte aligned", who);
+  const int ncols = plan->ncat * plan->dpad;
+  float* oprime = static_cast<float*>(workspace);
+  float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + align_up((size_t)nw * ncols * sizeof(float), 256));
+  const int nchunks = (int)((n + attend::WS_TOK - 1) / attend::WS_TOK);
+  for (int w0 = 0; w0 < nw; w0 += attend::WS_NW) {
+    attend::WsumArgs a;
+    a.W = W + (int64_t)w0 * ldw;
+    a.ldw = ldw;
+    a.nw = std::min(attend::WS_NW, nw - w0);
+    a.n = n;
+    a.idx = idx;
+    a.idx_rb = plan->idx_row_bytes;
+    a.qjl = qjl;
+    a.qjl_rb = plan->qjl_row_bytes;
+    a.gamma = gamma;
+    a.norms = norms;
+    a.cb = plan->cb;
+    a.d = plan->d;
+    a.dpad = plan->dpad;
+    a.ncols = ncols;
+    a.coef = plan->coef;
+    a.partial = partial;
+    const dim3 grid((unsigned)nchunks, (unsigned)((plan->d + 127) / 128));
+    // columns the partial kernel never writes (pad coordinates) must read as zero
+    TQ_CHECK_CUDA(cudaMemsetAsync(partial, 0, (size_t)nchunks * a.nw * ncols * sizeof(float), st), who);
+    cudaError_t e;
+    switch (plan->mse_bits) {
+      case 0: e = launch_wsum_partial<0>(plan, a, grid, st); break;
+      case 1: e = launch_wsum_partial<1>(plan, a, grid, st); break;
+      case 2: e = launch_wsum_partial<2>(plan, a, grid, st); break;
+      case 3: e = launch_wsum_partial<3>(plan, a, grid, st); break;
+      default: e = launch_wsum_partial<4>(plan, a, grid, st); break;
+    }
+    TQ_CHECK_CUDA(e, who);
+    attend::wsum_reduce_kernel<<<(unsigned)((a.nw * ncols + 255) / 256), 256, 0, st>>>(partial, nchunks, a.nw, ncols,
+                                                                                        oprime + (size_t)w0 * ncols);
+    count_launches(1);
+    TQ_CHECK_CUDA(cudaGetLastError(), who);
+  }
+  // out = o' [Pi ; S]
+  simt::RowsF32 A{oprime, ncols, nw, ncols};
+  simt::RowsF32 B{plan->dBackT, ncols, plan->d, ncols};
+  simt::EpStore ep{out, ldo, nullptr, nullptr};
+  TQ_CHECK_CUDA(simt::launch_gemm(A, B, ep, (int64_t)nw, (int64_t)plan->d, ncols, st), who);
+  return TQ_OK;
+}
+
+extern "C" int tq_softmax(const float* s1, const float* s2, int nw, int64_t n, int64_t lds, float scale, float* W,
+                          int64_t ldw, void* stream) {
+  const char* who = "tq_softmax";
+  TQ_REQUIRE(nw >= 0 && n >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
+  if (nw == 0 || n == 0) return TQ_OK;
+  TQ_REQUIRE(s1 != nullptr && W != nullptr, TQ_ERR_INVALID_ARG, "%s: s1 / W is NULL", who);
+  TQ_REQUIRE(lds >= n && ldw >= n, TQ_ERR_INVALID_ARG, "%s: row stride smaller than n", who);
+  attend::softmax_rows_kernel<<<nw, 1024, 0, static_cast<cudaStream_t>(stream)>>>(s1, s2, lds, n, scale, W, ldw);
+  count_launches(1);
+  TQ_CHECK_CUDA(cudaGetLastError(), who);
+  return TQ_OK;
 }
 
 // ======================================================================================

@@ -1,0 +1,130 @@
+"""KV-cache decode over a compressed cache (third evaluation configuration): K quantised with
+TurboQuant_prod, V with TurboQuant_mse, 128 channels per head split into 64 outlier channels at 3
+bits and 64 regular channels at 2 bits, 32 query heads (4 per KV head), softmax(q K^T / sqrt(128)) V.
+GPU: tq_quantize_*, tq_score, tq_softmax, tq_wsum.  Oracle: dequantise the same codes, textbook
+attention in fp64."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2504_19874_b200 as tq
+import tq_workloads as wl
+from oracle import turboquant_oracle as orc
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+HEAD_DIM, GROUP = 128, 64
+
+
+def split_channels(Xh: torch.Tensor):
+    """Outlier / regular channel lists of one head (harness rule: largest energy over tokens)."""
+    out = orc.select_outlier_channels(Xh.double().cpu().numpy(), GROUP)
+    rest = np.setdiff1d(np.arange(HEAD_DIM), out)
+    return torch.from_numpy(out).to(DEV), torch.from_numpy(rest).to(DEV)
+
+
+def attend_gpu(groupsK, groupsV, Kh, Vh, Qh):
+    """One KV head: returns out [4, 128] fp32 and everything the oracle needs to redo it."""
+    T = Kh.shape[0]
+    scores, rec = [], {"K": [], "V": []}
+    chK, chV = split_channels(Kh), split_channels(Vh)
+    for su, ch in zip(groupsK, chK):
+        Xg = Kh[:, ch].contiguous()
+        codes = su.quantize(Xg)
+        rec["K"].append((su, ch, Xg, codes))
+        scores.append(su.score(Qh[:, ch].contiguous(), T, *codes))
+    W = torch.empty_like(scores[0])
+    tq.tq_softmax(scores[0], scores[1], 1.0 / math.sqrt(HEAD_DIM), W)
+    out = torch.zeros((Qh.shape[0], HEAD_DIM), device=DEV)
+    for su, ch in zip(groupsV, chV):
+        Xg = Vh[:, ch].contiguous()
+        codes = su.quantize(Xg)
+        rec["V"].append((su, ch, Xg, codes))
+        og = torch.empty((Qh.shape[0], GROUP), device=DEV)
+        ws = torch.empty(tq.tq_workspace_bytes(su.plan, tq.TQ_OP_WSUM, T, Qh.shape[0]), dtype=torch.uint8, device=DEV)
+        tq.tq_wsum(su.plan, W, T, *codes, og, ws)
+        out[:, ch] = og
+    torch.cuda.synchronize()
+    return out, W, rec
+
+
+def attend_oracle(rec, Qh):
+    T = rec["K"][0][2].shape[0]
+    Khat, Vhat = np.zeros((T, HEAD_DIM)), np.zeros((T, HEAD_DIM))
+    for su, ch, _, codes in rec["K"]:
+        Khat[:, ch.cpu().numpy()] = P.oracle_dequant(su, *codes)
+    for su, ch, _, codes in rec["V"]:
+        Vhat[:, ch.cpu().numpy()] = P.oracle_dequant(su, *codes)
+    s = orc.score(P.as_f64(Qh), Khat)
+    return orc.attend(s, Vhat, 1.0 / math.sqrt(HEAD_DIM)), s
+
+
+@pytest.fixture(scope="module")
+def groups():
+    gK = (P.Setup(GROUP, 3, tq.TQ_PROD, 72, 73), P.Setup(GROUP, 2, tq.TQ_PROD, 74, 75))
+    gV = (P.Setup(GROUP, 3, tq.TQ_MSE, 76, 77), P.Setup(GROUP, 2, tq.TQ_MSE, 78, 79))
+    return gK, gV
+
+
+def test_kv_decode_full_shape(groups):
+    gK, gV = groups
+    K, V, Q = wl.kv_cache(device=DEV)                      # [8, 32768, 128] x2, [32, 128], bf16
+    heads, T, _ = K.shape
+    worst = 0.0
+    for h in range(heads):
+        Qh = Q[4 * h:4 * h + 4]
+        out, W, rec = attend_gpu(gK, gV, K[h], V[h], Qh)
+        ref, s = attend_oracle(rec, Qh)
+        # softmax weights against the oracle's, then the output rows
+        p = np.exp(s / math.sqrt(HEAD_DIM) - (s / math.sqrt(HEAD_DIM)).max(axis=1, keepdims=True))
+        p /= p.sum(axis=1, keepdims=True)
+        assert np.allclose(P.as_f64(W), p, rtol=2e-3, atol=1e-9)
+        err = np.linalg.norm(P.as_f64(out) - ref, axis=1) / np.linalg.norm(ref, axis=1)
+        worst = max(worst, float(err.max()))
+        if h == 0:   # codes of the four groups of one head against the oracle's quantiser
+            for kind in ("K", "V"):
+                for su, _, Xg, codes in rec[kind]:
+                    st = P.check_quantize(su, Xg, *codes)
+                    assert st["idx_mismatch"] == 0
+    # logits carry the fp32 score error (<= 1e-4 of ||q|| nu) times 1/sqrt(128); weights and outputs inherit it
+    assert worst <= 1e-3, worst
+
+
+def test_wsum_matches_dequantised_sum_all_modes():
+    g = torch.Generator(device="cpu").manual_seed(11)
+    for d, bits, mode, n, nw in [(64, 3, tq.TQ_PROD, 1000, 4), (64, 2, tq.TQ_MSE, 129, 1), (200, 4, tq.TQ_PROD, 515, 11),
+                                 (24, 1, tq.TQ_PROD, 70, 3), (128, 4, tq.TQ_MSE, 300, 9)]:
+        su = P.Setup(d, bits, mode)
+        X = (torch.randn((n, d), generator=g) * 2).to(DEV)
+        codes = su.quantize(X)
+        W = torch.randn((nw, n), generator=g).to(DEV)
+        out = torch.empty((nw, d), device=DEV)
+        ws = torch.empty(tq.tq_workspace_bytes(su.plan, tq.TQ_OP_WSUM, n, nw), dtype=torch.uint8, device=DEV)
+        tq.tq_wsum(su.plan, W, n, *codes, out, ws)
+        out2 = torch.empty_like(out)
+        tq.tq_wsum(su.plan, W, n, *codes, out2, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(out, out2)
+        ref = P.as_f64(W) @ P.oracle_dequant(su, *codes)
+        scale = np.abs(P.as_f64(W)) @ np.linalg.norm(P.oracle_dequant(su, *codes), axis=1)
+        assert np.all(np.linalg.norm(P.as_f64(out) - ref, axis=1) <= P.RTOL * scale)
+
+
+def test_softmax_rows_and_empty_inputs():
+    g = torch.Generator(device="cpu").manual_seed(12)
+    s1 = (torch.randn((5, 3001), generator=g) * 20).to(DEV)
+    s2 = (torch.randn((5, 3001), generator=g) * 20).to(DEV)
+    W = torch.empty_like(s1)
+    tq.tq_softmax(s1, s2, 0.37, W)
+    ref = torch.softmax((s1.double() + s2.double()) * 0.37, dim=1)
+    assert torch.allclose(W.double(), ref, rtol=1e-4, atol=1e-12)
+    tq.tq_softmax(s1, None, 1.0, W)
+    assert torch.allclose(W.double(), torch.softmax(s1.double(), dim=1), rtol=1e-4, atol=1e-12)
+    su = P.Setup(64, 2, tq.TQ_MSE)
+    out = torch.full((2, 64), 7.0, device=DEV)
+    tq.tq_wsum(su.plan, None, 0, None, None, None, None, out, None)     # n = 0: zeros
+    torch.cuda.synchronize()
+    assert not bool(out.any())
