@@ -213,6 +213,19 @@ int tq_topk(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq
             float* top_scores, int32_t* top_ids, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The k best of m candidate (score, id) pairs per query, sorted like tq_topk's output (descending
+ * score, equal scores by ascending id).  This is the merge step of a sharded search: every shard
+ * returns its local top-k (the search of Section 4.4 is independent per database vector), the lists
+ * are concatenated per query and reduced to the global top-k here.  Pairs with a negative id are
+ * empty slots and are ignored; ids must be distinct within a query.
+ *   cand_scores, cand_ids  device, nq rows of m entries, row stride ld
+ *   k 1..TQ_MAX_K;  top_scores / top_ids device out [nq, k] (may not alias the candidates);
+ *   if fewer than k candidates exist the tail is filled with (-inf, -1)
+ */
+int tq_select_topk(const float* cand_scores, const int32_t* cand_ids, int nq, int64_t m, int64_t ld, int k,
+                   float* top_scores, int32_t* top_ids, void* stream);
+
+/*
  * Weighted sum of dequantised vectors (the value side of attention over a compressed cache,
  * Section 4.3):   out[w, :] = sum_t W[w, t] * Xhat_t,   Xhat_t as in tq_dequantize.
  * Formed in the code domain -- sum_t W nu c[idx_t] and coef * sum_t W nu gamma z_t per coordinate,

@@ -40,6 +40,7 @@ _SIGNATURES = {
                                 c_void_p, c_int64, c_void_p]),
     "tq_topk": (c_int, [c_void_p, c_void_p, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                         c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "tq_select_topk": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_int, c_void_p, c_void_p, c_void_p]),
     "tq_softmax": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, ctypes.c_float, c_void_p, c_int64, c_void_p]),
     "tq_wsum": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                         c_void_p, c_int64, c_void_p, c_size_t, c_void_p]),
@@ -228,3 +229,11 @@ def tq_softmax(s1, s2, scale: float, W):
     if s2 is not None and (_rows(s2)[1] != lds or s2.shape != s1.shape):
         raise ValueError("s2 must have the shape and row stride of s1")
     _check(lib().tq_softmax(_dev(s1), _dev(s2), nw, n, lds, scale, _dev(W), ldw, _stream()))
+
+
+def tq_select_topk(cand_scores, cand_ids, k: int, top_scores, top_ids):
+    nq, ld = _rows(cand_scores)
+    if _rows(cand_ids)[1] != ld or cand_ids.shape != cand_scores.shape:
+        raise ValueError("cand_ids must have the shape and row stride of cand_scores")
+    _check(lib().tq_select_topk(_dev(cand_scores), _dev(cand_ids), nq, cand_scores.shape[1], ld, k, _dev(top_scores),
+                                _dev(top_ids), _stream()))

@@ -777,6 +777,21 @@ extern "C" int tq_wsum(const tq_plan* plan, const float* W, int nw, int64_t ldw,
   return TQ_OK;
 }
 
+extern "C" int tq_select_topk(const float* cand_scores, const int32_t* cand_ids, int nq, int64_t m, int64_t ld, int k,
+                              float* top_scores, int32_t* top_ids, void* stream) {
+  const char* who = "tq_select_topk";
+  TQ_REQUIRE(nq >= 0 && m >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
+  TQ_REQUIRE(k >= 1 && k <= TQ_MAX_K, TQ_ERR_UNSUPPORTED, "%s: k=%d outside 1..%d", who, k, TQ_MAX_K);
+  TQ_REQUIRE(m <= 0x7fffffffLL && ld <= 0x7fffffffLL, TQ_ERR_UNSUPPORTED, "%s: m / ld too large", who);
+  if (nq == 0) return TQ_OK;
+  TQ_REQUIRE(top_scores != nullptr && top_ids != nullptr, TQ_ERR_INVALID_ARG, "%s: output is NULL", who);
+  TQ_REQUIRE(m == 0 || (cand_scores != nullptr && cand_ids != nullptr && ld >= m), TQ_ERR_INVALID_ARG,
+             "%s: candidates are NULL or ld < m", who);
+  TQ_CHECK_CUDA(mscan::select_pairs(cand_scores, cand_ids, (int)ld, (int)m, nq, k, top_scores, top_ids,
+                                    static_cast<cudaStream_t>(stream)), who);
+  return TQ_OK;
+}
+
 extern "C" int tq_softmax(const float* s1, const float* s2, int nw, int64_t n, int64_t lds, float scale, float* W,
                           int64_t ldw, void* stream) {
   const char* who = "tq_softmax";

@@ -554,7 +554,10 @@ __global__ void __launch_bounds__(1024) select_kernel(SelArgs a) {
   const float* src_s = a.cand_s + (int64_t)q * a.cap;
   const int* src_i = a.cand_i ? a.cand_i + (int64_t)q * a.cap : nullptr;
   auto key_at = [&](int i) -> unsigned long long {
-    if (i < m_new) return make_key(src_s[i], src_i ? src_i[i] : a.id0 + i);
+    if (i < m_new) {
+      const int id = src_i ? src_i[i] : a.id0 + i;
+      return id < 0 ? 0ull : make_key(src_s[i], id);
+    }
     const int j = i - m_new;
     const int id = a.top_i[(int64_t)q * a.k + j];
     if (id < 0) return 0ull;   // an empty slot of the previous list
@@ -902,6 +905,11 @@ cudaError_t select_topk(const float* cand_s, const int* cand_i, const int* count
   select_kernel<<<nq, 1024, 0, st>>>(a);
   count_launches(1);
   return cudaGetLastError();
+}
+
+cudaError_t select_pairs(const float* cand_s, const int* cand_i, int ld, int m, int nq, int k, float* top_s, int* top_i,
+                         cudaStream_t st) {
+  return select_topk(cand_s, cand_i, nullptr, ld, m, 0, nq, k, 0, top_s, top_i, nullptr, nullptr, nullptr, st);
 }
 
 }  // namespace mscan

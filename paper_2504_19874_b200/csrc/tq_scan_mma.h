@@ -42,5 +42,9 @@ cudaError_t select_topk(const float* cand_s, const int* cand_i, const int* count
                         int merge, float* top_s, int* top_i, float* kth, int* overflow, const int* run_if,
                         cudaStream_t st);
 
+// The k best of m candidate pairs per query (row stride ld); pairs with id < 0 are skipped.
+cudaError_t select_pairs(const float* cand_s, const int* cand_i, int ld, int m, int nq, int k, float* top_s, int* top_i,
+                         cudaStream_t st);
+
 }  // namespace mscan
 }  // namespace tq
