@@ -396,6 +396,12 @@ extern "C" int tq_plan_create(int d, int bits, int mode, const float* Pi, const 
     PLAN_CUDA(tc::build_matrix_limbs(p->dPi, d, d, p->dpad, p->tc_bn, &p->pi_limbs), "bf16 limbs of Pi");
     if (mode == TQ_PROD)
       PLAN_CUDA(tc::build_matrix_limbs(p->dSp, d, d, p->dpad, p->tc_bn, &p->sp_limbs), "bf16 limbs of S'");
+    PLAN_CUDA(cudaStreamCreateWithFlags(&p->aux_stream, cudaStreamNonBlocking), "aux stream");
+    PLAN_CUDA(cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming), "event");
+    for (int i = 0; i < 2; ++i) {
+      PLAN_CUDA(cudaEventCreateWithFlags(&p->ev_split[i], cudaEventDisableTiming), "event");
+      PLAN_CUDA(cudaEventCreateWithFlags(&p->ev_gemm[i], cudaEventDisableTiming), "event");
+    }
     p->tc_ok = 1;
   }
   mscan::plan_init(p);
@@ -412,6 +418,12 @@ extern "C" int tq_plan_destroy(tq_plan* plan) {
   cudaFree(plan->dRotCat);
   cudaFree(plan->dBackT);
   cudaFree(plan->d_status);
+  if (plan->aux_stream) cudaStreamDestroy(plan->aux_stream);
+  if (plan->ev_fork) cudaEventDestroy(plan->ev_fork);
+  for (int i = 0; i < 2; ++i) {
+    if (plan->ev_split[i]) cudaEventDestroy(plan->ev_split[i]);
+    if (plan->ev_gemm[i]) cudaEventDestroy(plan->ev_gemm[i]);
+  }
   tc::free_matrix_limbs(&plan->pi_limbs);
   tc::free_matrix_limbs(&plan->sp_limbs);
   delete plan;
@@ -439,7 +451,9 @@ extern "C" size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int
     case TQ_OP_QUANTIZE:
       if (n == 0) return 0;
       if (plan->tc_ok)
-        return align_up((size_t)std::min<int64_t>(round_up64(n, 128), kTensorChunk) * tc::scratch_bytes_per_row(plan), 256);
+        return align_up((size_t)std::min<int64_t>(round_up64(n, 128), kTensorChunk) * tc::scratch_bytes_per_row(plan) +
+                            (n > kTensorChunk ? (size_t)kTensorChunk * plan->dpad * 4 : 0),   // second set of X limbs: lets blocks overlap
+                        256);
       if (plan->mode != TQ_PROD) return 0;
       return align_up((size_t)std::min<int64_t>(n, kResidualChunk) * plan->dpad * sizeof(float), 256);
     case TQ_OP_SCORE:

@@ -21,7 +21,7 @@ namespace {
 constexpr int BM = 128;          // rows of X per tile = TMEM lanes
 constexpr int BK = 64;           // bf16 elements per 128-byte swizzled row
 constexpr int UMMA_K = 16;
-constexpr int NTHREADS = 192;    // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+constexpr int NTHREADS = 320;    // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue (two per TMEM lane group)
 
 template <int BN>
 struct Cfg {
@@ -41,7 +41,7 @@ struct GemmArgs {
   __nv_bfloat16* E1;     // MODE 1: residual limbs, pitch ldE
   __nv_bfloat16* E2;
   int64_t ldE;
-  float* gpart;          // MODE 1: [tiles_n][Mpad] partial sums of e^2
+  float* gpart;          // MODE 1: [2 * tiles_n][Mpad] partial sums of e^2 (one per half column tile)
   int64_t Mpad;
   const float* nu;       // MODE 1: per-row norm (row with nu == 0 has residual 0); nullable
   int* status;
@@ -79,7 +79,7 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&tfull[i], 1);
-      mbar_init(&tempty[i], 4);
+      mbar_init(&tempty[i], 8);
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -160,8 +160,9 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------ epilogue (4 warps, 128 TMEM lanes)
+    // ------------------------------------------------------------ epilogue (8 warps: 4 TMEM lane groups x 2 column halves)
     const int lg = warp & 3;   // TMEM lane group this warp may read
+    const int half = (warp - 2) >> 2;   // which half of the tile's columns this warp takes
     bool ok = true;
     int64_t it = 0;
     for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
@@ -178,7 +179,7 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
       uint32_t* out_row = reinterpret_cast<uint32_t*>(a.out + (size_t)(row_ok ? row : 0) * a.out_rb);
       const size_t row_words = a.out_rb / 4;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
         const int col0 = n0 + c * 32;
         if (col0 >= a.N) break;   // uniform across the CTA: nothing but zero padding beyond
         uint32_t v[32];
@@ -255,9 +256,9 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tempty[acc]);
-      if (MODE == 1 && row_ok) a.gpart[(int64_t)tn * a.Mpad + row] = gsum;
+      if (MODE == 1 && row_ok) a.gpart[(int64_t)(2 * tn + half) * a.Mpad + row] = gsum;
       // pad words past the last tile's columns (rows whose stride exceeds the tiles' coverage)
-      if (tn == a.tiles_n - 1 && row_ok) {
+      if (tn == a.tiles_n - 1 && half == 1 && row_ok) {
         constexpr int kBitsPerCoord = (MODE == 2) ? 1 : BITS;
         if (kBitsPerCoord > 0) {
           const size_t covered = (size_t)((a.N + 31) >> 5) * kBitsPerCoord;
@@ -465,7 +466,7 @@ void free_matrix_limbs(MatrixLimbs* m) {
 size_t scratch_bytes_per_row(const tq_plan* plan) {
   const int tiles_n = (plan->d + plan->tc_bn - 1) / plan->tc_bn;
   size_t per = (size_t)plan->dpad * 2 * 2 + sizeof(float);                            // X limbs + nu
-  if (plan->mode == TQ_PROD) per += (size_t)plan->dpad * 2 * 2 + (size_t)tiles_n * 4;  // E limbs + partial sums
+  if (plan->mode == TQ_PROD) per += (size_t)plan->dpad * 2 * 2 + (size_t)tiles_n * 8;  // E limbs + partial sums (two per column tile)
   return per;
 }
 
@@ -487,34 +488,66 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
   if (prod) {
     EL1 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
     EL2 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
-    gpart = reinterpret_cast<float*>(p); p += (size_t)R * tiles_n * 4;
+    gpart = reinterpret_cast<float*>(p); p += (size_t)R * tiles_n * 8;
   }
-  float* nu_scratch = reinterpret_cast<float*>(p);
+  p += (size_t)R * sizeof(float);
   const size_t xsz = (x_dtype == TQ_F32) ? 4 : 2;
-
-  for (int64_t r0 = 0; r0 < n; r0 += R) {
+  // With room for a second set of X limbs, the split of block i+1 (HBM-bound) runs on the plan's
+  // second stream while the GEMMs of block i (tensor-bound) run on the caller's.
+  const bool pipelined = n > R && plan->aux_stream != nullptr &&
+                         scratch_bytes >= (size_t)R * per_row + (size_t)R * dpad * 4;
+  __nv_bfloat16* XLb[2][2] = {{XL1, XL2}, {XL1, XL2}};
+  if (pipelined) {
+    XLb[1][0] = reinterpret_cast<__nv_bfloat16*>(p);
+    XLb[1][1] = reinterpret_cast<__nv_bfloat16*>(p + (size_t)R * dpad * 2);
+  }
+  auto launch_split = [&](int64_t r0, int b, cudaStream_t s) -> cudaError_t {
     const int64_t rows = std::min(R, n - r0);
     const void* Xc = static_cast<const char*>(X) + (size_t)r0 * ldx * xsz;
     float* nu_out = norms ? norms + r0 : nullptr;
     const int blocks = (int)std::min<int64_t>((rows + 7) / 8, (int64_t)sm_count() * 8);
-    // 1. nu, u = x / nu, bf16 limbs of u
+    __nv_bfloat16 *L1 = XLb[b][0], *L2 = XLb[b][1];
     if (norms) {
       if (x_dtype == TQ_F32)
-        split_rows_kernel<float, true><<<blocks, 256, 0, st>>>(static_cast<const float*>(Xc), ldx, rows, d, dpad, XL1, XL2, nu_out);
+        split_rows_kernel<float, true><<<blocks, 256, 0, s>>>(static_cast<const float*>(Xc), ldx, rows, d, dpad, L1, L2, nu_out);
       else
-        split_rows_kernel<__nv_bfloat16, true><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(Xc), ldx, rows, d, dpad, XL1, XL2, nu_out);
+        split_rows_kernel<__nv_bfloat16, true><<<blocks, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(Xc), ldx, rows, d, dpad, L1, L2, nu_out);
     } else {
       if (x_dtype == TQ_F32)
-        split_rows_kernel<float, false><<<blocks, 256, 0, st>>>(static_cast<const float*>(Xc), ldx, rows, d, dpad, XL1, XL2, nullptr);
+        split_rows_kernel<float, false><<<blocks, 256, 0, s>>>(static_cast<const float*>(Xc), ldx, rows, d, dpad, L1, L2, nullptr);
       else
-        split_rows_kernel<__nv_bfloat16, false><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(Xc), ldx, rows, d, dpad, XL1, XL2, nullptr);
+        split_rows_kernel<__nv_bfloat16, false><<<blocks, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(Xc), ldx, rows, d, dpad, L1, L2, nullptr);
     }
     count_launches(1);
-    TQ_CHECK_CUDA(cudaGetLastError(), who);
-    (void)nu_scratch;
+    return cudaGetLastError();
+  };
+  if (pipelined) {
+    TQ_CHECK_CUDA(cudaEventRecord(plan->ev_fork, st), who);              // the second stream starts after the caller's work so far
+    TQ_CHECK_CUDA(cudaStreamWaitEvent(plan->aux_stream, plan->ev_fork, 0), who);
+    TQ_CHECK_CUDA(launch_split(0, 0, st), who);
+  }
+
+  int64_t blk = 0;
+  for (int64_t r0 = 0; r0 < n; r0 += R, ++blk) {
+    const int64_t rows = std::min(R, n - r0);
+    const int b = pipelined ? (int)(blk & 1) : 0;
+    float* nu_out = norms ? norms + r0 : nullptr;
+    // 1. nu, u = x / nu, bf16 limbs of u
+    if (!pipelined) {
+      TQ_CHECK_CUDA(launch_split(r0, 0, st), who);
+    } else {
+      if (r0 + R < n) {
+        const int nb = (int)((blk + 1) & 1);
+        if (blk >= 1) TQ_CHECK_CUDA(cudaStreamWaitEvent(plan->aux_stream, plan->ev_gemm[nb], 0), who);   // its last reader is done
+        TQ_CHECK_CUDA(launch_split(r0 + R, nb, plan->aux_stream), who);
+        TQ_CHECK_CUDA(cudaEventRecord(plan->ev_split[nb], plan->aux_stream), who);
+      }
+      if (blk >= 1) TQ_CHECK_CUDA(cudaStreamWaitEvent(st, plan->ev_split[b], 0), who);
+    }
+    __nv_bfloat16 *XLc1 = XLb[b][0], *XLc2 = XLb[b][1];
 
     CUtensorMap mA1, mA2;
-    TQ_REQUIRE(make_map(&mA1, XL1, rows, d, dpad, BM) && make_map(&mA2, XL2, rows, d, dpad, BM), TQ_ERR_CUDA,
+    TQ_REQUIRE(make_map(&mA1, XLc1, rows, d, dpad, BM) && make_map(&mA2, XLc2, rows, d, dpad, BM), TQ_ERR_CUDA,
                "%s: cuTensorMapEncodeTiled failed", who);
     GemmArgs g;
     g.M = rows;
@@ -535,11 +568,13 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     // 2. y = Pi u, idx (+ residual limbs and partial norms)
     if (!prod) {
       TQ_CHECK_CUDA(launch_gemm<0>(bn, plan->mse_bits, mA1, mA2, plan->pi_limbs.map_hi, plan->pi_limbs.map_lo, g, st), who);
+      if (pipelined) TQ_CHECK_CUDA(cudaEventRecord(plan->ev_gemm[b], st), who);
       continue;
     }
     TQ_CHECK_CUDA(launch_gemm<1>(bn, plan->mse_bits, mA1, mA2, plan->pi_limbs.map_hi, plan->pi_limbs.map_lo, g, st), who);
+    if (pipelined) TQ_CHECK_CUDA(cudaEventRecord(plan->ev_gemm[b], st), who);
     // 3. gamma = ||e||
-    gamma_finish_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(gpart, R, tiles_n, rows, gamma + r0);
+    gamma_finish_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(gpart, R, 2 * tiles_n, rows, gamma + r0);
     count_launches(1);
     TQ_CHECK_CUDA(cudaGetLastError(), who);
     // 4. qjl = sign(S' e)
