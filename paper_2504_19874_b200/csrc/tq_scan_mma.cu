@@ -50,7 +50,7 @@ __host__ __device__ constexpr int a_words(int bm) { return idx_words(bm) + der_w
 __host__ __device__ constexpr int ks_a(int bm) { return a_words(bm) / 2 * 8; }
 __host__ __device__ constexpr int ks_s(bool prod) { return prod ? 16 : 0; }
 
-// Per-query constants produced by qstats_kernel.
+// Per-query constants (computed inside bprep_kernel).
 struct QConst {
   double sa, ca;   // a = T_a * sa + ca   (MSE term)
   double ss, cs;   // s = T_s * ss + cs   (QJL term)
@@ -92,75 +92,75 @@ __host__ __device__ inline int s_slot(int r, int t4, int word, int bitpos) {
   return (r * 64 + t4 * 16 + 4 * word) * 8 + bitpos;
 }
 
-// ------------------------------------------------------------------ query statistics
-struct QStatArgs {
-  const float* Qcat;
-  int64_t ldq;
-  int d, dpad, prod;
-  double amax, csum;   // max |alpha_T|; alpha_empty - sum_T alpha_T
-  QConst* out;
-};
-
-__global__ void __launch_bounds__(256) qstats_kernel(QStatArgs a) {
-  __shared__ double red[4][8];
-  const float* q = a.Qcat + (int64_t)blockIdx.x * a.ldq;
-  double mx1 = 0.0, sm1 = 0.0, mx2 = 0.0, sm2 = 0.0;
-  for (int j = threadIdx.x; j < a.d; j += blockDim.x) {
-    const double v = (double)q[j];
-    mx1 = fmax(mx1, fabs(v));
-    sm1 += v;
-    if (a.prod) {
-      const double u = (double)q[a.dpad + j];
-      mx2 = fmax(mx2, fabs(u));
-      sm2 += u;
-    }
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    mx1 = fmax(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
-    mx2 = fmax(mx2, __shfl_xor_sync(0xffffffffu, mx2, o));
-    sm1 += __shfl_xor_sync(0xffffffffu, sm1, o);
-    sm2 += __shfl_xor_sync(0xffffffffu, sm2, o);
-  }
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (lane == 0) {
-    red[0][warp] = mx1; red[1][warp] = sm1; red[2][warp] = mx2; red[3][warp] = sm2;
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    for (int w = 1; w < 8; ++w) {
-      mx1 = fmax(mx1, red[0][w]); sm1 += red[1][w];
-      mx2 = fmax(mx2, red[2][w]); sm2 += red[3][w];
-    }
-    QConst c;
-    // |W| < 2^e with W = 2 alpha q'  ->  |W| 2^(29-e) < 2^29 (operands are differences of two such values)
-    auto expo = [](double wmax) {
-      if (!(wmax > 0.0) || !isfinite(wmax)) return 0;
-      int e;
-      frexp(wmax, &e);
-      return 29 - e;
-    };
-    c.fa = expo(2.0 * a.amax * mx1);
-    c.fs = expo(2.0 * mx2);
-    c.sa = ldexp(1.0, -c.fa);
-    c.ss = ldexp(1.0, -c.fs);
-    c.ca = a.csum * sm1;
-    c.cs = -sm2;
-    c.pad[0] = c.pad[1] = 0;
-    a.out[blockIdx.x] = c;
-  }
-}
-
 // ------------------------------------------------------------------ B operand
 struct BPrepArgs {
   const float* Qcat;   // rotated queries of this pass: row q at Qcat + q*ldq
   int64_t ldq;
-  const QConst* qc;
+  QConst* qc;          // out: per-query constants of this pass (written by block 0)
   int nq_pass;         // valid queries in this pass
   int d, dpad, bm, prod, R, NT;
   double alpha[8];
+  double amax, csum;   // max |alpha_T|; alpha_empty - sum_T alpha_T
   uint2* out;          // [NT][R][KS][32]
 };
+
+constexpr int kMaxPassQueries = 4;
+
+// Per-query scale and constants.  Every block derives them itself (a few thousand loads from L2),
+// in the same order, so that no separate launch is needed; block 0 publishes them for the scan.
+__device__ void query_constants(const BPrepArgs& a, QConst* sc /* shared, [kMaxPassQueries] */) {
+  __shared__ double red[4][8];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int ql = 0; ql < a.nq_pass; ++ql) {
+    const float* q = a.Qcat + (int64_t)ql * a.ldq;
+    double mx1 = 0.0, sm1 = 0.0, mx2 = 0.0, sm2 = 0.0;
+    for (int j = threadIdx.x; j < a.d; j += blockDim.x) {
+      const double v = (double)q[j];
+      mx1 = fmax(mx1, fabs(v));
+      sm1 += v;
+      if (a.prod) {
+        const double u = (double)q[a.dpad + j];
+        mx2 = fmax(mx2, fabs(u));
+        sm2 += u;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      mx1 = fmax(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+      mx2 = fmax(mx2, __shfl_xor_sync(0xffffffffu, mx2, o));
+      sm1 += __shfl_xor_sync(0xffffffffu, sm1, o);
+      sm2 += __shfl_xor_sync(0xffffffffu, sm2, o);
+    }
+    if (lane == 0) {
+      red[0][warp] = mx1; red[1][warp] = sm1; red[2][warp] = mx2; red[3][warp] = sm2;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int w = 1; w < 8; ++w) {
+        mx1 = fmax(mx1, red[0][w]); sm1 += red[1][w];
+        mx2 = fmax(mx2, red[2][w]); sm2 += red[3][w];
+      }
+      // |W| < 2^e with W = 2 alpha q'  ->  |W| 2^(29-e) < 2^29 (operands are differences of two such values)
+      auto expo = [](double wmax) {
+        if (!(wmax > 0.0) || !isfinite(wmax)) return 0;
+        int e;
+        frexp(wmax, &e);
+        return 29 - e;
+      };
+      QConst c;
+      c.fa = expo(2.0 * a.amax * mx1);
+      c.fs = expo(2.0 * mx2);
+      c.sa = ldexp(1.0, -c.fa);
+      c.ss = ldexp(1.0, -c.fs);
+      c.ca = a.csum * sm1;
+      c.cs = -sm2;
+      c.pad[0] = c.pad[1] = 0;
+      sc[ql] = c;
+      if (blockIdx.x == 0) a.qc[ql] = c;
+    }
+    __syncthreads();
+  }
+}
 
 __device__ __forceinline__ int digit_of(long long J, int limb) {
   int dg = 0;
@@ -172,6 +172,8 @@ __device__ __forceinline__ int digit_of(long long J, int limb) {
 }
 
 __global__ void __launch_bounds__(256) bprep_kernel(BPrepArgs a) {
+  __shared__ QConst sc[kMaxPassQueries];
+  query_constants(a, sc);
   const int ksa = ks_a(a.bm), kss = ks_s(a.prod != 0), KS = ksa + kss;
   const int64_t total = (int64_t)a.NT * a.R * KS * 32;
   const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -185,7 +187,7 @@ __global__ void __launch_bounds__(256) bprep_kernel(BPrepArgs a) {
   uint32_t out[2] = {0u, 0u};
   if (ql < a.nq_pass) {
     const float* q = a.Qcat + (int64_t)ql * a.ldq;
-    const QConst c = a.qc[ql];
+    const QConst c = sc[ql];
     const bool is_s = ks >= ksa;
     const int kk = is_s ? ks - ksa : ks;
     const int p = kk >> 3, k = kk & 7;
@@ -563,6 +565,16 @@ __global__ void __launch_bounds__(1024) select_kernel(SelArgs a) {
     if (id < 0) return 0ull;   // an empty slot of the previous list
     return make_key(a.top_s[(int64_t)q * a.k + j], id);
   };
+  // up to 16 keys per thread stay in registers for all rounds (lists up to 16,384 entries)
+  const bool cached = total <= 16 * 1024;
+  unsigned long long kc[16];
+  if (cached) {
+#pragma unroll
+    for (int u = 0; u < 16; ++u) {
+      const int i = u * 1024 + tid;
+      kc[u] = (i < total) ? key_at(i) : 0ull;
+    }
+  }
   int kk = min(a.k, total);
   unsigned long long prefix = 0ull;
   int shift = 56;
@@ -571,23 +583,27 @@ __global__ void __launch_bounds__(1024) select_kernel(SelArgs a) {
       shift = 56 - 8 * round;
       if (tid < 256) hist[tid] = 0;
       __syncthreads();
-      // batches of 8 independent loads per thread, then the (convergent) histogram updates
-      for (int base = 0; base < total; base += 8 * blockDim.x) {
-        unsigned long long keys[8];
+      auto tally = [&](unsigned long long key, bool valid) {
+        const bool in = valid && (round == 0 || (key >> (shift + 8)) == prefix);
+        // lanes with the same digit add once (scores of one query crowd into a few bins)
+        const int dg = in ? (int)((key >> shift) & 255ull) : -1;
+        const unsigned peers = __match_any_sync(0xffffffffu, dg);
+        if (in && (int)(__ffs(peers) - 1) == (tid & 31)) atomicAdd(&hist[dg], __popc(peers));
+      };
+      if (cached) {
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int i = base + u * blockDim.x + tid;
-          keys[u] = (i < total) ? key_at(i) : 0ull;
-        }
+        for (int u = 0; u < 16; ++u) tally(kc[u], u * 1024 + tid < total);
+      } else {
+        // batches of 8 independent loads per thread, then the (convergent) histogram updates
+        for (int base = 0; base < total; base += 8 * blockDim.x) {
+          unsigned long long keys[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int i = base + u * blockDim.x + tid;
-          const unsigned long long key = keys[u];
-          const bool in = i < total && (round == 0 || (key >> (shift + 8)) == prefix);
-          // lanes with the same digit add once (scores of one query crowd into a few bins)
-          const int dg = in ? (int)((key >> shift) & 255ull) : -1;
-          const unsigned peers = __match_any_sync(0xffffffffu, dg);
-          if (in && (int)(__ffs(peers) - 1) == (tid & 31)) atomicAdd(&hist[dg], __popc(peers));
+          for (int u = 0; u < 8; ++u) {
+            const int i = base + u * blockDim.x + tid;
+            keys[u] = (i < total) ? key_at(i) : 0ull;
+          }
+#pragma unroll
+          for (int u = 0; u < 8; ++u) tally(keys[u], base + u * (int)blockDim.x + tid < total);
         }
       }
       __syncthreads();
@@ -631,19 +647,25 @@ __global__ void __launch_bounds__(1024) select_kernel(SelArgs a) {
   skey[tid] = 0ull;
   __syncthreads();
   if (min(a.k, total) > 0) {
-    for (int base = 0; base < total; base += 8 * blockDim.x) {
-      unsigned long long keys[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int i = base + u * blockDim.x + tid;
-        keys[u] = (i < total) ? key_at(i) : 0ull;
+    auto keep = [&](unsigned long long key) {
+      if ((key >> shift) >= prefix && key != 0ull) {
+        const int slot = atomicAdd(&s_cnt, 1);
+        if (slot < 1024) skey[slot] = key;
       }
+    };
+    if (cached) {
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        if ((keys[u] >> shift) >= prefix && keys[u] != 0ull) {
-          const int slot = atomicAdd(&s_cnt, 1);
-          if (slot < 1024) skey[slot] = keys[u];
+      for (int u = 0; u < 16; ++u) keep(kc[u]);
+    } else {
+      for (int base = 0; base < total; base += 8 * blockDim.x) {
+        unsigned long long keys[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int i = base + u * blockDim.x + tid;
+          keys[u] = (i < total) ? key_at(i) : 0ull;
         }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) keep(keys[u]);
       }
     }
   }
@@ -724,6 +746,8 @@ cudaError_t launch_cfg(const Config& c, bool filter, const CUtensorMap& mi, cons
                        cudaStream_t st) {
   if (c.NW == 16 && c.NT == 1)
     return filter ? launch_t<BM, PROD, 16, 1, 1, 1>(mi, mq, args, c.smem, st) : launch_t<BM, PROD, 16, 1, 1, 0>(mi, mq, args, c.smem, st);
+  if (c.NW == 12 && c.NT == 2)
+    return filter ? launch_t<BM, PROD, 12, 1, 2, 1>(mi, mq, args, c.smem, st) : launch_t<BM, PROD, 12, 1, 2, 0>(mi, mq, args, c.smem, st);
   if (c.NT == 2)
     return filter ? launch_t<BM, PROD, 8, 1, 2, 1>(mi, mq, args, c.smem, st) : launch_t<BM, PROD, 8, 1, 2, 0>(mi, mq, args, c.smem, st);
   return filter ? launch_t<BM, PROD, 8, 1, 1, 1>(mi, mq, args, c.smem, st) : launch_t<BM, PROD, 8, 1, 1, 0>(mi, mq, args, c.smem, st);
@@ -741,10 +765,11 @@ cudaError_t launch_scan(const tq_plan* plan, const Config& c, bool filter, const
   }
 }
 
-// nq <= 2: one column tile, 16 consumer warps of 16 vectors; nq > 2: two column tiles, 8 warps.
+// nq <= 2: one column tile, 16 consumer warps of 16 vectors; nq > 2: two column tiles, 12 (else 8) warps.
 // Falls back to the smallest shape when the B operand leaves no room for two stages.
 Config config_for(const tq_plan* plan, int nq) {
   Config c{8, 1, 1, 2, 0};
+  if (nq > 2 && pick_config(plan, 12, 1, 2, &c)) return c;
   if (nq > 2 && pick_config(plan, 8, 1, 2, &c)) return c;
   if (pick_config(plan, 16, 1, 1, &c)) return c;
   pick_config(plan, 8, 1, 1, &c);
@@ -812,22 +837,12 @@ int prepare(const tq_plan* plan, const float* Qcat, int nqp, void* workspace, cu
   const int ncols = plan->ncat * plan->dpad;
   QConst* qc = static_cast<QConst*>(workspace);
   uint2* bfrag = reinterpret_cast<uint2*>(static_cast<char*>(workspace) + kQConstBytes);
-  QStatArgs qa;
-  qa.Qcat = Qcat;
-  qa.ldq = ncols;
-  qa.d = plan->d;
-  qa.dpad = plan->dpad;
-  qa.prod = prod ? 1 : 0;
-  qa.amax = plan->ms.amax;
-  qa.csum = plan->ms.csum;
-  qa.out = qc;
-  qstats_kernel<<<nqp, 256, 0, st>>>(qa);
-  count_launches(1);
-  TQ_CHECK_CUDA(cudaGetLastError(), who);
   BPrepArgs ba;
   ba.Qcat = Qcat;
   ba.ldq = ncols;
   ba.qc = qc;
+  ba.amax = plan->ms.amax;
+  ba.csum = plan->ms.csum;
   ba.nq_pass = nqp;
   ba.d = plan->d;
   ba.dpad = plan->dpad;
