@@ -153,50 +153,67 @@ bool has_pad_words(int d, int bits, size_t row_bytes) {
   return bits > 0 && (size_t)((d + 31) / 32) * bits * 4 < row_bytes;
 }
 
-// Few queries: one warp per output column j forms <Rot[j, :], q> for up to 8 queries at a time, with
-// the queries staged in shared memory (the matrix is read once per 8 queries); each lane sums its
-// d/32 products in fp32 and the 32 partial sums are added in fp64.
-constexpr int kRotQ = 8, kRotChunk = 1024;
+// Few queries: one warp per output column j forms <Rot[j, :], q> for up to 8 queries at a time.  The
+// warp's slice of the matrix row goes to registers first, so that its latency overlaps the staging
+// of the queries in shared memory; each lane sums its products in fp32, the 32 partial sums are
+// added in fp64.  The matrix is read once per 8 queries.
+constexpr int kRotQ = 8, kRotChunk = 2048;   // 64 KB of queries per chunk (dynamic shared memory)
 
 template <typename T>
 __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __restrict__ Rot, int nrows, int d,
                                                              const T* __restrict__ Q, int64_t ldq, int nq,
                                                              float* __restrict__ Qcat, int64_t ldo) {
-  __shared__ __align__(16) float qs[kRotQ][kRotChunk];
+  extern __shared__ __align__(16) float qs_raw[];
+  float (*qs)[kRotChunk] = reinterpret_cast<float (*)[kRotChunk]>(qs_raw);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int j = blockIdx.x * 8 + warp;
   const float* row = Rot + (size_t)min(j, nrows - 1) * d;
+  const bool vec = (d & 3) == 0;   // rows are 16-byte aligned
   for (int q0 = 0; q0 < nq; q0 += kRotQ) {
     float acc[kRotQ];
 #pragma unroll
     for (int qq = 0; qq < kRotQ; ++qq) acc[qq] = 0.f;
     for (int c0 = 0; c0 < d; c0 += kRotChunk) {
       const int len = min(kRotChunk, d - c0);
-      __syncthreads();
-      for (int e = threadIdx.x; e < kRotQ * kRotChunk; e += blockDim.x) {
-        const int qq = e / kRotChunk, c = e % kRotChunk;
-        float v = 0.f;
-        if (q0 + qq < nq && c < len) v = scan::to_f32<T>(Q[(int64_t)(q0 + qq) * ldq + c0 + c]);
-        qs[qq][c] = v;
+      float4 r[kRotChunk / 128];
+      if (vec) {
+        const float4* row4 = reinterpret_cast<const float4*>(row + c0);
+#pragma unroll
+        for (int i = 0; i < kRotChunk / 128; ++i) {
+          const int c4 = lane + 32 * i;
+          r[i] = (4 * c4 < len) ? __ldg(row4 + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
       }
       __syncthreads();
-      if ((d & 3) == 0) {   // rows are 16-byte aligned: 128-bit loads, four in flight per lane
-        const float4* row4 = reinterpret_cast<const float4*>(row + c0);
-        const int len4 = len >> 2;
-#pragma unroll 4
-        for (int c4 = lane; c4 < len4; c4 += 32) {
-          const float4 r = __ldg(row4 + c4);
+      for (int e = threadIdx.x; e < kRotQ * (kRotChunk / 4); e += blockDim.x) {
+        const int qq = e / (kRotChunk / 4), c = 4 * (e % (kRotChunk / 4));
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        if (q0 + qq < nq && c < len) {
+          const T* src = Q + (int64_t)(q0 + qq) * ldq + c0 + c;
 #pragma unroll
-          for (int qq = 0; qq < kRotQ; ++qq) {
-            const float4 v = *reinterpret_cast<const float4*>(&qs[qq][4 * c4]);
-            acc[qq] = fmaf(r.x, v.x, fmaf(r.y, v.y, fmaf(r.z, v.z, fmaf(r.w, v.w, acc[qq]))));
+          for (int t = 0; t < 4; ++t)
+            if (c + t < len) v[t] = scan::to_f32<T>(src[t]);
+        }
+        *reinterpret_cast<float4*>(&qs[qq][c]) = make_float4(v[0], v[1], v[2], v[3]);
+      }
+      __syncthreads();
+      if (vec) {
+#pragma unroll
+        for (int i = 0; i < kRotChunk / 128; ++i) {
+          const int c4 = lane + 32 * i;
+          if (4 * c4 < len) {
+#pragma unroll
+            for (int qq = 0; qq < kRotQ; ++qq) {
+              const float4 v = *reinterpret_cast<const float4*>(&qs[qq][4 * c4]);
+              acc[qq] = fmaf(r[i].x, v.x, fmaf(r[i].y, v.y, fmaf(r[i].z, v.z, fmaf(r[i].w, v.w, acc[qq]))));
+            }
           }
         }
       } else {
         for (int c = lane; c < len; c += 32) {
-          const float r = __ldg(row + c0 + c);
+          const float rv = __ldg(row + c0 + c);
 #pragma unroll
-          for (int qq = 0; qq < kRotQ; ++qq) acc[qq] = fmaf(r, qs[qq][c], acc[qq]);
+          for (int qq = 0; qq < kRotQ; ++qq) acc[qq] = fmaf(rv, qs[qq][c], acc[qq]);
         }
       }
     }
@@ -210,18 +227,28 @@ __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __rest
   }
 }
 
+template <typename T>
+cudaError_t launch_rotate_queries(const tq_plan* plan, const T* Q, int64_t ldq, int nq, float* Qcat, cudaStream_t st) {
+  const int ncols = plan->ncat * plan->dpad;
+  constexpr int smem = kRotQ * kRotChunk * (int)sizeof(float);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(rotate_queries_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  rotate_queries_kernel<T><<<(unsigned)((ncols + 7) / 8), 256, smem, st>>>(plan->dRotCat, ncols, plan->d, Q, ldq, nq, Qcat, ncols);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
 // Q' = Q Pi^T and Q'' = Q S^T side by side: Qcat[nq, ncat*dpad].
 cudaError_t prepare_queries(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, float* Qcat,
                             cudaStream_t st) {
   const int ncols = plan->ncat * plan->dpad;
   if (nq <= 64) {
-    const unsigned blocks = (unsigned)((ncols + 7) / 8);
-    if (q_dtype == TQ_F32)
-      rotate_queries_kernel<float><<<blocks, 256, 0, st>>>(plan->dRotCat, ncols, plan->d, static_cast<const float*>(Q), ldq, nq, Qcat, ncols);
-    else
-      rotate_queries_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(plan->dRotCat, ncols, plan->d, static_cast<const __nv_bfloat16*>(Q), ldq, nq, Qcat, ncols);
-    count_launches(1);
-    return cudaGetLastError();
+    if (q_dtype == TQ_F32) return launch_rotate_queries(plan, static_cast<const float*>(Q), ldq, nq, Qcat, st);
+    return launch_rotate_queries(plan, static_cast<const __nv_bfloat16*>(Q), ldq, nq, Qcat, st);
   }
   simt::RowsF32 B{plan->dRotCat, plan->d, ncols, plan->d};
   simt::EpStore ep{Qcat, ncols, nullptr, nullptr};
