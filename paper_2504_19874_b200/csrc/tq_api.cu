@@ -11,6 +11,7 @@
 #include "tq_quantize_tc.h"
 #include "tq_scan_mma.h"
 #include "tq_scan_simt.cuh"
+#include "tq_scan_tc.h"
 
 using namespace tq;
 
@@ -92,13 +93,53 @@ constexpr int64_t kTopkBlockMin = 4096, kTopkBlockPref = 65536;
 constexpr int kFewQueries = 16;  // up to this many queries the code scan is bandwidth-bound
 // top-k on the tensor-path scan: candidate pairs kept per query, queries per pass, dense-buffer rows
 constexpr int kCandCap = 32768;
-constexpr int kPassQueries = 4;
 constexpr int64_t kFilterMinN = 65536;
-constexpr int64_t kDenseRowsPref = 1 << 20, kDenseRowsMin = 4096;
+constexpr int64_t kDenseRowsMin = 4096;
+constexpr int kGroupQueries = tscan::kQueriesPerPass * tscan::kPassesPerGroup;
 
-size_t ms_score_fixed(const tq_plan* plan, int nq) { return qcat_bytes(plan, nq) + mscan::workspace_bytes(plan); }
+// The two engines behind the bit-plane scan: register-fed integer MMA (2 or 4 queries per pass) for few
+// queries, tcgen05 (32 queries per pass) from 16 queries on (measured at d = 1536, b = 4, n = 10^6: one
+// tcgen05 pass 1.29 ms, one register-fed pass of 4 queries 0.39 ms).
+struct ScanEngine {
+  const tq_plan* plan;
+  bool tc;
+  int qpp;                  // queries per pass
+  int64_t dense_rows_pref;  // rows of the dense score buffer that keep the rescue pass to a few launches
+  size_t ws_bytes;          // engine workspace (constants + B operand)
+};
+
+ScanEngine pick_engine(const tq_plan* plan, int nq) {
+  ScanEngine e;
+  e.plan = plan;
+  e.tc = nq >= 16 && tscan::available(plan);
+  e.qpp = e.tc ? tscan::kQueriesPerPass : mscan::queries_per_pass(plan, nq);
+  e.dense_rows_pref = e.tc ? (1 << 18) : (1 << 20);
+  e.ws_bytes = e.tc ? tscan::workspace_bytes(plan) : mscan::workspace_bytes(plan);
+  return e;
+}
+
+// Prepares what the pass starting at query q0 needs (the tcgen05 engine builds 256 queries at a time).
+int engine_prepare(const ScanEngine& e, const float* Qcat, int q0, int nq, void* ws, cudaStream_t st, const char* who) {
+  const int ncols = e.plan->ncat * e.plan->dpad;
+  if (e.tc) {
+    if (q0 % kGroupQueries != 0) return TQ_OK;
+    return tscan::prepare_group(e.plan, Qcat + (size_t)q0 * ncols, std::min(kGroupQueries, nq - q0), ws, st, who);
+  }
+  return mscan::prepare(e.plan, Qcat + (size_t)q0 * ncols, std::min(e.qpp, nq - q0), ws, st, who);
+}
+
+int engine_run(const ScanEngine& e, int q0, int nqp, int64_t n, const uint8_t* idx, const uint8_t* qjl, const float* gamma,
+               const float* norms, float* scores, int64_t lds, const mscan::Filter* filter, const int* run_if, const void* ws,
+               cudaStream_t st, const char* who) {
+  if (e.tc)
+    return tscan::run_pass(e.plan, (q0 % kGroupQueries) / tscan::kQueriesPerPass, nqp, n, idx, qjl, gamma, norms, scores, lds,
+                           filter, run_if, ws, st, who);
+  return mscan::run(e.plan, nqp, n, idx, qjl, gamma, norms, scores, lds, filter, run_if, ws, st, who);
+}
+
+size_t ms_score_fixed(const tq_plan* plan, int nq) { return qcat_bytes(plan, nq) + align_up(pick_engine(plan, nq).ws_bytes, 256); }
 size_t ms_topk_fixed(const tq_plan* plan, int nq) {
-  return ms_score_fixed(plan, nq) + 256 /* tau, count, overflow */ + (size_t)kPassQueries * kCandCap * 8;
+  return ms_score_fixed(plan, nq) + 512 /* tau, count, overflow */ + (size_t)pick_engine(plan, nq).qpp * kCandCap * 8;
 }
 
 template <typename T>
@@ -158,6 +199,7 @@ bool has_pad_words(int d, int bits, size_t row_bytes) {
 // of the queries in shared memory; each lane sums its products in fp32, the 32 partial sums are
 // added in fp64.  The matrix is read once per 8 queries.
 constexpr int kRotQ = 8, kRotChunk = 2048;   // 64 KB of queries per chunk (dynamic shared memory)
+constexpr int kRotQPerBlock = 64;            // queries per CTA (grid.y covers the rest)
 
 template <typename T>
 __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __restrict__ Rot, int nrows, int d,
@@ -169,7 +211,8 @@ __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __rest
   const int j = blockIdx.x * 8 + warp;
   const float* row = Rot + (size_t)min(j, nrows - 1) * d;
   const bool vec = (d & 3) == 0;   // rows are 16-byte aligned
-  for (int q0 = 0; q0 < nq; q0 += kRotQ) {
+  const int q_begin = blockIdx.y * kRotQPerBlock, q_end = min(nq, q_begin + kRotQPerBlock);
+  for (int q0 = q_begin; q0 < q_end; q0 += kRotQ) {
     float acc[kRotQ];
 #pragma unroll
     for (int qq = 0; qq < kRotQ; ++qq) acc[qq] = 0.f;
@@ -188,7 +231,7 @@ __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __rest
       for (int e = threadIdx.x; e < kRotQ * (kRotChunk / 4); e += blockDim.x) {
         const int qq = e / (kRotChunk / 4), c = 4 * (e % (kRotChunk / 4));
         float v[4] = {0.f, 0.f, 0.f, 0.f};
-        if (q0 + qq < nq && c < len) {
+        if (q0 + qq < q_end && c < len) {
           const T* src = Q + (int64_t)(q0 + qq) * ldq + c0 + c;
 #pragma unroll
           for (int t = 0; t < 4; ++t)
@@ -222,7 +265,7 @@ __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __rest
       double v = (double)acc[qq];
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      if (lane == 0 && j < nrows && q0 + qq < nq) Qcat[(int64_t)(q0 + qq) * ldo + j] = (float)v;
+      if (lane == 0 && j < nrows && q0 + qq < q_end) Qcat[(int64_t)(q0 + qq) * ldo + j] = (float)v;
     }
   }
 }
@@ -237,7 +280,8 @@ cudaError_t launch_rotate_queries(const tq_plan* plan, const T* Q, int64_t ldq, 
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  rotate_queries_kernel<T><<<(unsigned)((ncols + 7) / 8), 256, smem, st>>>(plan->dRotCat, ncols, plan->d, Q, ldq, nq, Qcat, ncols);
+  const dim3 grid((unsigned)((ncols + 7) / 8), (unsigned)((nq + kRotQPerBlock - 1) / kRotQPerBlock));
+  rotate_queries_kernel<T><<<grid, 256, smem, st>>>(plan->dRotCat, ncols, plan->d, Q, ldq, nq, Qcat, ncols);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -246,18 +290,11 @@ cudaError_t launch_rotate_queries(const tq_plan* plan, const T* Q, int64_t ldq, 
 cudaError_t prepare_queries(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, float* Qcat,
                             cudaStream_t st) {
   const int ncols = plan->ncat * plan->dpad;
-  if (nq <= 64) {
-    if (q_dtype == TQ_F32) return launch_rotate_queries(plan, static_cast<const float*>(Q), ldq, nq, Qcat, st);
-    return launch_rotate_queries(plan, static_cast<const __nv_bfloat16*>(Q), ldq, nq, Qcat, st);
-  }
-  simt::RowsF32 B{plan->dRotCat, plan->d, ncols, plan->d};
-  simt::EpStore ep{Qcat, ncols, nullptr, nullptr};
-  if (q_dtype == TQ_F32) {
-    simt::RowsF32 A{static_cast<const float*>(Q), ldq, nq, plan->d};
-    return simt::launch_gemm(A, B, ep, (int64_t)nq, (int64_t)ncols, plan->d, st);
-  }
-  simt::RowsBF16 A{static_cast<const __nv_bfloat16*>(Q), ldq, nq, plan->d};
-  return simt::launch_gemm(A, B, ep, (int64_t)nq, (int64_t)ncols, plan->d, st);
+  (void)ncols;
+  // One kernel for every query count, so that a query's rotated form (and hence its estimates) does not
+  // depend on how many other queries came with it.
+  if (q_dtype == TQ_F32) return launch_rotate_queries(plan, static_cast<const float*>(Q), ldq, nq, Qcat, st);
+  return launch_rotate_queries(plan, static_cast<const __nv_bfloat16*>(Q), ldq, nq, Qcat, st);
 }
 
 template <int BITS, bool PROD>
@@ -488,7 +525,9 @@ extern "C" size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int
     case TQ_OP_TOPK:
       if (plan->ms.ok)
         return ms_topk_fixed(plan, nq) +
-               align_up((size_t)kPassQueries * std::max<int64_t>(std::min<int64_t>(n, kDenseRowsPref), kDenseRowsMin) * sizeof(float), 256);
+               align_up((size_t)pick_engine(plan, nq).qpp *
+                            std::max<int64_t>(std::min<int64_t>(n, pick_engine(plan, nq).dense_rows_pref), kDenseRowsMin) * sizeof(float),
+                        256);
       return qcat_bytes(plan, nq) + align_up((size_t)nq * std::min<int64_t>(n, kTopkBlockPref) * sizeof(float), 256);
     case TQ_OP_WSUM: {
       const size_t ncols = (size_t)plan->ncat * plan->dpad;
@@ -630,12 +669,11 @@ extern "C" int tq_score(const tq_plan* plan, const void* Q, int q_dtype, int nq,
   TQ_CHECK_CUDA(prepare_queries(plan, Q, q_dtype, nq, ldq, Qcat, st), who);
   if (plan->ms.ok) {
     void* msw = static_cast<char*>(workspace) + qcat_bytes(plan, nq);
-    const int ncols = plan->ncat * plan->dpad;
-    const int qpp = mscan::queries_per_pass(plan, nq);
-    for (int q0 = 0; q0 < nq; q0 += qpp) {
-      const int nqp = std::min(qpp, nq - q0);
-      if ((rc = mscan::prepare(plan, Qcat + (size_t)q0 * ncols, nqp, msw, st, who))) return rc;
-      if ((rc = mscan::run(plan, nqp, n, idx, qjl, gamma, norms, scores + (int64_t)q0 * lds, lds, nullptr, nullptr, msw, st, who)))
+    const ScanEngine eng = pick_engine(plan, nq);
+    for (int q0 = 0; q0 < nq; q0 += eng.qpp) {
+      const int nqp = std::min(eng.qpp, nq - q0);
+      if ((rc = engine_prepare(eng, Qcat, q0, nq, msw, st, who))) return rc;
+      if ((rc = engine_run(eng, q0, nqp, n, idx, qjl, gamma, norms, scores + (int64_t)q0 * lds, lds, nullptr, nullptr, msw, st, who)))
         return rc;
     }
     return TQ_OK;
@@ -653,36 +691,36 @@ static int topk_ms(const tq_plan* plan, const float* Qcat, int nq, int64_t n, co
                    const float* gamma, const float* norms, int k, float* top_scores, int32_t* top_ids, char* ws,
                    size_t ws_bytes, cudaStream_t st, const char* who) {
   int rc;
+  const ScanEngine eng = pick_engine(plan, nq);
   void* msw = ws;
-  char* p = ws + mscan::workspace_bytes(plan);
-  float* tau = reinterpret_cast<float*>(p);
-  int* count = reinterpret_cast<int*>(p + 64);
-  int* overflow = reinterpret_cast<int*>(p + 128);
-  p += 256;
+  char* p = ws + align_up(eng.ws_bytes, 256);
+  float* tau = reinterpret_cast<float*>(p);          // [qpp] (qpp <= 32: 128 bytes)
+  int* count = reinterpret_cast<int*>(p + 128);      // [qpp], then the overflow flag
+  int* overflow = count + eng.qpp;
+  p += 512;
   float* cand_s = reinterpret_cast<float*>(p);
-  int* cand_i = reinterpret_cast<int*>(p + (size_t)kPassQueries * kCandCap * 4);
-  p += (size_t)kPassQueries * kCandCap * 8;
+  int* cand_i = reinterpret_cast<int*>(p + (size_t)eng.qpp * kCandCap * 4);
+  p += (size_t)eng.qpp * kCandCap * 8;
   float* dense = reinterpret_cast<float*>(p);
   const int64_t dense_floats = (int64_t)((ws + ws_bytes - p) / sizeof(float));
-  const int ncols = plan->ncat * plan->dpad;
-  const int qpp = mscan::queries_per_pass(plan, nq);
+  const int qpp = eng.qpp;
   const size_t xrb = plan->idx_row_bytes, qrb = plan->qjl_row_bytes;
   for (int q0 = 0; q0 < nq; q0 += qpp) {
     const int nqp = std::min(qpp, nq - q0);
     float* ts = top_scores + (size_t)q0 * k;
     int32_t* ti = top_ids + (size_t)q0 * k;
-    if ((rc = mscan::prepare(plan, Qcat + (size_t)q0 * ncols, nqp, msw, st, who))) return rc;
-    const int64_t dense_rows = dense_floats / nqp;
-    const bool use_filter = n >= kFilterMinN && dense_rows >= std::min<int64_t>(n, kDenseRowsPref);
+    if ((rc = engine_prepare(eng, Qcat, q0, nq, msw, st, who))) return rc;
+    const int64_t dense_rows = dense_floats / qpp;
+    const bool use_filter = n >= kFilterMinN && dense_rows >= std::min<int64_t>(n, eng.dense_rows_pref);
     const int* guard = nullptr;
     if (use_filter) {
       int64_t m = std::max<int64_t>(round_up64(n / 64, 256), round_up64(std::max(k, 4096), 256));
       m = std::min<int64_t>(m, std::min<int64_t>(dense_rows / 256 * 256, n));
-      if ((rc = mscan::run(plan, nqp, m, idx, qjl, gamma, norms, dense, m, nullptr, nullptr, msw, st, who))) return rc;
+      if ((rc = engine_run(eng, q0, nqp, m, idx, qjl, gamma, norms, dense, m, nullptr, nullptr, msw, st, who))) return rc;
       TQ_CHECK_CUDA(mscan::select_topk(dense, nullptr, nullptr, (int)m, (int)m, 0, nqp, k, 0, ts, ti, tau, nullptr, nullptr, st), who);
-      TQ_CHECK_CUDA(cudaMemsetAsync(count, 0, 128, st), who);   // counters and the overflow flag
+      TQ_CHECK_CUDA(cudaMemsetAsync(count, 0, (size_t)(qpp + 1) * sizeof(int), st), who);   // counters and the overflow flag
       mscan::Filter f{tau, count, cand_s, cand_i, kCandCap};
-      if ((rc = mscan::run(plan, nqp, n, idx, qjl, gamma, norms, nullptr, 0, &f, nullptr, msw, st, who))) return rc;
+      if ((rc = engine_run(eng, q0, nqp, n, idx, qjl, gamma, norms, nullptr, 0, &f, nullptr, msw, st, who))) return rc;
       TQ_CHECK_CUDA(mscan::select_topk(cand_s, cand_i, count, kCandCap, 0, 0, nqp, k, 0, ts, ti, nullptr, overflow, nullptr, st), who);
       guard = overflow;
     }
@@ -691,7 +729,7 @@ static int topk_ms(const tq_plan* plan, const float* Qcat, int nq, int64_t n, co
     if (block < n) block = block / 256 * 256;
     for (int64_t v0 = 0; v0 < n; v0 += block) {
       const int64_t cn = std::min(block, n - v0);
-      if ((rc = mscan::run(plan, nqp, cn, idx ? idx + (size_t)v0 * xrb : nullptr, qjl ? qjl + (size_t)v0 * qrb : nullptr,
+      if ((rc = engine_run(eng, q0, nqp, cn, idx ? idx + (size_t)v0 * xrb : nullptr, qjl ? qjl + (size_t)v0 * qrb : nullptr,
                            gamma ? gamma + v0 : nullptr, norms ? norms + v0 : nullptr, dense, block, nullptr, guard, msw, st, who)))
         return rc;
       TQ_CHECK_CUDA(mscan::select_topk(dense, nullptr, nullptr, (int)block, (int)cn, (int)v0, nqp, k, v0 > 0 ? 1 : 0, ts, ti,
@@ -715,7 +753,7 @@ extern "C" int tq_topk(const tq_plan* plan, const void* Q, int q_dtype, int nq, 
   if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
   TQ_REQUIRE(top_scores != nullptr && top_ids != nullptr, TQ_ERR_INVALID_ARG, "%s: output is NULL", who);
   const size_t qb = qcat_bytes(plan, nq);
-  const size_t need = plan->ms.ok ? ms_topk_fixed(plan, nq) + (size_t)kPassQueries * kDenseRowsMin * sizeof(float)
+  const size_t need = plan->ms.ok ? ms_topk_fixed(plan, nq) + (size_t)pick_engine(plan, nq).qpp * kDenseRowsMin * sizeof(float)
                                   : qb + align_up((size_t)nq * std::min<int64_t>(n, kTopkBlockMin) * sizeof(float), 256);
   TQ_REQUIRE(workspace != nullptr && workspace_bytes >= need, TQ_ERR_WORKSPACE, "%s: workspace of %zu bytes, %zu needed",
              who, workspace_bytes, need);

@@ -1,0 +1,648 @@
+// Many-query packed-code scan on tcgen05: the same bit-plane form of the estimator as in
+// tq_scan_mma.cu (codebook expanded over the index bits, raw bits and parity words as a 0/1 matrix,
+// query weights as fixed-point radix-256 digits), but with the multiply-accumulate on the 5th-generation
+// tensor cores:   D[128 vectors, 128 columns] += A[128, 32] * B[128, 32]^T,  kind::i8, s32 in TMEM.
+// 128 columns hold 32 queries x 4 digits, so one pass over the codes serves 32 queries and the decode
+// (one AND per four bits, done once per vector) is amortised over all of them.  A tcgen05 MMA of this
+// shape costs the same 64 cycles for any N <= 128, which is why this path is for many queries and the
+// register-fed mma.sync path for few.  The byte-expanded A tiles go through shared memory (TMEM is
+// full of accumulators), and that traffic -- per k-block 32 KB written + 32 KB read for A, 16 KB written
+// + 32 KB read for B = 896 cycles at 128 B/clk against 512 cycles of MMA -- is what bounds this kernel.
+//
+// CTA (one per SM, persistent over pairs of 128-vector tiles):
+//   warp 0      TMA producer of B: per k-block (128 K-bytes) one [128 rows x 128 B] box, 128-byte swizzle
+//   warp 1      MMA issuer and TMEM owner: per k-block 4 MMAs (K = 32) for each of the two tiles
+//   warps 2..9  transform + epilogue: thread = one vector row.  Per k-block it loads the row's 4 packed
+//               words (3 index words + their parity word at b_m = 3), expands them into 32 registers
+//               (w & (0x01010101 << k)) and stores them as the row's 128 bytes of the A tile in the
+//               swizzled K-major layout the UMMA descriptor expects; after the last k-block it reads
+//               its row of the accumulators from TMEM, recombines the digits and emits the estimates.
+// Two tiles share every B box (halves the L2 traffic of B); their accumulators (MSE part and QJL part,
+// 128 columns each, per tile) fill the 512 TMEM columns.  Rings: 3 stages of (A0, A1) = 32 KB and 4 stages of
+// B = 16 KB, each with full / empty mbarriers (empty =
+// tcgen05.commit); accumulator full / empty.  All waits are bounded.
+#include <algorithm>
+#include <cmath>
+
+#include "tq_quantize_tc.h"
+#include "tq_scan_tc.h"
+#include "tq_tc.cuh"
+
+namespace tq {
+namespace tscan {
+
+namespace {
+
+constexpr int TILE = 128;              // vectors per M tile = TMEM lanes
+constexpr int NCOL = 128;              // MMA N: 32 queries x 4 digits
+constexpr int LIMBS = 4;
+constexpr int KB_BYTES = 128;          // K extent of one k-block (one swizzled row)
+constexpr int A_STAGES = 3;            // ring of A tile pairs (written by the transform warps: short latency)
+constexpr int B_STAGES = 4;            // ring of B tiles (TMA from L2)
+constexpr int TILE_BYTES = TILE * KB_BYTES;          // 16 KB
+constexpr int A_STAGE_BYTES = 2 * TILE_BYTES;        // A (tile 0), A (tile 1)
+constexpr int A_RING_BYTES = A_STAGES * A_STAGE_BYTES;
+constexpr int NTHREADS = 320;
+constexpr int TMEM_COLS = 512;
+constexpr size_t kConstBytes = 256 * 48;             // per-query constants of one group
+
+struct QConst {
+  double sa, ca;   // a = T_a * sa + ca   (MSE term)
+  double ss, cs;   // s = T_s * ss + cs   (QJL term)
+  int fa, fs;
+  int pad[2];
+};
+
+struct Geo {
+  int bm, d, dpad;
+  int widx, wq;    // 32-bit words per idx / qjl row
+  int kba, kbs;    // k-blocks of the MSE part and of the QJL part
+};
+
+__host__ __device__ inline int div_up(int a, int b) { return (a + b - 1) / b; }
+
+Geo make_geo(const tq_plan* plan) {
+  Geo g;
+  g.bm = plan->mse_bits;
+  g.d = plan->d;
+  g.dpad = plan->dpad;
+  g.widx = (int)(plan->idx_row_bytes / 4);
+  g.wq = (plan->mode == TQ_PROD) ? (int)(plan->qjl_row_bytes / 4) : 0;
+  g.kba = g.bm == 0 ? 0 : g.bm == 3 ? div_up(g.widx, 3) : g.bm == 4 ? div_up(g.widx, 2) : div_up(g.widx, 4);
+  g.kbs = div_up(g.wq, 4);
+  return g;
+}
+
+// K slot (part, k-block, word wl of the block, bit of the word) -> (coordinate, Walsh term).
+// MSE part, b_m = 1, 2: four index words per block.  b_m = 3: the three words of one 96-bit group of 32
+// coordinates and their parity word.  b_m = 4: two index words and their two words of 3-subset parities.
+struct Slot {
+  int coord, term;
+};
+__device__ inline Slot slot_a(const Geo& g, int kb, int wl, int bit) {
+  if (g.bm <= 2) {
+    const int P = 32 * (4 * kb + wl) + bit;
+    return {P / g.bm, P % g.bm};
+  }
+  if (g.bm == 3) {
+    if (wl < 3) {
+      const int P = 32 * (3 * kb + wl) + bit;
+      return {P / 3, P % 3};
+    }
+    const int m = bit % 3;
+    const int c = (m == 0) ? bit / 3 : (m == 1) ? (32 + bit) / 3 : (64 + bit) / 3;
+    return {32 * kb + c, 4};
+  }
+  if (wl < 2) {
+    const int P = 32 * (2 * kb + wl) + bit;
+    return {P / 4, P % 4};
+  }
+  return {8 * (2 * kb + wl - 2) + bit / 4, 4 + (bit & 3)};
+}
+
+// ------------------------------------------------------------------ per-query constants
+struct StatArgs {
+  const float* Qcat;
+  int64_t ldq;
+  int d, dpad, prod;
+  double amax, csum;
+  QConst* out;
+};
+
+__global__ void __launch_bounds__(256) tstats_kernel(StatArgs a) {
+  __shared__ double red[4][8];
+  const float* q = a.Qcat + (int64_t)blockIdx.x * a.ldq;
+  double mx1 = 0.0, sm1 = 0.0, mx2 = 0.0, sm2 = 0.0;
+  for (int j = threadIdx.x; j < a.d; j += blockDim.x) {
+    const double v = (double)q[j];
+    mx1 = fmax(mx1, fabs(v));
+    sm1 += v;
+    if (a.prod) {
+      const double u = (double)q[a.dpad + j];
+      mx2 = fmax(mx2, fabs(u));
+      sm2 += u;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mx1 = fmax(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+    mx2 = fmax(mx2, __shfl_xor_sync(0xffffffffu, mx2, o));
+    sm1 += __shfl_xor_sync(0xffffffffu, sm1, o);
+    sm2 += __shfl_xor_sync(0xffffffffu, sm2, o);
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) {
+    red[0][warp] = mx1; red[1][warp] = sm1; red[2][warp] = mx2; red[3][warp] = sm2;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) {
+      mx1 = fmax(mx1, red[0][w]); sm1 += red[1][w];
+      mx2 = fmax(mx2, red[2][w]); sm2 += red[3][w];
+    }
+    // |W| < 2^e with W = 2 alpha q'  ->  |W| 2^(29-e) < 2^29: four signed radix-256 digits hold it.  The same
+    // exponent as in the register-fed scan, so that both engines form identical integers and estimates.
+    auto expo = [](double wmax) {
+      if (!(wmax > 0.0) || !isfinite(wmax)) return 0;
+      int e;
+      frexp(wmax, &e);
+      return 29 - e;
+    };
+    QConst c;
+    c.fa = expo(2.0 * a.amax * mx1);
+    c.fs = expo(2.0 * mx2);
+    c.sa = ldexp(1.0, -c.fa);
+    c.ss = ldexp(1.0, -c.fs);
+    c.ca = a.csum * sm1;
+    c.cs = -sm2;
+    c.pad[0] = c.pad[1] = 0;
+    a.out[blockIdx.x] = c;
+  }
+}
+
+// ------------------------------------------------------------------ B matrices
+// Ba[pass*128 + n][kba*128], Bs[pass*128 + n][kbs*128], n = 4 * (query in pass) + digit; K-major int8.
+// Byte kappa of a k-block = (2 wl + k / 4) * 16 + (k % 4) * 4 + i  <->  bit 8 i + k of word wl: the order in
+// which the transform threads lay out their registers.
+struct BPrepArgs {
+  const float* Qcat;
+  int64_t ldq;
+  const QConst* qc;
+  int nqg;
+  Geo g;
+  double alpha[8];
+  uint8_t* Ba;
+  uint8_t* Bs;
+};
+
+__device__ __forceinline__ int digit_of(long long J, int limb) {
+  int dg = 0;
+  for (int l = 0; l <= limb; ++l) {
+    dg = (int)(((J + 128) & 255) - 128);
+    J = (J - dg) >> 8;
+  }
+  return dg;
+}
+
+__global__ void __launch_bounds__(256) tbprep_kernel(BPrepArgs a, int part, int rows) {
+  const int nkb = part ? a.g.kbs : a.g.kba;
+  const int64_t total = (int64_t)rows * nkb * 4;
+  const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (tid >= total) return;
+  const int wl = (int)(tid & 3);
+  const int kb = (int)((tid >> 2) % nkb);
+  const int row = (int)((tid >> 2) / nkb);      // pass * 128 + n
+  const int ql = (row / NCOL) * kQueriesPerPass + (row % NCOL) / LIMBS, limb = row % LIMBS;
+  uint32_t out[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+  if (ql < a.nqg) {
+    const float* q = a.Qcat + (int64_t)ql * a.ldq;
+    const QConst c = a.qc[ql];
+    for (int k = 0; k < 8; ++k) {
+      for (int i = 0; i < 4; ++i) {
+        const int bit = 8 * i + k;
+        double W = 0.0;
+        int f;
+        if (!part) {
+          const Slot s = slot_a(a.g, kb, wl, bit);
+          if (s.coord < a.g.d) W = 2.0 * a.alpha[s.term] * (double)q[s.coord];
+          f = c.fa;
+        } else {
+          const int j = 32 * (4 * kb + wl) + bit;
+          if (j < a.g.d) W = 2.0 * (double)q[a.g.dpad + j];
+          f = c.fs;
+        }
+        double Jd = rint(ldexp(W, f - k));
+        if (!(fabs(Jd) <= 1073741824.0)) Jd = 0.0;   // non-finite query entries contribute nothing
+        out[k] |= (uint32_t)(digit_of((long long)Jd, limb) & 255) << (8 * i);
+      }
+    }
+  }
+  uint8_t* dst = (part ? a.Bs : a.Ba) + (size_t)row * nkb * KB_BYTES + (size_t)kb * KB_BYTES + wl * 32;
+  *reinterpret_cast<uint4*>(dst) = make_uint4(out[0], out[1], out[2], out[3]);
+  *reinterpret_cast<uint4*>(dst + 16) = make_uint4(out[4], out[5], out[6], out[7]);
+}
+
+// ------------------------------------------------------------------ scan kernel
+struct ScanArgs {
+  int64_t n, npairs;
+  Geo g;
+  int pass, nqp;
+  const QConst* qc;        // constants of this pass's queries
+  const uint8_t* idx;
+  size_t idx_rb;
+  const uint8_t* qjl;
+  size_t qjl_rb;
+  const float* gamma;
+  const float* norms;
+  float coef;
+  float* scores;
+  int64_t lds;
+  const float* tau;
+  int* count;
+  float* cand_s;
+  int* cand_i;
+  int cap;
+  const int* run_if;
+  int* status;
+};
+
+__device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// kind::i8: D = s32, A = unsigned 8-bit, B = signed 8-bit, both K-major.
+__host__ __device__ constexpr uint32_t idesc_i8(int M, int N) {
+  return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+template <int BM, int MODE>
+__global__ void __launch_bounds__(NTHREADS, 1)
+scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__ CUtensorMap tmBs, ScanArgs a) {
+  if (a.run_if != nullptr && *a.run_if == 0) return;
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* bring = smem + A_RING_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(bring + B_STAGES * TILE_BYTES);
+  uint64_t* afull = bars;                           // [A_STAGES]  transform warps -> MMA
+  uint64_t* aempty = afull + A_STAGES;              // [A_STAGES]  MMA -> transform warps
+  uint64_t* bfull = aempty + A_STAGES;              // [B_STAGES]  TMA -> MMA
+  uint64_t* bempty = bfull + B_STAGES;              // [B_STAGES]  MMA -> TMA producer
+  uint64_t* dfull = bempty + B_STAGES;              // accumulators complete -> epilogue
+  uint64_t* dempty = dfull + 1;                     // accumulators read -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(dempty + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  QConst* qcs = reinterpret_cast<QConst*>(dempty + 3);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nkb_total = a.g.kba + a.g.kbs;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < A_STAGES; ++s) {
+      tc::mbar_init(&afull[s], 8);
+      tc::mbar_init(&aempty[s], 1);
+    }
+    for (int s = 0; s < B_STAGES; ++s) {
+      tc::mbar_init(&bfull[s], 1);
+      tc::mbar_init(&bempty[s], 1);
+    }
+    tc::mbar_init(dfull, 1);
+    tc::mbar_init(dempty, 8);
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+    if (a.g.kba > 0) tc::tma_prefetch_desc(&tmBa);
+    if (a.g.kbs > 0) tc::tma_prefetch_desc(&tmBs);
+  }
+  if (threadIdx.x < kQueriesPerPass) {
+    QConst c = {1.0, 0.0, 1.0, 0.0, 0, 0, {0, 0}};
+    if ((int)threadIdx.x < a.nqp) c = a.qc[threadIdx.x];
+    qcs[threadIdx.x] = c;
+  }
+  if (warp == 1) tc::tmem_alloc(tmem_slot, TMEM_COLS);
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer of B
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int64_t pair = blockIdx.x; pair < a.npairs && ok; pair += gridDim.x) {
+        for (int f = 0; f < nkb_total; ++f) {
+          if (!(ok = tc::mbar_wait(&bempty[stage], phase ^ 1u, abort_flag, a.status))) break;
+          const bool part_s = f >= a.g.kba;
+          const int kb = part_s ? f - a.g.kba : f;
+          tc::mbar_arrive_expect_tx(&bfull[stage], TILE_BYTES);
+          tc::tma_load_2d(bring + stage * TILE_BYTES, part_s ? &tmBs : &tmBa, &bfull[stage], kb * KB_BYTES, a.pass * NCOL);
+          if (++stage == B_STAGES) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+      if (!ok) {
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);   // let copies in flight land
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_i8(TILE, NCOL);
+      int stage = 0, bstage = 0;
+      uint32_t phase = 0, bphase = 0;
+      bool ok = true;
+      int64_t it = 0;
+      for (int64_t pair = blockIdx.x; pair < a.npairs && ok; pair += gridDim.x, ++it) {
+        if (!(ok = tc::mbar_wait(dempty, (uint32_t)(it & 1) ^ 1u, abort_flag, a.status))) break;
+        tc::tc_fence_after();
+        for (int f = 0; f < nkb_total; ++f) {
+          if (!(ok = tc::mbar_wait(&bfull[bstage], bphase, abort_flag, a.status))) break;
+          if (!(ok = tc::mbar_wait(&afull[stage], phase, abort_flag, a.status))) break;
+          tc::tc_fence_after();
+          const bool part_s = f >= a.g.kba;
+          const int kb = part_s ? f - a.g.kba : f;
+          const uint32_t sb = tc::smem_u32(smem + stage * A_STAGE_BYTES);
+          const uint64_t bdesc = tc::smem_desc_sw128(tc::smem_u32(bring + bstage * TILE_BYTES));
+#pragma unroll
+          for (int t = 0; t < 2; ++t) {
+            const uint64_t adesc = tc::smem_desc_sw128(sb + t * TILE_BYTES);
+            const uint32_t d_tmem = tmem_base + (uint32_t)(t * 256 + (part_s ? NCOL : 0));
+#pragma unroll
+            for (int step = 0; step < 4; ++step)   // 32 K-bytes per MMA: +32 bytes inside the swizzled row
+              umma_i8(d_tmem, adesc + 2 * step, bdesc + 2 * step, idesc, (kb | step) != 0 ? 1u : 0u);
+          }
+          tc::umma_commit(&aempty[stage]);   // both stages reusable once these MMAs have read them
+          tc::umma_commit(&bempty[bstage]);
+          if (++stage == A_STAGES) {
+            stage = 0;
+            phase ^= 1u;
+          }
+          if (++bstage == B_STAGES) {
+            bstage = 0;
+            bphase ^= 1u;
+          }
+        }
+        if (ok) tc::umma_commit(dfull);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------------------------------------------------------- transform + epilogue (thread = vector row)
+    const int e = warp - 2;
+    const int t = e >> 2;                   // which tile of the pair
+    const int quad = warp & 3;              // TMEM lane group this warp may access
+    const int r = quad * 32 + lane;         // row inside the tile
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    int64_t it = 0;
+    for (int64_t pair = blockIdx.x; pair < a.npairs && ok; pair += gridDim.x, ++it) {
+      const int64_t row = pair * (2 * TILE) + t * TILE + r;
+      const bool row_ok = row < a.n;
+      const uint32_t* irow = reinterpret_cast<const uint32_t*>(a.idx + (size_t)(row_ok ? row : 0) * a.idx_rb);
+      const uint32_t* qrow = reinterpret_cast<const uint32_t*>(a.qjl + (size_t)(row_ok ? row : 0) * a.qjl_rb);
+      const float nu = (row_ok && a.norms != nullptr) ? __ldg(a.norms + row) : 1.f;
+      const float gm = (row_ok && a.g.kbs > 0) ? a.coef * __ldg(a.gamma + row) : 0.f;
+
+      // the row's packed words of k-block f (index words first, parity words derived later)
+      auto load_words = [&](int f, uint32_t (&w)[4]) {
+        w[0] = w[1] = w[2] = w[3] = 0u;
+        if (!row_ok || f >= nkb_total) return;
+        if (f >= a.g.kba) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(qrow) + (f - a.g.kba));
+          w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+        } else if (BM <= 2) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(irow) + f);
+          w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+        } else if (BM == 3) {
+#pragma unroll
+          for (int i = 0; i < 3; ++i)
+            if (3 * f + i < a.g.widx) w[i] = __ldg(irow + 3 * f + i);
+        } else {
+          const uint2 v = __ldg(reinterpret_cast<const uint2*>(irow) + f);
+          w[0] = v.x; w[1] = v.y;
+        }
+      };
+      // expands one k-block's words into the row's 128 bytes of the A tile of the current stage
+      auto emit = [&](uint32_t (&w)[4], int f) -> bool {
+        if (f >= nkb_total) return true;
+        if (f < a.g.kba) {
+          if (BM == 3) {
+            const uint32_t p0 = w[0] ^ __funnelshift_r(w[0], w[1], 1) ^ __funnelshift_r(w[0], w[1], 2);
+            const uint32_t p1 = w[1] ^ __funnelshift_r(w[1], w[2], 1) ^ __funnelshift_r(w[1], w[2], 2);
+            const uint32_t p2 = w[2] ^ (w[2] >> 1) ^ (w[2] >> 2);
+            w[3] = (p0 & 0x49249249u) | (p1 & 0x92492492u) | (p2 & 0x24924924u);
+          } else if (BM == 4) {
+            const uint32_t M = 0x11111111u;
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+              const uint32_t x = w[i], s1 = x >> 1, s2 = x >> 2, s3 = x >> 3;
+              w[2 + i] = ((x ^ s1 ^ s2) & M) | (((x ^ s1 ^ s3) & M) << 1) | (((x ^ s2 ^ s3) & M) << 2) | (((s1 ^ s2 ^ s3) & M) << 3);
+            }
+          }
+        }
+        if (!tc::mbar_wait(&aempty[stage], phase ^ 1u, abort_flag, a.status)) return false;
+        // 16-byte chunk c goes to position c ^ (r & 7) (128-byte swizzle)
+        unsigned char* arow = smem + stage * A_STAGE_BYTES + t * TILE_BYTES + r * KB_BYTES;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint32_t x = w[c >> 1];
+          const int k0 = (c & 1) * 4;
+          const uint4 v = make_uint4(x & (0x01010101u << k0), x & (0x01010101u << (k0 + 1)), x & (0x01010101u << (k0 + 2)),
+                                     x & (0x01010101u << (k0 + 3)));
+          *reinterpret_cast<uint4*>(arow + ((c ^ (r & 7)) << 4)) = v;
+        }
+        fence_async_smem();   // make the generic-proxy stores visible to the tensor core's reads
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&afull[stage]);
+        if (++stage == A_STAGES) {
+          stage = 0;
+          phase ^= 1u;
+        }
+        return true;
+      };
+      // two register sets of four k-blocks each: the loads of one set (the codes stream from HBM) are in flight
+      // while the other set is expanded
+      constexpr int PF = 4;
+      uint32_t wa[PF][4], wb[PF][4];
+#pragma unroll
+      for (int j = 0; j < PF; ++j) load_words(j, wa[j]);
+      for (int f0 = 0; f0 < nkb_total && ok; f0 += 2 * PF) {
+#pragma unroll
+        for (int j = 0; j < PF; ++j) load_words(f0 + PF + j, wb[j]);
+#pragma unroll
+        for (int j = 0; j < PF; ++j) ok = ok && emit(wa[j], f0 + j);
+#pragma unroll
+        for (int j = 0; j < PF; ++j) load_words(f0 + 2 * PF + j, wa[j]);
+#pragma unroll
+        for (int j = 0; j < PF; ++j) ok = ok && emit(wb[j], f0 + PF + j);
+      }
+      if (!ok) break;
+
+      // ---- epilogue: this thread's row of the four accumulators
+      if (!(ok = tc::mbar_wait(dfull, (uint32_t)(it & 1), abort_flag, a.status))) break;
+      tc::tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(t * 256);
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {   // 32 columns = 8 queries per chunk
+        uint32_t va[32], vs[32];
+        if (a.g.kba > 0) tc::tmem_ld32(taddr + ch * 32, va);
+        if (a.g.kbs > 0) tc::tmem_ld32(taddr + NCOL + ch * 32, vs);
+        tc::tmem_ld_wait();
+#pragma unroll
+        for (int qq = 0; qq < 8; ++qq) {
+          const int ql = ch * 8 + qq;
+          long long Ta = 0, Ts = 0;
+#pragma unroll
+          for (int l = 0; l < LIMBS; ++l) {
+            if (a.g.kba > 0) Ta += (long long)(int)va[4 * qq + l] << (8 * l);
+            if (a.g.kbs > 0) Ts += (long long)(int)vs[4 * qq + l] << (8 * l);
+          }
+          const QConst c = qcs[ql];
+          const double av = (a.g.kba > 0) ? (double)Ta * c.sa + c.ca : 0.0;
+          const double sv = (a.g.kbs > 0) ? (double)Ts * c.ss + c.cs : 0.0;
+          const float est = (float)((double)nu * (av + (double)gm * sv));
+          if (row_ok && ql < a.nqp) {
+            if (MODE == 0) {
+              a.scores[(int64_t)ql * a.lds + row] = est;
+            } else if (est >= __ldg(a.tau + ql)) {
+              const int slot = atomicAdd(a.count + ql, 1);
+              if (slot < a.cap) {
+                a.cand_s[(int64_t)ql * a.cap + slot] = est;
+                a.cand_i[(int64_t)ql * a.cap + slot] = (int)row;
+              }
+            }
+          }
+        }
+      }
+      tc::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(dempty);
+    }
+  }
+
+  tc::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc::tc_fence_after();
+    tc::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+constexpr size_t kSmemBytes = A_RING_BYTES + B_STAGES * TILE_BYTES + 1024 + 256 + kQueriesPerPass * sizeof(QConst);
+
+template <int BM, int MODE>
+cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& ms, const ScanArgs& args, cudaStream_t st) {
+  auto kern = scan_tc_kernel<BM, MODE>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int grid = (int)std::min<int64_t>(args.npairs, tc::sm_count());
+  kern<<<grid, NTHREADS, kSmemBytes, st>>>(ma, ms, args);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+template <int MODE>
+cudaError_t launch_bm(int bm, const CUtensorMap& ma, const CUtensorMap& ms, const ScanArgs& args, cudaStream_t st) {
+  switch (bm) {
+    case 0: return launch_t<0, MODE>(ma, ms, args, st);
+    case 1: return launch_t<1, MODE>(ma, ms, args, st);
+    case 2: return launch_t<2, MODE>(ma, ms, args, st);
+    case 3: return launch_t<3, MODE>(ma, ms, args, st);
+    default: return launch_t<4, MODE>(ma, ms, args, st);
+  }
+}
+
+size_t b_bytes(const Geo& g, int part) {
+  return (size_t)kPassesPerGroup * NCOL * (part ? g.kbs : g.kba) * KB_BYTES;
+}
+
+}  // namespace
+
+bool available(const tq_plan* plan) { return plan->ms.ok != 0; }
+
+size_t workspace_bytes(const tq_plan* plan) {
+  if (!available(plan)) return 0;
+  const Geo g = make_geo(plan);
+  return kConstBytes + b_bytes(g, 0) + b_bytes(g, 1);
+}
+
+int prepare_group(const tq_plan* plan, const float* Qcat, int nqg, void* workspace, cudaStream_t st, const char* who) {
+  const Geo g = make_geo(plan);
+  const int ncols = plan->ncat * plan->dpad;
+  QConst* qc = static_cast<QConst*>(workspace);
+  uint8_t* Ba = static_cast<uint8_t*>(workspace) + kConstBytes;
+  uint8_t* Bs = Ba + b_bytes(g, 0);
+  StatArgs sa;
+  sa.Qcat = Qcat;
+  sa.ldq = ncols;
+  sa.d = plan->d;
+  sa.dpad = plan->dpad;
+  sa.prod = plan->mode == TQ_PROD ? 1 : 0;
+  sa.amax = plan->ms.amax;
+  sa.csum = plan->ms.csum;
+  sa.out = qc;
+  tstats_kernel<<<nqg, 256, 0, st>>>(sa);
+  count_launches(1);
+  TQ_CHECK_CUDA(cudaGetLastError(), who);
+  BPrepArgs ba;
+  ba.Qcat = Qcat;
+  ba.ldq = ncols;
+  ba.qc = qc;
+  ba.nqg = nqg;
+  ba.g = g;
+  for (int i = 0; i < 8; ++i) ba.alpha[i] = plan->ms.alpha[i];
+  ba.Ba = Ba;
+  ba.Bs = Bs;
+  const int passes = (nqg + kQueriesPerPass - 1) / kQueriesPerPass;
+  const int rows = passes * NCOL;
+  for (int part = 0; part < 2; ++part) {
+    const int nkb = part ? g.kbs : g.kba;
+    if (nkb == 0) continue;
+    const int64_t total = (int64_t)rows * nkb * 4;
+    tbprep_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(ba, part, rows);
+    count_launches(1);
+    TQ_CHECK_CUDA(cudaGetLastError(), who);
+  }
+  return TQ_OK;
+}
+
+int run_pass(const tq_plan* plan, int pass, int nqp, int64_t n, const uint8_t* idx, const uint8_t* qjl, const float* gamma,
+             const float* norms, float* scores, int64_t lds, const mscan::Filter* filter, const int* run_if,
+             const void* workspace, cudaStream_t st, const char* who) {
+  const Geo g = make_geo(plan);
+  const QConst* qc = static_cast<const QConst*>(workspace);
+  const uint8_t* Ba = static_cast<const uint8_t*>(workspace) + kConstBytes;
+  const uint8_t* Bs = Ba + b_bytes(g, 0);
+  CUtensorMap ma, ms;
+  const uint64_t rows = (uint64_t)kPassesPerGroup * NCOL;
+  if (g.kba > 0)
+    TQ_REQUIRE(tc::make_byte_map(&ma, Ba, rows, (uint64_t)g.kba * KB_BYTES, (uint64_t)g.kba * KB_BYTES, KB_BYTES, NCOL, true),
+               TQ_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (B, MSE part)", who);
+  if (g.kbs > 0)
+    TQ_REQUIRE(tc::make_byte_map(&ms, Bs, rows, (uint64_t)g.kbs * KB_BYTES, (uint64_t)g.kbs * KB_BYTES, KB_BYTES, NCOL, true),
+               TQ_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (B, QJL part)", who);
+  if (g.kba == 0) ma = ms;
+  if (g.kbs == 0) ms = ma;
+  ScanArgs a;
+  a.n = n;
+  a.npairs = (n + 2 * TILE - 1) / (2 * TILE);
+  a.g = g;
+  a.pass = pass;
+  a.nqp = nqp;
+  a.qc = qc + (size_t)pass * kQueriesPerPass;
+  a.idx = idx;
+  a.idx_rb = plan->idx_row_bytes;
+  a.qjl = qjl;
+  a.qjl_rb = plan->qjl_row_bytes;
+  a.gamma = gamma;
+  a.norms = norms;
+  a.coef = plan->coef;
+  a.scores = scores;
+  a.lds = lds;
+  a.tau = filter ? filter->tau : nullptr;
+  a.count = filter ? filter->count : nullptr;
+  a.cand_s = filter ? filter->cand_s : nullptr;
+  a.cand_i = filter ? filter->cand_i : nullptr;
+  a.cap = filter ? filter->cap : 0;
+  a.run_if = run_if;
+  a.status = plan->d_status;
+  TQ_CHECK_CUDA(filter ? launch_bm<1>(g.bm, ma, ms, a, st) : launch_bm<0>(g.bm, ma, ms, a, st), who);
+  return TQ_OK;
+}
+
+}  // namespace tscan
+}  // namespace tq

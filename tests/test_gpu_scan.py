@@ -49,6 +49,44 @@ def test_scores_every_pass_shape_and_determinism(nq):
     P.check_topk(ref, P.score_tolerance(su, Q, codes[3], n), ts, ti, 37)
 
 
+@pytest.mark.parametrize("d,bits,mode", [(128, 1, tq.TQ_MSE), (200, 2, tq.TQ_MSE), (520, 3, tq.TQ_MSE), (264, 4, tq.TQ_MSE),
+                                          (128, 1, tq.TQ_PROD), (200, 2, tq.TQ_PROD), (1536, 3, tq.TQ_PROD),
+                                          (520, 4, tq.TQ_PROD), (264, 5, tq.TQ_PROD)])
+def test_many_query_engine_every_bit_width(d, bits, mode):
+    """16 or more queries take the tcgen05 engine (32 queries per pass); its estimates equal the
+    few-query engine's bit for bit, and both match the oracle."""
+    su = P.Setup(d, bits, mode)
+    n, nq = 700, 37
+    X, Q = _data(d, n, nq, 31 * d + bits + mode)
+    codes = su.quantize(X)
+    sc = su.score(Q, n, *codes)
+    P.check_scores(su, sc, Q, *codes)
+    few = su.score(Q[:3].contiguous(), n, *codes)
+    assert torch.equal(few, sc[:3])
+    last = su.score(Q[nq - 2:].contiguous(), n, *codes)
+    assert torch.equal(last, sc[nq - 2:])
+    ts, ti = su.topk(Q, n, *codes, 25)
+    for q in (0, 17, nq - 1):
+        vals, order = torch.sort(sc[q], descending=True, stable=True)
+        assert torch.equal(ti[q].long(), order[:25]) and torch.equal(ts[q], vals[:25])
+
+
+def test_many_query_engine_groups_of_256_and_filter_flow():
+    cfg = wl.CONFIGS["c2"]
+    su = P.Setup(cfg.d, 3, tq.TQ_PROD, cfg.pi_seed, cfg.s_seed)
+    n, nq, k = 66000, 300, 10            # two groups of B operands (256 + 44 queries), thresholded top-k
+    X, Q = wl.database(cfg, n, device=DEV), wl.queries(cfg, nq, device=DEV)
+    codes = su.quantize(X)
+    sc = su.score(Q, n, *codes)
+    ts, ti = su.topk(Q, n, *codes, k)
+    for q in (0, 31, 32, 255, 256, 299):
+        one = su.score(Q[q:q + 1].contiguous(), n, *codes)
+        assert torch.equal(one[0], sc[q])
+        vals, order = torch.sort(sc[q], descending=True, stable=True)
+        assert torch.equal(ti[q].long(), order[:k]) and torch.equal(ts[q], vals[:k])
+    P.check_scores(su, sc[:4, :2000].contiguous(), Q[:4].contiguous(), *(None if t is None else t[:2000].contiguous() for t in codes))
+
+
 def test_zero_and_huge_queries_and_unit_norm_codes():
     d = 200
     su = P.Setup(d, 3, tq.TQ_PROD)
