@@ -272,6 +272,16 @@ def run_b200(args):
                              "score_codes_gbs": code_bytes / (ms_score * 1e-3) / 1e9,
                              "topk_codes_gbs": code_bytes / (ms_topk * 1e-3) / 1e9})
     del scores_buf
+    # many queries: 256 queries through the tcgen05 engine (32 per pass), top-k with the thresholded flow
+    mq = 256
+    Qm = wl.make_vectors(cfg, mq, cfg.query_seed + 7, dev)
+    ws_m = torch.empty(max(tq.tq_workspace_bytes(plan, tq.TQ_OP_TOPK, n, mq, k), 16), dtype=torch.uint8, device=dev)
+    tsm = torch.empty((mq, k), dtype=torch.float32, device=dev)
+    tim = torch.empty((mq, k), dtype=torch.int32, device=dev)
+    ms_many = time_call(lambda: tq.tq_topk(plan, Qm, n, idx, qjl, gamma, norms, k, tsm, tim, ws_m), reps=2)
+    many_queries = {"nq": mq, "passes": mq // 32, "topk_ms": ms_many, "queries_per_s": mq / (ms_many * 1e-3),
+                    "codes_gbs_times_passes": code_bytes * (mq // 32) / (ms_many * 1e-3) / 1e9}
+    del ws_m, Qm
 
     # ---- end to end: inputs start in pinned host memory, codes and top-k go back to the host ----
     e2e = None
@@ -383,7 +393,7 @@ def run_b200(args):
             "quantize_vectors_per_s": n / (q_ms * 1e-3), "quantize_ms": q_ms,
             "scan_ms": s_ms, "scan_codes_gbs": scan_gbs, "scan_frac_hbm": scan_gbs / peaks["hbm_gbs"],
             "scan_queries_per_s": nq / (s_ms * 1e-3),
-            "scan_regimes": scan_regimes, "roofline": roofline, "roofline_scan": roofline_scan, "clocks": clocks,
+            "scan_regimes": scan_regimes, "scan_many_queries": many_queries, "roofline": roofline, "roofline_scan": roofline_scan, "clocks": clocks,
             "e2e": e2e, "gpu_launches": int(launches)}
     if not args.no_cpu_baseline:
         sample = 32768
