@@ -369,19 +369,23 @@ bool make_map(CUtensorMap* map, const __nv_bfloat16* base, int64_t rows, int col
 
 }  // namespace
 
-// Byte matrix [rows, row_bytes] with row pitch `pitch` bytes; box = box_bytes x box_rows; no swizzle, or the
-// 128-byte swizzle (box_bytes must then be 128) that the UMMA shared-memory descriptors expect.
+// Byte matrix [rows, row_bytes] with row pitch `pitch` bytes; box = box_bytes x box_rows; `swizzle` = 0 (plain
+// rows in shared memory) or 32 / 64 / 128 (that swizzle span; box_bytes must not exceed it).
 bool make_byte_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes, uint64_t pitch,
-                   uint32_t box_bytes, uint32_t box_rows, bool swizzle128) {
+                   uint32_t box_bytes, uint32_t box_rows, int swizzle) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)pitch};
   const cuuint32_t box[2] = {(cuuint32_t)box_bytes, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
+  const CUtensorMapSwizzle sw = swizzle == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                : swizzle == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                : swizzle == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
+                                                : CU_TENSOR_MAP_SWIZZLE_NONE;
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 int sm_count() {

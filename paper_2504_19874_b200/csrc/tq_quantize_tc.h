@@ -18,10 +18,10 @@ size_t scratch_bytes_per_row(const tq_plan* plan);
 
 int sm_count();                // SMs of the current device
 // TMA descriptor of a byte matrix [rows, row_bytes] (row pitch `pitch` bytes), box = box_bytes x box_rows
-// bytes, zero fill outside the matrix; plain layout in shared memory, or the 128-byte swizzle (box_bytes = 128).
+// bytes, zero fill outside the matrix; swizzle = 0 (plain rows in shared memory) or 32 / 64 / 128.
 // False when the driver offers no tensor maps.
 bool make_byte_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes, uint64_t pitch,
-                   uint32_t box_bytes, uint32_t box_rows, bool swizzle128 = false);
+                   uint32_t box_bytes, uint32_t box_rows, int swizzle = 0);
 
 // Quant_mse / Quant_prod of n rows through the tcgen05 GEMMs (qjl, gamma unused for TQ_MSE).
 int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t ldx, uint8_t* idx, uint8_t* qjl,

@@ -140,12 +140,14 @@ __device__ void query_constants(const BPrepArgs& a, QConst* sc /* shared, [kMaxP
         mx1 = fmax(mx1, red[0][w]); sm1 += red[1][w];
         mx2 = fmax(mx2, red[2][w]); sm2 += red[3][w];
       }
-      // |W| < 2^e with W = 2 alpha q'  ->  |W| 2^(29-e) < 2^29 (operands are differences of two such values)
+      // |W| < 2^e with W = 2 alpha q'  ->  |W| 2^(22-e) < 2^22: the fixed-point integers (and their pairwise
+      // differences, < 2^23) fit three signed radix-256 digits, the format the tcgen05 engine uses, so that
+      // both engines form identical sums; the fourth digit column of this engine stays zero.
       auto expo = [](double wmax) {
         if (!(wmax > 0.0) || !isfinite(wmax)) return 0;
         int e;
         frexp(wmax, &e);
-        return 29 - e;
+        return 22 - e;
       };
       QConst c;
       c.fa = expo(2.0 * a.amax * mx1);
@@ -212,7 +214,7 @@ __global__ void __launch_bounds__(256) bprep_kernel(BPrepArgs a) {
         const double W7 = weight(8 * byte + 7, &f);
         double Jd = rint(ldexp(W7, f - 7));
         if (k < 7) Jd = rint(ldexp(weight(8 * byte + k, &f), f - k)) - Jd;
-        if (!(fabs(Jd) <= 1073741824.0)) Jd = 0.0;   // non-finite query entries contribute nothing
+        if (!(fabs(Jd) <= 8388608.0)) Jd = 0.0;   // non-finite query entries contribute nothing
         const int dg = digit_of((long long)Jd, limb);
         out[which] |= (uint32_t)(dg & 255) << (8 * byte);
       }

@@ -1,26 +1,32 @@
 // Many-query packed-code scan on tcgen05: the same bit-plane form of the estimator as in
 // tq_scan_mma.cu (codebook expanded over the index bits, raw bits and parity words as a 0/1 matrix,
-// query weights as fixed-point radix-256 digits), but with the multiply-accumulate on the 5th-generation
-// tensor cores:   D[128 vectors, 128 columns] += A[128, 32] * B[128, 32]^T,  kind::i8, s32 in TMEM.
-// 128 columns hold 32 queries x 4 digits, so one pass over the codes serves 32 queries and the decode
-// (one AND per four bits, done once per vector) is amortised over all of them.  A tcgen05 MMA of this
-// shape costs the same 64 cycles for any N <= 128, which is why this path is for many queries and the
-// register-fed mma.sync path for few.  The byte-expanded A tiles go through shared memory (TMEM is
-// full of accumulators), and that traffic -- per k-block 32 KB written + 32 KB read for A, 16 KB written
-// + 32 KB read for B = 896 cycles at 128 B/clk against 512 cycles of MMA -- is what bounds this kernel.
+// query weights as fixed-point radix-256 digits, identical integers), but with the multiply-accumulate
+// on the 5th-generation tensor cores:
+//     D[128 vectors, 96 columns] += A[128, 32] * B[96, 32]^T,   kind::i8, s32 accumulators in TMEM.
+// 96 columns hold 32 queries x 3 digits, so one pass over the codes serves 32 queries and the decode
+// (one AND per four bits, once per vector) is amortised over all of them.  A tcgen05 MMA of this shape
+// costs about the same 55-64 cycles for any N <= 128, which is why this path is for many queries and
+// the register-fed mma.sync path for few.
+//
+// The A operand never touches shared memory: byte-expanded bit planes are 8x the packed codes, and
+// writing + reading them there would cost more shared-memory cycles than the MMAs take.  Each
+// transform thread owns one vector row = one TMEM lane; it expands the row's four packed words of a
+// k-block into 32 registers and stores them with tcgen05.st into the 32 TMEM columns of that k-block,
+// from where the MMA takes A directly.
 //
 // CTA (one per SM, persistent over pairs of 128-vector tiles):
-//   warp 0      TMA producer of B: per k-block (128 K-bytes) one [128 rows x 128 B] box, 128-byte swizzle
+//   warp 0      TMA producer: per k-block (128 K-bytes) one [96 rows x 128 B] box of B (128-byte swizzle); per
+//               four k-blocks the packed rows of the pair ([256 rows x 32..64 B], swizzled for row-per-thread reads)
 //   warp 1      MMA issuer and TMEM owner: per k-block 4 MMAs (K = 32) for each of the two tiles
-//   warps 2..9  transform + epilogue: thread = one vector row.  Per k-block it loads the row's 4 packed
-//               words (3 index words + their parity word at b_m = 3), expands them into 32 registers
-//               (w & (0x01010101 << k)) and stores them as the row's 128 bytes of the A tile in the
-//               swizzled K-major layout the UMMA descriptor expects; after the last k-block it reads
-//               its row of the accumulators from TMEM, recombines the digits and emits the estimates.
-// Two tiles share every B box (halves the L2 traffic of B); their accumulators (MSE part and QJL part,
-// 128 columns each, per tile) fill the 512 TMEM columns.  Rings: 3 stages of (A0, A1) = 32 KB and 4 stages of
-// B = 16 KB, each with full / empty mbarriers (empty =
-// tcgen05.commit); accumulator full / empty.  All waits are bounded.
+//   warps 2..9  transform + epilogue (thread = vector row): the row's packed bytes from shared memory; per
+//               k-block 3 index words + their parity
+//               word (b_m = 3) -> 32 x (w & (0x01010101 << k)) -> tcgen05.st; after the last k-block the
+//               row's accumulators are read back (tcgen05.ld), the digits recombined, estimates emitted.
+// TMEM (512 columns): tile t: MSE-part accumulator at 192 t + [0, 96), QJL-part at 192 t + [96, 192);
+// A: two k-block slots of 32 columns per tile at 384 + 64 t.  The two tiles share every B box (halves
+// the L2 traffic of B).  Rings: 2 A slots (TMEM), 6 B stages and 4 packed-row stages (shared memory) with
+// full mbarriers; one tcgen05.commit per k-block releases both the A slot and the B stage; accumulator
+// full / empty.  All waits are bounded.
 #include <algorithm>
 #include <cmath>
 
@@ -34,14 +40,16 @@ namespace tscan {
 namespace {
 
 constexpr int TILE = 128;              // vectors per M tile = TMEM lanes
-constexpr int NCOL = 128;              // MMA N: 32 queries x 4 digits
-constexpr int LIMBS = 4;
+constexpr int LIMBS = 3;               // signed radix-256 digits per weight (|J| < 2^23)
+constexpr int NCOL = 96;               // MMA N: 3 digits x 32 queries, digit-major (column = 32 digit + query)
 constexpr int KB_BYTES = 128;          // K extent of one k-block (one swizzled row)
-constexpr int A_STAGES = 3;            // ring of A tile pairs (written by the transform warps: short latency)
-constexpr int B_STAGES = 4;            // ring of B tiles (TMA from L2)
-constexpr int TILE_BYTES = TILE * KB_BYTES;          // 16 KB
-constexpr int A_STAGE_BYTES = 2 * TILE_BYTES;        // A (tile 0), A (tile 1)
-constexpr int A_RING_BYTES = A_STAGES * A_STAGE_BYTES;
+constexpr int A_SLOTS = 2;             // k-blocks of A per tile resident in TMEM
+constexpr int B_STAGES = 6;            // ring of B tiles in shared memory (TMA from L2)
+constexpr int BTILE_BYTES = NCOL * KB_BYTES;         // 12 KB
+constexpr int P_STAGES = 4;            // ring of packed-row groups (4 k-blocks of the pair's 256 rows each)
+constexpr int PTILE_BYTES = 2 * TILE * 64;           // 16 KB: 256 rows x at most 64 bytes
+constexpr int D_COLS = 2 * NCOL;                     // accumulator columns per tile (MSE part, QJL part)
+constexpr int A_COL0 = 2 * D_COLS;                   // first TMEM column of the A slots
 constexpr int NTHREADS = 320;
 constexpr int TMEM_COLS = 512;
 constexpr size_t kConstBytes = 256 * 48;             // per-query constants of one group
@@ -60,6 +68,8 @@ struct Geo {
 };
 
 __host__ __device__ inline int div_up(int a, int b) { return (a + b - 1) / b; }
+// packed idx bytes of one row consumed by a group of four k-blocks
+__host__ __device__ constexpr int group_bytes(int bm) { return bm == 3 ? 48 : bm == 4 ? 32 : 64; }
 
 Geo make_geo(const tq_plan* plan) {
   Geo g;
@@ -140,13 +150,13 @@ __global__ void __launch_bounds__(256) tstats_kernel(StatArgs a) {
       mx1 = fmax(mx1, red[0][w]); sm1 += red[1][w];
       mx2 = fmax(mx2, red[2][w]); sm2 += red[3][w];
     }
-    // |W| < 2^e with W = 2 alpha q'  ->  |W| 2^(29-e) < 2^29: four signed radix-256 digits hold it.  The same
+    // |W| < 2^e with W = 2 alpha q'  ->  |W| 2^(22-e) < 2^22: three signed radix-256 digits hold it.  The same
     // exponent as in the register-fed scan, so that both engines form identical integers and estimates.
     auto expo = [](double wmax) {
       if (!(wmax > 0.0) || !isfinite(wmax)) return 0;
       int e;
       frexp(wmax, &e);
-      return 29 - e;
+      return 22 - e;
     };
     QConst c;
     c.fa = expo(2.0 * a.amax * mx1);
@@ -161,7 +171,7 @@ __global__ void __launch_bounds__(256) tstats_kernel(StatArgs a) {
 }
 
 // ------------------------------------------------------------------ B matrices
-// Ba[pass*128 + n][kba*128], Bs[pass*128 + n][kbs*128], n = 4 * (query in pass) + digit; K-major int8.
+// Ba[pass*96 + n][kba*128], Bs[pass*96 + n][kbs*128], n = 32 * digit + (query in pass); K-major int8.
 // Byte kappa of a k-block = (2 wl + k / 4) * 16 + (k % 4) * 4 + i  <->  bit 8 i + k of word wl: the order in
 // which the transform threads lay out their registers.
 struct BPrepArgs {
@@ -191,8 +201,8 @@ __global__ void __launch_bounds__(256) tbprep_kernel(BPrepArgs a, int part, int 
   if (tid >= total) return;
   const int wl = (int)(tid & 3);
   const int kb = (int)((tid >> 2) % nkb);
-  const int row = (int)((tid >> 2) / nkb);      // pass * 128 + n
-  const int ql = (row / NCOL) * kQueriesPerPass + (row % NCOL) / LIMBS, limb = row % LIMBS;
+  const int row = (int)((tid >> 2) / nkb);      // pass * 96 + n
+  const int ql = (row / NCOL) * kQueriesPerPass + (row % NCOL) % kQueriesPerPass, limb = (row % NCOL) / kQueriesPerPass;
   uint32_t out[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
   if (ql < a.nqg) {
     const float* q = a.Qcat + (int64_t)ql * a.ldq;
@@ -212,7 +222,7 @@ __global__ void __launch_bounds__(256) tbprep_kernel(BPrepArgs a, int part, int 
           f = c.fs;
         }
         double Jd = rint(ldexp(W, f - k));
-        if (!(fabs(Jd) <= 1073741824.0)) Jd = 0.0;   // non-finite query entries contribute nothing
+        if (!(fabs(Jd) <= 8388608.0)) Jd = 0.0;   // non-finite query entries contribute nothing
         out[k] |= (uint32_t)(digit_of((long long)Jd, limb) & 255) << (8 * i);
       }
     }
@@ -246,34 +256,39 @@ struct ScanArgs {
   int* status;
 };
 
-__device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+// D[tmem] (+)= A[tmem] * B[smem]^T: A is taken from TMEM (row = lane, 4 K-bytes per 32-bit column).
+__device__ __forceinline__ void umma_i8_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // kind::i8: D = s32, A = unsigned 8-bit, B = signed 8-bit, both K-major.
 __host__ __device__ constexpr uint32_t idesc_i8(int M, int N) {
   return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 template <int BM, int MODE>
 __global__ void __launch_bounds__(NTHREADS, 1)
-scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__ CUtensorMap tmBs, ScanArgs a) {
+scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__ CUtensorMap tmBs,
+               const __grid_constant__ CUtensorMap tmPa, const __grid_constant__ CUtensorMap tmPs, ScanArgs a) {
   if (a.run_if != nullptr && *a.run_if == 0) return;
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  unsigned char* bring = smem + A_RING_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(bring + B_STAGES * TILE_BYTES);
-  uint64_t* afull = bars;                           // [A_STAGES]  transform warps -> MMA
-  uint64_t* aempty = afull + A_STAGES;              // [A_STAGES]  MMA -> transform warps
-  uint64_t* bfull = aempty + A_STAGES;              // [B_STAGES]  TMA -> MMA
-  uint64_t* bempty = bfull + B_STAGES;              // [B_STAGES]  MMA -> TMA producer
-  uint64_t* dfull = bempty + B_STAGES;              // accumulators complete -> epilogue
+  unsigned char* bring = smem;
+  unsigned char* pring = smem + B_STAGES * BTILE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(pring + P_STAGES * PTILE_BYTES);
+  uint64_t* afull = bars;                           // [A_SLOTS]   transform warps -> MMA
+  uint64_t* bfull = afull + A_SLOTS;                // [B_STAGES]  TMA -> MMA
+  // One tcgen05.commit per k-block: the issuing thread pays ~350 cycles per commit (measured), so the release
+  // of the A slot (2 k-blocks later) and of the B stage (6 k-blocks later) share one ring of barriers.
+  uint64_t* kdone = bfull + B_STAGES;               // [B_STAGES]  MMAs of k-block f complete
+  uint64_t* pfull = kdone + B_STAGES;               // [P_STAGES]  TMA (packed rows) -> transform warps
+  uint64_t* pempty = pfull + P_STAGES;              // [P_STAGES]  transform warps -> TMA producer
+  uint64_t* dfull = pempty + P_STAGES;              // accumulators complete -> epilogue
   uint64_t* dempty = dfull + 1;                     // accumulators read -> MMA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(dempty + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -283,13 +298,14 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
   const int nkb_total = a.g.kba + a.g.kbs;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < A_STAGES; ++s) {
-      tc::mbar_init(&afull[s], 8);
-      tc::mbar_init(&aempty[s], 1);
-    }
+    for (int s = 0; s < A_SLOTS; ++s) tc::mbar_init(&afull[s], 8);
     for (int s = 0; s < B_STAGES; ++s) {
       tc::mbar_init(&bfull[s], 1);
-      tc::mbar_init(&bempty[s], 1);
+      tc::mbar_init(&kdone[s], 1);
+    }
+    for (int s = 0; s < P_STAGES; ++s) {
+      tc::mbar_init(&pfull[s], 1);
+      tc::mbar_init(&pempty[s], 8);
     }
     tc::mbar_init(dfull, 1);
     tc::mbar_init(dempty, 8);
@@ -297,6 +313,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
     tc::fence_barrier_init();
     if (a.g.kba > 0) tc::tma_prefetch_desc(&tmBa);
     if (a.g.kbs > 0) tc::tma_prefetch_desc(&tmBs);
+    if (a.g.kba > 0) tc::tma_prefetch_desc(&tmPa);
+    if (a.g.kbs > 0) tc::tma_prefetch_desc(&tmPs);
   }
   if (threadIdx.x < kQueriesPerPass) {
     QConst c = {1.0, 0.0, 1.0, 0.0, 0, 0, {0, 0}};
@@ -312,16 +330,29 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of B
     if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
+      int stage = 0, pstage = 0;
+      uint32_t phase = 0, pphase = 0;
       bool ok = true;
+      long long kc = 0;   // k-blocks issued so far by this CTA
       for (int64_t pair = blockIdx.x; pair < a.npairs && ok; pair += gridDim.x) {
-        for (int f = 0; f < nkb_total; ++f) {
-          if (!(ok = tc::mbar_wait(&bempty[stage], phase ^ 1u, abort_flag, a.status))) break;
+        for (int f = 0; f < nkb_total; ++f, ++kc) {
           const bool part_s = f >= a.g.kba;
           const int kb = part_s ? f - a.g.kba : f;
-          tc::mbar_arrive_expect_tx(&bfull[stage], TILE_BYTES);
-          tc::tma_load_2d(bring + stage * TILE_BYTES, part_s ? &tmBs : &tmBa, &bfull[stage], kb * KB_BYTES, a.pass * NCOL);
+          if ((kb & 3) == 0) {   // the packed rows of the pair for the next four k-blocks
+            if (!(ok = tc::mbar_wait(&pempty[pstage], pphase ^ 1u, abort_flag, a.status))) break;
+            const int gb = part_s ? 64 : group_bytes(BM);
+            tc::mbar_arrive_expect_tx(&pfull[pstage], (uint32_t)(2 * TILE * gb));
+            tc::tma_load_2d(pring + pstage * PTILE_BYTES, part_s ? &tmPs : &tmPa, &pfull[pstage], (kb >> 2) * gb,
+                            (int)(pair * (2 * TILE)));
+            if (++pstage == P_STAGES) {
+              pstage = 0;
+              pphase ^= 1u;
+            }
+          }
+          // B stage kc % B_STAGES was last read by the MMAs of k-block kc - B_STAGES
+          if (kc >= B_STAGES && !(ok = tc::mbar_wait(&kdone[stage], phase ^ 1u, abort_flag, a.status))) break;
+          tc::mbar_arrive_expect_tx(&bfull[stage], BTILE_BYTES);
+          tc::tma_load_2d(bring + stage * BTILE_BYTES, part_s ? &tmBs : &tmBa, &bfull[stage], kb * KB_BYTES, a.pass * NCOL);
           if (++stage == B_STAGES) {
             stage = 0;
             phase ^= 1u;
@@ -350,19 +381,17 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
           tc::tc_fence_after();
           const bool part_s = f >= a.g.kba;
           const int kb = part_s ? f - a.g.kba : f;
-          const uint32_t sb = tc::smem_u32(smem + stage * A_STAGE_BYTES);
-          const uint64_t bdesc = tc::smem_desc_sw128(tc::smem_u32(bring + bstage * TILE_BYTES));
+          const uint64_t bdesc = tc::smem_desc_sw128(tc::smem_u32(bring + bstage * BTILE_BYTES));
 #pragma unroll
           for (int t = 0; t < 2; ++t) {
-            const uint64_t adesc = tc::smem_desc_sw128(sb + t * TILE_BYTES);
-            const uint32_t d_tmem = tmem_base + (uint32_t)(t * 256 + (part_s ? NCOL : 0));
+            const uint32_t a_tmem = tmem_base + (uint32_t)(A_COL0 + t * (A_SLOTS * 32) + stage * 32);
+            const uint32_t d_tmem = tmem_base + (uint32_t)(t * D_COLS + (part_s ? NCOL : 0));
 #pragma unroll
-            for (int step = 0; step < 4; ++step)   // 32 K-bytes per MMA: +32 bytes inside the swizzled row
-              umma_i8(d_tmem, adesc + 2 * step, bdesc + 2 * step, idesc, (kb | step) != 0 ? 1u : 0u);
+            for (int step = 0; step < 4; ++step)   // 32 K-bytes per MMA: 8 TMEM columns of A, +32 bytes inside B's swizzled row
+              umma_i8_ts(d_tmem, a_tmem + 8 * step, bdesc + 2 * step, idesc, (kb | step) != 0 ? 1u : 0u);
           }
-          tc::umma_commit(&aempty[stage]);   // both stages reusable once these MMAs have read them
-          tc::umma_commit(&bempty[bstage]);
-          if (++stage == A_STAGES) {
+          tc::umma_commit(&kdone[bstage]);   // A slot and B stage reusable once these MMAs have read them
+          if (++stage == A_SLOTS) {
             stage = 0;
             phase ^= 1u;
           }
@@ -381,37 +410,17 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
     const int t = e >> 2;                   // which tile of the pair
     const int quad = warp & 3;              // TMEM lane group this warp may access
     const int r = quad * 32 + lane;         // row inside the tile
-    int stage = 0;
-    uint32_t phase = 0;
+    int stage = 0, pstage_keep = 0;
+    uint32_t pphase_keep = 0;
+    long long kt = 0;   // k-blocks expanded so far by this warp
     bool ok = true;
     int64_t it = 0;
     for (int64_t pair = blockIdx.x; pair < a.npairs && ok; pair += gridDim.x, ++it) {
       const int64_t row = pair * (2 * TILE) + t * TILE + r;
       const bool row_ok = row < a.n;
-      const uint32_t* irow = reinterpret_cast<const uint32_t*>(a.idx + (size_t)(row_ok ? row : 0) * a.idx_rb);
-      const uint32_t* qrow = reinterpret_cast<const uint32_t*>(a.qjl + (size_t)(row_ok ? row : 0) * a.qjl_rb);
       const float nu = (row_ok && a.norms != nullptr) ? __ldg(a.norms + row) : 1.f;
       const float gm = (row_ok && a.g.kbs > 0) ? a.coef * __ldg(a.gamma + row) : 0.f;
 
-      // the row's packed words of k-block f (index words first, parity words derived later)
-      auto load_words = [&](int f, uint32_t (&w)[4]) {
-        w[0] = w[1] = w[2] = w[3] = 0u;
-        if (!row_ok || f >= nkb_total) return;
-        if (f >= a.g.kba) {
-          const uint4 v = __ldg(reinterpret_cast<const uint4*>(qrow) + (f - a.g.kba));
-          w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-        } else if (BM <= 2) {
-          const uint4 v = __ldg(reinterpret_cast<const uint4*>(irow) + f);
-          w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-        } else if (BM == 3) {
-#pragma unroll
-          for (int i = 0; i < 3; ++i)
-            if (3 * f + i < a.g.widx) w[i] = __ldg(irow + 3 * f + i);
-        } else {
-          const uint2 v = __ldg(reinterpret_cast<const uint2*>(irow) + f);
-          w[0] = v.x; w[1] = v.y;
-        }
-      };
       // expands one k-block's words into the row's 128 bytes of the A tile of the current stage
       auto emit = [&](uint32_t (&w)[4], int f) -> bool {
         if (f >= nkb_total) return true;
@@ -430,62 +439,105 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
             }
           }
         }
-        if (!tc::mbar_wait(&aempty[stage], phase ^ 1u, abort_flag, a.status)) return false;
-        // 16-byte chunk c goes to position c ^ (r & 7) (128-byte swizzle)
-        unsigned char* arow = smem + stage * A_STAGE_BYTES + t * TILE_BYTES + r * KB_BYTES;
+        // the row's 128 A bytes of this k-block: register 4 c + e = (word c / 2, bit 4 (c % 2) + e of every byte)
+        uint32_t v[32];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
           const uint32_t x = w[c >> 1];
           const int k0 = (c & 1) * 4;
-          const uint4 v = make_uint4(x & (0x01010101u << k0), x & (0x01010101u << (k0 + 1)), x & (0x01010101u << (k0 + 2)),
-                                     x & (0x01010101u << (k0 + 3)));
-          *reinterpret_cast<uint4*>(arow + ((c ^ (r & 7)) << 4)) = v;
+#pragma unroll
+          for (int e2 = 0; e2 < 4; ++e2) v[4 * c + e2] = x & (0x01010101u << (k0 + e2));
         }
-        fence_async_smem();   // make the generic-proxy stores visible to the tensor core's reads
+        // A slot kt % 2 was last read by the MMAs of k-block kt - 2: completion number (kt - 2) / B_STAGES of its barrier
+        if (kt >= A_SLOTS) {
+          const long long kp = kt - A_SLOTS;
+          if (!tc::mbar_wait(&kdone[(int)(kp % B_STAGES)], (uint32_t)((kp / B_STAGES) & 1), abort_flag, a.status)) return false;
+        }
+        tc::tc_fence_after();
+        tc::tmem_st32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(A_COL0 + t * (A_SLOTS * 32) + stage * 32), v);
+        tc::tmem_st_wait();
+        tc::tc_fence_before();
         __syncwarp();
         if (lane == 0) tc::mbar_arrive(&afull[stage]);
-        if (++stage == A_STAGES) {
-          stage = 0;
-          phase ^= 1u;
-        }
+        if (++stage == A_SLOTS) stage = 0;
+        ++kt;
         return true;
       };
-      // two register sets of four k-blocks each: the loads of one set (the codes stream from HBM) are in flight
-      // while the other set is expanded
-      constexpr int PF = 4;
-      uint32_t wa[PF][4], wb[PF][4];
+      // groups of four k-blocks: the pair's packed rows arrive by TMA ([256 rows x group bytes], swizzled so that
+      // row-per-thread 16-byte reads are conflict-free); the thread copies its row's bytes to registers, frees the
+      // stage and expands the four k-blocks
+      const int prow = t * TILE + r;   // row inside the pair
+      int pstage = pstage_keep;
+      uint32_t pphase = pphase_keep;
+      for (int f0 = 0; f0 < nkb_total && ok; f0 += 4) {
+        // a part boundary inside a group cannot happen: each part starts a new group
+        const bool part_s = f0 >= a.g.kba;
+        if (!(ok = tc::mbar_wait(&pfull[pstage], pphase, abort_flag, a.status))) break;
+        const unsigned char* ps = pring + pstage * PTILE_BYTES;
+        uint32_t w[4][4];
 #pragma unroll
-      for (int j = 0; j < PF; ++j) load_words(j, wa[j]);
-      for (int f0 = 0; f0 < nkb_total && ok; f0 += 2 * PF) {
+        for (int j = 0; j < 4; ++j) w[j][0] = w[j][1] = w[j][2] = w[j][3] = 0u;
+        if (part_s || BM <= 2) {           // 64 bytes per row, 64-byte swizzle: chunk c at c ^ ((row >> 1) & 3)
 #pragma unroll
-        for (int j = 0; j < PF; ++j) load_words(f0 + PF + j, wb[j]);
+          for (int j = 0; j < 4; ++j) {
+            const uint4 v = *reinterpret_cast<const uint4*>(ps + prow * 64 + ((j ^ ((prow >> 1) & 3)) << 4));
+            w[j][0] = v.x; w[j][1] = v.y; w[j][2] = v.z; w[j][3] = v.w;
+          }
+        } else if (BM == 3) {              // 48 bytes per row, plain: three words per k-block
+          uint32_t x[12];
 #pragma unroll
-        for (int j = 0; j < PF; ++j) ok = ok && emit(wa[j], f0 + j);
+          for (int j = 0; j < 3; ++j) {
+            const uint4 v = *reinterpret_cast<const uint4*>(ps + prow * 48 + j * 16);
+            x[4 * j] = v.x; x[4 * j + 1] = v.y; x[4 * j + 2] = v.z; x[4 * j + 3] = v.w;
+          }
 #pragma unroll
-        for (int j = 0; j < PF; ++j) load_words(f0 + 2 * PF + j, wa[j]);
+          for (int j = 0; j < 4; ++j) {
+            w[j][0] = x[3 * j]; w[j][1] = x[3 * j + 1]; w[j][2] = x[3 * j + 2];
+          }
+        } else {                           // b_m = 4: 32 bytes per row, 32-byte swizzle: chunk c at c ^ ((row >> 2) & 1)
 #pragma unroll
-        for (int j = 0; j < PF; ++j) ok = ok && emit(wb[j], f0 + PF + j);
+          for (int j = 0; j < 2; ++j) {
+            const uint4 v = *reinterpret_cast<const uint4*>(ps + prow * 32 + ((j ^ ((prow >> 2) & 1)) << 4));
+            w[2 * j][0] = v.x; w[2 * j][1] = v.y; w[2 * j + 1][0] = v.z; w[2 * j + 1][1] = v.w;
+          }
+        }
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&pempty[pstage]);
+        if (++pstage == P_STAGES) {
+          pstage = 0;
+          pphase ^= 1u;
+        }
+        const int fend = part_s ? nkb_total : a.g.kba;   // k-blocks of this part end here
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (f0 + j < fend) ok = ok && emit(w[j], f0 + j);
+        if (!part_s && f0 + 4 >= a.g.kba) f0 = a.g.kba - 4;   // the next group starts the QJL part
       }
+      pstage_keep = pstage;
+      pphase_keep = pphase;
       if (!ok) break;
 
       // ---- epilogue: this thread's row of the four accumulators
       if (!(ok = tc::mbar_wait(dfull, (uint32_t)(it & 1), abort_flag, a.status))) break;
       tc::tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(t * 256);
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(t * D_COLS);
 #pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {   // 32 columns = 8 queries per chunk
-        uint32_t va[32], vs[32];
-        if (a.g.kba > 0) tc::tmem_ld32(taddr + ch * 32, va);
-        if (a.g.kbs > 0) tc::tmem_ld32(taddr + NCOL + ch * 32, vs);
+      for (int h = 0; h < 2; ++h) {   // 16 queries per half: digit l of query 16 h + qq sits in column 32 l + 16 h + qq
+        uint32_t va[LIMBS][16], vs[LIMBS][16];
+#pragma unroll
+        for (int l = 0; l < LIMBS; ++l) {
+          if (a.g.kba > 0) tc::tmem_ld16(taddr + l * 32 + h * 16, va[l]);
+          if (a.g.kbs > 0) tc::tmem_ld16(taddr + NCOL + l * 32 + h * 16, vs[l]);
+        }
         tc::tmem_ld_wait();
 #pragma unroll
-        for (int qq = 0; qq < 8; ++qq) {
-          const int ql = ch * 8 + qq;
+        for (int qq = 0; qq < 16; ++qq) {
+          const int ql = h * 16 + qq;
           long long Ta = 0, Ts = 0;
 #pragma unroll
           for (int l = 0; l < LIMBS; ++l) {
-            if (a.g.kba > 0) Ta += (long long)(int)va[4 * qq + l] << (8 * l);
-            if (a.g.kbs > 0) Ts += (long long)(int)vs[4 * qq + l] << (8 * l);
+            if (a.g.kba > 0) Ta += (long long)(int)va[l][qq] << (8 * l);
+            if (a.g.kbs > 0) Ts += (long long)(int)vs[l][qq] << (8 * l);
           }
           const QConst c = qcs[ql];
           const double av = (a.g.kba > 0) ? (double)Ta * c.sa + c.ca : 0.0;
@@ -518,10 +570,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
   }
 }
 
-constexpr size_t kSmemBytes = A_RING_BYTES + B_STAGES * TILE_BYTES + 1024 + 256 + kQueriesPerPass * sizeof(QConst);
+// at least 120 KB so that a second CTA can never share the SM (the kernel allocates all of TMEM)
+constexpr size_t kSmemUsed = B_STAGES * BTILE_BYTES + P_STAGES * PTILE_BYTES + 1024 + 512 + kQueriesPerPass * sizeof(QConst);
+constexpr size_t kSmemBytes = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;
 
 template <int BM, int MODE>
-cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& ms, const ScanArgs& args, cudaStream_t st) {
+cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
+                     const ScanArgs& args, cudaStream_t st) {
   auto kern = scan_tc_kernel<BM, MODE>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -530,19 +585,20 @@ cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& ms, const ScanArg
     attr_set = true;
   }
   const int grid = (int)std::min<int64_t>(args.npairs, tc::sm_count());
-  kern<<<grid, NTHREADS, kSmemBytes, st>>>(ma, ms, args);
+  kern<<<grid, NTHREADS, kSmemBytes, st>>>(ma, ms, pa, ps, args);
   count_launches(1);
   return cudaGetLastError();
 }
 
 template <int MODE>
-cudaError_t launch_bm(int bm, const CUtensorMap& ma, const CUtensorMap& ms, const ScanArgs& args, cudaStream_t st) {
+cudaError_t launch_bm(int bm, const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
+                      const ScanArgs& args, cudaStream_t st) {
   switch (bm) {
-    case 0: return launch_t<0, MODE>(ma, ms, args, st);
-    case 1: return launch_t<1, MODE>(ma, ms, args, st);
-    case 2: return launch_t<2, MODE>(ma, ms, args, st);
-    case 3: return launch_t<3, MODE>(ma, ms, args, st);
-    default: return launch_t<4, MODE>(ma, ms, args, st);
+    case 0: return launch_t<0, MODE>(ma, ms, pa, ps, args, st);
+    case 1: return launch_t<1, MODE>(ma, ms, pa, ps, args, st);
+    case 2: return launch_t<2, MODE>(ma, ms, pa, ps, args, st);
+    case 3: return launch_t<3, MODE>(ma, ms, pa, ps, args, st);
+    default: return launch_t<4, MODE>(ma, ms, pa, ps, args, st);
   }
 }
 
@@ -610,13 +666,25 @@ int run_pass(const tq_plan* plan, int pass, int nqp, int64_t n, const uint8_t* i
   CUtensorMap ma, ms;
   const uint64_t rows = (uint64_t)kPassesPerGroup * NCOL;
   if (g.kba > 0)
-    TQ_REQUIRE(tc::make_byte_map(&ma, Ba, rows, (uint64_t)g.kba * KB_BYTES, (uint64_t)g.kba * KB_BYTES, KB_BYTES, NCOL, true),
+    TQ_REQUIRE(tc::make_byte_map(&ma, Ba, rows, (uint64_t)g.kba * KB_BYTES, (uint64_t)g.kba * KB_BYTES, KB_BYTES, NCOL, 128),
                TQ_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (B, MSE part)", who);
   if (g.kbs > 0)
-    TQ_REQUIRE(tc::make_byte_map(&ms, Bs, rows, (uint64_t)g.kbs * KB_BYTES, (uint64_t)g.kbs * KB_BYTES, KB_BYTES, NCOL, true),
+    TQ_REQUIRE(tc::make_byte_map(&ms, Bs, rows, (uint64_t)g.kbs * KB_BYTES, (uint64_t)g.kbs * KB_BYTES, KB_BYTES, NCOL, 128),
                TQ_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (B, QJL part)", who);
   if (g.kba == 0) ma = ms;
   if (g.kbs == 0) ms = ma;
+  // packed rows: boxes of [256 rows x group bytes]; 64- and 32-byte boxes are swizzled (row-per-thread reads)
+  CUtensorMap pa, ps;
+  const int gb = group_bytes(g.bm);
+  if (g.kba > 0)
+    TQ_REQUIRE(tc::make_byte_map(&pa, idx, (uint64_t)n, plan->idx_row_bytes, plan->idx_row_bytes, gb, 2 * TILE,
+                                 gb == 64 ? 64 : gb == 32 ? 32 : 0),
+               TQ_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (idx rows)", who);
+  if (g.kbs > 0)
+    TQ_REQUIRE(tc::make_byte_map(&ps, qjl, (uint64_t)n, plan->qjl_row_bytes, plan->qjl_row_bytes, 64, 2 * TILE, 64), TQ_ERR_CUDA,
+               "%s: cuTensorMapEncodeTiled failed (qjl rows)", who);
+  if (g.kba == 0) pa = ps;
+  if (g.kbs == 0) ps = pa;
   ScanArgs a;
   a.n = n;
   a.npairs = (n + 2 * TILE - 1) / (2 * TILE);
@@ -640,7 +708,7 @@ int run_pass(const tq_plan* plan, int pass, int nqp, int64_t n, const uint8_t* i
   a.cap = filter ? filter->cap : 0;
   a.run_if = run_if;
   a.status = plan->d_status;
-  TQ_CHECK_CUDA(filter ? launch_bm<1>(g.bm, ma, ms, a, st) : launch_bm<0>(g.bm, ma, ms, a, st), who);
+  TQ_CHECK_CUDA(filter ? launch_bm<1>(g.bm, ma, ms, pa, ps, a, st) : launch_bm<0>(g.bm, ma, ms, pa, ps, a, st), who);
   return TQ_OK;
 }
 
