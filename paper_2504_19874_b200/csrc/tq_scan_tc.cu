@@ -44,13 +44,15 @@ constexpr int LIMBS = 3;               // signed radix-256 digits per weight (|J
 constexpr int NCOL = 96;               // MMA N: 3 digits x 32 queries, digit-major (column = 32 digit + query)
 constexpr int KB_BYTES = 128;          // K extent of one k-block (one swizzled row)
 constexpr int A_SLOTS = 2;             // k-blocks of A per tile resident in TMEM
-constexpr int B_STAGES = 6;            // ring of B tiles in shared memory (TMA from L2)
+constexpr int B_STAGES = 8;            // ring of B tiles in shared memory (TMA from L2); a power of two, so that ring
+                                       // positions and phases of 32-bit counters are masks and shifts
 constexpr int BTILE_BYTES = NCOL * KB_BYTES;         // 12 KB
 constexpr int P_STAGES = 4;            // ring of packed-row groups (4 k-blocks of the pair's 256 rows each)
 constexpr int PTILE_BYTES = 2 * TILE * 64;           // 16 KB: 256 rows x at most 64 bytes
 constexpr int D_COLS = 2 * NCOL;                     // accumulator columns per tile (MSE part, QJL part)
 constexpr int A_COL0 = 2 * D_COLS;                   // first TMEM column of the A slots
-constexpr int NTHREADS = 320;
+constexpr int N_ISSUERS = 2;             // MMA-issuing warps (a tcgen05.commit stalls its thread; a second issuer hides it)
+constexpr int NTHREADS = 32 * (1 + N_ISSUERS + 8);
 constexpr int TMEM_COLS = 512;
 constexpr size_t kConstBytes = 256 * 48;             // per-query constants of one group
 
@@ -289,10 +291,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
   uint64_t* pfull = kdone + B_STAGES;               // [P_STAGES]  TMA (packed rows) -> transform warps
   uint64_t* pempty = pfull + P_STAGES;              // [P_STAGES]  transform warps -> TMA producer
   uint64_t* dfull = pempty + P_STAGES;              // accumulators complete -> epilogue
-  uint64_t* dempty = dfull + 1;                     // accumulators read -> MMA
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(dempty + 1);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(dfull + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  QConst* qcs = reinterpret_cast<QConst*>(dempty + 3);
+  QConst* qcs = reinterpret_cast<QConst*>(dfull + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nkb_total = a.g.kba + a.g.kbs;
@@ -307,8 +308,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
       tc::mbar_init(&pfull[s], 1);
       tc::mbar_init(&pempty[s], 8);
     }
-    tc::mbar_init(dfull, 1);
-    tc::mbar_init(dempty, 8);
+    tc::mbar_init(dfull, N_ISSUERS);
     *abort_flag = 0;
     tc::fence_barrier_init();
     if (a.g.kba > 0) tc::tma_prefetch_desc(&tmBa);
@@ -364,55 +364,52 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
-    // ---------------------------------------------------------------- MMA issuer
+  } else if (warp <= N_ISSUERS) {
+    // ---------------------------------------------------------------- MMA issuers
+    // The k-blocks are dealt in turn to the issuing warps: 8 MMAs (4 per tile) + one commit each.  The
+    // accumulators are zeroed by the transform warps, every MMA accumulates, and integer sums do not depend
+    // on the order in which the k-blocks of different threads reach the tensor pipe.
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_i8(TILE, NCOL);
-      int stage = 0, bstage = 0;
-      uint32_t phase = 0, bphase = 0;
+      const int me = warp - 1;
       bool ok = true;
-      int64_t it = 0;
-      for (int64_t pair = blockIdx.x; pair < a.npairs && ok; pair += gridDim.x, ++it) {
-        if (!(ok = tc::mbar_wait(dempty, (uint32_t)(it & 1) ^ 1u, abort_flag, a.status))) break;
-        tc::tc_fence_after();
-        for (int f = 0; f < nkb_total; ++f) {
-          if (!(ok = tc::mbar_wait(&bfull[bstage], bphase, abort_flag, a.status))) break;
-          if (!(ok = tc::mbar_wait(&afull[stage], phase, abort_flag, a.status))) break;
+      uint32_t kc = 0;    // k-blocks of this CTA so far
+      int turn = 0;       // whose k-block comes next
+      const uint64_t bdesc0 = tc::smem_desc_sw128(tc::smem_u32(bring));
+      for (int64_t pair = blockIdx.x; pair < a.npairs && ok; pair += gridDim.x) {
+        for (int f = 0; f < nkb_total; ++f, ++kc) {
+          const bool mine = turn == me;
+          if (++turn == N_ISSUERS) turn = 0;
+          if (!mine) continue;
+          const uint32_t bstage = kc & (B_STAGES - 1), stage = kc & (A_SLOTS - 1);
+          if (!(ok = tc::mbar_wait(&bfull[bstage], (kc / B_STAGES) & 1u, abort_flag, a.status))) break;
+          if (!(ok = tc::mbar_wait(&afull[stage], (kc / A_SLOTS) & 1u, abort_flag, a.status))) break;
           tc::tc_fence_after();
           const bool part_s = f >= a.g.kba;
-          const int kb = part_s ? f - a.g.kba : f;
-          const uint64_t bdesc = tc::smem_desc_sw128(tc::smem_u32(bring + bstage * BTILE_BYTES));
+          const uint64_t bdesc = bdesc0 + (uint64_t)(bstage * (BTILE_BYTES >> 4));
 #pragma unroll
           for (int t = 0; t < 2; ++t) {
             const uint32_t a_tmem = tmem_base + (uint32_t)(A_COL0 + t * (A_SLOTS * 32) + stage * 32);
             const uint32_t d_tmem = tmem_base + (uint32_t)(t * D_COLS + (part_s ? NCOL : 0));
 #pragma unroll
             for (int step = 0; step < 4; ++step)   // 32 K-bytes per MMA: 8 TMEM columns of A, +32 bytes inside B's swizzled row
-              umma_i8_ts(d_tmem, a_tmem + 8 * step, bdesc + 2 * step, idesc, (kb | step) != 0 ? 1u : 0u);
+              umma_i8_ts(d_tmem, a_tmem + 8 * step, bdesc + 2 * step, idesc, 1u);
           }
           tc::umma_commit(&kdone[bstage]);   // A slot and B stage reusable once these MMAs have read them
-          if (++stage == A_SLOTS) {
-            stage = 0;
-            phase ^= 1u;
-          }
-          if (++bstage == B_STAGES) {
-            bstage = 0;
-            bphase ^= 1u;
-          }
         }
-        if (ok) tc::umma_commit(dfull);
+        if (ok) tc::umma_commit(dfull);   // all MMAs this thread issued for the pair
       }
     }
     __syncwarp();
   } else {
     // ---------------------------------------------------------------- transform + epilogue (thread = vector row)
-    const int e = warp - 2;
+    const int e = warp - 1 - N_ISSUERS;
     const int t = e >> 2;                   // which tile of the pair
     const int quad = warp & 3;              // TMEM lane group this warp may access
     const int r = quad * 32 + lane;         // row inside the tile
     int stage = 0, pstage_keep = 0;
     uint32_t pphase_keep = 0;
-    long long kt = 0;   // k-blocks expanded so far by this warp
+    uint32_t kt = 0;    // k-blocks expanded so far by this warp
     bool ok = true;
     int64_t it = 0;
     for (int64_t pair = blockIdx.x; pair < a.npairs && ok; pair += gridDim.x, ++it) {
@@ -420,6 +417,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
       const bool row_ok = row < a.n;
       const float nu = (row_ok && a.norms != nullptr) ? __ldg(a.norms + row) : 1.f;
       const float gm = (row_ok && a.g.kbs > 0) ? a.coef * __ldg(a.gamma + row) : 0.f;
+
+      // this row's accumulators start from zero (the previous pair's epilogue, by this same thread, has read
+      // them; the stores complete before the row's first A tile is announced)
+#pragma unroll
+      for (int c = 0; c < D_COLS; c += 16) tc::tmem_fill16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(t * D_COLS + c), 0u);
 
       // expands one k-block's words into the row's 128 bytes of the A tile of the current stage
       auto emit = [&](uint32_t (&w)[4], int f) -> bool {
@@ -450,8 +452,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
         }
         // A slot kt % 2 was last read by the MMAs of k-block kt - 2: completion number (kt - 2) / B_STAGES of its barrier
         if (kt >= A_SLOTS) {
-          const long long kp = kt - A_SLOTS;
-          if (!tc::mbar_wait(&kdone[(int)(kp % B_STAGES)], (uint32_t)((kp / B_STAGES) & 1), abort_flag, a.status)) return false;
+          const uint32_t kp = kt - A_SLOTS;
+          if (!tc::mbar_wait(&kdone[kp & (B_STAGES - 1)], (kp / B_STAGES) & 1u, abort_flag, a.status)) return false;
         }
         tc::tc_fence_after();
         tc::tmem_st32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(A_COL0 + t * (A_SLOTS * 32) + stage * 32), v);
@@ -557,8 +559,6 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
         }
       }
       tc::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) tc::mbar_arrive(dempty);
     }
   }
 

@@ -43,8 +43,7 @@ constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2-3 s of SM clock
 
 // Bounded wait.  `abort_flag` lives in shared memory; once any thread of the CTA gives up,
 // every other wait of that CTA returns false at its next check.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  if (mbar_try_wait(bar, parity)) return true;
+static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
   const long long t0 = clock64();
   uint32_t polls = 0;
   while (true) {
@@ -58,6 +57,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       }
     }
   }
+}
+// The polling loop is kept out of line: the waits sit in hot loops whose code should stay small.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status);
 }
 
 // ---------------------------------------------------------------- TMA
@@ -118,6 +122,13 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
         "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(taddr)
+      : "memory");
+}
+// Stores one value into 16 consecutive columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_fill16(uint32_t taddr, uint32_t x) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};" ::"r"(taddr), "r"(x)
       : "memory");
 }
 // Stores 32 registers into 32 consecutive columns of this thread's TMEM lane.
