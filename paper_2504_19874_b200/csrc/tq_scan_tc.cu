@@ -15,18 +15,25 @@
 // from where the MMA takes A directly.
 //
 // CTA (one per SM, persistent over pairs of 128-vector tiles):
-//   warp 0      TMA producer: per k-block (128 K-bytes) one [96 rows x 128 B] box of B (128-byte swizzle); per
-//               four k-blocks the packed rows of the pair ([256 rows x 32..64 B], swizzled for row-per-thread reads)
-//   warp 1      MMA issuer and TMEM owner: per k-block 4 MMAs (K = 32) for each of the two tiles
-//   warps 2..9  transform + epilogue (thread = vector row): the row's packed bytes from shared memory; per
-//               k-block 3 index words + their parity
-//               word (b_m = 3) -> 32 x (w & (0x01010101 << k)) -> tcgen05.st; after the last k-block the
-//               row's accumulators are read back (tcgen05.ld), the digits recombined, estimates emitted.
+//   warp 0       TMA producer: per k-block (128 K-bytes) one [96 rows x 128 B] box of B (128-byte swizzle); per
+//                four k-blocks the packed rows of the pair ([256 rows x 32..64 B], swizzled for row-per-thread reads)
+//   warps 1..2   MMA issuers (warp 1 owns TMEM): k-blocks alternate between them, 8 MMAs (K = 32, 4 per tile)
+//                + one commit each.  A tcgen05.commit keeps its thread for ~350 cycles while the 8 MMAs take
+//                ~420, so a single issuer leaves the tensor pipe idle half of the time (measured: 95 cycles
+//                per MMA with one issuing thread, 70 with two).
+//   warps 3..10  transform + epilogue (thread = vector row): zero the row's accumulators (tcgen05.st), then per
+//                k-block the row's packed bytes from shared memory, 3 index words + their parity word (b_m = 3)
+//                -> 32 x (w & (0x01010101 << k)) -> tcgen05.st; after the last k-block the row's accumulators
+//                are read back (tcgen05.ld), the digits recombined, estimates emitted.
+// Every MMA accumulates onto the zeroed accumulators; the sums are integers, so the order in which the
+// k-blocks of the two issuers reach the pipe does not matter.
 // TMEM (512 columns): tile t: MSE-part accumulator at 192 t + [0, 96), QJL-part at 192 t + [96, 192);
 // A: two k-block slots of 32 columns per tile at 384 + 64 t.  The two tiles share every B box (halves
-// the L2 traffic of B).  Rings: 2 A slots (TMEM), 6 B stages and 4 packed-row stages (shared memory) with
-// full mbarriers; one tcgen05.commit per k-block releases both the A slot and the B stage; accumulator
-// full / empty.  All waits are bounded.
+// the L2 traffic of B).  Rings: 2 A slots (TMEM), 8 B stages and 4 packed-row stages (shared memory) with
+// full mbarriers; one tcgen05.commit per k-block releases both the A slot and the B stage; accumulator-full
+// barrier (one commit per issuer).  Ring positions and phases are masks and shifts of 32-bit counters: the
+// single-lane roles run dependent instruction chains, where 64-bit division costs real time.  All waits
+// are bounded.
 #include <algorithm>
 #include <cmath>
 
@@ -286,7 +293,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
   uint64_t* afull = bars;                           // [A_SLOTS]   transform warps -> MMA
   uint64_t* bfull = afull + A_SLOTS;                // [B_STAGES]  TMA -> MMA
   // One tcgen05.commit per k-block: the issuing thread pays ~350 cycles per commit (measured), so the release
-  // of the A slot (2 k-blocks later) and of the B stage (6 k-blocks later) share one ring of barriers.
+  // of the A slot (2 k-blocks later) and of the B stage (8 k-blocks later) share one ring of barriers.
   uint64_t* kdone = bfull + B_STAGES;               // [B_STAGES]  MMAs of k-block f complete
   uint64_t* pfull = kdone + B_STAGES;               // [P_STAGES]  TMA (packed rows) -> transform warps
   uint64_t* pempty = pfull + P_STAGES;              // [P_STAGES]  transform warps -> TMA producer

@@ -7,7 +7,7 @@
 namespace tq {
 namespace tscan {
 
-constexpr int kQueriesPerPass = 32;    // 128 MMA columns = 32 queries x 4 radix-256 digits
+constexpr int kQueriesPerPass = 32;    // 96 MMA columns = 32 queries x 3 radix-256 digits
 constexpr int kPassesPerGroup = 8;     // B operands are built for up to 8 passes (256 queries) at a time
 
 // Whether the plan can use this path (same conditions as the bit-plane scan, plus shared-memory room).
