@@ -216,6 +216,7 @@ __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __rest
     float acc[kRotQ];
 #pragma unroll
     for (int qq = 0; qq < kRotQ; ++qq) acc[qq] = 0.f;
+    const int nact = min(kRotQ, q_end - q0);   // queries of this round: the others are neither staged nor summed
     for (int c0 = 0; c0 < d; c0 += kRotChunk) {
       const int len = min(kRotChunk, d - c0);
       float4 r[kRotChunk / 128];
@@ -228,7 +229,7 @@ __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __rest
         }
       }
       __syncthreads();
-      for (int e = threadIdx.x; e < kRotQ * (kRotChunk / 4); e += blockDim.x) {
+      for (int e = threadIdx.x; e < nact * (kRotChunk / 4); e += blockDim.x) {
         const int qq = e / (kRotChunk / 4), c = 4 * (e % (kRotChunk / 4));
         float v[4] = {0.f, 0.f, 0.f, 0.f};
         if (q0 + qq < q_end && c < len) {
@@ -247,8 +248,10 @@ __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __rest
           if (4 * c4 < len) {
 #pragma unroll
             for (int qq = 0; qq < kRotQ; ++qq) {
-              const float4 v = *reinterpret_cast<const float4*>(&qs[qq][4 * c4]);
-              acc[qq] = fmaf(r[i].x, v.x, fmaf(r[i].y, v.y, fmaf(r[i].z, v.z, fmaf(r[i].w, v.w, acc[qq]))));
+              if (qq < nact) {
+                const float4 v = *reinterpret_cast<const float4*>(&qs[qq][4 * c4]);
+                acc[qq] = fmaf(r[i].x, v.x, fmaf(r[i].y, v.y, fmaf(r[i].z, v.z, fmaf(r[i].w, v.w, acc[qq]))));
+              }
             }
           }
         }
@@ -256,12 +259,14 @@ __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __rest
         for (int c = lane; c < len; c += 32) {
           const float rv = __ldg(row + c0 + c);
 #pragma unroll
-          for (int qq = 0; qq < kRotQ; ++qq) acc[qq] = fmaf(rv, qs[qq][c], acc[qq]);
+          for (int qq = 0; qq < kRotQ; ++qq)
+            if (qq < nact) acc[qq] = fmaf(rv, qs[qq][c], acc[qq]);
         }
       }
     }
 #pragma unroll
     for (int qq = 0; qq < kRotQ; ++qq) {
+      if (qq >= nact) break;
       double v = (double)acc[qq];
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

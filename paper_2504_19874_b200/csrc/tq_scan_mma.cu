@@ -164,6 +164,12 @@ __device__ void query_constants(const BPrepArgs& a, QConst* sc /* shared, [kMaxP
   }
 }
 
+// 2^e as a double; multiplying by it is the exact scaling ldexp performs, at the cost of one multiply.
+__device__ __forceinline__ double pow2_of(int e) {
+  if (e < -1000 || e > 1000) return ldexp(1.0, e);
+  return __hiloint2double((e + 1023) << 20, 0);
+}
+
 __device__ __forceinline__ int digit_of(long long J, int limb) {
   int dg = 0;
   for (int l = 0; l <= limb; ++l) {
@@ -173,13 +179,17 @@ __device__ __forceinline__ int digit_of(long long J, int limb) {
   return dg;
 }
 
+// One thread per output byte (8 per uint2 element): the chain of fp64 and index arithmetic behind a digit is
+// long, and this kernel sits in front of every scan call; the 8 bytes meet by a shuffle-OR.
 __global__ void __launch_bounds__(256) bprep_kernel(BPrepArgs a) {
   __shared__ QConst sc[kMaxPassQueries];
   query_constants(a, sc);
   const int ksa = ks_a(a.bm), kss = ks_s(a.prod != 0), KS = ksa + kss;
   const int64_t total = (int64_t)a.NT * a.R * KS * 32;
-  const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (tid >= total) return;
+  const int64_t tid8 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t tid = tid8 >> 3;
+  if (tid >= total) return;   // total * 8 is a multiple of 256: whole warps leave together
+  const int which = (int)(tid8 >> 2) & 1, byte = (int)tid8 & 3;
   const int lane = (int)(tid & 31);
   const int ks = (int)((tid >> 5) % KS);
   const int r = (int)((tid >> 5) / KS % a.R);
@@ -193,34 +203,33 @@ __global__ void __launch_bounds__(256) bprep_kernel(BPrepArgs a) {
     const bool is_s = ks >= ksa;
     const int kk = is_s ? ks - ksa : ks;
     const int p = kk >> 3, k = kk & 7;
-    for (int which = 0; which < 2; ++which) {
-      for (int byte = 0; byte < 4; ++byte) {
-        // Slot (byte, k) and the slot of bit 7 of the same byte: the k = 7 operand is the raw byte
-        // (sum_j 2^j bit_j), so the operand of k < 7 carries J_k - J_7.
-        auto weight = [&](int bp, int* f_out) -> double {
-          double W = 0.0;
-          if (!is_s) {
-            const Slot s = a_slot(a.bm, r, t4, 2 * p + which, bp);
-            if (s.coord < a.d) W = 2.0 * a.alpha[s.term] * (double)q[s.coord];
-            *f_out = c.fa;
-          } else {
-            const int j = s_slot(r, t4, 2 * p + which, bp);
-            if (j < a.d) W = 2.0 * (double)q[a.dpad + j];
-            *f_out = c.fs;
-          }
-          return W;
-        };
-        int f = 0;
-        const double W7 = weight(8 * byte + 7, &f);
-        double Jd = rint(ldexp(W7, f - 7));
-        if (k < 7) Jd = rint(ldexp(weight(8 * byte + k, &f), f - k)) - Jd;
-        if (!(fabs(Jd) <= 8388608.0)) Jd = 0.0;   // non-finite query entries contribute nothing
-        const int dg = digit_of((long long)Jd, limb);
-        out[which] |= (uint32_t)(dg & 255) << (8 * byte);
+    const int fexp = is_s ? c.fs : c.fa;
+    const double scale7 = pow2_of(fexp - 7), scalek = pow2_of(fexp - k);
+    // Slot (byte, k) and the slot of bit 7 of the same byte: the k = 7 operand is the raw byte
+    // (sum_j 2^j bit_j), so the operand of k < 7 carries J_k - J_7.
+    auto weight = [&](int bp) -> double {
+      double W = 0.0;
+      if (!is_s) {
+        const Slot s = a_slot(a.bm, r, t4, 2 * p + which, bp);
+        if (s.coord < a.d) W = 2.0 * a.alpha[s.term] * (double)q[s.coord];
+      } else {
+        const int j = s_slot(r, t4, 2 * p + which, bp);
+        if (j < a.d) W = 2.0 * (double)q[a.dpad + j];
       }
-    }
+      return W;
+    };
+    double Jd = rint(weight(8 * byte + 7) * scale7);
+    if (k < 7) Jd = rint(weight(8 * byte + k) * scalek) - Jd;
+    if (!(fabs(Jd) <= 8388608.0)) Jd = 0.0;   // non-finite query entries contribute nothing
+    const int dg = digit_of((long long)Jd, limb);
+    out[which] = (uint32_t)(dg & 255) << (8 * byte);
   }
-  a.out[tid] = make_uint2(out[0], out[1]);
+#pragma unroll
+  for (int o = 1; o < 8; o <<= 1) {
+    out[0] |= __shfl_xor_sync(0xffffffffu, out[0], o);
+    out[1] |= __shfl_xor_sync(0xffffffffu, out[1], o);
+  }
+  if ((tid8 & 7) == 0) a.out[tid] = make_uint2(out[0], out[1]);
 }
 
 // ------------------------------------------------------------------ scan kernel
@@ -855,7 +864,7 @@ int prepare(const tq_plan* plan, const float* Qcat, int nqp, void* workspace, cu
   for (int i = 0; i < 8; ++i) ba.alpha[i] = plan->ms.alpha[i];
   ba.out = bfrag;
   const int64_t total = (int64_t)c.NT * plan->ms.R * (ks_a(bm) + ks_s(prod)) * 32;
-  bprep_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(ba);
+  bprep_kernel<<<(unsigned)((total * 8 + 255) / 256), 256, 0, st>>>(ba);
   count_launches(1);
   TQ_CHECK_CUDA(cudaGetLastError(), who);
   return TQ_OK;
