@@ -61,6 +61,7 @@ constexpr int A_COL0 = 2 * D_COLS;                   // first TMEM column of the
 constexpr int N_ISSUERS = 2;             // MMA-issuing warps (a tcgen05.commit stalls its thread; a second issuer hides it)
 constexpr int NTHREADS = 32 * (1 + N_ISSUERS + 8);
 constexpr int TMEM_COLS = 512;
+constexpr int LBUF = 128;              // candidates per query a CTA collects in shared memory before it appends them
 constexpr size_t kConstBytes = 256 * 48;             // per-query constants of one group
 
 struct QConst {
@@ -301,6 +302,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(dfull + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   QConst* qcs = reinterpret_cast<QConst*>(dfull + 4);
+  float* taus = reinterpret_cast<float*>(qcs + kQueriesPerPass);   // [32] admission thresholds (filter mode)
+  // Filter mode: admitted pairs are collected per CTA and appended to the global lists in one piece per query at
+  // the end: one atomic per (CTA, query) instead of one per pair on 32 contended counters.
+  int* lcnt = reinterpret_cast<int*>(taus + kQueriesPerPass);       // [32]
+  uint2* lbuf = reinterpret_cast<uint2*>(lcnt + kQueriesPerPass);   // [32][LBUF] (score bits, row)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nkb_total = a.g.kba + a.g.kbs;
@@ -327,6 +333,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
     QConst c = {1.0, 0.0, 1.0, 0.0, 0, 0, {0, 0}};
     if ((int)threadIdx.x < a.nqp) c = a.qc[threadIdx.x];
     qcs[threadIdx.x] = c;
+    taus[threadIdx.x] = (MODE == 1 && (int)threadIdx.x < a.nqp) ? a.tau[threadIdx.x] : 0.f;
+    lcnt[threadIdx.x] = 0;
   }
   if (warp == 1) tc::tmem_alloc(tmem_slot, TMEM_COLS);
   tc::tc_fence_before();
@@ -419,11 +427,22 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
     uint32_t kt = 0;    // k-blocks expanded so far by this warp
     bool ok = true;
     int64_t it = 0;
+    // the row's scalars are requested one pair ahead, so that their latency hides behind a pair's k-blocks
+    auto load_nu = [&](int64_t pr) -> float {
+      const int64_t rw = pr * (2 * TILE) + t * TILE + r;
+      return (pr < a.npairs && rw < a.n && a.norms != nullptr) ? __ldg(a.norms + rw) : 1.f;
+    };
+    auto load_gm = [&](int64_t pr) -> float {
+      const int64_t rw = pr * (2 * TILE) + t * TILE + r;
+      return (pr < a.npairs && rw < a.n && a.g.kbs > 0) ? a.coef * __ldg(a.gamma + rw) : 0.f;
+    };
+    float nu_next = load_nu(blockIdx.x), gm_next = load_gm(blockIdx.x);
     for (int64_t pair = blockIdx.x; pair < a.npairs && ok; pair += gridDim.x, ++it) {
       const int64_t row = pair * (2 * TILE) + t * TILE + r;
       const bool row_ok = row < a.n;
-      const float nu = (row_ok && a.norms != nullptr) ? __ldg(a.norms + row) : 1.f;
-      const float gm = (row_ok && a.g.kbs > 0) ? a.coef * __ldg(a.gamma + row) : 0.f;
+      const float nu = nu_next, gm = gm_next;
+      nu_next = load_nu(pair + gridDim.x);
+      gm_next = load_gm(pair + gridDim.x);
 
       // this row's accumulators start from zero (the previous pair's epilogue, by this same thread, has read
       // them; the stores complete before the row's first A tile is announced)
@@ -555,11 +574,16 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
           if (row_ok && ql < a.nqp) {
             if (MODE == 0) {
               a.scores[(int64_t)ql * a.lds + row] = est;
-            } else if (est >= __ldg(a.tau + ql)) {
-              const int slot = atomicAdd(a.count + ql, 1);
-              if (slot < a.cap) {
-                a.cand_s[(int64_t)ql * a.cap + slot] = est;
-                a.cand_i[(int64_t)ql * a.cap + slot] = (int)row;
+            } else if (est >= taus[ql]) {
+              const int ls = atomicAdd(&lcnt[ql], 1);
+              if (ls < LBUF) {
+                lbuf[ql * LBUF + ls] = make_uint2(__float_as_uint(est), (uint32_t)row);
+              } else {   // the CTA's buffer is full: straight to the global list
+                const int slot = atomicAdd(a.count + ql, 1);
+                if (slot < a.cap) {
+                  a.cand_s[(int64_t)ql * a.cap + slot] = est;
+                  a.cand_i[(int64_t)ql * a.cap + slot] = (int)row;
+                }
               }
             }
           }
@@ -575,10 +599,27 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
     tc::tc_fence_after();
     tc::tmem_dealloc(tmem_base, TMEM_COLS);
   }
+  if (MODE == 1 && warp > N_ISSUERS) {   // the eight transform warps append four queries' collected pairs each
+    for (int ql = (warp - 1 - N_ISSUERS) * 4; ql < (warp - N_ISSUERS) * 4; ++ql) {
+      const int m = min(lcnt[ql], LBUF);
+      if (m == 0 || ql >= a.nqp) continue;
+      int base = 0;
+      if (lane == 0) base = atomicAdd(a.count + ql, m);
+      base = __shfl_sync(0xffffffffu, base, 0);
+      for (int i = lane; i < m; i += 32) {
+        const int slot = base + i;
+        if (slot < a.cap) {
+          const uint2 e = lbuf[ql * LBUF + i];
+          a.cand_s[(int64_t)ql * a.cap + slot] = __uint_as_float(e.x);
+          a.cand_i[(int64_t)ql * a.cap + slot] = (int)e.y;
+        }
+      }
+    }
+  }
 }
 
 // at least 120 KB so that a second CTA can never share the SM (the kernel allocates all of TMEM)
-constexpr size_t kSmemUsed = B_STAGES * BTILE_BYTES + P_STAGES * PTILE_BYTES + 1024 + 512 + kQueriesPerPass * sizeof(QConst);
+constexpr size_t kSmemUsed = B_STAGES * BTILE_BYTES + P_STAGES * PTILE_BYTES + 1024 + 512 + kQueriesPerPass * (sizeof(QConst) + sizeof(float) + sizeof(int) + LBUF * sizeof(uint2));
 constexpr size_t kSmemBytes = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;
 
 template <int BM, int MODE>
