@@ -249,6 +249,50 @@ int tq_wsum(const tq_plan* plan, const float* W, int nw, int64_t ldw, int64_t n,
 int tq_softmax(const float* s1, const float* s2, int nw, int64_t n, int64_t lds, float scale,
                float* W, int64_t ldw, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Decode attention over a compressed KV cache, all KV heads of a layer in one call (the use of the
+ * two quantisers in Section 4.3: keys with TurboQuant_prod so that q.k is estimated without bias,
+ * values with TurboQuant_mse; channels of a head may be split into groups of different bit widths,
+ * the outlier treatment of that section).  For query head r = h * q_per_kv + j of KV head h:
+ *     logit_t = scale * sum_groups  estimate of < q_r[channels of the group], k_t[those channels] >
+ *               (estimator of Section 3.2 on the group's codes; Algorithm 1 when the key plan is _mse),
+ *     out_r   = sum_t softmax(logit)_t * v~_t,   v~_t = DeQuant_mse of the value codes (Algorithm 1),
+ * evaluated on the packed codes: nothing is dequantised per token, Pi_V^T is applied once per output
+ * row.  Equal to tq_score per (head, group) + tq_softmax + tq_wsum within fp32 rounding.
+ *
+ * One tq_kv_group per channel group.  All plans share one dimension d (a multiple of 8, <= 128) and
+ * one device; the key plan may be TQ_PROD or TQ_MSE, the value plan is TQ_MSE.  Code arrays hold the
+ * rows of all heads, head-major: row h * tokens + t.  All pointers are device pointers owned by the
+ * caller; nothing is retained after the call.
+ */
+#define TQ_MAX_KV_GROUPS 4
+typedef struct tq_kv_group {
+  const tq_plan* plan_k;
+  const tq_plan* plan_v;
+  const uint8_t* k_idx;       /* [heads*tokens, tq_idx_row_bytes(d, b_m of plan_k)], 4-byte aligned; NULL if b_m = 0 */
+  const uint8_t* k_qjl;       /* [heads*tokens, tq_qjl_row_bytes(d)] (TQ_PROD), 4-byte aligned, else NULL */
+  const float* k_gamma;       /* [heads*tokens] residual norms (TQ_PROD), else NULL */
+  const float* k_norms;       /* [heads*tokens] key norms, or NULL for unit norms */
+  const uint8_t* v_idx;       /* [heads*tokens, tq_idx_row_bytes(d, b of plan_v)] */
+  const float* v_norms;       /* [heads*tokens] value norms, or NULL */
+  const int32_t* k_channels;  /* [heads, d] column of Q that is coordinate c of this group for KV head h */
+  const int32_t* v_channels;  /* [heads, d] column of out that receives coordinate c of this group */
+} tq_kv_group;
+
+/* Bytes of workspace tq_attend_decode needs (rotated queries + per-slice partial results). */
+size_t tq_attend_decode_workspace_bytes(int ngroups, int heads, int64_t tokens, int d);
+
+/*   groups     host array of ngroups (1..TQ_MAX_KV_GROUPS) descriptors
+ *   Q          device, [heads*q_per_kv rows, row stride ldq elements] of q_dtype (TQ_F32 / TQ_BF16); 1 <= q_per_kv <= 4
+ *   out        device fp32, [heads*q_per_kv rows, row stride ldo]; only the columns named by v_channels are written
+ *   workspace  device, 256-byte aligned, >= tq_attend_decode_workspace_bytes(...)
+ * tokens == 0 writes zeros to those columns.  Results do not depend on timing (fixed reduction orders).
+ * Errors: TQ_ERR_INVALID_ARG / _UNSUPPORTED / _ALIGNMENT / _WORKSPACE / _CUDA as for the other calls.
+ */
+int tq_attend_decode(const tq_kv_group* groups, int ngroups, int heads, int64_t tokens, int q_per_kv,
+                     const void* Q, int q_dtype, int64_t ldq, float scale, float* out, int64_t ldo,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -44,7 +44,16 @@ _SIGNATURES = {
     "tq_softmax": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, ctypes.c_float, c_void_p, c_int64, c_void_p]),
     "tq_wsum": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                         c_void_p, c_int64, c_void_p, c_size_t, c_void_p]),
+    "tq_attend_decode_workspace_bytes": (c_size_t, [c_int, c_int, c_int64, c_int]),
+    "tq_attend_decode": (c_int, [c_void_p, c_int, c_int, c_int64, c_int, c_void_p, c_int, c_int64, ctypes.c_float,
+                                 c_void_p, c_int64, c_void_p, c_size_t, c_void_p]),
 }
+
+
+class KvGroup(ctypes.Structure):
+    """struct tq_kv_group of include/tq.h (one channel group of a compressed KV layer)."""
+    _fields_ = [(name, c_void_p) for name in ("plan_k", "plan_v", "k_idx", "k_qjl", "k_gamma", "k_norms", "v_idx", "v_norms",
+                                              "k_channels", "v_channels")]
 
 
 class TqError(RuntimeError):
@@ -229,6 +238,27 @@ def tq_softmax(s1, s2, scale: float, W):
     if s2 is not None and (_rows(s2)[1] != lds or s2.shape != s1.shape):
         raise ValueError("s2 must have the shape and row stride of s1")
     _check(lib().tq_softmax(_dev(s1), _dev(s2), nw, n, lds, scale, _dev(W), ldw, _stream()))
+
+
+def tq_attend_decode_workspace_bytes(ngroups: int, heads: int, tokens: int, d: int) -> int:
+    return lib().tq_attend_decode_workspace_bytes(ngroups, heads, tokens, d)
+
+
+def tq_attend_decode(groups, heads: int, tokens: int, q_per_kv: int, Q, scale: float, out, workspace):
+    """groups: sequence of dicts with keys plan_k, plan_v (Plan) and k_idx, k_qjl, k_gamma, k_norms, v_idx,
+    v_norms, k_channels, v_channels (CUDA tensors or None); rows of all heads head-major."""
+    arr = (KvGroup * len(groups))()
+    for dst, g in zip(arr, groups):
+        dst.plan_k, dst.plan_v = g["plan_k"].handle, g["plan_v"].handle
+        for name in ("k_idx", "k_qjl", "k_gamma", "k_norms", "v_idx", "v_norms", "k_channels", "v_channels"):
+            setattr(dst, name, _dev(g.get(name)))
+        for name in ("k_channels", "v_channels"):
+            if g[name].dtype != torch.int32 or not g[name].is_contiguous():
+                raise ValueError(f"{name} must be a contiguous int32 tensor")
+    _, ldq = _rows(Q)
+    _, ldo = _rows(out)
+    _check(lib().tq_attend_decode(ctypes.cast(arr, c_void_p), len(groups), heads, tokens, q_per_kv, _dev(Q), _dtype_code(Q),
+                                  ldq, scale, _dev(out), ldo, *_scratch_args(workspace), _stream()))
 
 
 def tq_select_topk(cand_scores, cand_ids, k: int, top_scores, top_ids):

@@ -1,0 +1,490 @@
+// Decode attention over a compressed KV cache in two launches (plus a small query-preparation
+// launch): scores of the Section 3.2 estimator on the packed K codes, softmax over the tokens, and
+// the weighted sum of the dequantised V vectors taken in the code domain (Section 4.3 use of the
+// quantisers), for all KV heads and channel groups of a layer at once.
+//
+//   prepare_kernel   per (head, group): gathers the group's channels of the head's queries and forms
+//                    q' = Pi q, q'' = S q.
+//   partial_kernel   per (head, slice of <= 1024 tokens), flash-decode style:
+//                    A) thread = token.  The MSE term sum_c q'_c c[idx_c] and the QJL term
+//                       sum_i q''_i z_i are sums of table entries: four index bits (4, 2 or 1
+//                       coordinates; one coordinate for 3-bit indices) select one float4 holding the
+//                       partial sums of up to four queries, built per CTA from q', q'' and the codebook.
+//                       logit = scale * sum_groups nu (mse + coef gamma qjl).
+//                    B) slice maximum, p = exp(logit - max), sum of p.
+//                    C) thread = output coordinate: acc[c] = sum_t p_t nu^V_t c_V[idx^V_{t,c}], walked
+//                       in a fixed order, so results do not depend on timing.
+//   merge_kernel     per (head, query): combines the slices (max / sum rescaling), divides by the sum and
+//                    applies x~ = Pi_V^T y' per group, scattering to the group's channels.
+//
+// Work per token is ~50 warp instructions, i.e. CUDA-core bound at roughly 10x the time the code
+// bytes take from HBM; the unfused path (tq_score, tq_softmax, tq_wsum per head and group) is two
+// orders of magnitude slower at 32k tokens because each of its 88 launches serves one head.
+#include <algorithm>
+#include <cfloat>
+#include <cstring>
+
+#include "tq_internal.h"
+
+namespace tq {
+namespace kvdec {
+
+constexpr int MAXG = TQ_MAX_KV_GROUPS;
+constexpr int MAXQ = 4;          // queries per KV head (one float4 of partial sums)
+constexpr int MAXD = 128;        // channels per group
+constexpr int SLICE = 512;       // tokens per CTA
+constexpr int NT = 256;          // threads per CTA
+
+struct GroupDev {
+  const uint8_t* k_idx;
+  const uint8_t* k_qjl;
+  const float* k_gamma;
+  const float* k_norms;
+  const uint8_t* v_idx;
+  const float* v_norms;
+  const int32_t* k_channels;
+  const int32_t* v_channels;
+  const float* k_rotcat;   // [ncat*dpad, d]
+  const float* v_pi;       // [d, d]
+  float k_cent[16], v_cent[16];
+  int k_bits, v_bits, k_prod;
+  int k_idx_rb, k_qjl_rb, v_idx_rb;
+  int k_dpad;
+  float coef;
+  int lut_mse_off, lut_qjl_off;   // float4 offsets of this group's tables in shared memory
+  int k_idx_soff, k_qjl_soff, v_idx_soff;   // byte offsets of the staged code rows inside their shared-memory buffers
+};
+
+struct Args {
+  GroupDev g[MAXG];
+  int ngroups, heads, qpk, d, nslices;
+  int64_t tokens;
+  float scale;
+  float* qrot;      // [heads, ngroups, MAXQ, 2*MAXD]
+  float* part_ml;   // [heads, nslices, 2, MAXQ]      slice maximum, slice sum of exponentials
+  float* part_acc;  // [heads, nslices, ngroups*d, MAXQ]
+  int lut_float4;   // float4 entries of all tables
+  int kbuf_bytes, vbuf_bytes;   // shared-memory room for the slice's K and V code rows
+};
+
+__host__ __device__ inline int mse_lookups(int d, int bits) {   // table rows of the MSE term
+  return bits == 0 ? 0 : bits == 1 ? d / 4 : bits == 2 ? d / 2 : d;
+}
+__host__ __device__ inline int mse_entries(int bits) { return bits == 3 ? 8 : 16; }
+
+// ------------------------------------------------------------------ query preparation
+template <typename T>
+__global__ void __launch_bounds__(128) prepare_kernel(Args a, const T* __restrict__ Q, int64_t ldq) {
+  __shared__ float qs[MAXQ][MAXD];
+  const int h = blockIdx.x / a.ngroups, gi = blockIdx.x % a.ngroups;
+  const GroupDev& g = a.g[gi];
+  const int d = a.d;
+  for (int e = threadIdx.x; e < MAXQ * d; e += blockDim.x) {
+    const int j = e / d, c = e % d;
+    float v = 0.f;
+    if (j < a.qpk) {
+      const int ch = g.k_channels[h * d + c];
+      v = (float)Q[(int64_t)(h * a.qpk + j) * ldq + ch];
+    }
+    qs[j][c] = v;
+  }
+  __syncthreads();
+  float* out = a.qrot + (size_t)(h * a.ngroups + gi) * MAXQ * 2 * MAXD;
+  const int nrows = (g.k_prod ? 2 : 1) * g.k_dpad;
+  for (int o = threadIdx.x; o < nrows; o += blockDim.x) {
+    const int half = o / g.k_dpad, r = o % g.k_dpad;
+    float acc[MAXQ] = {0.f, 0.f, 0.f, 0.f};
+    if (r < d) {
+      const float* row = g.k_rotcat + (size_t)o * d;
+#pragma unroll 8
+      for (int c = 0; c < d; ++c) {
+        const float m = row[c];
+#pragma unroll
+        for (int j = 0; j < MAXQ; ++j) acc[j] = fmaf(m, qs[j][c], acc[j]);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < MAXQ; ++j) out[(size_t)j * 2 * MAXD + half * MAXD + r] = acc[j];
+  }
+}
+
+// ------------------------------------------------------------------ per-slice scores, weights, V sums
+__device__ __forceinline__ void add4(float4& a, const float4 b) {
+  a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+}
+
+// Asynchronous copy of a contiguous run of code rows into shared memory (the whole CTA takes part).
+// Rows are 4-byte aligned; 16-byte pieces are used where the source allows.
+__device__ __forceinline__ void stage_rows(unsigned char* dst, const unsigned char* src, int bytes) {
+  const uint32_t d0 = (uint32_t)__cvta_generic_to_shared(dst);
+  int done = 0;
+  if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+    done = bytes & ~15;
+    for (int i = threadIdx.x * 16; i < done; i += NT * 16)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d0 + i), "l"(src + i) : "memory");
+  }
+  for (int i = done + threadIdx.x * 4; i < bytes; i += NT * 4)
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d0 + i), "l"(src + i) : "memory");
+}
+
+__global__ void __launch_bounds__(NT) partial_kernel(Args a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float4* lut = reinterpret_cast<float4*>(smem_raw);                       // [lut_float4]
+  float4* lg = lut + a.lut_float4;                                         // [SLICE] logits, then p
+  float4* wvg = lg + SLICE;                                                // [ngroups][SLICE] p * nu^V of the group
+  float* qs = reinterpret_cast<float*>(wvg);                               // rotated queries while the tables are built
+  unsigned char* kbuf = reinterpret_cast<unsigned char*>(wvg + a.ngroups * SLICE);
+  unsigned char* vbuf = kbuf + a.kbuf_bytes;
+  float* vcent = reinterpret_cast<float*>(vbuf + a.vbuf_bytes);            // [MAXG][16]
+  float* red = vcent + MAXG * 16;                                          // [NT/32][MAXQ] + [MAXQ]
+  float4* accred = reinterpret_cast<float4*>(red + (NT / 32 + 1) * MAXQ);  // [NT] partial sums of phase C
+  const int h = blockIdx.x / a.nslices, sl = blockIdx.x % a.nslices;
+  const int64_t t0 = (int64_t)sl * SLICE;
+  const int ntok = (int)min((int64_t)SLICE, a.tokens - t0);
+  const int64_t row0 = (int64_t)h * a.tokens + t0;
+  const int d = a.d, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  // ---- the slice's code rows travel to shared memory while the tables are built: every row is touched once,
+  //      and a thread that waited for its own row would see one DRAM latency per token
+  for (int gi = 0; gi < a.ngroups; ++gi) {
+    const GroupDev& g = a.g[gi];
+    if (g.k_bits > 0) stage_rows(kbuf + g.k_idx_soff, g.k_idx + (size_t)row0 * g.k_idx_rb, ntok * g.k_idx_rb);
+    if (g.k_prod) stage_rows(kbuf + g.k_qjl_soff, g.k_qjl + (size_t)row0 * g.k_qjl_rb, ntok * g.k_qjl_rb);
+    stage_rows(vbuf + g.v_idx_soff, g.v_idx + (size_t)row0 * g.v_idx_rb, ntok * g.v_idx_rb);
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  {
+    const float* q = a.qrot + (size_t)h * a.ngroups * MAXQ * 2 * MAXD;
+    for (int e = tid; e < a.ngroups * MAXQ * 2 * MAXD; e += NT) qs[e] = q[e];
+  }
+  __syncthreads();
+
+  // ---- tables: entry (lookup L, value v) = sum over the coordinates the L-th field covers
+  for (int gi = 0; gi < a.ngroups; ++gi) {
+    const GroupDev& g = a.g[gi];
+    const float* q = qs + (size_t)gi * MAXQ * 2 * MAXD;
+    const int nl = mse_lookups(d, g.k_bits), ne = mse_entries(g.k_bits);
+    const int cpl = g.k_bits == 1 ? 4 : g.k_bits == 2 ? 2 : 1;   // coordinates per lookup
+    for (int e = tid; e < nl * ne; e += NT) {
+      const int L = e / ne, v = e % ne;
+      float s[MAXQ] = {0.f, 0.f, 0.f, 0.f};
+      for (int u = 0; u < cpl; ++u) {
+        const int c = L * cpl + u;
+        const float cent = g.k_cent[(v >> (u * g.k_bits)) & ((1 << g.k_bits) - 1)];
+#pragma unroll
+        for (int j = 0; j < MAXQ; ++j) s[j] = fmaf(q[j * 2 * MAXD + c], cent, s[j]);
+      }
+      lut[g.lut_mse_off + e] = make_float4(s[0], s[1], s[2], s[3]);
+    }
+    if (g.k_prod) {
+      for (int e = tid; e < (d / 4) * 16; e += NT) {
+        const int L = e >> 4, v = e & 15;
+        float s[MAXQ] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float sg = ((v >> u) & 1) ? 1.f : -1.f;
+#pragma unroll
+          for (int j = 0; j < MAXQ; ++j) s[j] = fmaf(sg, q[j * 2 * MAXD + MAXD + 4 * L + u], s[j]);
+        }
+        lut[g.lut_qjl_off + e] = make_float4(s[0], s[1], s[2], s[3]);
+      }
+    }
+    if (tid < 16) vcent[gi * 16 + tid] = g.v_cent[tid];
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+
+  // ---- A: logits of this slice's tokens (thread = token)
+  float mx[MAXQ] = {-FLT_MAX, -FLT_MAX, -FLT_MAX, -FLT_MAX};
+  for (int tl = tid; tl < ntok; tl += NT) {
+    const int64_t row = row0 + tl;
+    float4 score = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int gi = 0; gi < a.ngroups; ++gi) {
+      const GroupDev& g = a.g[gi];
+      const float nu = g.k_norms ? __ldg(g.k_norms + row) : 1.f;
+      const float cg = g.k_prod ? g.coef * __ldg(g.k_gamma + row) : 0.f;
+      float4 am = make_float4(0.f, 0.f, 0.f, 0.f), aq = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (g.k_bits == 3) {          // 8 coordinates per 3 bytes
+        const uint8_t* p = kbuf + g.k_idx_soff + (size_t)tl * g.k_idx_rb;
+        const float4* tb = lut + g.lut_mse_off;
+        for (int c8 = 0; c8 < d / 8; ++c8) {
+          const uint32_t x = (uint32_t)p[3 * c8] | ((uint32_t)p[3 * c8 + 1] << 8) | ((uint32_t)p[3 * c8 + 2] << 16);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) add4(am, tb[(c8 * 8 + u) * 8 + ((x >> (3 * u)) & 7u)]);
+        }
+      } else if (g.k_bits > 0) {    // nibbles never straddle a word
+        const uint32_t* p = reinterpret_cast<const uint32_t*>(kbuf + g.k_idx_soff + (size_t)tl * g.k_idx_rb);
+        const float4* tb = lut + g.lut_mse_off;
+        const int nw = d * g.k_bits / 32;
+        for (int w = 0; w < nw; ++w) {
+          const uint32_t x = p[w];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) add4(am, tb[(w * 8 + u) * 16 + ((x >> (4 * u)) & 15u)]);
+        }
+      }
+      if (g.k_prod) {
+        const uint32_t* p = reinterpret_cast<const uint32_t*>(kbuf + g.k_qjl_soff + (size_t)tl * g.k_qjl_rb);
+        const float4* tb = lut + g.lut_qjl_off;
+        for (int w = 0; w < d / 32; ++w) {
+          const uint32_t x = p[w];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) add4(aq, tb[(w * 8 + u) * 16 + ((x >> (4 * u)) & 15u)]);
+        }
+      }
+      score.x += nu * fmaf(cg, aq.x, am.x);
+      score.y += nu * fmaf(cg, aq.y, am.y);
+      score.z += nu * fmaf(cg, aq.z, am.z);
+      score.w += nu * fmaf(cg, aq.w, am.w);
+    }
+    const float4 l4 = make_float4(a.scale * score.x, a.scale * score.y, a.scale * score.z, a.scale * score.w);
+    lg[tl] = l4;
+    mx[0] = fmaxf(mx[0], l4.x); mx[1] = fmaxf(mx[1], l4.y); mx[2] = fmaxf(mx[2], l4.z); mx[3] = fmaxf(mx[3], l4.w);
+  }
+
+  // ---- B: slice maximum, exponentials, their sum (fixed reduction order)
+#pragma unroll
+  for (int j = 0; j < MAXQ; ++j) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx[j] = fmaxf(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], o));
+    if (lane == 0) red[warp * MAXQ + j] = mx[j];
+  }
+  __syncthreads();
+  if (tid < MAXQ) {
+    float m = red[tid];
+    for (int w = 1; w < NT / 32; ++w) m = fmaxf(m, red[w * MAXQ + tid]);
+    red[(NT / 32) * MAXQ + tid] = m;
+  }
+  __syncthreads();
+  float smax[MAXQ], sum[MAXQ] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int j = 0; j < MAXQ; ++j) smax[j] = red[(NT / 32) * MAXQ + j];
+  __syncthreads();
+  for (int tl = tid; tl < ntok; tl += NT) {
+    const float4 l4 = lg[tl];
+    const float4 p = make_float4(expf(l4.x - smax[0]), expf(l4.y - smax[1]), expf(l4.z - smax[2]), expf(l4.w - smax[3]));
+    sum[0] += p.x; sum[1] += p.y; sum[2] += p.z; sum[3] += p.w;
+    for (int gi = 0; gi < a.ngroups; ++gi) {
+      const float nv = a.g[gi].v_norms ? __ldg(a.g[gi].v_norms + row0 + tl) : 1.f;
+      wvg[gi * SLICE + tl] = make_float4(p.x * nv, p.y * nv, p.z * nv, p.w * nv);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < MAXQ; ++j) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum[j] += __shfl_xor_sync(0xffffffffu, sum[j], o);
+    if (lane == 0) red[warp * MAXQ + j] = sum[j];
+  }
+  __syncthreads();
+  float* ml = a.part_ml + (size_t)(h * a.nslices + sl) * 2 * MAXQ;
+  if (tid < MAXQ) {
+    float s = 0.f;
+    for (int w = 0; w < NT / 32; ++w) s += red[w * MAXQ + tid];
+    ml[tid] = smax[tid];
+    ml[MAXQ + tid] = s;
+  }
+
+  // ---- C: acc[oc] = sum_t p_t nu^V_t c_V[idx^V_{t,c}]   (thread = output coordinate x token phase)
+  const int ncoord = a.ngroups * d;
+  const int nrep = max(1, NT / ncoord);          // token phases that share the CTA
+  float4* out = reinterpret_cast<float4*>(a.part_acc) + (size_t)(h * a.nslices + sl) * ncoord;
+  for (int base = 0; base < ncoord; base += NT) {   // one round unless ngroups * d > 256
+    const int item = tid;
+    const int oc = base + (nrep > 1 ? item % ncoord : item), ph = nrep > 1 ? item / ncoord : 0;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const bool live = oc < ncoord && ph < nrep;
+    if (live) {
+      const int gi = oc / d, c = oc % d;
+      const GroupDev& g = a.g[gi];
+      const int bit = c * g.v_bits, bo = bit >> 3, sh = bit & 7, rb = g.v_idx_rb;
+      const uint32_t mask = (1u << g.v_bits) - 1u;
+      const bool two = sh + g.v_bits > 8;
+      const float* ct = vcent + gi * 16;
+      const unsigned char* vb = vbuf + g.v_idx_soff + bo;
+      const float4* wg = wvg + gi * SLICE;
+#pragma unroll 4
+      for (int tl = ph; tl < ntok; tl += nrep) {
+        const unsigned char* p = vb + (size_t)tl * rb;
+        uint32_t x = p[0];
+        if (two) x |= (uint32_t)p[1] << 8;
+        const float cv = ct[(x >> sh) & mask];
+        const float4 w = wg[tl];
+        acc.x = fmaf(w.x, cv, acc.x); acc.y = fmaf(w.y, cv, acc.y); acc.z = fmaf(w.z, cv, acc.z); acc.w = fmaf(w.w, cv, acc.w);
+      }
+    }
+    if (nrep > 1) {   // add the token phases in a fixed order
+      accred[tid] = acc;
+      __syncthreads();
+      if (tid < ncoord) {
+        float4 s = accred[tid];
+        for (int r = 1; r < nrep; ++r) add4(s, accred[r * ncoord + tid]);
+        out[tid] = s;
+      }
+      __syncthreads();
+    } else if (live) {
+      out[oc] = acc;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ merge of the slices + inverse rotation
+__global__ void __launch_bounds__(128) merge_kernel(Args a, float* __restrict__ out, int64_t ldo) {
+  __shared__ float yp[MAXG * MAXD];
+  __shared__ float wsl[64];
+  __shared__ float stat[2];
+  const int h = blockIdx.x / a.qpk, j = blockIdx.x % a.qpk;
+  const int ncoord = a.ngroups * a.d, d = a.d;
+  const float* ml = a.part_ml + (size_t)h * a.nslices * 2 * MAXQ;
+  if (threadIdx.x == 0) {
+    float M = -FLT_MAX;
+    for (int s = 0; s < a.nslices; ++s) M = fmaxf(M, ml[s * 2 * MAXQ + j]);
+    double L = 0.0;
+    for (int s = 0; s < a.nslices; ++s) L += (double)ml[s * 2 * MAXQ + MAXQ + j] * (double)expf(ml[s * 2 * MAXQ + j] - M);
+    stat[0] = M;
+    stat[1] = (float)(1.0 / L);
+  }
+  __syncthreads();
+  const float M = stat[0], inv = stat[1];
+  const float* acc = a.part_acc + (size_t)h * a.nslices * ncoord * MAXQ;
+  for (int oc = threadIdx.x; oc < ncoord; oc += blockDim.x) yp[oc] = 0.f;
+  for (int s0 = 0; s0 < a.nslices; s0 += 64) {   // slice weights in chunks of 64, slices added in order
+    const int ns = min(64, a.nslices - s0);
+    __syncthreads();
+    if ((int)threadIdx.x < ns) wsl[threadIdx.x] = expf(ml[(s0 + threadIdx.x) * 2 * MAXQ + j] - M) * inv;
+    __syncthreads();
+    for (int oc = threadIdx.x; oc < ncoord; oc += blockDim.x) {
+      float v = yp[oc];
+#pragma unroll 8
+      for (int s = 0; s < ns; ++s) v = fmaf(wsl[s], acc[((size_t)(s0 + s) * ncoord + oc) * MAXQ + j], v);
+      yp[oc] = v;
+    }
+  }
+  __syncthreads();
+  // x~_k = sum_c Pi[c][k] y'_c per group, scattered to the group's channels of this head
+  for (int ok = threadIdx.x; ok < ncoord; ok += blockDim.x) {
+    const int gi = ok / d, k = ok % d;
+    const GroupDev& g = a.g[gi];
+    float v = 0.f;
+#pragma unroll 8
+    for (int c = 0; c < d; ++c) v = fmaf(g.v_pi[(size_t)c * d + k], yp[gi * d + c], v);
+    out[(int64_t)(h * a.qpk + j) * ldo + g.v_channels[h * d + k]] = v;
+  }
+}
+
+size_t workspace_bytes(int ngroups, int heads, int64_t tokens, int d) {
+  const int64_t nslices = std::max<int64_t>(1, (tokens + SLICE - 1) / SLICE);
+  size_t b = (size_t)heads * ngroups * MAXQ * 2 * MAXD * sizeof(float);
+  b += (size_t)heads * nslices * 2 * MAXQ * sizeof(float);
+  b = (b + 255) / 256 * 256;
+  b += (size_t)heads * nslices * ngroups * d * MAXQ * sizeof(float);
+  return (b + 255) / 256 * 256;
+}
+
+}  // namespace kvdec
+}  // namespace tq
+
+extern "C" size_t tq_attend_decode_workspace_bytes(int ngroups, int heads, int64_t tokens, int d) {
+  if (ngroups <= 0 || heads <= 0 || tokens < 0 || d <= 0) return 0;
+  return tq::kvdec::workspace_bytes(ngroups, heads, tokens, d);
+}
+
+extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int heads, int64_t tokens, int q_per_kv,
+                                const void* Q, int q_dtype, int64_t ldq, float scale, float* out, int64_t ldo,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  using namespace tq;
+  using namespace tq::kvdec;
+  const char* who = "tq_attend_decode";
+  TQ_REQUIRE(groups != nullptr && ngroups >= 1 && ngroups <= MAXG, TQ_ERR_INVALID_ARG, "%s: 1..%d channel groups", who, MAXG);
+  TQ_REQUIRE(heads >= 0 && tokens >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
+  TQ_REQUIRE(q_per_kv >= 1 && q_per_kv <= MAXQ, TQ_ERR_UNSUPPORTED, "%s: 1..%d queries per KV head", who, MAXQ);
+  TQ_REQUIRE(q_dtype == TQ_F32 || q_dtype == TQ_BF16, TQ_ERR_UNSUPPORTED, "%s: unknown query dtype %d", who, q_dtype);
+  if (heads == 0) return TQ_OK;
+  TQ_REQUIRE(out != nullptr && Q != nullptr, TQ_ERR_INVALID_ARG, "%s: Q or out is NULL", who);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Args a;
+  std::memset(&a, 0, sizeof(a));
+  const int d = groups[0].plan_k ? groups[0].plan_k->d : 0;
+  TQ_REQUIRE(d >= 8 && d <= MAXD && d % 8 == 0, TQ_ERR_UNSUPPORTED, "%s: group dimension %d (multiples of 8 up to %d)", who, d, MAXD);
+  TQ_REQUIRE(ldq >= 1 && ldo >= 1, TQ_ERR_INVALID_ARG, "%s: bad row stride", who);
+  int lut = 0, kbytes = 0, vbytes = 0;
+  for (int gi = 0; gi < ngroups; ++gi) {
+    const tq_kv_group& s = groups[gi];
+    TQ_REQUIRE(s.plan_k && s.plan_v, TQ_ERR_INVALID_ARG, "%s: group %d has no plan", who, gi);
+    TQ_REQUIRE(s.plan_k->d == d && s.plan_v->d == d, TQ_ERR_UNSUPPORTED, "%s: all groups must share one dimension", who);
+    TQ_REQUIRE(s.plan_v->mode == TQ_MSE && s.plan_v->mse_bits >= 1, TQ_ERR_UNSUPPORTED,
+               "%s: values must be quantised with TurboQuant_mse", who);
+    TQ_REQUIRE(s.plan_k->device == s.plan_v->device, TQ_ERR_INVALID_ARG, "%s: plans of different devices", who);
+    const bool prod = s.plan_k->mode == TQ_PROD;
+    TQ_REQUIRE(s.k_channels && s.v_channels && s.v_idx, TQ_ERR_INVALID_ARG, "%s: group %d: NULL channel list or codes", who, gi);
+    TQ_REQUIRE(s.plan_k->mse_bits == 0 || s.k_idx, TQ_ERR_INVALID_ARG, "%s: group %d: k_idx is NULL", who, gi);
+    TQ_REQUIRE(!prod || (s.k_qjl && s.k_gamma), TQ_ERR_INVALID_ARG, "%s: group %d: k_qjl / k_gamma is NULL", who, gi);
+    TQ_REQUIRE((reinterpret_cast<uintptr_t>(s.k_idx) & 3) == 0 && (reinterpret_cast<uintptr_t>(s.k_qjl) & 3) == 0,
+               TQ_ERR_ALIGNMENT, "%s: group %d: codes are not 4-byte aligned", who, gi);
+    GroupDev& g = a.g[gi];
+    g.k_idx = s.k_idx; g.k_qjl = s.k_qjl; g.k_gamma = s.k_gamma; g.k_norms = s.k_norms;
+    g.v_idx = s.v_idx; g.v_norms = s.v_norms;
+    g.k_channels = s.k_channels; g.v_channels = s.v_channels;
+    g.k_rotcat = s.plan_k->dRotCat; g.v_pi = s.plan_v->dPi;
+    for (int i = 0; i < 16; ++i) { g.k_cent[i] = s.plan_k->cb.c[i]; g.v_cent[i] = s.plan_v->cb.c[i]; }
+    g.k_bits = s.plan_k->mse_bits; g.v_bits = s.plan_v->mse_bits; g.k_prod = prod ? 1 : 0;
+    g.k_idx_rb = (int)s.plan_k->idx_row_bytes; g.k_qjl_rb = (int)s.plan_k->qjl_row_bytes; g.v_idx_rb = (int)s.plan_v->idx_row_bytes;
+    g.k_dpad = s.plan_k->dpad;
+    g.coef = s.plan_k->coef;
+    g.lut_mse_off = lut;
+    lut += mse_lookups(d, g.k_bits) * mse_entries(g.k_bits);
+    g.lut_qjl_off = lut;
+    if (prod) lut += (d / 4) * 16;
+    g.k_idx_soff = kbytes;
+    kbytes += (g.k_bits > 0 ? SLICE * g.k_idx_rb + 15 : 0) / 16 * 16;
+    g.k_qjl_soff = kbytes;
+    kbytes += (prod ? SLICE * g.k_qjl_rb + 15 : 0) / 16 * 16;
+    g.v_idx_soff = vbytes;
+    vbytes += (SLICE * g.v_idx_rb + 15) / 16 * 16;
+  }
+  if (tokens == 0) {   // no tokens: the output rows are zero
+    TQ_CHECK_CUDA(cudaMemset2DAsync(out, (size_t)ldo * sizeof(float), 0, (size_t)ngroups * d * sizeof(float),
+                                    (size_t)heads * q_per_kv, st), who);
+    return TQ_OK;
+  }
+  const int64_t nslices = (tokens + SLICE - 1) / SLICE;
+  TQ_REQUIRE((int64_t)heads * nslices < (1 << 30), TQ_ERR_UNSUPPORTED, "%s: too many (head, slice) pairs", who);
+  const size_t need = kvdec::workspace_bytes(ngroups, heads, tokens, d);
+  TQ_REQUIRE(workspace != nullptr && workspace_bytes >= need, TQ_ERR_WORKSPACE, "%s: workspace of %zu bytes, %zu needed", who,
+             workspace_bytes, need);
+  TQ_REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255) == 0, TQ_ERR_ALIGNMENT, "%s: workspace is not 256-byte aligned", who);
+  a.ngroups = ngroups; a.heads = heads; a.qpk = q_per_kv; a.d = d; a.nslices = (int)nslices;
+  a.tokens = tokens; a.scale = scale; a.lut_float4 = lut;
+  a.kbuf_bytes = kbytes; a.vbuf_bytes = vbytes;
+  char* w = static_cast<char*>(workspace);
+  a.qrot = reinterpret_cast<float*>(w);
+  size_t off = (size_t)heads * ngroups * MAXQ * 2 * MAXD * sizeof(float);
+  a.part_ml = reinterpret_cast<float*>(w + off);
+  off += (size_t)heads * nslices * 2 * MAXQ * sizeof(float);
+  off = (off + 255) / 256 * 256;
+  a.part_acc = reinterpret_cast<float*>(w + off);
+
+  int dev = 0;
+  TQ_CHECK_CUDA(cudaGetDevice(&dev), who);
+  TQ_REQUIRE(dev == groups[0].plan_k->device, TQ_ERR_INVALID_ARG, "%s: the plans belong to device %d, current device is %d", who,
+             groups[0].plan_k->device, dev);
+  if (q_dtype == TQ_F32)
+    prepare_kernel<float><<<heads * ngroups, 128, 0, st>>>(a, static_cast<const float*>(Q), ldq);
+  else
+    prepare_kernel<__nv_bfloat16><<<heads * ngroups, 128, 0, st>>>(a, static_cast<const __nv_bfloat16*>(Q), ldq);
+  TQ_CHECK_CUDA(cudaGetLastError(), who);
+  const size_t smem = (size_t)lut * sizeof(float4) + (size_t)(1 + ngroups) * SLICE * sizeof(float4) + kbytes + vbytes +
+                      MAXG * 16 * sizeof(float) + (NT / 32 + 1) * MAXQ * sizeof(float) + NT * sizeof(float4);
+  TQ_REQUIRE(smem <= 220 * 1024, TQ_ERR_UNSUPPORTED, "%s: %zu bytes of shared memory needed (too many wide groups)", who, smem);
+  static size_t smem_set[16] = {0};
+  if (dev < 16 && smem > smem_set[dev]) {
+    TQ_CHECK_CUDA(cudaFuncSetAttribute(partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), who);
+    smem_set[dev] = smem;
+  } else if (dev >= 16) {
+    TQ_CHECK_CUDA(cudaFuncSetAttribute(partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), who);
+  }
+  partial_kernel<<<(unsigned)(heads * nslices), NT, smem, st>>>(a);
+  TQ_CHECK_CUDA(cudaGetLastError(), who);
+  merge_kernel<<<heads * q_per_kv, 128, 0, st>>>(a, out, ldo);
+  TQ_CHECK_CUDA(cudaGetLastError(), who);
+  count_launches(3);
+  return TQ_OK;
+}

@@ -128,3 +128,90 @@ def test_softmax_rows_and_empty_inputs():
     tq.tq_wsum(su.plan, None, 0, None, None, None, None, out, None)     # n = 0: zeros
     torch.cuda.synchronize()
     assert not bool(out.any())
+
+
+# ---------------------------------------------------------------------------------------------
+# tq_attend_decode: the same computation for all KV heads and channel groups of a layer in one call
+
+
+def _fused_layer(groupsK, groupsV, recs, Q, heads, T, qpk):
+    """Concatenates the per-head codes of `recs` head-major and runs tq_attend_decode."""
+    groups = []
+    for gi in range(len(groupsK)):
+        cat = lambda kind, i: (None if recs[0][kind][gi][3][i] is None
+                               else torch.cat([recs[h][kind][gi][3][i] for h in range(heads)]).contiguous())
+        groups.append({
+            "plan_k": groupsK[gi].plan, "plan_v": groupsV[gi].plan,
+            "k_idx": cat("K", 0), "k_qjl": cat("K", 1), "k_gamma": cat("K", 2), "k_norms": cat("K", 3),
+            "v_idx": cat("V", 0), "v_norms": cat("V", 3),
+            "k_channels": torch.stack([recs[h]["K"][gi][1] for h in range(heads)]).to(torch.int32).contiguous(),
+            "v_channels": torch.stack([recs[h]["V"][gi][1] for h in range(heads)]).to(torch.int32).contiguous(),
+        })
+    d = groupsK[0].d
+    ws = torch.empty(tq.tq_attend_decode_workspace_bytes(len(groups), heads, T, d), dtype=torch.uint8, device=DEV)
+    out = torch.full((heads * qpk, HEAD_DIM), float("nan"), device=DEV)
+    tq.tq_attend_decode(groups, heads, T, qpk, Q, 1.0 / math.sqrt(HEAD_DIM), out, ws)
+    out2 = torch.full_like(out, float("nan"))
+    tq.tq_attend_decode(groups, heads, T, qpk, Q, 1.0 / math.sqrt(HEAD_DIM), out2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)          # fixed reduction orders: repeatable bit for bit
+    return out
+
+
+def test_fused_decode_full_shape_against_the_separate_calls(groups):
+    gK, gV = groups
+    K, V, Q = wl.kv_cache(device=DEV)
+    heads, T, _ = K.shape
+    outs, recs = [], []
+    for h in range(heads):
+        out, _, rec = attend_gpu(gK, gV, K[h], V[h], Q[4 * h:4 * h + 4])
+        outs.append(out)
+        recs.append(rec)
+    ref = torch.cat(outs)
+    fused = _fused_layer(gK, gV, recs, Q, heads, T, 4)
+    err = (fused - ref).norm(dim=1) / ref.norm(dim=1)
+    assert float(err.max()) <= 2e-4, float(err.max())
+
+
+@pytest.mark.parametrize("heads,T,qpk", [(2, 2500, 3), (1, 1024, 1), (3, 77, 4)])
+def test_fused_decode_against_the_oracle(groups, heads, T, qpk):
+    gK, gV = groups
+    K, V, Q = wl.kv_cache(heads=heads, tokens=T, q_per_kv=qpk, seed=5 + T, device=DEV)
+    recs, refs = [], []
+    for h in range(heads):
+        Qh = Q[qpk * h:qpk * h + qpk]
+        _, _, rec = attend_gpu(gK, gV, K[h], V[h], Qh)
+        recs.append(rec)
+        refs.append(attend_oracle(rec, Qh)[0])
+    ref = np.concatenate(refs)
+    fused = P.as_f64(_fused_layer(gK, gV, recs, Q, heads, T, qpk))
+    err = np.linalg.norm(fused - ref, axis=1) / np.linalg.norm(ref, axis=1)
+    assert float(err.max()) <= 1e-3, float(err.max())
+
+
+def test_fused_decode_other_bit_widths_and_argument_checks():
+    # one group of 128 channels: keys TurboQuant_mse 4-bit (no QJL part), values 4-bit; then keys prod 4-bit (3-bit indices)
+    for kbits, kmode in ((4, tq.TQ_MSE), (4, tq.TQ_PROD), (1, tq.TQ_PROD)):
+        gK = (P.Setup(HEAD_DIM, kbits, kmode, 81, 82),)
+        gV = (P.Setup(HEAD_DIM, 4, tq.TQ_MSE, 83, 84),)
+        heads, T, qpk = 2, 1500, 2
+        K, V, Q = wl.kv_cache(heads=heads, tokens=T, q_per_kv=qpk, seed=9, device=DEV)
+        ch = torch.arange(HEAD_DIM, device=DEV)
+        recs, refs = [], []
+        for h in range(heads):
+            rec = {"K": [], "V": []}
+            Kh, Vh = K[h].float().contiguous(), V[h].float().contiguous()
+            rec["K"].append((gK[0], ch, Kh, gK[0].quantize(Kh)))
+            rec["V"].append((gV[0], ch, Vh, gV[0].quantize(Vh)))
+            recs.append(rec)
+            refs.append(attend_oracle(rec, Q[qpk * h:qpk * h + qpk])[0])
+        fused = P.as_f64(_fused_layer(gK, gV, recs, Q, heads, T, qpk))
+        ref = np.concatenate(refs)
+        err = np.linalg.norm(fused - ref, axis=1) / np.linalg.norm(ref, axis=1)
+        assert float(err.max()) <= 1e-3, (kbits, kmode, float(err.max()))
+    with pytest.raises(tq.TqError):     # a workspace that is too small is refused
+        g = {"plan_k": gK[0].plan, "plan_v": gV[0].plan, "k_idx": recs[0]["K"][0][3][0], "k_qjl": recs[0]["K"][0][3][1],
+             "k_gamma": recs[0]["K"][0][3][2], "k_norms": recs[0]["K"][0][3][3], "v_idx": recs[0]["V"][0][3][0],
+             "v_norms": recs[0]["V"][0][3][3], "k_channels": ch.to(torch.int32).repeat(1, 1), "v_channels": ch.to(torch.int32).repeat(1, 1)}
+        tq.tq_attend_decode([g], 1, T, qpk, Q, 1.0, torch.empty((qpk, HEAD_DIM), device=DEV),
+                            torch.empty(256, dtype=torch.uint8, device=DEV))
