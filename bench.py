@@ -304,6 +304,67 @@ def run_b200(args):
               "score_frac_hbm": code_bytes2 / (ms_s2 * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     del idx2, norms2, scratch2, ws2, sc2, plan2
 
+    # ---- KV-cache decode (config c3): one layer = 8 KV heads x 32768 tokens, 2.5 bits per channel, 32 query heads;
+    #      32 layer copies so that the codes (0.94 GB) exceed L2; tq_attend_decode, one call per layer ----
+    kv = None
+    if n == WORKLOAD["n"]:
+        import math
+        Kc, Vc, Qc = wl.kv_cache(device=dev)
+        Hh, Tt, hd = Kc.shape
+        grp = 64
+
+        def kv_plan(b, mode, ps, ss):
+            cent_g, _ = tq.tq_codebook(grp, b - 1 if mode == tq.TQ_PROD else b)
+            return tq.Plan(grp, b, mode, tq.tq_rotation(grp, ps), tq.tq_rotation(grp, ss, tq.TQ_GAUSSIAN) if mode == tq.TQ_PROD else None, cent_g)
+
+        pk = (kv_plan(3, tq.TQ_PROD, 72, 73), kv_plan(2, tq.TQ_PROD, 74, 75))
+        pv = (kv_plan(3, tq.TQ_MSE, 76, 77), kv_plan(2, tq.TQ_MSE, 78, 79))
+
+        def split(Xh):   # harness rule: the 64 channels of largest energy form the outlier group
+            o = torch.topk(Xh.float().pow(2).sum(0), grp).indices.sort().values
+            m = torch.ones(hd, dtype=torch.bool, device=dev)
+            m[o] = False
+            return o, torch.nonzero(m).flatten()
+
+        chk = [split(Kc[h]) for h in range(Hh)]
+        chv = [split(Vc[h]) for h in range(Hh)]
+        groups = []
+        for g in range(2):
+            Xk = torch.cat([Kc[h][:, chk[h][g]] for h in range(Hh)]).contiguous()
+            Xv = torch.cat([Vc[h][:, chv[h][g]] for h in range(Hh)]).contiguous()
+            rows = Xk.shape[0]
+            gd = {"plan_k": pk[g], "plan_v": pv[g],
+                  "k_idx": torch.empty((rows, pk[g].idx_row_bytes), dtype=torch.uint8, device=dev),
+                  "k_qjl": torch.empty((rows, pk[g].qjl_row_bytes), dtype=torch.uint8, device=dev),
+                  "k_gamma": torch.empty(rows, device=dev), "k_norms": torch.empty(rows, device=dev),
+                  "v_idx": torch.empty((rows, pv[g].idx_row_bytes), dtype=torch.uint8, device=dev),
+                  "v_norms": torch.empty(rows, device=dev),
+                  "k_channels": torch.stack([chk[h][g] for h in range(Hh)]).to(torch.int32).contiguous(),
+                  "v_channels": torch.stack([chv[h][g] for h in range(Hh)]).to(torch.int32).contiguous()}
+            sk = torch.empty(max(tq.tq_workspace_bytes(pk[g], tq.TQ_OP_QUANTIZE, rows), 16), dtype=torch.uint8, device=dev)
+            tq.tq_quantize_prod(pk[g], Xk, gd["k_idx"], gd["k_qjl"], gd["k_gamma"], gd["k_norms"], sk)
+            tq.tq_quantize_mse(pv[g], Xv, gd["v_idx"], gd["v_norms"], sk)
+            groups.append(gd)
+        code_keys = ("k_idx", "k_qjl", "k_gamma", "k_norms", "v_idx", "v_norms")
+        layer_bytes = sum(gd[key].numel() * gd[key].element_size() for gd in groups for key in code_keys)
+        n_layers = 32
+        layers = [[{key: (val.clone() if key in code_keys else val) for key, val in gd.items()} for gd in groups]
+                  for _ in range(n_layers)]
+        ws_kv = torch.empty(tq.tq_attend_decode_workspace_bytes(2, Hh, Tt, grp), dtype=torch.uint8, device=dev)
+        out_kv = torch.zeros((Hh * 4, hd), dtype=torch.float32, device=dev)
+
+        def decode_all_layers():
+            for lay in layers:
+                tq.tq_attend_decode(lay, Hh, Tt, 4, Qc, 1.0 / math.sqrt(hd), out_kv, ws_kv)
+
+        ms_model = time_call(decode_all_layers, reps=3)
+        us_layer = ms_model * 1e3 / n_layers
+        kv = {"workload": f"c3: {Hh} KV heads x {Tt} tokens x {hd} channels (64 at 3 bits + 64 at 2 bits), K prod / V mse, 32 query heads",
+              "layers": n_layers, "us_per_layer": us_layer, "code_bytes_per_layer": layer_bytes,
+              "codes_gbs": layer_bytes / (us_layer * 1e-6) / 1e9, "frac_hbm": layer_bytes / (us_layer * 1e-6) / 1e9 / peaks["hbm_gbs"],
+              "launches_per_layer": 3}
+        del layers, groups, Kc, Vc
+
     # ---- end to end: inputs start in pinned host memory, codes and top-k go back to the host ----
     e2e = None
     if not args.no_e2e:
@@ -414,7 +475,7 @@ def run_b200(args):
             "quantize_vectors_per_s": n / (q_ms * 1e-3), "quantize_ms": q_ms,
             "scan_ms": s_ms, "scan_codes_gbs": scan_gbs, "scan_frac_hbm": scan_gbs / peaks["hbm_gbs"],
             "scan_queries_per_s": nq / (s_ms * 1e-3),
-            "scan_regimes": scan_regimes, "scan_many_queries": many_queries, "mse_b2": mse_b2, "roofline": roofline, "roofline_scan": roofline_scan, "clocks": clocks,
+            "scan_regimes": scan_regimes, "scan_many_queries": many_queries, "mse_b2": mse_b2, "kv_decode": kv, "roofline": roofline, "roofline_scan": roofline_scan, "clocks": clocks,
             "e2e": e2e, "gpu_launches": int(launches)}
     if not args.no_cpu_baseline:
         sample = 32768

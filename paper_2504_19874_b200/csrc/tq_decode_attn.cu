@@ -44,7 +44,7 @@ struct GroupDev {
   const float* v_norms;
   const int32_t* k_channels;
   const int32_t* v_channels;
-  const float* k_rotcat;   // [ncat*dpad, d]
+  const float* k_backt;    // [d, ncat*dpad]: column o = row o of [Pi ; S]
   const float* v_pi;       // [d, d]
   float k_cent[16], v_cent[16];
   int k_bits, v_bits, k_prod;
@@ -95,10 +95,10 @@ __global__ void __launch_bounds__(128) prepare_kernel(Args a, const T* __restric
     const int half = o / g.k_dpad, r = o % g.k_dpad;
     float acc[MAXQ] = {0.f, 0.f, 0.f, 0.f};
     if (r < d) {
-      const float* row = g.k_rotcat + (size_t)o * d;
+      const float* col = g.k_backt + o;   // consecutive threads read consecutive addresses
 #pragma unroll 8
       for (int c = 0; c < d; ++c) {
-        const float m = row[c];
+        const float m = col[(size_t)c * nrows];
 #pragma unroll
         for (int j = 0; j < MAXQ; ++j) acc[j] = fmaf(m, qs[j][c], acc[j]);
       }
@@ -327,45 +327,55 @@ __global__ void __launch_bounds__(NT) partial_kernel(Args a) {
 }
 
 // ------------------------------------------------------------------ merge of the slices + inverse rotation
-__global__ void __launch_bounds__(128) merge_kernel(Args a, float* __restrict__ out, int64_t ldo) {
-  __shared__ float yp[MAXG * MAXD];
+__global__ void __launch_bounds__(256) merge_kernel(Args a, float* __restrict__ out, int64_t ldo) {
+  __shared__ float yp[2][MAXG * MAXD];
   __shared__ float wsl[64];
   __shared__ float stat[2];
   const int h = blockIdx.x / a.qpk, j = blockIdx.x % a.qpk;
   const int ncoord = a.ngroups * a.d, d = a.d;
   const float* ml = a.part_ml + (size_t)h * a.nslices * 2 * MAXQ;
-  if (threadIdx.x == 0) {
+  if (threadIdx.x < 32) {   // global maximum and sum: lanes take slices in turn, combined in a fixed order
+    const int lane = threadIdx.x;
     float M = -FLT_MAX;
-    for (int s = 0; s < a.nslices; ++s) M = fmaxf(M, ml[s * 2 * MAXQ + j]);
+    for (int s = lane; s < a.nslices; s += 32) M = fmaxf(M, ml[s * 2 * MAXQ + j]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     double L = 0.0;
-    for (int s = 0; s < a.nslices; ++s) L += (double)ml[s * 2 * MAXQ + MAXQ + j] * (double)expf(ml[s * 2 * MAXQ + j] - M);
-    stat[0] = M;
-    stat[1] = (float)(1.0 / L);
+    for (int s = lane; s < a.nslices; s += 32) L += (double)ml[s * 2 * MAXQ + MAXQ + j] * (double)expf(ml[s * 2 * MAXQ + j] - M);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+    if (lane == 0) {
+      stat[0] = M;
+      stat[1] = (float)(1.0 / L);
+    }
   }
   __syncthreads();
   const float M = stat[0], inv = stat[1];
   const float* acc = a.part_acc + (size_t)h * a.nslices * ncoord * MAXQ;
-  for (int oc = threadIdx.x; oc < ncoord; oc += blockDim.x) yp[oc] = 0.f;
-  for (int s0 = 0; s0 < a.nslices; s0 += 64) {   // slice weights in chunks of 64, slices added in order
+  const int half = threadIdx.x >> 7, t = threadIdx.x & 127;   // each half of the CTA adds every other slice
+  for (int oc = t; oc < ncoord; oc += 128) yp[half][oc] = 0.f;
+  for (int s0 = 0; s0 < a.nslices; s0 += 64) {   // slice weights in chunks of 64
     const int ns = min(64, a.nslices - s0);
     __syncthreads();
     if ((int)threadIdx.x < ns) wsl[threadIdx.x] = expf(ml[(s0 + threadIdx.x) * 2 * MAXQ + j] - M) * inv;
     __syncthreads();
-    for (int oc = threadIdx.x; oc < ncoord; oc += blockDim.x) {
-      float v = yp[oc];
-#pragma unroll 8
-      for (int s = 0; s < ns; ++s) v = fmaf(wsl[s], acc[((size_t)(s0 + s) * ncoord + oc) * MAXQ + j], v);
-      yp[oc] = v;
+    for (int oc = t; oc < ncoord; oc += 128) {
+      float v = yp[half][oc];
+#pragma unroll 16
+      for (int s = half; s < ns; s += 2) v = fmaf(wsl[s], acc[((size_t)(s0 + s) * ncoord + oc) * MAXQ + j], v);
+      yp[half][oc] = v;
     }
   }
+  __syncthreads();
+  for (int oc = threadIdx.x; oc < ncoord; oc += blockDim.x) yp[0][oc] += yp[1][oc];
   __syncthreads();
   // x~_k = sum_c Pi[c][k] y'_c per group, scattered to the group's channels of this head
   for (int ok = threadIdx.x; ok < ncoord; ok += blockDim.x) {
     const int gi = ok / d, k = ok % d;
     const GroupDev& g = a.g[gi];
     float v = 0.f;
-#pragma unroll 8
-    for (int c = 0; c < d; ++c) v = fmaf(g.v_pi[(size_t)c * d + k], yp[gi * d + c], v);
+#pragma unroll 16
+    for (int c = 0; c < d; ++c) v = fmaf(g.v_pi[(size_t)c * d + k], yp[0][gi * d + c], v);
     out[(int64_t)(h * a.qpk + j) * ldo + g.v_channels[h * d + k]] = v;
   }
 }
@@ -423,7 +433,7 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
     g.k_idx = s.k_idx; g.k_qjl = s.k_qjl; g.k_gamma = s.k_gamma; g.k_norms = s.k_norms;
     g.v_idx = s.v_idx; g.v_norms = s.v_norms;
     g.k_channels = s.k_channels; g.v_channels = s.v_channels;
-    g.k_rotcat = s.plan_k->dRotCat; g.v_pi = s.plan_v->dPi;
+    g.k_backt = s.plan_k->dBackT; g.v_pi = s.plan_v->dPi;
     for (int i = 0; i < 16; ++i) { g.k_cent[i] = s.plan_k->cb.c[i]; g.v_cent[i] = s.plan_v->cb.c[i]; }
     g.k_bits = s.plan_k->mse_bits; g.v_bits = s.plan_v->mse_bits; g.k_prod = prod ? 1 : 0;
     g.k_idx_rb = (int)s.plan_k->idx_row_bytes; g.k_qjl_rb = (int)s.plan_k->qjl_row_bytes; g.v_idx_rb = (int)s.plan_v->idx_row_bytes;
@@ -483,7 +493,7 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   }
   partial_kernel<<<(unsigned)(heads * nslices), NT, smem, st>>>(a);
   TQ_CHECK_CUDA(cudaGetLastError(), who);
-  merge_kernel<<<heads * q_per_kv, 128, 0, st>>>(a, out, ldo);
+  merge_kernel<<<heads * q_per_kv, 256, 0, st>>>(a, out, ldo);
   TQ_CHECK_CUDA(cudaGetLastError(), who);
   count_launches(3);
   return TQ_OK;
