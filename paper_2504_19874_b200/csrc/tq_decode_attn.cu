@@ -52,6 +52,7 @@ struct GroupDev {
   int k_dpad;
   float coef;
   int lut_mse_off, lut_qjl_off;   // float4 offsets of this group's tables in shared memory
+  int vunit0;   // first of this group's units (runs of coordinates sharing bytes of the value row)
   int k_idx_soff, k_qjl_soff, v_idx_soff;   // byte offsets of the staged code rows inside their shared-memory buffers
 };
 
@@ -64,6 +65,7 @@ struct Args {
   float* part_ml;   // [heads, nslices, 2, MAXQ]      slice maximum, slice sum of exponentials
   float* part_acc;  // [heads, nslices, ngroups*d, MAXQ]
   int lut_float4;   // float4 entries of all tables
+  int vunits, region0;   // units of all groups; float4 entries of the first shared-memory region
   int kbuf_bytes, vbuf_bytes;   // shared-memory room for the slice's K and V code rows
 };
 
@@ -127,17 +129,46 @@ __device__ __forceinline__ void stage_rows(unsigned char* dst, const unsigned ch
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d0 + i), "l"(src + i) : "memory");
 }
 
+__host__ __device__ inline int vunits_of(int d, int bits) { return (bits == 1 || bits == 3) ? d / 8 : d / 4; }
+
+// Value sums of one unit: BV-bit indices of CU consecutive coordinates sit in NB bytes of the row.
+template <int BV>
+__device__ __forceinline__ void vsum_unit(const unsigned char* vb, int rb, const float4* __restrict__ wg,
+                                          const float* __restrict__ ct, int ph, int nrep, int ntok, float4* dst) {
+  constexpr int CU = (BV == 1 || BV == 3) ? 8 : 4;
+  constexpr int NB = BV == 3 ? 3 : (BV == 4 ? 2 : 1);
+  float4 acc[CU];
+#pragma unroll
+  for (int u = 0; u < CU; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+  for (int tl = ph; tl < ntok; tl += nrep) {
+    const unsigned char* p = vb + (size_t)tl * rb;
+    uint32_t x = p[0];
+    if (NB > 1) x |= (uint32_t)p[1] << 8;
+    if (NB > 2) x |= (uint32_t)p[2] << 16;
+    const float4 w = wg[tl];
+#pragma unroll
+    for (int u = 0; u < CU; ++u) {
+      const float cv = ct[(x >> (BV * u)) & ((1u << BV) - 1u)];
+      acc[u].x = fmaf(w.x, cv, acc[u].x); acc[u].y = fmaf(w.y, cv, acc[u].y);
+      acc[u].z = fmaf(w.z, cv, acc[u].z); acc[u].w = fmaf(w.w, cv, acc[u].w);
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < CU; ++u) dst[u] = acc[u];
+}
+
 __global__ void __launch_bounds__(NT) partial_kernel(Args a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float4* lut = reinterpret_cast<float4*>(smem_raw);                       // [lut_float4]
   float4* lg = lut + a.lut_float4;                                         // [SLICE] logits, then p
-  float4* wvg = lg + SLICE;                                                // [ngroups][SLICE] p * nu^V of the group
+  // region0 (float4) >= tables + logits and >= the per-phase sums of phase C, which reuse that room
+  float4* wvg = lut + a.region0;                                           // [ngroups][SLICE] p * nu^V of the group
   float* qs = reinterpret_cast<float*>(wvg);                               // rotated queries while the tables are built
   unsigned char* kbuf = reinterpret_cast<unsigned char*>(wvg + a.ngroups * SLICE);
   unsigned char* vbuf = kbuf + a.kbuf_bytes;
   float* vcent = reinterpret_cast<float*>(vbuf + a.vbuf_bytes);            // [MAXG][16]
   float* red = vcent + MAXG * 16;                                          // [NT/32][MAXQ] + [MAXQ]
-  float4* accred = reinterpret_cast<float4*>(red + (NT / 32 + 1) * MAXQ);  // [NT] partial sums of phase C
   const int h = blockIdx.x / a.nslices, sl = blockIdx.x % a.nslices;
   const int64_t t0 = (int64_t)sl * SLICE;
   const int ntok = (int)min((int64_t)SLICE, a.tokens - t0);
@@ -283,46 +314,36 @@ __global__ void __launch_bounds__(NT) partial_kernel(Args a) {
     ml[MAXQ + tid] = s;
   }
 
-  // ---- C: acc[oc] = sum_t p_t nu^V_t c_V[idx^V_{t,c}]   (thread = output coordinate x token phase)
+  // ---- C: acc[oc] = sum_t p_t nu^V_t c_V[idx^V_{t,c}].  A thread owns the 4 or 8 coordinates that share 1-3 bytes
+  //      of the value row (so that one load and one weight fetch serve all of them) and one of nrep token phases;
+  //      the phases are added in a fixed order afterwards.  The tables and logits are dead by now: their room
+  //      holds the per-phase sums.
   const int ncoord = a.ngroups * d;
-  const int nrep = max(1, NT / ncoord);          // token phases that share the CTA
+  const int nrep = max(1, NT / a.vunits);
+  float4* rbuf = lut;   // [nrep][ncoord]
+  if (tid < nrep * a.vunits) {
+    int gi = 0;
+    while (gi + 1 < a.ngroups && tid >= nrep * a.g[gi + 1].vunit0) ++gi;
+    const GroupDev& g = a.g[gi];
+    const int local = tid - nrep * g.vunit0, nu_g = vunits_of(d, g.v_bits);
+    const int ph = local / nu_g, u = local % nu_g;
+    const float* ct = vcent + gi * 16;
+    const float4* wg = wvg + gi * SLICE;
+    const unsigned char* vb = vbuf + g.v_idx_soff;
+    float4* dst = rbuf + (size_t)ph * ncoord + gi * d;
+    switch (g.v_bits) {
+      case 1: vsum_unit<1>(vb + u, g.v_idx_rb, wg, ct, ph, nrep, ntok, dst + u * 8); break;
+      case 2: vsum_unit<2>(vb + u, g.v_idx_rb, wg, ct, ph, nrep, ntok, dst + u * 4); break;
+      case 3: vsum_unit<3>(vb + 3 * u, g.v_idx_rb, wg, ct, ph, nrep, ntok, dst + u * 8); break;
+      default: vsum_unit<4>(vb + 2 * u, g.v_idx_rb, wg, ct, ph, nrep, ntok, dst + u * 4); break;
+    }
+  }
+  __syncthreads();
   float4* out = reinterpret_cast<float4*>(a.part_acc) + (size_t)(h * a.nslices + sl) * ncoord;
-  for (int base = 0; base < ncoord; base += NT) {   // one round unless ngroups * d > 256
-    const int item = tid;
-    const int oc = base + (nrep > 1 ? item % ncoord : item), ph = nrep > 1 ? item / ncoord : 0;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    const bool live = oc < ncoord && ph < nrep;
-    if (live) {
-      const int gi = oc / d, c = oc % d;
-      const GroupDev& g = a.g[gi];
-      const int bit = c * g.v_bits, bo = bit >> 3, sh = bit & 7, rb = g.v_idx_rb;
-      const uint32_t mask = (1u << g.v_bits) - 1u;
-      const bool two = sh + g.v_bits > 8;
-      const float* ct = vcent + gi * 16;
-      const unsigned char* vb = vbuf + g.v_idx_soff + bo;
-      const float4* wg = wvg + gi * SLICE;
-#pragma unroll 4
-      for (int tl = ph; tl < ntok; tl += nrep) {
-        const unsigned char* p = vb + (size_t)tl * rb;
-        uint32_t x = p[0];
-        if (two) x |= (uint32_t)p[1] << 8;
-        const float cv = ct[(x >> sh) & mask];
-        const float4 w = wg[tl];
-        acc.x = fmaf(w.x, cv, acc.x); acc.y = fmaf(w.y, cv, acc.y); acc.z = fmaf(w.z, cv, acc.z); acc.w = fmaf(w.w, cv, acc.w);
-      }
-    }
-    if (nrep > 1) {   // add the token phases in a fixed order
-      accred[tid] = acc;
-      __syncthreads();
-      if (tid < ncoord) {
-        float4 s = accred[tid];
-        for (int r = 1; r < nrep; ++r) add4(s, accred[r * ncoord + tid]);
-        out[tid] = s;
-      }
-      __syncthreads();
-    } else if (live) {
-      out[oc] = acc;
-    }
+  for (int oc = tid; oc < ncoord; oc += NT) {
+    float4 sacc = rbuf[oc];
+    for (int r = 1; r < nrep; ++r) add4(sacc, rbuf[(size_t)r * ncoord + oc]);
+    out[oc] = sacc;
   }
 }
 
@@ -415,7 +436,7 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   const int d = groups[0].plan_k ? groups[0].plan_k->d : 0;
   TQ_REQUIRE(d >= 8 && d <= MAXD && d % 8 == 0, TQ_ERR_UNSUPPORTED, "%s: group dimension %d (multiples of 8 up to %d)", who, d, MAXD);
   TQ_REQUIRE(ldq >= 1 && ldo >= 1, TQ_ERR_INVALID_ARG, "%s: bad row stride", who);
-  int lut = 0, kbytes = 0, vbytes = 0;
+  int lut = 0, kbytes = 0, vbytes = 0, vunits = 0;
   for (int gi = 0; gi < ngroups; ++gi) {
     const tq_kv_group& s = groups[gi];
     TQ_REQUIRE(s.plan_k && s.plan_v, TQ_ERR_INVALID_ARG, "%s: group %d has no plan", who, gi);
@@ -447,6 +468,8 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
     kbytes += (g.k_bits > 0 ? SLICE * g.k_idx_rb + 15 : 0) / 16 * 16;
     g.k_qjl_soff = kbytes;
     kbytes += (prod ? SLICE * g.k_qjl_rb + 15 : 0) / 16 * 16;
+    g.vunit0 = vunits;
+    vunits += vunits_of(d, g.v_bits);
     g.v_idx_soff = vbytes;
     vbytes += (SLICE * g.v_idx_rb + 15) / 16 * 16;
   }
@@ -464,6 +487,8 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   a.ngroups = ngroups; a.heads = heads; a.qpk = q_per_kv; a.d = d; a.nslices = (int)nslices;
   a.tokens = tokens; a.scale = scale; a.lut_float4 = lut;
   a.kbuf_bytes = kbytes; a.vbuf_bytes = vbytes;
+  a.vunits = vunits;
+  a.region0 = std::max(lut + SLICE, std::max(1, NT / vunits) * ngroups * d);
   char* w = static_cast<char*>(workspace);
   a.qrot = reinterpret_cast<float*>(w);
   size_t off = (size_t)heads * ngroups * MAXQ * 2 * MAXD * sizeof(float);
@@ -481,8 +506,8 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   else
     prepare_kernel<__nv_bfloat16><<<heads * ngroups, 128, 0, st>>>(a, static_cast<const __nv_bfloat16*>(Q), ldq);
   TQ_CHECK_CUDA(cudaGetLastError(), who);
-  const size_t smem = (size_t)lut * sizeof(float4) + (size_t)(1 + ngroups) * SLICE * sizeof(float4) + kbytes + vbytes +
-                      MAXG * 16 * sizeof(float) + (NT / 32 + 1) * MAXQ * sizeof(float) + NT * sizeof(float4);
+  const size_t smem = (size_t)a.region0 * sizeof(float4) + (size_t)ngroups * SLICE * sizeof(float4) + kbytes + vbytes +
+                      MAXG * 16 * sizeof(float) + (NT / 32 + 1) * MAXQ * sizeof(float);
   TQ_REQUIRE(smem <= 220 * 1024, TQ_ERR_UNSUPPORTED, "%s: %zu bytes of shared memory needed (too many wide groups)", who, smem);
   static size_t smem_set[16] = {0};
   if (dev < 16 && smem > smem_set[dev]) {
