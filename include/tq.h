@@ -262,19 +262,20 @@ int tq_softmax(const float* s1, const float* s2, int nw, int64_t n, int64_t lds,
  *
  * One tq_kv_group per channel group.  All plans share one dimension d (a multiple of 8, <= 128) and
  * one device; the key plan may be TQ_PROD or TQ_MSE, the value plan is TQ_MSE.  Code arrays hold the
- * rows of all heads, head-major: row h * tokens + t.  All pointers are device pointers owned by the
- * caller; nothing is retained after the call.
+ * rows of all heads, head-major: row h * head_stride + t, head_stride >= tokens being the capacity of
+ * the cache.  All pointers are device pointers owned by the caller; nothing is retained after the call.
+ * tq_attend_decode only reads the code arrays, tq_kv_append writes one row per head.
  */
 #define TQ_MAX_KV_GROUPS 4
 typedef struct tq_kv_group {
   const tq_plan* plan_k;
   const tq_plan* plan_v;
-  const uint8_t* k_idx;       /* [heads*tokens, tq_idx_row_bytes(d, b_m of plan_k)], 4-byte aligned; NULL if b_m = 0 */
-  const uint8_t* k_qjl;       /* [heads*tokens, tq_qjl_row_bytes(d)] (TQ_PROD), 4-byte aligned, else NULL */
-  const float* k_gamma;       /* [heads*tokens] residual norms (TQ_PROD), else NULL */
-  const float* k_norms;       /* [heads*tokens] key norms, or NULL for unit norms */
-  const uint8_t* v_idx;       /* [heads*tokens, tq_idx_row_bytes(d, b of plan_v)] */
-  const float* v_norms;       /* [heads*tokens] value norms, or NULL */
+  uint8_t* k_idx;       /* [heads*head_stride, tq_idx_row_bytes(d, b_m of plan_k)], 4-byte aligned; NULL if b_m = 0 */
+  uint8_t* k_qjl;       /* [heads*head_stride, tq_qjl_row_bytes(d)] (TQ_PROD), 4-byte aligned, else NULL */
+  float* k_gamma;       /* [heads*head_stride] residual norms (TQ_PROD), else NULL */
+  float* k_norms;       /* [heads*head_stride] key norms, or NULL for unit norms */
+  uint8_t* v_idx;       /* [heads*head_stride, tq_idx_row_bytes(d, b of plan_v)] */
+  float* v_norms;       /* [heads*head_stride] value norms, or NULL */
   const int32_t* k_channels;  /* [heads, d] column of Q that is coordinate c of this group for KV head h */
   const int32_t* v_channels;  /* [heads, d] column of out that receives coordinate c of this group */
 } tq_kv_group;
@@ -283,15 +284,28 @@ typedef struct tq_kv_group {
 size_t tq_attend_decode_workspace_bytes(int ngroups, int heads, int64_t tokens, int d);
 
 /*   groups     host array of ngroups (1..TQ_MAX_KV_GROUPS) descriptors
+ *   tokens     tokens attended to (rows 0 .. tokens-1 of every head); head_stride >= tokens
  *   Q          device, [heads*q_per_kv rows, row stride ldq elements] of q_dtype (TQ_F32 / TQ_BF16); 1 <= q_per_kv <= 4
  *   out        device fp32, [heads*q_per_kv rows, row stride ldo]; only the columns named by v_channels are written
  *   workspace  device, 256-byte aligned, >= tq_attend_decode_workspace_bytes(...)
  * tokens == 0 writes zeros to those columns.  Results do not depend on timing (fixed reduction orders).
  * Errors: TQ_ERR_INVALID_ARG / _UNSUPPORTED / _ALIGNMENT / _WORKSPACE / _CUDA as for the other calls.
  */
-int tq_attend_decode(const tq_kv_group* groups, int ngroups, int heads, int64_t tokens, int q_per_kv,
+int tq_attend_decode(const tq_kv_group* groups, int ngroups, int heads, int64_t tokens, int64_t head_stride, int q_per_kv,
                      const void* Q, int q_dtype, int64_t ldq, float scale, float* out, int64_t ldo,
                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* Appends one token to a compressed KV cache (the streaming use of Section 4.3: keys and values are
+ * quantised as they are generated): for every KV head h and channel group, Quant_prod / Quant_mse
+ * (Algorithms 2 / 1) of the group's channels of K[h] and V[h], written to row h * head_stride + position
+ * of the group's code arrays (idx, qjl, gamma, norms; norms arrays may be NULL when unit norms are
+ * implied).  Same comparisons as tq_quantize_*: codes agree with them up to fp32 summation order.
+ *   K, V   device, [heads rows, row strides ldk / ldv elements] of kv_dtype (TQ_F32 / TQ_BF16), full head rows
+ * Errors: TQ_ERR_INVALID_ARG (NULL pointers, position outside [0, head_stride)), TQ_ERR_UNSUPPORTED,
+ * TQ_ERR_ALIGNMENT, TQ_ERR_CUDA.
+ */
+int tq_kv_append(const tq_kv_group* groups, int ngroups, int heads, int64_t head_stride, int64_t position,
+                 const void* K, const void* V, int kv_dtype, int64_t ldk, int64_t ldv, void* stream);
 
 #ifdef __cplusplus
 }

@@ -45,8 +45,9 @@ _SIGNATURES = {
     "tq_wsum": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                         c_void_p, c_int64, c_void_p, c_size_t, c_void_p]),
     "tq_attend_decode_workspace_bytes": (c_size_t, [c_int, c_int, c_int64, c_int]),
-    "tq_attend_decode": (c_int, [c_void_p, c_int, c_int, c_int64, c_int, c_void_p, c_int, c_int64, ctypes.c_float,
+    "tq_attend_decode": (c_int, [c_void_p, c_int, c_int, c_int64, c_int64, c_int, c_void_p, c_int, c_int64, ctypes.c_float,
                                  c_void_p, c_int64, c_void_p, c_size_t, c_void_p]),
+    "tq_kv_append": (c_int, [c_void_p, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p]),
 }
 
 
@@ -244,9 +245,7 @@ def tq_attend_decode_workspace_bytes(ngroups: int, heads: int, tokens: int, d: i
     return lib().tq_attend_decode_workspace_bytes(ngroups, heads, tokens, d)
 
 
-def tq_attend_decode(groups, heads: int, tokens: int, q_per_kv: int, Q, scale: float, out, workspace):
-    """groups: sequence of dicts with keys plan_k, plan_v (Plan) and k_idx, k_qjl, k_gamma, k_norms, v_idx,
-    v_norms, k_channels, v_channels (CUDA tensors or None); rows of all heads head-major."""
+def _kv_groups(groups):
     arr = (KvGroup * len(groups))()
     for dst, g in zip(arr, groups):
         dst.plan_k, dst.plan_v = g["plan_k"].handle, g["plan_v"].handle
@@ -255,10 +254,30 @@ def tq_attend_decode(groups, heads: int, tokens: int, q_per_kv: int, Q, scale: f
         for name in ("k_channels", "v_channels"):
             if g[name].dtype != torch.int32 or not g[name].is_contiguous():
                 raise ValueError(f"{name} must be a contiguous int32 tensor")
+    return arr
+
+
+def tq_attend_decode(groups, heads: int, tokens: int, q_per_kv: int, Q, scale: float, out, workspace, head_stride=None):
+    """groups: sequence of dicts with keys plan_k, plan_v (Plan) and k_idx, k_qjl, k_gamma, k_norms, v_idx,
+    v_norms, k_channels, v_channels (CUDA tensors or None); rows of all heads head-major, head_stride rows
+    per head (default: tokens)."""
+    arr = _kv_groups(groups)
     _, ldq = _rows(Q)
     _, ldo = _rows(out)
-    _check(lib().tq_attend_decode(ctypes.cast(arr, c_void_p), len(groups), heads, tokens, q_per_kv, _dev(Q), _dtype_code(Q),
+    _check(lib().tq_attend_decode(ctypes.cast(arr, c_void_p), len(groups), heads, tokens,
+                                  tokens if head_stride is None else head_stride, q_per_kv, _dev(Q), _dtype_code(Q),
                                   ldq, scale, _dev(out), ldo, *_scratch_args(workspace), _stream()))
+
+
+def tq_kv_append(groups, heads: int, head_stride: int, position: int, K, V):
+    """Quantises one new token per KV head (K, V: [heads, head_dim]) into row `position` of every head."""
+    arr = _kv_groups(groups)
+    _, ldk = _rows(K)
+    _, ldv = _rows(V)
+    if K.dtype != V.dtype:
+        raise ValueError("K and V must have one dtype")
+    _check(lib().tq_kv_append(ctypes.cast(arr, c_void_p), len(groups), heads, head_stride, position, _dev(K), _dev(V),
+                              _dtype_code(K), ldk, ldv, _stream()))
 
 
 def tq_select_topk(cand_scores, cand_ids, k: int, top_scores, top_ids):

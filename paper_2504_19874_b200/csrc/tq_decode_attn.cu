@@ -60,6 +60,7 @@ struct Args {
   GroupDev g[MAXG];
   int ngroups, heads, qpk, d, nslices;
   int64_t tokens;
+  int64_t head_stride;   // rows between consecutive heads in the code arrays (>= tokens)
   float scale;
   float* qrot;      // [heads, ngroups, MAXQ, 2*MAXD]
   float* part_ml;   // [heads, nslices, 2, MAXQ]      slice maximum, slice sum of exponentials
@@ -172,7 +173,7 @@ __global__ void __launch_bounds__(NT) partial_kernel(Args a) {
   const int h = blockIdx.x / a.nslices, sl = blockIdx.x % a.nslices;
   const int64_t t0 = (int64_t)sl * SLICE;
   const int ntok = (int)min((int64_t)SLICE, a.tokens - t0);
-  const int64_t row0 = (int64_t)h * a.tokens + t0;
+  const int64_t row0 = (int64_t)h * a.head_stride + t0;
   const int d = a.d, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   // ---- the slice's code rows travel to shared memory while the tables are built: every row is touched once,
@@ -401,6 +402,90 @@ __global__ void __launch_bounds__(256) merge_kernel(Args a, float* __restrict__ 
   }
 }
 
+
+// ------------------------------------------------------------------ append of one token per head
+struct AppendGroup {
+  uint8_t* k_idx; uint8_t* k_qjl; float* k_gamma; float* k_norms;
+  uint8_t* v_idx; float* v_norms;
+  const int32_t* k_channels; const int32_t* v_channels;
+  const float* k_backt; const float* k_sp; const float* v_backt;   // [d, ncat*dpad] (column j = row j of Pi), S' [d, d]
+  Codebook k_cb, v_cb;
+  int k_prod, k_idx_rb, k_qjl_rb, v_idx_rb, k_ncols, v_ncols;
+};
+struct AppendArgs {
+  AppendGroup g[MAXG];
+  int ngroups, heads, d;
+  int64_t head_stride, position;
+};
+
+// Quant_mse / Quant_prod (Algorithms 1, 2) of one d-vector by one CTA, thread j = rotated coordinate j, with the
+// comparisons the batch quantiser makes: y = Pi x, idx_j = #{i : y_j > t_i nu}, e = y / nu - c[idx],
+// z = sign(S' e), gamma = ||e||.
+template <typename T>
+__global__ void __launch_bounds__(MAXD) append_kernel(AppendArgs a, const T* __restrict__ K, int64_t ldk,
+                                                      const T* __restrict__ V, int64_t ldv) {
+  __shared__ float xs[MAXD], es[MAXD], red[4];
+  __shared__ uint32_t words[MAXD * 4 / 32 + 1];
+  const int h = blockIdx.x / a.ngroups, gi = blockIdx.x % a.ngroups, isv = blockIdx.y;
+  const AppendGroup& g = a.g[gi];
+  const int d = a.d, j = threadIdx.x, lane = j & 31, warp = j >> 5;
+  const int64_t row = (int64_t)h * a.head_stride + a.position;
+  const Codebook& cb = isv ? g.v_cb : g.k_cb;
+  const bool prod = !isv && g.k_prod;
+  const int bm = cb.bits;
+  auto block_sum = [&](float v) -> float {   // fixed order: lanes by shuffles, then the warps in turn
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    float s = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w];
+    return s;
+  };
+  float x = 0.f;
+  if (j < d) {
+    const int ch = (isv ? g.v_channels : g.k_channels)[h * d + j];
+    x = isv ? (float)V[(int64_t)h * ldv + ch] : (float)K[(int64_t)h * ldk + ch];
+  }
+  xs[j] = x;
+  if (j < (int)(sizeof(words) / sizeof(words[0]))) words[j] = 0u;
+  const float nu = sqrtf(block_sum(x * x));   // the sync inside also publishes xs and words
+  const float inv = nu > 0.f ? 1.f / nu : 0.f, vcmp = nu > 0.f ? nu : 1.f;
+  const float* bt = isv ? g.v_backt : g.k_backt;
+  const int ncols = isv ? g.v_ncols : g.k_ncols;
+  float y = 0.f;
+  if (j < d)
+    for (int c = 0; c < d; ++c) y = fmaf(bt[(size_t)c * ncols + j], xs[c], y);
+  int code = 0;
+  for (int t = 0; t < (1 << bm) - 1; ++t) code += (y > cb.t[t] * vcmp) ? 1 : 0;
+  if (j < d && bm > 0) {
+    const int bit = j * bm;
+    atomicOr(&words[bit >> 5], (uint32_t)code << (bit & 31));
+    if ((bit & 31) + bm > 32) atomicOr(&words[(bit >> 5) + 1], (uint32_t)code >> (32 - (bit & 31)));
+  }
+  const float e = (j < d && nu > 0.f) ? y * inv - cb.c[code] : 0.f;
+  es[j] = e;
+  float gamma = 0.f;
+  if (prod) gamma = sqrtf(block_sum(e * e)); else __syncthreads();
+  uint8_t* idx_row = (isv ? g.v_idx + (size_t)row * g.v_idx_rb : g.k_idx + (size_t)row * g.k_idx_rb);
+  const int idx_rb = isv ? g.v_idx_rb : g.k_idx_rb;
+  if (bm > 0 && j < idx_rb / 4) reinterpret_cast<uint32_t*>(idx_row)[j] = (j < (d * bm + 31) / 32) ? words[j] : 0u;
+  float* norms = isv ? g.v_norms : g.k_norms;
+  if (j == 0 && norms) norms[row] = nu;
+  if (prod) {
+    if (j == 0) g.k_gamma[row] = gamma;
+    float sp = 0.f;
+    if (j < d) {
+      const float* srow = g.k_sp + (size_t)j * d;
+      for (int c = 0; c < d; ++c) sp = fmaf(srow[c], es[c], sp);
+    }
+    const uint32_t bits = __ballot_sync(0xffffffffu, j < d && sp >= 0.f);
+    uint32_t* qrow = reinterpret_cast<uint32_t*>(g.k_qjl + (size_t)row * g.k_qjl_rb);
+    if (lane == 0 && warp < g.k_qjl_rb / 4) qrow[warp] = bits;
+  }
+}
+
 size_t workspace_bytes(int ngroups, int heads, int64_t tokens, int d) {
   const int64_t nslices = std::max<int64_t>(1, (tokens + SLICE - 1) / SLICE);
   size_t b = (size_t)heads * ngroups * MAXQ * 2 * MAXD * sizeof(float);
@@ -418,7 +503,7 @@ extern "C" size_t tq_attend_decode_workspace_bytes(int ngroups, int heads, int64
   return tq::kvdec::workspace_bytes(ngroups, heads, tokens, d);
 }
 
-extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int heads, int64_t tokens, int q_per_kv,
+extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int heads, int64_t tokens, int64_t head_stride, int q_per_kv,
                                 const void* Q, int q_dtype, int64_t ldq, float scale, float* out, int64_t ldo,
                                 void* workspace, size_t workspace_bytes, void* stream) {
   using namespace tq;
@@ -426,6 +511,8 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   const char* who = "tq_attend_decode";
   TQ_REQUIRE(groups != nullptr && ngroups >= 1 && ngroups <= MAXG, TQ_ERR_INVALID_ARG, "%s: 1..%d channel groups", who, MAXG);
   TQ_REQUIRE(heads >= 0 && tokens >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
+  TQ_REQUIRE(head_stride >= tokens, TQ_ERR_INVALID_ARG, "%s: head_stride %lld is smaller than tokens %lld", who,
+             (long long)head_stride, (long long)tokens);
   TQ_REQUIRE(q_per_kv >= 1 && q_per_kv <= MAXQ, TQ_ERR_UNSUPPORTED, "%s: 1..%d queries per KV head", who, MAXQ);
   TQ_REQUIRE(q_dtype == TQ_F32 || q_dtype == TQ_BF16, TQ_ERR_UNSUPPORTED, "%s: unknown query dtype %d", who, q_dtype);
   if (heads == 0) return TQ_OK;
@@ -485,7 +572,7 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
              workspace_bytes, need);
   TQ_REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255) == 0, TQ_ERR_ALIGNMENT, "%s: workspace is not 256-byte aligned", who);
   a.ngroups = ngroups; a.heads = heads; a.qpk = q_per_kv; a.d = d; a.nslices = (int)nslices;
-  a.tokens = tokens; a.scale = scale; a.lut_float4 = lut;
+  a.tokens = tokens; a.head_stride = head_stride; a.scale = scale; a.lut_float4 = lut;
   a.kbuf_bytes = kbytes; a.vbuf_bytes = vbytes;
   a.vunits = vunits;
   a.region0 = std::max(lut + SLICE, std::max(1, NT / vunits) * ngroups * d);
@@ -521,5 +608,56 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   merge_kernel<<<heads * q_per_kv, 256, 0, st>>>(a, out, ldo);
   TQ_CHECK_CUDA(cudaGetLastError(), who);
   count_launches(3);
+  return TQ_OK;
+}
+
+extern "C" int tq_kv_append(const tq_kv_group* groups, int ngroups, int heads, int64_t head_stride, int64_t position,
+                            const void* K, const void* V, int kv_dtype, int64_t ldk, int64_t ldv, void* stream) {
+  using namespace tq;
+  using namespace tq::kvdec;
+  const char* who = "tq_kv_append";
+  TQ_REQUIRE(groups != nullptr && ngroups >= 1 && ngroups <= MAXG, TQ_ERR_INVALID_ARG, "%s: 1..%d channel groups", who, MAXG);
+  TQ_REQUIRE(heads >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
+  TQ_REQUIRE(position >= 0 && position < head_stride, TQ_ERR_INVALID_ARG, "%s: position %lld outside [0, head_stride %lld)", who,
+             (long long)position, (long long)head_stride);
+  TQ_REQUIRE(kv_dtype == TQ_F32 || kv_dtype == TQ_BF16, TQ_ERR_UNSUPPORTED, "%s: unknown dtype %d", who, kv_dtype);
+  if (heads == 0) return TQ_OK;
+  TQ_REQUIRE(K != nullptr && V != nullptr, TQ_ERR_INVALID_ARG, "%s: K or V is NULL", who);
+  AppendArgs a;
+  std::memset(&a, 0, sizeof(a));
+  const int d = groups[0].plan_k ? groups[0].plan_k->d : 0;
+  TQ_REQUIRE(d >= 8 && d <= MAXD && d % 8 == 0, TQ_ERR_UNSUPPORTED, "%s: group dimension %d (multiples of 8 up to %d)", who, d, MAXD);
+  for (int gi = 0; gi < ngroups; ++gi) {
+    const tq_kv_group& s = groups[gi];
+    TQ_REQUIRE(s.plan_k && s.plan_v, TQ_ERR_INVALID_ARG, "%s: group %d has no plan", who, gi);
+    TQ_REQUIRE(s.plan_k->d == d && s.plan_v->d == d, TQ_ERR_UNSUPPORTED, "%s: all groups must share one dimension", who);
+    TQ_REQUIRE(s.plan_v->mode == TQ_MSE && s.plan_v->mse_bits >= 1, TQ_ERR_UNSUPPORTED,
+               "%s: values must be quantised with TurboQuant_mse", who);
+    const bool prod = s.plan_k->mode == TQ_PROD;
+    TQ_REQUIRE(s.k_channels && s.v_channels && s.v_idx, TQ_ERR_INVALID_ARG, "%s: group %d: NULL channel list or codes", who, gi);
+    TQ_REQUIRE(s.plan_k->mse_bits == 0 || s.k_idx, TQ_ERR_INVALID_ARG, "%s: group %d: k_idx is NULL", who, gi);
+    TQ_REQUIRE(!prod || (s.k_qjl && s.k_gamma), TQ_ERR_INVALID_ARG, "%s: group %d: k_qjl / k_gamma is NULL", who, gi);
+    TQ_REQUIRE(((reinterpret_cast<uintptr_t>(s.k_idx) | reinterpret_cast<uintptr_t>(s.k_qjl) | reinterpret_cast<uintptr_t>(s.v_idx)) & 3) == 0,
+               TQ_ERR_ALIGNMENT, "%s: group %d: codes are not 4-byte aligned", who, gi);
+    AppendGroup& g = a.g[gi];
+    g.k_idx = s.k_idx; g.k_qjl = s.k_qjl; g.k_gamma = s.k_gamma; g.k_norms = s.k_norms;
+    g.v_idx = s.v_idx; g.v_norms = s.v_norms;
+    g.k_channels = s.k_channels; g.v_channels = s.v_channels;
+    g.k_backt = s.plan_k->dBackT; g.k_sp = s.plan_k->dSp; g.v_backt = s.plan_v->dBackT;
+    g.k_cb = s.plan_k->cb; g.v_cb = s.plan_v->cb;
+    g.k_prod = prod ? 1 : 0;
+    g.k_idx_rb = (int)s.plan_k->idx_row_bytes; g.k_qjl_rb = (int)s.plan_k->qjl_row_bytes; g.v_idx_rb = (int)s.plan_v->idx_row_bytes;
+    g.k_ncols = s.plan_k->ncat * s.plan_k->dpad; g.v_ncols = s.plan_v->ncat * s.plan_v->dpad;
+  }
+  a.ngroups = ngroups; a.heads = heads; a.d = d; a.head_stride = head_stride; a.position = position;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const dim3 grid((unsigned)(heads * ngroups), 2);
+  if (kv_dtype == TQ_F32)
+    append_kernel<float><<<grid, MAXD, 0, st>>>(a, static_cast<const float*>(K), ldk, static_cast<const float*>(V), ldv);
+  else
+    append_kernel<__nv_bfloat16><<<grid, MAXD, 0, st>>>(a, static_cast<const __nv_bfloat16*>(K), ldk,
+                                                         static_cast<const __nv_bfloat16*>(V), ldv);
+  TQ_CHECK_CUDA(cudaGetLastError(), who);
+  count_launches(1);
   return TQ_OK;
 }

@@ -215,3 +215,65 @@ def test_fused_decode_other_bit_widths_and_argument_checks():
              "v_norms": recs[0]["V"][0][3][3], "k_channels": ch.to(torch.int32).repeat(1, 1), "v_channels": ch.to(torch.int32).repeat(1, 1)}
         tq.tq_attend_decode([g], 1, T, qpk, Q, 1.0, torch.empty((qpk, HEAD_DIM), device=DEV),
                             torch.empty(256, dtype=torch.uint8, device=DEV))
+
+
+def test_streaming_append_then_decode(groups):
+    """A cache of capacity 300 tokens per head: 200 tokens quantised in one batch, 10 more appended one at a
+    time with tq_kv_append; the appended rows against the oracle's quantiser and the batch quantiser, then
+    decode attention over the 210 tokens against the oracle."""
+    gK, gV = groups
+    heads, T0, T1, cap, qpk = 2, 200, 210, 300, 4
+    K, V, Q = wl.kv_cache(heads=heads, tokens=T1, q_per_kv=qpk, seed=21, device=DEV)
+    chK = [split_channels(K[h][:T0]) for h in range(heads)]
+    chV = [split_channels(V[h][:T0]) for h in range(heads)]
+    gds = []
+    for gi in range(2):
+        suk, suv = gK[gi], gV[gi]
+        gd = {"plan_k": suk.plan, "plan_v": suv.plan,
+              "k_idx": torch.zeros((heads * cap, suk.idx_rb), dtype=torch.uint8, device=DEV),
+              "k_qjl": torch.zeros((heads * cap, suk.qjl_rb), dtype=torch.uint8, device=DEV),
+              "k_gamma": torch.zeros(heads * cap, device=DEV), "k_norms": torch.zeros(heads * cap, device=DEV),
+              "v_idx": torch.zeros((heads * cap, suv.idx_rb), dtype=torch.uint8, device=DEV),
+              "v_norms": torch.zeros(heads * cap, device=DEV),
+              "k_channels": torch.stack([chK[h][gi] for h in range(heads)]).to(torch.int32).contiguous(),
+              "v_channels": torch.stack([chV[h][gi] for h in range(heads)]).to(torch.int32).contiguous()}
+        for h in range(heads):
+            ck = suk.quantize(K[h][:T0][:, chK[h][gi]].contiguous())
+            cv = suv.quantize(V[h][:T0][:, chV[h][gi]].contiguous())
+            r = slice(h * cap, h * cap + T0)
+            gd["k_idx"][r], gd["k_qjl"][r], gd["k_gamma"][r], gd["k_norms"][r] = ck
+            gd["v_idx"][r], gd["v_norms"][r] = cv[0], cv[3]
+        gds.append(gd)
+    for t in range(T0, T1):
+        tq.tq_kv_append(gds, heads, cap, t, K[:, t].contiguous(), V[:, t].contiguous())
+    torch.cuda.synchronize()
+    # the appended rows: against the oracle's quantiser (same criteria as the batch path) and the batch quantiser
+    recs = []
+    for h in range(heads):
+        rec = {"K": [], "V": []}
+        for gi in range(2):
+            suk, suv = gK[gi], gV[gi]
+            new = slice(h * cap + T0, h * cap + T1)
+            Xk = K[h][T0:T1][:, chK[h][gi]].contiguous()
+            Xv = V[h][T0:T1][:, chV[h][gi]].contiguous()
+            app_k = (gds[gi]["k_idx"][new].contiguous(), gds[gi]["k_qjl"][new].contiguous(),
+                     gds[gi]["k_gamma"][new].contiguous(), gds[gi]["k_norms"][new].contiguous())
+            app_v = (gds[gi]["v_idx"][new].contiguous(), None, None, gds[gi]["v_norms"][new].contiguous())
+            P.check_quantize(suk, Xk, *app_k)
+            P.check_quantize(suv, Xv, *app_v)
+            bk, bv = suk.quantize(Xk), suv.quantize(Xv)
+            assert (bk[0] != app_k[0]).float().mean() <= 0.01 and (bv[0] != app_v[0]).float().mean() <= 0.01
+            assert torch.allclose(bk[3], app_k[3], rtol=1e-6) and torch.allclose(bk[2], app_k[2], rtol=1e-4)
+            allr = slice(h * cap, h * cap + T1)
+            rec["K"].append((suk, chK[h][gi], K[h][:T1][:, chK[h][gi]], tuple(gds[gi][k][allr].contiguous() for k in ("k_idx", "k_qjl", "k_gamma", "k_norms"))))
+            rec["V"].append((suv, chV[h][gi], V[h][:T1][:, chV[h][gi]], (gds[gi]["v_idx"][allr].contiguous(), None, None, gds[gi]["v_norms"][allr].contiguous())))
+        recs.append(rec)
+    ws = torch.empty(tq.tq_attend_decode_workspace_bytes(2, heads, T1, GROUP), dtype=torch.uint8, device=DEV)
+    out = torch.zeros((heads * qpk, HEAD_DIM), device=DEV)
+    tq.tq_attend_decode(gds, heads, T1, qpk, Q, 1.0 / math.sqrt(HEAD_DIM), out, ws, head_stride=cap)
+    torch.cuda.synchronize()
+    ref = np.concatenate([attend_oracle(recs[h], Q[qpk * h:qpk * h + qpk])[0] for h in range(heads)])
+    err = np.linalg.norm(P.as_f64(out) - ref, axis=1) / np.linalg.norm(ref, axis=1)
+    assert float(err.max()) <= 1e-3, float(err.max())
+    with pytest.raises(tq.TqError):
+        tq.tq_kv_append(gds, heads, cap, cap, K[:, 0].contiguous(), V[:, 0].contiguous())   # position outside the cache
