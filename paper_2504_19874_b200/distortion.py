@@ -85,6 +85,37 @@ def measure(d: int = 1536, n: int = 20000, nq: int = 8, device: str = "cuda:0", 
     return out
 
 
+def recall_1_at_k(d: int = 1536, n: int = 100000, nq: int = 256, bits=(2, 4), ks=(1, 2, 4, 8, 16, 32, 64),
+                  device: str = "cuda:0", seed: int = 0):
+    """Recall 1@k of nearest-neighbour search by inner product (the measure of the paper's nearest-neighbour
+    experiments): the fraction of queries whose exact top-1 vector (fp32 scan of the original rows) is among the
+    k best of tq_topk on the TurboQuant_prod codes.  Returns {b: {k: recall}}."""
+    dev = torch.device(device)
+    Pi = tq.tq_rotation(d, 42 + seed)
+    S = tq.tq_rotation(d, 43 + seed, tq.TQ_GAUSSIAN)
+    X = _unit_rows(n, d, 1 + seed, dev)
+    Q = _unit_rows(nq, d, 1001 + seed, dev)
+    truth = torch.argmax(Q @ X.T, dim=1)
+    kmax = max(ks)
+    out = {}
+    for b in bits:
+        cent, _ = tq.tq_codebook(d, b - 1)
+        plan = tq.Plan(d, b, tq.TQ_PROD, Pi, S, cent)
+        idx = torch.empty((n, max(plan.idx_row_bytes, 1)), dtype=torch.uint8, device=dev)
+        qjl = torch.empty((n, plan.qjl_row_bytes), dtype=torch.uint8, device=dev)
+        gamma = torch.empty(n, device=dev)
+        norms = torch.empty(n, device=dev)
+        scratch = torch.empty(max(tq.tq_workspace_bytes(plan, tq.TQ_OP_QUANTIZE, n), 16), dtype=torch.uint8, device=dev)
+        tq.tq_quantize_prod(plan, X, idx, qjl, gamma, norms, scratch)
+        ts = torch.empty((nq, kmax), device=dev)
+        ti = torch.empty((nq, kmax), dtype=torch.int32, device=dev)
+        ws = torch.empty(max(tq.tq_workspace_bytes(plan, tq.TQ_OP_TOPK, n, nq, kmax), 16), dtype=torch.uint8, device=dev)
+        tq.tq_topk(plan, Q, n, idx, qjl, gamma, norms, kmax, ts, ti, ws)
+        hit = ti.long() == truth[:, None]
+        out[b] = {k: float(hit[:, :k].any(dim=1).float().mean()) for k in ks}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--d", type=int, default=1536)
@@ -97,6 +128,10 @@ def main():
     for b, v in r.items():
         print(f" {b}  {v['dmse']:.4f}  [{4.0 ** -b:.4f}, {2.7207 * 4.0 ** -b:.4f}]   {v['dprod_times_d']:8.4f}   "
               f"{v['prod_bias']:+.2e} ({v['prod_bias_sigma']:.1e})   {v['prod_slope']:.4f}      {v['mse_estimator_slope']:.4f}")
+    rec = recall_1_at_k(args.d)
+    print("recall 1@k of tq_topk on TurboQuant_prod codes (100,000 embedding-like rows, 256 queries):")
+    for b, v in rec.items():
+        print(f" b = {b}: " + "  ".join(f"1@{k} = {x:.3f}" for k, x in v.items()))
 
 
 if __name__ == "__main__":

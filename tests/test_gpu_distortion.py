@@ -52,3 +52,14 @@ def test_distortion_is_data_oblivious():
     for b in (1, 2, 3, 4):
         assert abs(ani[b]["dmse"] / iso[b]["dmse"] - 1) < 0.03
         assert abs(ani[b]["dprod_times_d"] / iso[b]["dprod_times_d"] - 1) < 0.15
+
+
+def test_recall_grows_with_k_and_with_bits():
+    """Recall 1@k of tq_topk against an exact fp32 scan (the measure of the paper's nearest-neighbour
+    experiments) on synthetic embedding-like rows: monotone in k, better with more bits, complete by k = 64 at 4 bits."""
+    rec = distortion.recall_1_at_k(d=1536, n=50000, nq=128)
+    for b in (2, 4):
+        vals = [rec[b][k] for k in sorted(rec[b])]
+        assert all(x <= y + 1e-9 for x, y in zip(vals, vals[1:]))
+    assert all(rec[4][k] >= rec[2][k] for k in rec[2])
+    assert rec[4][1] >= 0.6 and rec[4][64] == 1.0 and rec[2][64] >= 0.95
