@@ -44,6 +44,7 @@ def parse_args():
     ap.add_argument("--nq", type=int, default=WORKLOAD["nq"])
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kv", action="store_true", help="run the KV-cache decode leg even when --n is reduced (profiling runs)")
     return ap.parse_args()
 
 
@@ -307,7 +308,7 @@ def run_b200(args):
     # ---- KV-cache decode (config c3): one layer = 8 KV heads x 32768 tokens, 2.5 bits per channel, 32 query heads;
     #      32 layer copies so that the codes (0.94 GB) exceed L2; tq_attend_decode, one call per layer ----
     kv = None
-    if n == WORKLOAD["n"]:
+    if n == WORKLOAD["n"] or args.kv:
         import math
         Kc, Vc, Qc = wl.kv_cache(device=dev)
         Hh, Tt, hd = Kc.shape

@@ -32,7 +32,7 @@ namespace kvdec {
 constexpr int MAXG = TQ_MAX_KV_GROUPS;
 constexpr int MAXQ = 4;          // queries per KV head (one float4 of partial sums)
 constexpr int MAXD = 128;        // channels per group
-constexpr int SLICE = 512;       // tokens per CTA
+constexpr int SLICE = 256;       // tokens per CTA
 constexpr int NT = 256;          // threads per CTA
 
 struct GroupDev {
