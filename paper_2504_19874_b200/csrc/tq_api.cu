@@ -279,11 +279,14 @@ template <typename T>
 cudaError_t launch_rotate_queries(const tq_plan* plan, const T* Q, int64_t ldq, int nq, float* Qcat, cudaStream_t st) {
   const int ncols = plan->ncat * plan->dpad;
   constexpr int smem = kRotQ * kRotChunk * (int)sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
+  // function attributes are per device: remember the devices this launcher has prepared
+  static unsigned long long attr_devices = 0;
+  int attr_dev = 0;
+  if (cudaGetDevice(&attr_dev) != cudaSuccess) return cudaErrorInvalidDevice;
+  if (attr_dev >= 64 || !((attr_devices >> attr_dev) & 1ull)) {
     cudaError_t e = cudaFuncSetAttribute(rotate_queries_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    if (attr_dev < 64) attr_devices |= 1ull << attr_dev;
   }
   const dim3 grid((unsigned)((ncols + 7) / 8), (unsigned)((nq + kRotQPerBlock - 1) / kRotQPerBlock));
   rotate_queries_kernel<T><<<grid, 256, smem, st>>>(plan->dRotCat, ncols, plan->d, Q, ldq, nq, Qcat, ncols);

@@ -404,11 +404,14 @@ template <int BN, int MODE, int BITS>
 cudaError_t launch_gemm_t(const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b1, const CUtensorMap& b2,
                           const GemmArgs& args, cudaStream_t st) {
   auto kern = quantize_gemm_kernel<BN, MODE, BITS>;
-  static bool attr_set = false;
-  if (!attr_set) {
+  // function attributes are per device: remember the devices this launcher has prepared
+  static unsigned long long attr_devices = 0;
+  int attr_dev = 0;
+  if (cudaGetDevice(&attr_dev) != cudaSuccess) return cudaErrorInvalidDevice;
+  if (attr_dev >= 64 || !((attr_devices >> attr_dev) & 1ull)) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    if (attr_dev < 64) attr_devices |= 1ull << attr_dev;
   }
   const int64_t tiles = (int64_t)args.tiles_m * args.tiles_n;
   const int grid = (int)std::min<int64_t>(tiles, sm_count());

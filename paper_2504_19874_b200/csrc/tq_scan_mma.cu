@@ -740,11 +740,14 @@ bool pick_config(const tq_plan* plan, int NW, int MT, int NT, Config* out) {
 template <int BM, bool PROD, int NW, int MT, int NT, int MODE>
 cudaError_t launch_t(const CUtensorMap& mi, const CUtensorMap& mq, const ScanArgs& args, size_t smem, cudaStream_t st) {
   auto kern = scan_mma_kernel<BM, PROD, NW, MT, NT, MODE>;
-  static size_t attr = 0;
-  if (smem > attr) {
+  // function attributes are per device: the largest size set so far, per device
+  static size_t attr[64] = {0};
+  int attr_dev = 0;
+  if (cudaGetDevice(&attr_dev) != cudaSuccess) return cudaErrorInvalidDevice;
+  if (attr_dev >= 64 || smem > attr[attr_dev]) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr = smem;
+    if (attr_dev < 64) attr[attr_dev] = smem;
   }
   const int grid = (int)std::min<int64_t>(args.ntiles, tc::sm_count());
   kern<<<grid, 32 * (NW + 1), smem, st>>>(mi, mq, args);

@@ -626,11 +626,14 @@ template <int BM, int MODE>
 cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
                      const ScanArgs& args, cudaStream_t st) {
   auto kern = scan_tc_kernel<BM, MODE>;
-  static bool attr_set = false;
-  if (!attr_set) {
+  // function attributes are per device: remember the devices this launcher has prepared
+  static unsigned long long attr_devices = 0;
+  int attr_dev = 0;
+  if (cudaGetDevice(&attr_dev) != cudaSuccess) return cudaErrorInvalidDevice;
+  if (attr_dev >= 64 || !((attr_devices >> attr_dev) & 1ull)) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    if (attr_dev < 64) attr_devices |= 1ull << attr_dev;
   }
   const int grid = (int)std::min<int64_t>(args.npairs, tc::sm_count());
   kern<<<grid, NTHREADS, kSmemBytes, st>>>(ma, ms, pa, ps, args);
