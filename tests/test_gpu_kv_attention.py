@@ -191,9 +191,9 @@ def test_fused_decode_against_the_oracle(groups, heads, T, qpk):
 
 def test_fused_decode_other_bit_widths_and_argument_checks():
     # one group of 128 channels: keys TurboQuant_mse 4-bit (no QJL part), values 4-bit; then keys prod 4-bit (3-bit indices)
-    for kbits, kmode in ((4, tq.TQ_MSE), (4, tq.TQ_PROD), (1, tq.TQ_PROD)):
+    for kbits, kmode, vbits in ((4, tq.TQ_MSE, 4), (4, tq.TQ_PROD, 1), (1, tq.TQ_PROD, 2), (2, tq.TQ_MSE, 3)):
         gK = (P.Setup(HEAD_DIM, kbits, kmode, 81, 82),)
-        gV = (P.Setup(HEAD_DIM, 4, tq.TQ_MSE, 83, 84),)
+        gV = (P.Setup(HEAD_DIM, vbits, tq.TQ_MSE, 83, 84),)
         heads, T, qpk = 2, 1500, 2
         K, V, Q = wl.kv_cache(heads=heads, tokens=T, q_per_kv=qpk, seed=9, device=DEV)
         ch = torch.arange(HEAD_DIM, device=DEV)
@@ -208,7 +208,7 @@ def test_fused_decode_other_bit_widths_and_argument_checks():
         fused = P.as_f64(_fused_layer(gK, gV, recs, Q, heads, T, qpk))
         ref = np.concatenate(refs)
         err = np.linalg.norm(fused - ref, axis=1) / np.linalg.norm(ref, axis=1)
-        assert float(err.max()) <= 1e-3, (kbits, kmode, float(err.max()))
+        assert float(err.max()) <= 1e-3, (kbits, kmode, vbits, float(err.max()))
     with pytest.raises(tq.TqError):     # a workspace that is too small is refused
         g = {"plan_k": gK[0].plan, "plan_v": gV[0].plan, "k_idx": recs[0]["K"][0][3][0], "k_qjl": recs[0]["K"][0][3][1],
              "k_gamma": recs[0]["K"][0][3][2], "k_norms": recs[0]["K"][0][3][3], "v_idx": recs[0]["V"][0][3][0],
