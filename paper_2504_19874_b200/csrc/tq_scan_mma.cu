@@ -52,8 +52,8 @@ __host__ __device__ constexpr int ks_s(bool prod) { return prod ? 16 : 0; }
 
 // Per-query constants (computed inside bprep_kernel).
 struct QConst {
-  double sa, ca;   // a = T_a * sa + ca   (MSE term)
-  double ss, cs;   // s = T_s * ss + cs   (QJL term)
+  float sa, ca;    // a = T_a * sa + ca   (MSE term)
+  float ss, cs;    // s = T_s * ss + cs   (QJL term)
   int fa, fs;      // fixed-point exponents
   int pad[2];
 };
@@ -152,10 +152,10 @@ __device__ void query_constants(const BPrepArgs& a, QConst* sc /* shared, [kMaxP
       QConst c;
       c.fa = expo(2.0 * a.amax * mx1);
       c.fs = expo(2.0 * mx2);
-      c.sa = ldexp(1.0, -c.fa);
-      c.ss = ldexp(1.0, -c.fs);
-      c.ca = a.csum * sm1;
-      c.cs = -sm2;
+      c.sa = (float)ldexp(1.0, -c.fa);
+      c.ss = (float)ldexp(1.0, -c.fs);
+      c.ca = (float)(a.csum * sm1);
+      c.cs = (float)(-sm2);
       c.pad[0] = c.pad[1] = 0;
       sc[ql] = c;
       if (blockIdx.x == 0) a.qc[ql] = c;
@@ -481,8 +481,10 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
 
     // ---------------------------------------------------------------- epilogue
     // Thread (g, t4) holds columns 2 t4, 2 t4 + 1 of rows g and g + 8: two of the four digits of
-    // query t4 / 2.  The lane pair (t4, t4 ^ 1) adds its halves; the even lane then finishes row g,
-    // the odd lane row g + 8.
+    // query t4 / 2.  The digit sums are recombined exactly (T = D0 + 256 D1 + 65536 D2 + ... as a 64-bit
+    // integer, the same T in both engines although their digit sums differ), then everything is fp32: one
+    // rounding of T (2^-24 of sum |W|, three orders below the tolerance) and three FMAs.  The even lane of a
+    // pair finishes row g, the odd lane row g + 8: one 64-bit shuffle hands each the other's half.
 #pragma unroll
     for (int m = 0; m < MT; ++m) {
       const int64_t row0 = tile * VT + cw * (MT * 16) + m * 16;
@@ -491,27 +493,24 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
       const float nu = nu_pre[m], gm = gm_pre[m];
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        long long ta[2], ts[2];
+        auto combine = [&](const int (&acc)[2][4]) -> float {
+          long long mine[2];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          long long pa = (long long)(accA[m][nt][0][2 * h] + accA[m][nt][1][2 * h]) +
-                         ((long long)(accA[m][nt][0][2 * h + 1] + accA[m][nt][1][2 * h + 1]) << 8);
-          long long ps = (long long)(accS[m][nt][0][2 * h] + accS[m][nt][1][2 * h]) +
-                         ((long long)(accS[m][nt][0][2 * h + 1] + accS[m][nt][1][2 * h + 1]) << 8);
-          if (t4 & 1) {
-            pa <<= 16;
-            ps <<= 16;
+          for (int h = 0; h < 2; ++h) {   // digits (0, 1) on the even lane, (2, 3) on the odd lane, as one integer
+            const int lo = acc[0][2 * h] + acc[1][2 * h], hi = acc[0][2 * h + 1] + acc[1][2 * h + 1];
+            mine[h] = (long long)hi * 256 + lo;
           }
-          ta[h] = pa + shfl_xor_ll(pa, 1);
-          ts[h] = PROD ? ps + shfl_xor_ll(ps, 1) : 0;
-        }
+          const long long recv = shfl_xor_ll((t4 & 1) ? mine[0] : mine[1], 1);
+          const long long T = (t4 & 1) ? mine[1] * 65536 + recv : recv * 65536 + mine[0];
+          return (float)T;   // one rounding of the exact integer: the same value in both engines
+        };
+        const float Ta = combine(accA[m][nt]);
+        const float Ts = PROD ? combine(accS[m][nt]) : 0.f;
         const int ql = nt * 2 + (t4 >> 1);
-        const long long Ta = (t4 & 1) ? ta[1] : ta[0];
-        const long long Ts = (t4 & 1) ? ts[1] : ts[0];
         const QConst c = qcs[ql];
-        const double av = (BM > 0) ? (double)Ta * c.sa + c.ca : 0.0;
-        const double sv = PROD ? (double)Ts * c.ss + c.cs : 0.0;
-        const float est = (float)((double)nu * (av + (double)gm * sv));
+        const float av = (BM > 0) ? fmaf(Ta, c.sa, c.ca) : 0.f;
+        const float sv = PROD ? fmaf(Ts, c.ss, c.cs) : 0.f;
+        const float est = __fmul_rn(nu, fmaf(gm, sv, av));
         if (row_ok && ql < a.nq_pass) {
           if (MODE == 0) {
             a.scores[(int64_t)ql * a.lds + row] = est;

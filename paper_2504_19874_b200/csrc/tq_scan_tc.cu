@@ -65,8 +65,8 @@ constexpr int LBUF = 128;              // candidates per query a CTA collects in
 constexpr size_t kConstBytes = 256 * 48;             // per-query constants of one group
 
 struct QConst {
-  double sa, ca;   // a = T_a * sa + ca   (MSE term)
-  double ss, cs;   // s = T_s * ss + cs   (QJL term)
+  float sa, ca;    // a = T_a * sa + ca   (MSE term)
+  float ss, cs;    // s = T_s * ss + cs   (QJL term)
   int fa, fs;
   int pad[2];
 };
@@ -171,10 +171,10 @@ __global__ void __launch_bounds__(256) tstats_kernel(StatArgs a) {
     QConst c;
     c.fa = expo(2.0 * a.amax * mx1);
     c.fs = expo(2.0 * mx2);
-    c.sa = ldexp(1.0, -c.fa);
-    c.ss = ldexp(1.0, -c.fs);
-    c.ca = a.csum * sm1;
-    c.cs = -sm2;
+    c.sa = (float)ldexp(1.0, -c.fa);
+    c.ss = (float)ldexp(1.0, -c.fs);
+    c.ca = (float)(a.csum * sm1);
+    c.cs = (float)(-sm2);
     c.pad[0] = c.pad[1] = 0;
     a.out[blockIdx.x] = c;
   }
@@ -330,7 +330,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
     if (a.g.kbs > 0) tc::tma_prefetch_desc(&tmPs);
   }
   if (threadIdx.x < kQueriesPerPass) {
-    QConst c = {1.0, 0.0, 1.0, 0.0, 0, 0, {0, 0}};
+    QConst c = {1.f, 0.f, 1.f, 0.f, 0, 0, {0, 0}};
     if ((int)threadIdx.x < a.nqp) c = a.qc[threadIdx.x];
     qcs[threadIdx.x] = c;
     taus[threadIdx.x] = (MODE == 1 && (int)threadIdx.x < a.nqp) ? a.tau[threadIdx.x] : 0.f;
@@ -561,16 +561,18 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
 #pragma unroll
         for (int qq = 0; qq < 16; ++qq) {
           const int ql = h * 16 + qq;
-          long long Ta = 0, Ts = 0;
-#pragma unroll
-          for (int l = 0; l < LIMBS; ++l) {
-            if (a.g.kba > 0) Ta += (long long)(int)va[l][qq] << (8 * l);
-            if (a.g.kbs > 0) Ts += (long long)(int)vs[l][qq] << (8 * l);
-          }
+          // digits recombined exactly (64-bit integer: the same T as in the register-fed engine), then fp32
           const QConst c = qcs[ql];
-          const double av = (a.g.kba > 0) ? (double)Ta * c.sa + c.ca : 0.0;
-          const double sv = (a.g.kbs > 0) ? (double)Ts * c.ss + c.cs : 0.0;
-          const float est = (float)((double)nu * (av + (double)gm * sv));
+          float av = 0.f, sv = 0.f;
+          if (a.g.kba > 0) {
+            const long long T = ((long long)(int)va[2][qq] * 256 + (int)va[1][qq]) * 256 + (int)va[0][qq];
+            av = fmaf((float)T, c.sa, c.ca);
+          }
+          if (a.g.kbs > 0) {
+            const long long T = ((long long)(int)vs[2][qq] * 256 + (int)vs[1][qq]) * 256 + (int)vs[0][qq];
+            sv = fmaf((float)T, c.ss, c.cs);
+          }
+          const float est = __fmul_rn(nu, fmaf(gm, sv, av));
           if (row_ok && ql < a.nqp) {
             if (MODE == 0) {
               a.scores[(int64_t)ql * a.lds + row] = est;
