@@ -229,7 +229,11 @@ __global__ void __launch_bounds__(256) bprep_kernel(BPrepArgs a) {
     out[0] |= __shfl_xor_sync(0xffffffffu, out[0], o);
     out[1] |= __shfl_xor_sync(0xffffffffu, out[1], o);
   }
-  if ((tid8 & 7) == 0) a.out[tid] = make_uint2(out[0], out[1]);
+  // k-steps 2j and 2j + 1 of a lane sit side by side, so that the scan fetches both with one 16-byte load
+  if ((tid8 & 7) == 0) {
+    const int64_t pairbase = (tid >> 5) / 2 * 64;   // (nt, r, ks / 2) block of 32 lanes x 2 k-steps
+    a.out[pairbase + lane * 2 + (ks & 1)] = make_uint2(out[0], out[1]);
+  }
 }
 
 // ------------------------------------------------------------------ scan kernel
@@ -433,9 +437,10 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
           }
         }
 
-      const uint2* Bb[NT];
+      uint4 b4[NT];
+      const uint4* Bb[NT];   // per lane: the operands of k-steps 2j, 2j + 1 as one 16-byte piece
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt) Bb[nt] = Bs + ((size_t)(nt * a.R + r) * KS) * 32 + lane;
+      for (int nt = 0; nt < NT; ++nt) Bb[nt] = reinterpret_cast<const uint4*>(Bs + ((size_t)(nt * a.R + r) * KS) * 32) + lane;
 
 #pragma unroll
       for (int p = 0; p < WA / 2; ++p)
@@ -444,7 +449,10 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
           const uint32_t mk = 0x01010101u << k;
           uint2 b[NT];
 #pragma unroll
-          for (int nt = 0; nt < NT; ++nt) b[nt] = Bb[nt][(p * 8 + k) * 32];
+          for (int nt = 0; nt < NT; ++nt) {
+            if ((k & 1) == 0) b4[nt] = Bb[nt][((p * 8 + k) >> 1) * 32];
+            b[nt] = (k & 1) ? make_uint2(b4[nt].z, b4[nt].w) : make_uint2(b4[nt].x, b4[nt].y);
+          }
 #pragma unroll
           for (int m = 0; m < MT; ++m) {
             // k = 7 feeds the whole word (all eight bits of every byte): B carries the difference
@@ -464,7 +472,10 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
             const uint32_t mk = 0x01010101u << k;
             uint2 b[NT];
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) b[nt] = Bb[nt][(KSA + p * 8 + k) * 32];
+            for (int nt = 0; nt < NT; ++nt) {
+              if ((k & 1) == 0) b4[nt] = Bb[nt][((KSA + p * 8 + k) >> 1) * 32];
+              b[nt] = (k & 1) ? make_uint2(b4[nt].z, b4[nt].w) : make_uint2(b4[nt].x, b4[nt].y);
+            }
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
               const uint32_t a0 = (k == 7) ? z[m][0][2 * p] : (z[m][0][2 * p] & mk);
