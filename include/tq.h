@@ -274,7 +274,7 @@ typedef struct tq_kv_group {
   uint8_t* k_qjl;       /* [heads*head_stride, tq_qjl_row_bytes(d)] (TQ_PROD), 4-byte aligned, else NULL */
   float* k_gamma;       /* [heads*head_stride] residual norms (TQ_PROD), else NULL */
   float* k_norms;       /* [heads*head_stride] key norms, or NULL for unit norms */
-  uint8_t* v_idx;       /* [heads*head_stride, tq_idx_row_bytes(d, b of plan_v)] */
+  uint8_t* v_idx;       /* [heads*head_stride, tq_idx_row_bytes(d, b of plan_v)], 4-byte aligned */
   float* v_norms;       /* [heads*head_stride] value norms, or NULL */
   const int32_t* k_channels;  /* [heads, d] column of Q that is coordinate c of this group for KV head h */
   const int32_t* v_channels;  /* [heads, d] column of out that receives coordinate c of this group */

@@ -535,7 +535,7 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
     TQ_REQUIRE(s.k_channels && s.v_channels && s.v_idx, TQ_ERR_INVALID_ARG, "%s: group %d: NULL channel list or codes", who, gi);
     TQ_REQUIRE(s.plan_k->mse_bits == 0 || s.k_idx, TQ_ERR_INVALID_ARG, "%s: group %d: k_idx is NULL", who, gi);
     TQ_REQUIRE(!prod || (s.k_qjl && s.k_gamma), TQ_ERR_INVALID_ARG, "%s: group %d: k_qjl / k_gamma is NULL", who, gi);
-    TQ_REQUIRE((reinterpret_cast<uintptr_t>(s.k_idx) & 3) == 0 && (reinterpret_cast<uintptr_t>(s.k_qjl) & 3) == 0,
+    TQ_REQUIRE(((reinterpret_cast<uintptr_t>(s.k_idx) | reinterpret_cast<uintptr_t>(s.k_qjl) | reinterpret_cast<uintptr_t>(s.v_idx)) & 3) == 0,
                TQ_ERR_ALIGNMENT, "%s: group %d: codes are not 4-byte aligned", who, gi);
     GroupDev& g = a.g[gi];
     g.k_idx = s.k_idx; g.k_qjl = s.k_qjl; g.k_gamma = s.k_gamma; g.k_norms = s.k_norms;

@@ -597,6 +597,7 @@ __global__ void __launch_bounds__(1024) select_kernel(SelArgs a) {
     }
   }
   int kk = min(a.k, total);
+  const int k_target = kk;
   unsigned long long prefix = 0ull;
   int shift = 56;
   if (kk > 0) {
@@ -649,7 +650,9 @@ __global__ void __launch_bounds__(1024) select_kernel(SelArgs a) {
             if (cum < kk && cum + c[e] >= kk) {
               s_prefix = (prefix << 8) | (unsigned long long)(255 - 8 * tid - e);
               s_kk = kk - cum;
-              s_done = (c[e] == kk - cum);
+              // stop when the bucket is exactly what is missing, or when everything at or above it fits the
+              // final sort, which then settles the order (further rounds would only narrow a small set)
+              s_done = (c[e] == kk - cum) || (k_target - (kk - cum) + c[e] <= 1024);
             }
             cum += c[e];
           }
