@@ -307,6 +307,45 @@ def run_b200(args):
               "score_frac_hbm": code_bytes2 / (ms_s2 * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     del idx2, norms2, scratch2, ws2, sc2, plan2
 
+    # ---- the other vector configurations at full size: quantise time and scan times (c2: d = 200, b = 3;
+    #      c5: d = 3072, b = 2 and 4), each with its own inputs ----
+    other = None
+    if n == WORKLOAD["n"] and world == 1:
+        other = []
+        for cname, cbits, ck in (("c2", 3, 100), ("c5", 2, 10), ("c5", 4, 100)):
+            cc = wl.CONFIGS[cname]
+            dd, nn = cc.d, cc.n
+            cent_c, _ = tq.tq_codebook(dd, cbits - 1)
+            plan_c = tq.Plan(dd, cbits, tq.TQ_PROD, tq.tq_rotation(dd, cc.pi_seed), tq.tq_rotation(dd, cc.s_seed, tq.TQ_GAUSSIAN), cent_c)
+            Xc = wl.make_vectors(cc, nn, cc.data_seed, dev)
+            Qc8 = wl.queries(cc, 8, dev)
+            Qc256 = wl.make_vectors(cc, 256, cc.query_seed + 7, dev)
+            ci = torch.empty((nn, max(plan_c.idx_row_bytes, 1)), dtype=torch.uint8, device=dev)
+            cq = torch.empty((nn, plan_c.qjl_row_bytes), dtype=torch.uint8, device=dev)
+            cg = torch.empty(nn, dtype=torch.float32, device=dev)
+            cn = torch.empty(nn, dtype=torch.float32, device=dev)
+            cs = torch.empty(max(tq.tq_workspace_bytes(plan_c, tq.TQ_OP_QUANTIZE, nn), 16), dtype=torch.uint8, device=dev)
+            cw = torch.empty(max(tq.tq_workspace_bytes(plan_c, tq.TQ_OP_TOPK, nn, 256, ck), 16), dtype=torch.uint8, device=dev)
+            ms_q = time_call(lambda: tq.tq_quantize_prod(plan_c, Xc, ci, cq, cg, cn, cs), reps=2)
+            torch.cuda.synchronize()
+            time.sleep(0.5)   # the scan is issue-bound: let the SM clock recover from the power-capped GEMMs before timing it
+            sc1 = torch.empty((1, nn), dtype=torch.float32, device=dev)
+            q1 = Qc8[:1].contiguous()
+            ms_s1 = time_call(lambda: tq.tq_score(plan_c, q1, nn, ci, cq, cg, cn, sc1, cw))
+            t_s = torch.empty((256, ck), dtype=torch.float32, device=dev)
+            t_i = torch.empty((256, ck), dtype=torch.int32, device=dev)
+            ms_t8 = time_call(lambda: tq.tq_topk(plan_c, Qc8, nn, ci, cq, cg, cn, ck, t_s[:8], t_i[:8], cw))
+            ms_t256 = time_call(lambda: tq.tq_topk(plan_c, Qc256, nn, ci, cq, cg, cn, ck, t_s, t_i, cw), reps=2)
+            cb = nn * (plan_c.idx_row_bytes + plan_c.qjl_row_bytes + 8)
+            other.append({"workload": f"{cname}: d={dd}, TurboQuant_prod b={cbits}, n={nn}, top-{ck}",
+                          "quantize_ms": ms_q, "quantize_vectors_per_s": nn / (ms_q * 1e-3),
+                          "quantize_frac_pass_adjusted": 3 * 4.0 * nn * dd * dd / (ms_q * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+                          "score_nq1_ms": ms_s1, "score_nq1_codes_gbs": cb / (ms_s1 * 1e-3) / 1e9,
+                          "score_nq1_frac_hbm": cb / (ms_s1 * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                          "topk_nq8_ms": ms_t8, "topk_nq256_ms": ms_t256, "topk_nq256_queries_per_s": 256 / (ms_t256 * 1e-3)})
+            del Xc, ci, cq, cg, cn, cs, cw, sc1, t_s, t_i, plan_c
+            torch.cuda.empty_cache()
+
     # ---- KV-cache decode (config c3): one layer = 8 KV heads x 32768 tokens, 2.5 bits per channel, 32 query heads;
     #      32 layer copies so that the codes (0.94 GB) exceed L2; tq_attend_decode, one call per layer ----
     kv = None
@@ -478,7 +517,7 @@ def run_b200(args):
             "quantize_vectors_per_s": n / (q_ms * 1e-3), "quantize_ms": q_ms,
             "scan_ms": s_ms, "scan_codes_gbs": scan_gbs, "scan_frac_hbm": scan_gbs / peaks["hbm_gbs"],
             "scan_queries_per_s": nq / (s_ms * 1e-3),
-            "scan_regimes": scan_regimes, "scan_many_queries": many_queries, "mse_b2": mse_b2, "kv_decode": kv, "roofline": roofline, "roofline_scan": roofline_scan, "clocks": clocks,
+            "scan_regimes": scan_regimes, "scan_many_queries": many_queries, "mse_b2": mse_b2, "kv_decode": kv, "other_configs": other, "roofline": roofline, "roofline_scan": roofline_scan, "clocks": clocks,
             "e2e": e2e, "gpu_launches": int(launches)}
     if not args.no_cpu_baseline:
         sample = 32768
