@@ -523,9 +523,14 @@ extern "C" size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int
     case TQ_OP_QUANTIZE:
       if (n == 0) return 0;
       if (plan->tc_ok)
-        return align_up((size_t)std::min<int64_t>(round_up64(n, 128), kTensorChunk) * tc::scratch_bytes_per_row(plan) +
-                            (n > kTensorChunk ? (size_t)kTensorChunk * plan->dpad * 4 : 0),   // second set of X limbs: lets blocks overlap
+      {
+        // rows per launch: 65,536 at d = 1536 and more for short rows (same scratch bytes), so that a launch of the
+        // persistent GEMM stays long against its prologue and the launch sequence
+        const int64_t chunk = std::min<int64_t>(kTensorChunk * std::max(1, 1536 / plan->dpad), 8 * kTensorChunk);
+        return align_up((size_t)std::min<int64_t>(round_up64(n, 128), chunk) * tc::scratch_bytes_per_row(plan) +
+                            (n > chunk ? (size_t)chunk * plan->dpad * 4 : 0),   // second set of X limbs: lets blocks overlap
                         256);
+      }
       if (plan->mode != TQ_PROD) return 0;
       return align_up((size_t)std::min<int64_t>(n, kResidualChunk) * plan->dpad * sizeof(float), 256);
     case TQ_OP_SCORE:
