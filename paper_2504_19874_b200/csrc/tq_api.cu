@@ -98,8 +98,9 @@ constexpr int64_t kDenseRowsMin = 4096;
 constexpr int kGroupQueries = tscan::kQueriesPerPass * tscan::kPassesPerGroup;
 
 // The two engines behind the bit-plane scan: register-fed integer MMA (2 or 4 queries per pass) for few
-// queries, tcgen05 (32 queries per pass) from 9 queries on (measured at d = 1536, b = 4, n = 10^6: one
-// tcgen05 pass 0.79 ms, one register-fed pass of 4 queries 0.39 ms, so three of those already cost more).
+// queries, tcgen05 (32 queries per pass) from 7 queries on (measured at d = 1536, b = 4, n = 10^6: a short
+// tcgen05 pass 0.69 ms, register-fed passes 0.24 ms for 1-2 queries and 0.37 ms for 3-4, so 4 + 3 queries
+// already cost more).
 struct ScanEngine {
   const tq_plan* plan;
   bool tc;
@@ -111,7 +112,7 @@ struct ScanEngine {
 ScanEngine pick_engine(const tq_plan* plan, int nq) {
   ScanEngine e;
   e.plan = plan;
-  e.tc = nq >= 9 && tscan::available(plan);
+  e.tc = nq >= 7 && tscan::available(plan);
   e.qpp = e.tc ? tscan::kQueriesPerPass : mscan::queries_per_pass(plan, nq);
   e.dense_rows_pref = e.tc ? (1 << 18) : (1 << 20);
   e.ws_bytes = e.tc ? tscan::workspace_bytes(plan) : mscan::workspace_bytes(plan);

@@ -551,6 +551,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(t * D_COLS);
 #pragma unroll 1
       for (int h = 0; h < 2; ++h) {   // 16 queries per half: digit l of query 16 h + qq sits in column 32 l + 16 h + qq
+        if (h * 16 >= a.nqp) break;   // a short last pass: columns of absent queries are not read
         uint32_t va[LIMBS][16], vs[LIMBS][16];
 #pragma unroll
         for (int l = 0; l < LIMBS; ++l) {
@@ -561,6 +562,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
 #pragma unroll
         for (int qq = 0; qq < 16; ++qq) {
           const int ql = h * 16 + qq;
+          if (ql >= a.nqp) break;
           // digits recombined exactly (64-bit integer: the same T as in the register-fed engine), then fp32
           const QConst c = qcs[ql];
           float av = 0.f, sv = 0.f;

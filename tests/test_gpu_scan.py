@@ -32,7 +32,7 @@ def test_scores_every_bit_width(d, bits, mode):
     P.check_scores(su, sc, Q, *codes)
 
 
-@pytest.mark.parametrize("nq", [1, 2, 3, 4, 7, 8, 9, 15])
+@pytest.mark.parametrize("nq", [1, 2, 3, 4, 6, 7, 8, 15])
 def test_scores_every_pass_shape_and_determinism(nq):
     d = 264
     su = P.Setup(d, 4, tq.TQ_PROD)
@@ -53,7 +53,7 @@ def test_scores_every_pass_shape_and_determinism(nq):
                                           (128, 1, tq.TQ_PROD), (200, 2, tq.TQ_PROD), (1536, 3, tq.TQ_PROD),
                                           (520, 4, tq.TQ_PROD), (264, 5, tq.TQ_PROD)])
 def test_many_query_engine_every_bit_width(d, bits, mode):
-    """Nine or more queries take the tcgen05 engine (32 queries per pass); its estimates equal the
+    """Seven or more queries take the tcgen05 engine (32 queries per pass); its estimates equal the
     few-query engine's bit for bit, and both match the oracle."""
     su = P.Setup(d, bits, mode)
     n, nq = 700, 37
