@@ -491,7 +491,8 @@ def run_b200(args):
     peaks = measured_peaks()
     q_ms = statistics.mean(phase_ms["quantize"])
     s_ms = statistics.mean(phase_ms["scan"])
-    passes = math.ceil(nq / (4 if nq > 2 else 2))  # the scan streams the codes once per tile of 2 (nq <= 2) or 4 queries
+    # the scan streams the codes once per pass: 2 queries (nq <= 2) or 4 (nq <= 6) on the register-fed engine, 32 on tcgen05
+    passes = math.ceil(nq / 32) if nq >= 7 else math.ceil(nq / (4 if nq > 2 else 2))
     scan_gbs = code_bytes * passes / (s_ms * 1e-3) / 1e9
     # Dominant kernels: the two d x d contractions of Quant_prod (4 n d^2 flops in all).
     gemm_flops = 4.0 * n * d * d
