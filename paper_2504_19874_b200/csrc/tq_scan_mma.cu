@@ -24,8 +24,8 @@
 // HBM -> shared memory in [rows x 64-byte] boxes (ring of stages, mbarrier full/empty, bounded
 // waits), each consumer thread pulls its 16-byte pieces into registers, frees the stage, derives the
 // parity words, and issues mma.sync.m16n8k32 (u8 x s8 -> s32) against B fragments resident in
-// shared memory.  The epilogue recombines the digit columns, applies gamma, nu and the per-query
-// constants in fp64 and either stores dense scores or appends (score, id) pairs that pass a
+// shared memory.  The epilogue recombines the digit columns exactly (64-bit integer), applies gamma, nu and
+// the per-query constants in fp32 and either stores dense scores or appends (score, id) pairs that pass a
 // per-query threshold to a candidate list (top-k).
 #include <algorithm>
 #include <cmath>
