@@ -20,7 +20,7 @@
 // permutation of the K axis is allowed as long as B is permuted alike, bits are consumed in
 // whatever order they sit in the registers; no coordinate is ever extracted.
 //
-// Kernel: persistent CTAs, one TMA producer warp + 8 consumer warps.  Packed rows travel
+// Kernel: persistent CTAs, one TMA producer warp + 12 or 16 consumer warps.  Packed rows travel
 // HBM -> shared memory in [rows x 64-byte] boxes (ring of stages, mbarrier full/empty, bounded
 // waits), each consumer thread pulls its 16-byte pieces into registers, frees the stage, derives the
 // parity words, and issues mma.sync.m16n8k32 (u8 x s8 -> s32) against B fragments resident in
