@@ -277,3 +277,43 @@ def test_streaming_append_then_decode(groups):
     assert float(err.max()) <= 1e-3, float(err.max())
     with pytest.raises(tq.TqError):
         tq.tq_kv_append(gds, heads, cap, cap, K[:, 0].contiguous(), V[:, 0].contiguous())   # position outside the cache
+
+
+def test_fused_decode_edge_cases(groups):
+    """No tokens (zero rows), fp32 queries with a row stride, an output with a row stride, and repeatability
+    across different head strides."""
+    gK, gV = groups
+    heads, T, qpk = 2, 300, 2
+    K, V, Q = wl.kv_cache(heads=heads, tokens=T, q_per_kv=qpk, seed=31, device=DEV)
+    recs = []
+    for h in range(heads):
+        _, _, rec = attend_gpu(gK, gV, K[h], V[h], Q[qpk * h:qpk * h + qpk])
+        recs.append(rec)
+    base = _fused_layer(gK, gV, recs, Q, heads, T, qpk)
+    # the same codes in a cache of larger capacity, fp32 queries inside a wider buffer, output inside a wider buffer
+    cap = 512
+    gds = []
+    for gi in range(2):
+        gd = {"plan_k": gK[gi].plan, "plan_v": gV[gi].plan}
+        for name, kind, i in (("k_idx", "K", 0), ("k_qjl", "K", 1), ("k_gamma", "K", 2), ("k_norms", "K", 3), ("v_idx", "V", 0), ("v_norms", "V", 3)):
+            src = [recs[h][kind][gi][3][i] for h in range(heads)]
+            buf = torch.zeros((heads * cap,) + tuple(src[0].shape[1:]), dtype=src[0].dtype, device=DEV)
+            for h in range(heads):
+                buf[h * cap:h * cap + T] = src[h]
+            gd[name] = buf
+        gd["k_channels"] = torch.stack([recs[h]["K"][gi][1] for h in range(heads)]).to(torch.int32).contiguous()
+        gd["v_channels"] = torch.stack([recs[h]["V"][gi][1] for h in range(heads)]).to(torch.int32).contiguous()
+        gds.append(gd)
+    Qw = torch.zeros((heads * qpk, HEAD_DIM + 24), device=DEV)
+    Qw[:, :HEAD_DIM] = Q.float()
+    outw = torch.full((heads * qpk, HEAD_DIM + 8), 5.0, device=DEV)
+    ws = torch.empty(tq.tq_attend_decode_workspace_bytes(2, heads, T, GROUP), dtype=torch.uint8, device=DEV)
+    tq.tq_attend_decode(gds, heads, T, qpk, Qw[:, :HEAD_DIM], 1.0 / math.sqrt(HEAD_DIM), outw[:, :HEAD_DIM], ws, head_stride=cap)
+    torch.cuda.synchronize()
+    assert torch.equal(outw[:, :HEAD_DIM], base)          # bf16 queries are exact in fp32: identical results
+    assert bool((outw[:, HEAD_DIM:] == 5.0).all())        # nothing written outside the named columns
+    out0 = torch.full((heads * qpk, HEAD_DIM), 3.0, device=DEV)
+    tq.tq_attend_decode(gds, heads, 0, qpk, Q, 1.0, out0, ws, head_stride=cap)
+    torch.cuda.synchronize()
+    assert not bool(out0.any())
+    tq.tq_attend_decode(gds, 0, T, qpk, Q, 1.0, out0, ws, head_stride=cap)   # no heads: nothing to do
