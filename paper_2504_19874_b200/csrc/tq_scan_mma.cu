@@ -241,6 +241,7 @@ struct ScanArgs {
   int64_t n;
   int64_t ntiles;
   int R, stages;
+  int idx_rb;              // bytes of one idx row (its tail may leave whole 64-byte blocks of the last range empty)
   const uint2* Bfrag;
   int bfrag_u2;            // uint2 elements of Bfrag (multiple of 32)
   const QConst* qc;        // constants of this pass's queries
@@ -442,8 +443,12 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) Bb[nt] = reinterpret_cast<const uint4*>(Bs + ((size_t)(nt * a.R + r) * KS) * 32) + lane;
 
+      // 64-byte blocks of this range that hold row bytes at all (short rows: d well below a multiple of 512);
+      // the others are zero fill, whose k-steps add nothing
+      const int nvalid = (BM == 3) ? BM : max(0, min(BM, (a.idx_rb - r * 64 * BM + 63) / 64));
 #pragma unroll
-      for (int p = 0; p < WA / 2; ++p)
+      for (int p = 0; p < WA / 2; ++p) {
+        if (BM != 3 && ((2 * p < NI ? 2 * p : 2 * p - NI) >> 2) >= nvalid) continue;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint32_t mk = 0x01010101u << k;
@@ -464,6 +469,7 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
             for (int nt = 0; nt < NT; ++nt) mma_u8s8(accA[m][nt][k & 1], a0, a1, a2, a3, b[nt].x, b[nt].y);
           }
         }
+      }
       if (PROD) {
 #pragma unroll
         for (int p = 0; p < 2; ++p)
@@ -906,6 +912,7 @@ int run(const tq_plan* plan, int nqp, int64_t n, const uint8_t* idx, const uint8
   sa.n = n;
   sa.ntiles = (n + VT - 1) / VT;
   sa.R = plan->ms.R;
+  sa.idx_rb = (int)plan->idx_row_bytes;
   sa.stages = c.stages;
   sa.Bfrag = reinterpret_cast<const uint2*>(static_cast<const char*>(workspace) + kQConstBytes);
   sa.bfrag_u2 = c.NT * plan->ms.R * (ks_a(bm) + ks_s(prod)) * 32;
