@@ -700,11 +700,13 @@ __global__ void __launch_bounds__(1024) select_kernel(SelArgs a) {
     }
   }
   __syncthreads();
-  // bitonic sort, descending
-  for (int kb = 2; kb <= 1024; kb <<= 1) {
+  // bitonic sort, descending, of the smallest power of two that holds the survivors (the rest of skey is zero)
+  int sort_n = 32;
+  while (sort_n < min(s_cnt, 1024)) sort_n <<= 1;
+  for (int kb = 2; kb <= sort_n; kb <<= 1) {
     for (int j = kb >> 1; j > 0; j >>= 1) {
       const int p = tid ^ j;
-      if (p > tid) {
+      if (p > tid && p < sort_n) {
         const unsigned long long x = skey[tid], y = skey[p];
         const bool desc = ((tid & kb) == 0);
         if (desc ? (x < y) : (x > y)) {
