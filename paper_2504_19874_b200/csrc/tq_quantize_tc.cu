@@ -21,7 +21,8 @@ namespace {
 constexpr int BM = 128;          // rows of X per tile = TMEM lanes
 constexpr int BK = 64;           // bf16 elements per 128-byte swizzled row
 constexpr int UMMA_K = 16;
-constexpr int NTHREADS = 320;    // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue (two per TMEM lane group)
+constexpr int EPS = 4;           // epilogue warps per TMEM lane group: each takes 1/EPS of the tile's columns
+constexpr int NTHREADS = 32 * (2 + 4 * EPS);   // warp 0: TMA, warp 1: MMA + TMEM owner, then the epilogue warps
 
 template <int BN>
 struct Cfg {
@@ -41,7 +42,7 @@ struct GemmArgs {
   __nv_bfloat16* E1;     // MODE 1: residual limbs, pitch ldE
   __nv_bfloat16* E2;
   int64_t ldE;
-  float* gpart;          // MODE 1: [2 * tiles_n][Mpad] partial sums of e^2 (one per half column tile)
+  float* gpart;          // MODE 1: [EPS * tiles_n][Mpad] partial sums of e^2 (one per epilogue warp's columns)
   int64_t Mpad;
   const float* nu;       // MODE 1: per-row norm (row with nu == 0 has residual 0); nullable
   int* status;
@@ -79,7 +80,7 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&tfull[i], 1);
-      mbar_init(&tempty[i], 8);
+      mbar_init(&tempty[i], 4 * EPS);
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -162,7 +163,7 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
   } else {
     // ------------------------------------------------------------ epilogue (8 warps: 4 TMEM lane groups x 2 column halves)
     const int lg = warp & 3;   // TMEM lane group this warp may read
-    const int half = (warp - 2) >> 2;   // which half of the tile's columns this warp takes
+    const int half = (warp - 2) >> 2;   // which part (of EPS) of the tile's columns this warp takes
     bool ok = true;
     int64_t it = 0;
     for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
@@ -179,7 +180,7 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
       uint32_t* out_row = reinterpret_cast<uint32_t*>(a.out + (size_t)(row_ok ? row : 0) * a.out_rb);
       const size_t row_words = a.out_rb / 4;
 #pragma unroll 1
-      for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
+      for (int c = half * (BN / 32 / EPS); c < (half + 1) * (BN / 32 / EPS); ++c) {
         const int col0 = n0 + c * 32;
         if (col0 >= a.N) break;   // uniform across the CTA: nothing but zero padding beyond
         uint32_t v[32];
@@ -256,9 +257,9 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tempty[acc]);
-      if (MODE == 1 && row_ok) a.gpart[(int64_t)(2 * tn + half) * a.Mpad + row] = gsum;
+      if (MODE == 1 && row_ok) a.gpart[(int64_t)(EPS * tn + half) * a.Mpad + row] = gsum;
       // pad words past the last tile's columns (rows whose stride exceeds the tiles' coverage)
-      if (tn == a.tiles_n - 1 && half == 1 && row_ok) {
+      if (tn == a.tiles_n - 1 && half == EPS - 1 && row_ok) {
         constexpr int kBitsPerCoord = (MODE == 2) ? 1 : BITS;
         if (kBitsPerCoord > 0) {
           const size_t covered = (size_t)((a.N + 31) >> 5) * kBitsPerCoord;
@@ -474,7 +475,7 @@ void free_matrix_limbs(MatrixLimbs* m) {
 size_t scratch_bytes_per_row(const tq_plan* plan) {
   const int tiles_n = (plan->d + plan->tc_bn - 1) / plan->tc_bn;
   size_t per = (size_t)plan->dpad * 2 * 2 + sizeof(float);                            // X limbs + nu
-  if (plan->mode == TQ_PROD) per += (size_t)plan->dpad * 2 * 2 + (size_t)tiles_n * 8;  // E limbs + partial sums (two per column tile)
+  if (plan->mode == TQ_PROD) per += (size_t)plan->dpad * 2 * 2 + (size_t)tiles_n * 4 * EPS;  // E limbs + partial sums (EPS per column tile)
   return per;
 }
 
@@ -496,7 +497,7 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
   if (prod) {
     EL1 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
     EL2 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
-    gpart = reinterpret_cast<float*>(p); p += (size_t)R * tiles_n * 8;
+    gpart = reinterpret_cast<float*>(p); p += (size_t)R * tiles_n * 4 * EPS;
   }
   p += (size_t)R * sizeof(float);
   const size_t xsz = (x_dtype == TQ_F32) ? 4 : 2;
@@ -582,7 +583,7 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     TQ_CHECK_CUDA(launch_gemm<1>(bn, plan->mse_bits, mA1, mA2, plan->pi_limbs.map_hi, plan->pi_limbs.map_lo, g, st), who);
     if (pipelined) TQ_CHECK_CUDA(cudaEventRecord(plan->ev_gemm[b], st), who);
     // 3. gamma = ||e||
-    gamma_finish_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(gpart, R, 2 * tiles_n, rows, gamma + r0);
+    gamma_finish_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(gpart, R, EPS * tiles_n, rows, gamma + r0);
     count_launches(1);
     TQ_CHECK_CUDA(cudaGetLastError(), who);
     // 4. qjl = sign(S' e)
