@@ -71,7 +71,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE,
+                                          "-lms", "25", "-i", str(self.gpu)], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -224,13 +224,15 @@ def run_b200(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    # the clock sampler starts before the warm-up steps (same work as the timed ones): nvidia-smi needs ~0.1 s to
+    # deliver its first sample, about as long as the timed region lasts
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     for _ in range(max(args.warmup, 3)):
         step(False)
     barrier()
     launches0 = tq.tq_launch_count()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     barrier()
     t_start = ev()
     t_end = ev()
