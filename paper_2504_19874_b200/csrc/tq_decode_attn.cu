@@ -115,6 +115,17 @@ __global__ void __launch_bounds__(128) prepare_kernel(Args a, const T* __restric
 __device__ __forceinline__ void add4(float4& a, const float4 b) {
   a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
 }
+// A table of E entries keeps the (x, y) halves of its float4 entries in one array of float2 and the (z, w) halves
+// in a second one behind it: lanes that read different entries of one table row then hit different banks
+// (16-byte entries collide pairwise), at the price of two loads per lookup.
+__device__ __forceinline__ void add_entry(float4& a, const float2* __restrict__ t2, int entries, int e) {
+  const float2 lo = t2[e], hi = t2[entries + e];
+  a.x += lo.x; a.y += lo.y; a.z += hi.x; a.w += hi.y;
+}
+__device__ __forceinline__ void put_entry(float2* t2, int entries, int e, float x, float y, float z, float w) {
+  t2[e] = make_float2(x, y);
+  t2[entries + e] = make_float2(z, w);
+}
 
 // Asynchronous copy of a contiguous run of code rows into shared memory (the whole CTA takes part).
 // Rows are 4-byte aligned; 16-byte pieces are used where the source allows.
@@ -206,7 +217,7 @@ __global__ void __launch_bounds__(NT) partial_kernel(Args a) {
 #pragma unroll
         for (int j = 0; j < MAXQ; ++j) s[j] = fmaf(q[j * 2 * MAXD + c], cent, s[j]);
       }
-      lut[g.lut_mse_off + e] = make_float4(s[0], s[1], s[2], s[3]);
+      put_entry(reinterpret_cast<float2*>(lut + g.lut_mse_off), nl * ne, e, s[0], s[1], s[2], s[3]);
     }
     if (g.k_prod) {
       for (int e = tid; e < (d / 4) * 16; e += NT) {
@@ -218,7 +229,7 @@ __global__ void __launch_bounds__(NT) partial_kernel(Args a) {
 #pragma unroll
           for (int j = 0; j < MAXQ; ++j) s[j] = fmaf(sg, q[j * 2 * MAXD + MAXD + 4 * L + u], s[j]);
         }
-        lut[g.lut_qjl_off + e] = make_float4(s[0], s[1], s[2], s[3]);
+        put_entry(reinterpret_cast<float2*>(lut + g.lut_qjl_off), (d / 4) * 16, e, s[0], s[1], s[2], s[3]);
       }
     }
     if (tid < 16) vcent[gi * 16 + tid] = g.v_cent[tid];
@@ -238,29 +249,31 @@ __global__ void __launch_bounds__(NT) partial_kernel(Args a) {
       float4 am = make_float4(0.f, 0.f, 0.f, 0.f), aq = make_float4(0.f, 0.f, 0.f, 0.f);
       if (g.k_bits == 3) {          // 8 coordinates per 3 bytes
         const uint8_t* p = kbuf + g.k_idx_soff + (size_t)tl * g.k_idx_rb;
-        const float4* tb = lut + g.lut_mse_off;
+        const float2* tb = reinterpret_cast<const float2*>(lut + g.lut_mse_off);
+        const int ent = d * 8;
         for (int c8 = 0; c8 < d / 8; ++c8) {
           const uint32_t x = (uint32_t)p[3 * c8] | ((uint32_t)p[3 * c8 + 1] << 8) | ((uint32_t)p[3 * c8 + 2] << 16);
 #pragma unroll
-          for (int u = 0; u < 8; ++u) add4(am, tb[(c8 * 8 + u) * 8 + ((x >> (3 * u)) & 7u)]);
+          for (int u = 0; u < 8; ++u) add_entry(am, tb, ent, (c8 * 8 + u) * 8 + (int)((x >> (3 * u)) & 7u));
         }
       } else if (g.k_bits > 0) {    // nibbles never straddle a word
         const uint32_t* p = reinterpret_cast<const uint32_t*>(kbuf + g.k_idx_soff + (size_t)tl * g.k_idx_rb);
-        const float4* tb = lut + g.lut_mse_off;
-        const int nw = d * g.k_bits / 32;
+        const float2* tb = reinterpret_cast<const float2*>(lut + g.lut_mse_off);
+        const int nw = d * g.k_bits / 32, ent = nw * 8 * 16;
         for (int w = 0; w < nw; ++w) {
           const uint32_t x = p[w];
 #pragma unroll
-          for (int u = 0; u < 8; ++u) add4(am, tb[(w * 8 + u) * 16 + ((x >> (4 * u)) & 15u)]);
+          for (int u = 0; u < 8; ++u) add_entry(am, tb, ent, (w * 8 + u) * 16 + (int)((x >> (4 * u)) & 15u));
         }
       }
       if (g.k_prod) {
         const uint32_t* p = reinterpret_cast<const uint32_t*>(kbuf + g.k_qjl_soff + (size_t)tl * g.k_qjl_rb);
-        const float4* tb = lut + g.lut_qjl_off;
+        const float2* tb = reinterpret_cast<const float2*>(lut + g.lut_qjl_off);
+        const int ent = (d / 4) * 16;
         for (int w = 0; w < d / 32; ++w) {
           const uint32_t x = p[w];
 #pragma unroll
-          for (int u = 0; u < 8; ++u) add4(aq, tb[(w * 8 + u) * 16 + ((x >> (4 * u)) & 15u)]);
+          for (int u = 0; u < 8; ++u) add_entry(aq, tb, ent, (w * 8 + u) * 16 + (int)((x >> (4 * u)) & 15u));
         }
       }
       score.x += nu * fmaf(cg, aq.x, am.x);
