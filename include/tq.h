@@ -260,7 +260,7 @@ int tq_softmax(const float* s1, const float* s2, int nw, int64_t n, int64_t lds,
  * evaluated on the packed codes: nothing is dequantised per token, Pi_V^T is applied once per output
  * row.  Equal to tq_score per (head, group) + tq_softmax + tq_wsum within fp32 rounding.
  *
- * One tq_kv_group per channel group.  All plans share one dimension d (a multiple of 8, <= 128) and
+ * One tq_kv_group per channel group.  All plans share one dimension d (a multiple of 32, <= 128) and
  * one device; the key plan may be TQ_PROD or TQ_MSE, the value plan is TQ_MSE.  Code arrays hold the
  * rows of all heads, head-major: row h * head_stride + t, head_stride >= tokens being the capacity of
  * the cache.  All pointers are device pointers owned by the caller; nothing is retained after the call.

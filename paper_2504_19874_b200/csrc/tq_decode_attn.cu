@@ -260,21 +260,35 @@ __global__ void __launch_bounds__(NT) partial_kernel(Args a) {
         const uint32_t* p = reinterpret_cast<const uint32_t*>(kbuf + g.k_idx_soff + (size_t)tl * g.k_idx_rb);
         const float2* tb = reinterpret_cast<const float2*>(lut + g.lut_mse_off);
         const int nw = d * g.k_bits / 32, ent = nw * 8 * 16;
-        for (int w = 0; w < nw; ++w) {
-          const uint32_t x = p[w];
+        auto word = [&](int w, uint32_t x) {
 #pragma unroll
           for (int u = 0; u < 8; ++u) add_entry(am, tb, ent, (w * 8 + u) * 16 + (int)((x >> (4 * u)) & 15u));
-        }
+        };
+        int w = 0;
+        if ((g.k_idx_rb & 7) == 0)   // 8-byte loads where the rows allow (4-byte loads at a 16-byte row stride collide 4-way)
+          for (; w + 1 < nw; w += 2) {
+            const uint2 xx = *reinterpret_cast<const uint2*>(p + w);
+            word(w, xx.x);
+            word(w + 1, xx.y);
+          }
+        for (; w < nw; ++w) word(w, p[w]);
       }
       if (g.k_prod) {
         const uint32_t* p = reinterpret_cast<const uint32_t*>(kbuf + g.k_qjl_soff + (size_t)tl * g.k_qjl_rb);
         const float2* tb = reinterpret_cast<const float2*>(lut + g.lut_qjl_off);
         const int ent = (d / 4) * 16;
-        for (int w = 0; w < d / 32; ++w) {
-          const uint32_t x = p[w];
+        auto word = [&](int w, uint32_t x) {
 #pragma unroll
           for (int u = 0; u < 8; ++u) add_entry(aq, tb, ent, (w * 8 + u) * 16 + (int)((x >> (4 * u)) & 15u));
-        }
+        };
+        int w = 0;
+        if ((g.k_qjl_rb & 7) == 0)
+          for (; w + 1 < d / 32; w += 2) {
+            const uint2 xx = *reinterpret_cast<const uint2*>(p + w);
+            word(w, xx.x);
+            word(w + 1, xx.y);
+          }
+        for (; w < d / 32; ++w) word(w, p[w]);
       }
       score.x += nu * fmaf(cg, aq.x, am.x);
       score.y += nu * fmaf(cg, aq.y, am.y);
@@ -534,7 +548,7 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   Args a;
   std::memset(&a, 0, sizeof(a));
   const int d = groups[0].plan_k ? groups[0].plan_k->d : 0;
-  TQ_REQUIRE(d >= 8 && d <= MAXD && d % 8 == 0, TQ_ERR_UNSUPPORTED, "%s: group dimension %d (multiples of 8 up to %d)", who, d, MAXD);
+  TQ_REQUIRE(d >= 32 && d <= MAXD && d % 32 == 0, TQ_ERR_UNSUPPORTED, "%s: group dimension %d (multiples of 32 up to %d)", who, d, MAXD);
   TQ_REQUIRE(ldq >= 1 && ldo >= 1, TQ_ERR_INVALID_ARG, "%s: bad row stride", who);
   int lut = 0, kbytes = 0, vbytes = 0, vunits = 0;
   for (int gi = 0; gi < ngroups; ++gi) {
@@ -639,7 +653,7 @@ extern "C" int tq_kv_append(const tq_kv_group* groups, int ngroups, int heads, i
   AppendArgs a;
   std::memset(&a, 0, sizeof(a));
   const int d = groups[0].plan_k ? groups[0].plan_k->d : 0;
-  TQ_REQUIRE(d >= 8 && d <= MAXD && d % 8 == 0, TQ_ERR_UNSUPPORTED, "%s: group dimension %d (multiples of 8 up to %d)", who, d, MAXD);
+  TQ_REQUIRE(d >= 32 && d <= MAXD && d % 32 == 0, TQ_ERR_UNSUPPORTED, "%s: group dimension %d (multiples of 32 up to %d)", who, d, MAXD);
   for (int gi = 0; gi < ngroups; ++gi) {
     const tq_kv_group& s = groups[gi];
     TQ_REQUIRE(s.plan_k && s.plan_v, TQ_ERR_INVALID_ARG, "%s: group %d has no plan", who, gi);
