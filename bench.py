@@ -499,9 +499,9 @@ def run_b200(args):
     # Dominant kernels: the two d x d contractions of Quant_prod (4 n d^2 flops in all).
     gemm_flops = 4.0 * n * d * d
     achieved_tf = gemm_flops / (q_ms * 1e-3) / 1e12
-    rows_per_launch = 98176   # what the quantiser's scratch (tq_workspace_bytes) holds at d = 1536, prod
+    rows_per_launch = 98304   # what the quantiser's scratch (tq_workspace_bytes) holds at d = 1536, prod
     launches_per_step = math.ceil(n / rows_per_launch)
-    roofline = {"bound": "tensor", "kernel": "tc::quantize_gemm_kernel (Y = U Pi^T and Z = E S'^T, one launch of each per 98,176 rows)",
+    roofline = {"bound": "tensor", "kernel": "tc::quantize_gemm_kernel (Y = U Pi^T and Z = E S'^T, one launch of each per 98,304 rows)",
                 "achieved": achieved_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                 "frac": achieved_tf / peaks["bf16_tflops_sustained"],
                 "frac_pass_adjusted": 3.0 * achieved_tf / peaks["bf16_tflops_sustained"],
@@ -510,7 +510,7 @@ def run_b200(args):
                 "note": "achieved = algorithmic flops 4 n d^2 of the step / CUDA-event time of the quantise phase "
                         f"({launches_per_step} launches of each GEMM + operand split); fp32 fidelity takes 3 bf16 MMA passes, "
                         "so frac_pass_adjusted = 3 x frac is the fraction of the binding tensor bound; traffic = DRAM bytes of "
-                        "one rotate + one project launch of 98,176 rows (ncu, profiles/ncu_quantize_gemm_c4_prod_b4.md)"}
+                        "one rotate + one project launch of 98,304 rows (ncu, profiles/ncu_quantize_gemm_c4_prod_b4.md)"}
     best = max(scan_regimes, key=lambda r: r["score_codes_gbs"])
     roofline_scan = {"bound": "hbm", "kernel": "mscan::scan_mma_kernel (packed-code scan, one pass, nq <= 2, dense scores)",
                      "achieved": best["score_codes_gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -469,12 +469,6 @@ extern "C" int tq_plan_create(int d, int bits, int mode, const float* Pi, const 
     PLAN_CUDA(tc::build_matrix_limbs(p->dPi, d, d, p->dpad, p->tc_bn, &p->pi_limbs), "bf16 limbs of Pi");
     if (mode == TQ_PROD)
       PLAN_CUDA(tc::build_matrix_limbs(p->dSp, d, d, p->dpad, p->tc_bn, &p->sp_limbs), "bf16 limbs of S'");
-    PLAN_CUDA(cudaStreamCreateWithFlags(&p->aux_stream, cudaStreamNonBlocking), "aux stream");
-    PLAN_CUDA(cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming), "event");
-    for (int i = 0; i < 2; ++i) {
-      PLAN_CUDA(cudaEventCreateWithFlags(&p->ev_split[i], cudaEventDisableTiming), "event");
-      PLAN_CUDA(cudaEventCreateWithFlags(&p->ev_gemm[i], cudaEventDisableTiming), "event");
-    }
     p->tc_ok = 1;
   }
   mscan::plan_init(p);
@@ -491,12 +485,6 @@ extern "C" int tq_plan_destroy(tq_plan* plan) {
   cudaFree(plan->dRotCat);
   cudaFree(plan->dBackT);
   cudaFree(plan->d_status);
-  if (plan->aux_stream) cudaStreamDestroy(plan->aux_stream);
-  if (plan->ev_fork) cudaEventDestroy(plan->ev_fork);
-  for (int i = 0; i < 2; ++i) {
-    if (plan->ev_split[i]) cudaEventDestroy(plan->ev_split[i]);
-    if (plan->ev_gemm[i]) cudaEventDestroy(plan->ev_gemm[i]);
-  }
   tc::free_matrix_limbs(&plan->pi_limbs);
   tc::free_matrix_limbs(&plan->sp_limbs);
   delete plan;
@@ -528,8 +516,10 @@ extern "C" size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int
         // rows per launch: 65,536 at d = 1536 and more for short rows (same scratch bytes), so that a launch of the
         // persistent GEMM stays long against its prologue and the launch sequence
         const int64_t chunk = std::min<int64_t>(kTensorChunk * std::max(1, 1536 / plan->dpad), 8 * kTensorChunk);
-        return align_up((size_t)std::min<int64_t>(round_up64(n, 128), chunk) * tc::scratch_bytes_per_row(plan) +
-                            (n > chunk ? (size_t)chunk * plan->dpad * 4 : 0),   // second set of X limbs: lets blocks overlap
+        // (half as many rows again when n exceeds the chunk: fewer, longer launches measured faster than 65,536-row
+        // ones, also than 65,536-row ones whose operand split ran beside the previous block's GEMMs)
+        return align_up((size_t)std::min<int64_t>(round_up64(n, 128), n > chunk ? chunk + chunk / 2 : chunk) *
+                            tc::scratch_bytes_per_row(plan),
                         256);
       }
       if (plan->mode != TQ_PROD) return 0;

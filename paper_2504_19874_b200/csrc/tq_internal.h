@@ -59,9 +59,6 @@ struct tq_plan {
   int tc_bn;       // N extent of its MMA tile
   tq::MatrixLimbs pi_limbs;   // Pi
   tq::MatrixLimbs sp_limbs;   // S' (TQ_PROD)
-  // second stream + events that let the operand split of block i+1 run beside the GEMMs of block i
-  cudaStream_t aux_stream;
-  cudaEvent_t ev_fork, ev_split[2], ev_gemm[2];
   // bit-plane scan on the integer tensor path (d >= 128, antisymmetric codebook)
   struct {
     int ok;            // 1 when this plan can use it

@@ -499,23 +499,13 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     EL2 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
     gpart = reinterpret_cast<float*>(p); p += (size_t)R * tiles_n * 4 * EPS;
   }
-  p += (size_t)R * sizeof(float);
   const size_t xsz = (x_dtype == TQ_F32) ? 4 : 2;
-  // With room for a second set of X limbs, the split of block i+1 (HBM-bound) runs on the plan's
-  // second stream while the GEMMs of block i (tensor-bound) run on the caller's.
-  const bool pipelined = n > R && plan->aux_stream != nullptr &&
-                         scratch_bytes >= (size_t)R * per_row + (size_t)R * dpad * 4;
-  __nv_bfloat16* XLb[2][2] = {{XL1, XL2}, {XL1, XL2}};
-  if (pipelined) {
-    XLb[1][0] = reinterpret_cast<__nv_bfloat16*>(p);
-    XLb[1][1] = reinterpret_cast<__nv_bfloat16*>(p + (size_t)R * dpad * 2);
-  }
-  auto launch_split = [&](int64_t r0, int b, cudaStream_t s) -> cudaError_t {
+  auto launch_split = [&](int64_t r0, cudaStream_t s) -> cudaError_t {
     const int64_t rows = std::min(R, n - r0);
     const void* Xc = static_cast<const char*>(X) + (size_t)r0 * ldx * xsz;
     float* nu_out = norms ? norms + r0 : nullptr;
     const int blocks = (int)std::min<int64_t>((rows + 7) / 8, (int64_t)sm_count() * 8);
-    __nv_bfloat16 *L1 = XLb[b][0], *L2 = XLb[b][1];
+    __nv_bfloat16 *L1 = XL1, *L2 = XL2;
     if (norms) {
       if (x_dtype == TQ_F32)
         split_rows_kernel<float, true><<<blocks, 256, 0, s>>>(static_cast<const float*>(Xc), ldx, rows, d, dpad, L1, L2, nu_out);
@@ -530,30 +520,12 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     count_launches(1);
     return cudaGetLastError();
   };
-  if (pipelined) {
-    TQ_CHECK_CUDA(cudaEventRecord(plan->ev_fork, st), who);              // the second stream starts after the caller's work so far
-    TQ_CHECK_CUDA(cudaStreamWaitEvent(plan->aux_stream, plan->ev_fork, 0), who);
-    TQ_CHECK_CUDA(launch_split(0, 0, st), who);
-  }
-
-  int64_t blk = 0;
-  for (int64_t r0 = 0; r0 < n; r0 += R, ++blk) {
+  for (int64_t r0 = 0; r0 < n; r0 += R) {
     const int64_t rows = std::min(R, n - r0);
-    const int b = pipelined ? (int)(blk & 1) : 0;
     float* nu_out = norms ? norms + r0 : nullptr;
     // 1. nu, u = x / nu, bf16 limbs of u
-    if (!pipelined) {
-      TQ_CHECK_CUDA(launch_split(r0, 0, st), who);
-    } else {
-      if (r0 + R < n) {
-        const int nb = (int)((blk + 1) & 1);
-        if (blk >= 1) TQ_CHECK_CUDA(cudaStreamWaitEvent(plan->aux_stream, plan->ev_gemm[nb], 0), who);   // its last reader is done
-        TQ_CHECK_CUDA(launch_split(r0 + R, nb, plan->aux_stream), who);
-        TQ_CHECK_CUDA(cudaEventRecord(plan->ev_split[nb], plan->aux_stream), who);
-      }
-      if (blk >= 1) TQ_CHECK_CUDA(cudaStreamWaitEvent(st, plan->ev_split[b], 0), who);
-    }
-    __nv_bfloat16 *XLc1 = XLb[b][0], *XLc2 = XLb[b][1];
+    TQ_CHECK_CUDA(launch_split(r0, st), who);
+    __nv_bfloat16 *XLc1 = XL1, *XLc2 = XL2;
 
     CUtensorMap mA1, mA2;
     TQ_REQUIRE(make_map(&mA1, XLc1, rows, d, dpad, BM) && make_map(&mA2, XLc2, rows, d, dpad, BM), TQ_ERR_CUDA,
@@ -577,11 +549,9 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     // 2. y = Pi u, idx (+ residual limbs and partial norms)
     if (!prod) {
       TQ_CHECK_CUDA(launch_gemm<0>(bn, plan->mse_bits, mA1, mA2, plan->pi_limbs.map_hi, plan->pi_limbs.map_lo, g, st), who);
-      if (pipelined) TQ_CHECK_CUDA(cudaEventRecord(plan->ev_gemm[b], st), who);
       continue;
     }
     TQ_CHECK_CUDA(launch_gemm<1>(bn, plan->mse_bits, mA1, mA2, plan->pi_limbs.map_hi, plan->pi_limbs.map_lo, g, st), who);
-    if (pipelined) TQ_CHECK_CUDA(cudaEventRecord(plan->ev_gemm[b], st), who);
     // 3. gamma = ||e||
     gamma_finish_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(gpart, R, EPS * tiles_n, rows, gamma + r0);
     count_launches(1);
