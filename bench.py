@@ -505,7 +505,7 @@ def run_b200(args):
                 "achieved": achieved_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                 "frac": achieved_tf / peaks["bf16_tflops_sustained"],
                 "frac_pass_adjusted": 3.0 * achieved_tf / peaks["bf16_tflops_sustained"],
-                "traffic": 1286.0e6 + 633.6e6 if d == 1536 else None,
+                "traffic": 1303.8e6 + 633.4e6 if d == 1536 else None,
                 "peak_source": f"bf16 sustained, of {peaks['source']}",
                 "note": "achieved = algorithmic flops 4 n d^2 of the step / CUDA-event time of the quantise phase "
                         f"({launches_per_step} launches of each GEMM + operand split); fp32 fidelity takes 3 bf16 MMA passes, "
