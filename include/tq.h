@@ -31,6 +31,15 @@
  *             ascending order (0-based).  Row stride tq_idx_row_bytes(d, b_m); pad bits are 0.
  *   qjl row : bit j = 1 iff (S r)_j >= 0 (sign(0) = +1).  Row stride tq_qjl_row_bytes(d).
  *   gamma, norms : float32 arrays of length n.
+ * This is TQ_LAYOUT_CANONICAL, the layout of every plan unless tq_plan_set_layout chose the other one:
+ *   TQ_LAYOUT_NIBBLE (TQ_PROD plans with b = 4 only): the three index bits and the sign bit of coordinate j
+ *             share nibble j of one combined row of ceil(d/2) bytes -- byte j >> 1, bits 4 (j & 1) .. 4 (j & 1) + 3,
+ *             index in the low three bits, sign bit on top.  The combined row is stored across the same two
+ *             arrays with the same strides: its first tq_idx_row_bytes(d, 3) bytes in the idx row, the
+ *             remaining bytes in the qjl row; unused nibbles are 0.  Same bytes per vector, an exact
+ *             permutation of the canonical bits (tq_convert_layout goes either way); the scan reads four
+ *             coordinates' centroids with one byte-permute instruction in this layout, which makes
+ *             tq_score / tq_topk about 1.5 times faster than on the bit streams.
  */
 #ifndef TQ_H_
 #define TQ_H_
@@ -55,6 +64,7 @@ enum {
 enum { TQ_MSE = 0, TQ_PROD = 1 };              /* plan mode                                   */
 enum { TQ_F32 = 0, TQ_BF16 = 1 };              /* element type of X / Q                       */
 enum { TQ_ORTHOGONAL = 0, TQ_GAUSSIAN = 1 };   /* tq_rotation kind                            */
+enum { TQ_LAYOUT_CANONICAL = 0, TQ_LAYOUT_NIBBLE = 1 };   /* arrangement of the code rows, see above */
 enum { TQ_OP_QUANTIZE = 0, TQ_OP_SCORE = 1, TQ_OP_TOPK = 2, TQ_OP_WSUM = 3, TQ_OP_DEQUANTIZE = 4 };
 
 #define TQ_MAX_D 8192
@@ -113,6 +123,27 @@ size_t tq_qjl_row_bytes(int d);
 int tq_plan_create(int d, int bits, int mode, const float* Pi, const float* S,
                    const float* centroids, tq_plan** out);
 int tq_plan_destroy(tq_plan* plan);
+
+/*
+ * Chooses the arrangement of the idx / qjl rows that this plan's calls write (tq_quantize_prod) and read
+ * (tq_score, tq_topk, tq_dequantize, tq_wsum, tq_score_static).  The paper fixes no layout ("b-bit integers",
+ * Algorithm 1), so this is the library's choice; the codes themselves are the same.
+ *   layout  TQ_LAYOUT_CANONICAL (default, every plan) or TQ_LAYOUT_NIBBLE (TQ_PROD, b = 4, d >= 128 and
+ *           small enough for the scan's shared-memory operand: d <= 4096 is always accepted)
+ * Returns TQ_ERR_UNSUPPORTED for a plan that cannot use the requested layout.  Host-side switch, no device
+ * work; arrays written under one layout must be converted before they are read under the other.
+ * tq_attend_decode / tq_kv_append take canonical plans only.
+ */
+int tq_plan_set_layout(tq_plan* plan, int layout);
+int tq_plan_layout(const tq_plan* plan);   /* TQ_LAYOUT_*; -1 for a NULL plan */
+
+/*
+ * Rewrites n rows of codes in place from layout `from` into layout `to` (TQ_LAYOUT_*): an exact permutation
+ * of the bits of each (idx row, qjl row) pair; gamma and norms are not touched.  from == to is a no-op.
+ *   idx, qjl  device, the arrays of tq_quantize_prod (same strides in both layouts)
+ * Errors: TQ_ERR_UNSUPPORTED when the plan cannot use TQ_LAYOUT_NIBBLE; the usual argument checks.
+ */
+int tq_convert_layout(const tq_plan* plan, int64_t n, uint8_t* idx, uint8_t* qjl, int from, int to, void* stream);
 
 /* Synchronises the device and reports whether any kernel launched for this plan since the
  * last call gave up one of its bounded device-side waits (TQ_ERR_TIMEOUT; the outputs of that

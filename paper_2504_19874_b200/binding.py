@@ -10,6 +10,7 @@ import torch
 TQ_MSE, TQ_PROD = 0, 1
 TQ_F32, TQ_BF16 = 0, 1
 TQ_ORTHOGONAL, TQ_GAUSSIAN = 0, 1
+TQ_LAYOUT_CANONICAL, TQ_LAYOUT_NIBBLE = 0, 1
 TQ_OP_QUANTIZE, TQ_OP_SCORE, TQ_OP_TOPK, TQ_OP_WSUM, TQ_OP_DEQUANTIZE = 0, 1, 2, 3, 4
 TQ_STATIC_SCRATCH_BYTES = 1 << 20
 
@@ -29,6 +30,9 @@ _SIGNATURES = {
     "tq_plan_create": (c_int, [c_int, c_int, c_int, _F, _F, _F, ctypes.POINTER(c_void_p)]),
     "tq_plan_destroy": (c_int, [c_void_p]),
     "tq_plan_status": (c_int, [c_void_p]),
+    "tq_plan_set_layout": (c_int, [c_void_p, c_int]),
+    "tq_plan_layout": (c_int, [c_void_p]),
+    "tq_convert_layout": (c_int, [c_void_p, c_int64, c_void_p, c_void_p, c_int, c_int, c_void_p]),
     "tq_workspace_bytes": (c_size_t, [c_void_p, c_int, c_int64, c_int, c_int]),
     "tq_quantize_mse": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "tq_quantize_prod": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -161,6 +165,14 @@ class Plan:
                                     ctypes.byref(h)))
         self.handle = h
 
+    def set_layout(self, layout: int) -> None:
+        """TQ_LAYOUT_CANONICAL or TQ_LAYOUT_NIBBLE (TQ_PROD with b = 4 only): arrangement of the code rows."""
+        _check(lib().tq_plan_set_layout(self.handle, layout))
+
+    @property
+    def layout(self) -> int:
+        return lib().tq_plan_layout(self.handle)
+
     def close(self):
         if getattr(self, "handle", None):
             lib().tq_plan_destroy(self.handle)
@@ -176,6 +188,11 @@ class Plan:
 def tq_plan_status(plan: Plan) -> None:
     """Synchronises and raises TqError(6) if a kernel of this plan gave up a bounded wait."""
     _check(lib().tq_plan_status(plan.handle))
+
+
+def tq_convert_layout(plan: Plan, n: int, idx, qjl, src: int, dst: int) -> None:
+    """Rewrites n rows of (idx, qjl) in place from layout `src` into layout `dst`."""
+    _check(lib().tq_convert_layout(plan.handle, n, _dev(idx), _dev(qjl), src, dst, _stream()))
 
 
 def tq_workspace_bytes(plan: Plan, op: int, n: int, nq: int = 0, k: int = 0) -> int:

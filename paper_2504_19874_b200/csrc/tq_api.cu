@@ -10,6 +10,7 @@
 #include "tq_internal.h"
 #include "tq_quantize_tc.h"
 #include "tq_scan_mma.h"
+#include "tq_scan_nib.h"
 #include "tq_scan_simt.cuh"
 #include "tq_scan_tc.h"
 
@@ -80,6 +81,7 @@ simt::Codes make_codes(const tq_plan* plan, int64_t n, const uint8_t* idx, const
   c.dpad = plan->dpad;
   c.coef = plan->coef;
   c.rows = n;
+  c.nibble = plan->layout == TQ_LAYOUT_NIBBLE;
   return c;
 }
 
@@ -104,6 +106,7 @@ constexpr int kGroupQueries = tscan::kQueriesPerPass * tscan::kPassesPerGroup;
 struct ScanEngine {
   const tq_plan* plan;
   bool tc;
+  bool nib;                 // table-lookup scan of the nibble layout (2 or 8 queries per pass)
   int qpp;                  // queries per pass
   int64_t dense_rows_pref;  // rows of the dense score buffer that keep the rescue pass to a few launches
   size_t ws_bytes;          // engine workspace (constants + B operand)
@@ -112,16 +115,18 @@ struct ScanEngine {
 ScanEngine pick_engine(const tq_plan* plan, int nq) {
   ScanEngine e;
   e.plan = plan;
-  e.tc = nq >= 7 && tscan::available(plan);
-  e.qpp = e.tc ? tscan::kQueriesPerPass : mscan::queries_per_pass(plan, nq);
+  e.nib = plan->layout == TQ_LAYOUT_NIBBLE;
+  e.tc = !e.nib && nq >= 7 && tscan::available(plan);
+  e.qpp = e.nib ? nscan::queries_per_pass(plan, nq) : e.tc ? tscan::kQueriesPerPass : mscan::queries_per_pass(plan, nq);
   e.dense_rows_pref = e.tc ? (1 << 18) : (1 << 20);
-  e.ws_bytes = e.tc ? tscan::workspace_bytes(plan) : mscan::workspace_bytes(plan);
+  e.ws_bytes = e.nib ? nscan::workspace_bytes(plan) : e.tc ? tscan::workspace_bytes(plan) : mscan::workspace_bytes(plan);
   return e;
 }
 
 // Prepares what the pass starting at query q0 needs (the tcgen05 engine builds 256 queries at a time).
 int engine_prepare(const ScanEngine& e, const float* Qcat, int q0, int nq, void* ws, cudaStream_t st, const char* who) {
   const int ncols = e.plan->ncat * e.plan->dpad;
+  if (e.nib) return nscan::prepare(e.plan, Qcat + (size_t)q0 * ncols, std::min(e.qpp, nq - q0), ws, st, who);
   if (e.tc) {
     if (q0 % kGroupQueries != 0) return TQ_OK;
     return tscan::prepare_group(e.plan, Qcat + (size_t)q0 * ncols, std::min(kGroupQueries, nq - q0), ws, st, who);
@@ -132,6 +137,7 @@ int engine_prepare(const ScanEngine& e, const float* Qcat, int q0, int nq, void*
 int engine_run(const ScanEngine& e, int q0, int nqp, int64_t n, const uint8_t* idx, const uint8_t* qjl, const float* gamma,
                const float* norms, float* scores, int64_t lds, const mscan::Filter* filter, const int* run_if, const void* ws,
                cudaStream_t st, const char* who) {
+  if (e.nib) return nscan::run(e.plan, nqp, n, idx, qjl, gamma, norms, scores, lds, filter, run_if, ws, true, st, who);
   if (e.tc)
     return tscan::run_pass(e.plan, (q0 % kGroupQueries) / tscan::kQueriesPerPass, nqp, n, idx, qjl, gamma, norms, scores, lds,
                            filter, run_if, ws, st, who);
@@ -208,6 +214,9 @@ __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __rest
                                                              float* __restrict__ Qcat, int64_t ldo) {
   extern __shared__ __align__(16) float qs_raw[];
   float (*qs)[kRotChunk] = reinterpret_cast<float (*)[kRotChunk]>(qs_raw);
+  // a successor launched as a programmatic dependent may be scheduled while this grid drains (it waits for
+  // this grid's completion before it reads Qcat)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int j = blockIdx.x * 8 + warp;
   const float* row = Rot + (size_t)min(j, nrows - 1) * d;
@@ -472,6 +481,7 @@ extern "C" int tq_plan_create(int d, int bits, int mode, const float* Pi, const 
     p->tc_ok = 1;
   }
   mscan::plan_init(p);
+  nscan::plan_init(p);
   PLAN_CUDA(cudaDeviceSynchronize(), "synchronize");
 #undef PLAN_CUDA
   *out = p;
@@ -489,6 +499,33 @@ extern "C" int tq_plan_destroy(tq_plan* plan) {
   tc::free_matrix_limbs(&plan->sp_limbs);
   delete plan;
   return TQ_OK;
+}
+
+extern "C" int tq_plan_set_layout(tq_plan* plan, int layout) {
+  const char* who = "tq_plan_set_layout";
+  TQ_REQUIRE(plan != nullptr, TQ_ERR_INVALID_ARG, "%s: plan is NULL", who);
+  TQ_REQUIRE(layout == TQ_LAYOUT_CANONICAL || layout == TQ_LAYOUT_NIBBLE, TQ_ERR_INVALID_ARG, "%s: unknown layout %d", who, layout);
+  TQ_REQUIRE(layout == TQ_LAYOUT_CANONICAL || plan->nb.ok, TQ_ERR_UNSUPPORTED,
+             "%s: the nibble layout needs a TQ_PROD plan with b = 4, d >= 128 (d=%d, b=%d, mode=%d)", who, plan->d, plan->bits,
+             plan->mode);
+  plan->layout = layout;
+  return TQ_OK;
+}
+
+extern "C" int tq_plan_layout(const tq_plan* plan) { return plan ? plan->layout : -1; }
+
+extern "C" int tq_convert_layout(const tq_plan* plan, int64_t n, uint8_t* idx, uint8_t* qjl, int from, int to, void* stream) {
+  const char* who = "tq_convert_layout";
+  int rc = check_plan(plan, who);
+  if (rc) return rc;
+  TQ_REQUIRE(n >= 0, TQ_ERR_INVALID_ARG, "%s: n is negative", who);
+  for (int l : {from, to})
+    TQ_REQUIRE(l == TQ_LAYOUT_CANONICAL || l == TQ_LAYOUT_NIBBLE, TQ_ERR_INVALID_ARG, "%s: unknown layout %d", who, l);
+  TQ_REQUIRE(plan->nb.ok, TQ_ERR_UNSUPPORTED, "%s: this plan has no nibble layout (TQ_PROD, b = 4, d >= 128 only)", who);
+  if (n == 0 || from == to) return TQ_OK;
+  TQ_REQUIRE(idx != nullptr && qjl != nullptr, TQ_ERR_INVALID_ARG, "%s: idx / qjl is NULL", who);
+  TQ_REQUIRE(aligned(idx, 16) && aligned(qjl, 16), TQ_ERR_ALIGNMENT, "%s: idx / qjl is not 16-byte aligned", who);
+  return nscan::convert(plan, n, idx, qjl, to, static_cast<cudaStream_t>(stream), who);
 }
 
 extern "C" int tq_plan_status(tq_plan* plan) {
@@ -588,7 +625,10 @@ extern "C" int tq_quantize_prod(const tq_plan* plan, const void* X, int x_dtype,
     TQ_REQUIRE(scratch != nullptr && scratch_bytes >= least, TQ_ERR_WORKSPACE,
                "%s: scratch of %zu bytes, at least %zu needed", who, scratch_bytes, least);
     TQ_REQUIRE(aligned(scratch, 256), TQ_ERR_ALIGNMENT, "%s: scratch is not 256-byte aligned", who);
-    return tc::quantize(plan, X, x_dtype, n, ldx, idx, qjl, gamma, norms, scratch, scratch_bytes, st, who);
+    if ((rc = tc::quantize(plan, X, x_dtype, n, ldx, idx, qjl, gamma, norms, scratch, scratch_bytes, st, who))) return rc;
+    // the GEMM epilogues write the bit streams; the nibble layout is an in-place permutation of each row
+    if (plan->layout == TQ_LAYOUT_NIBBLE) return nscan::convert(plan, n, idx, qjl, TQ_LAYOUT_NIBBLE, st, who);
+    return TQ_OK;
   }
   const size_t need = tq_workspace_bytes(plan, TQ_OP_QUANTIZE, n, 0, 0);
   TQ_REQUIRE(scratch != nullptr && scratch_bytes >= need, TQ_ERR_WORKSPACE, "%s: scratch of %zu bytes, %zu needed", who,
@@ -834,6 +874,7 @@ extern "C" int tq_wsum(const tq_plan* plan, const float* W, int nw, int64_t ldw,
     a.dpad = plan->dpad;
     a.ncols = ncols;
     a.coef = plan->coef;
+    a.nibble = plan->layout == TQ_LAYOUT_NIBBLE;
     a.partial = partial;
     const dim3 grid((unsigned)nchunks, (unsigned)((plan->d + 127) / 128));
     // columns the partial kernel never writes (pad coordinates) must read as zero

@@ -70,6 +70,7 @@ struct WsumArgs {
   Codebook cb;
   int d, dpad, ncols;
   float coef;
+  bool nibble;          // TQ_LAYOUT_NIBBLE (BITS = 3, PROD): nibble j of [idx row | qjl row] = index | sign << 3
   float* partial;       // [nchunks, nw, ncols]
 };
 
@@ -101,6 +102,18 @@ __global__ void __launch_bounds__(128) wsum_partial_kernel(WsumArgs a) {
   const int bitpos = j * BITS, byte0 = bitpos >> 3, sh = bitpos & 7;
   for (int tt = 0; tt < ntok; ++tt) {
     const int64_t t = t0 + tt;
+    if (a.nibble) {
+      const size_t byte = (size_t)j >> 1;
+      const uint32_t x = byte < a.idx_rb ? a.idx[(size_t)t * a.idx_rb + byte] : a.qjl[(size_t)t * a.qjl_rb + (byte - a.idx_rb)];
+      const uint32_t nib = (x >> (4 * (j & 1))) & 15u;
+      const float c = a.cb.c[nib & 7u];
+#pragma unroll
+      for (int w = 0; w < WS_NW; ++w) {
+        acc[w] = fmaf(wn[w][tt], c, acc[w]);
+        if (PROD) accs[w] += (nib & 8u) ? wg[w][tt] : -wg[w][tt];
+      }
+      continue;
+    }
     if (BITS > 0) {
       const uint8_t* row = a.idx + (size_t)t * a.idx_rb;
       uint32_t v = row[byte0];

@@ -555,6 +555,8 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
     const tq_kv_group& s = groups[gi];
     TQ_REQUIRE(s.plan_k && s.plan_v, TQ_ERR_INVALID_ARG, "%s: group %d has no plan", who, gi);
     TQ_REQUIRE(s.plan_k->d == d && s.plan_v->d == d, TQ_ERR_UNSUPPORTED, "%s: all groups must share one dimension", who);
+    TQ_REQUIRE(s.plan_k->layout == TQ_LAYOUT_CANONICAL && s.plan_v->layout == TQ_LAYOUT_CANONICAL, TQ_ERR_UNSUPPORTED,
+               "%s: group %d: plans must use the canonical code layout", who, gi);
     TQ_REQUIRE(s.plan_v->mode == TQ_MSE && s.plan_v->mse_bits >= 1, TQ_ERR_UNSUPPORTED,
                "%s: values must be quantised with TurboQuant_mse", who);
     TQ_REQUIRE(s.plan_k->device == s.plan_v->device, TQ_ERR_INVALID_ARG, "%s: plans of different devices", who);
@@ -658,6 +660,8 @@ extern "C" int tq_kv_append(const tq_kv_group* groups, int ngroups, int heads, i
     const tq_kv_group& s = groups[gi];
     TQ_REQUIRE(s.plan_k && s.plan_v, TQ_ERR_INVALID_ARG, "%s: group %d has no plan", who, gi);
     TQ_REQUIRE(s.plan_k->d == d && s.plan_v->d == d, TQ_ERR_UNSUPPORTED, "%s: all groups must share one dimension", who);
+    TQ_REQUIRE(s.plan_k->layout == TQ_LAYOUT_CANONICAL && s.plan_v->layout == TQ_LAYOUT_CANONICAL, TQ_ERR_UNSUPPORTED,
+               "%s: group %d: plans must use the canonical code layout", who, gi);
     TQ_REQUIRE(s.plan_v->mode == TQ_MSE && s.plan_v->mse_bits >= 1, TQ_ERR_UNSUPPORTED,
                "%s: values must be quantised with TurboQuant_mse", who);
     const bool prod = s.plan_k->mode == TQ_PROD;

@@ -78,10 +78,26 @@ struct Codes {
   int d, dpad;
   float coef;
   int64_t rows;
+  bool nibble;   // TQ_LAYOUT_NIBBLE: nibble j of the combined row [idx row | qjl row] = index | sign << 3
   __device__ __forceinline__ void load(int64_t r, int k0, float (&v)[8]) const {
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = 0.f;
     if (r >= rows) return;
+    if (nibble) {   // k0 is a multiple of 8: one 32-bit word of the combined row holds the eight coordinates
+      const int j0 = k0 < dpad ? k0 : k0 - dpad;
+      if (j0 >= d) return;
+      const size_t byte = (size_t)j0 >> 1;
+      const uint8_t* s = byte < idx_rb ? idx + (size_t)r * idx_rb + byte : qjl + (size_t)r * qjl_rb + (byte - idx_rb);
+      const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(s));
+      const float g = k0 < dpad ? 0.f : coef * __ldg(gamma + r);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (j0 + i >= d) break;
+        const uint32_t nib = (w >> (4 * i)) & 15u;
+        v[i] = k0 < dpad ? cb.c[nib & 7u] : ((nib & 8u) ? g : -g);
+      }
+      return;
+    }
     if (k0 < dpad) {
       const int bits = cb.bits;
       if (bits == 0 || k0 >= d) return;

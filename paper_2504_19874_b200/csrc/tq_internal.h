@@ -67,6 +67,14 @@ struct tq_plan {
     double amax;       // max |alpha|
     double csum;       // mean term minus the sum of alpha: constant part of sum_j q'_j c[idx_j]
   } ms;
+  // nibble layout of the codes and the table-lookup scan (TQ_PROD with a 3-bit MSE stage)
+  int layout;      // TQ_LAYOUT_*: arrangement of the idx / qjl rows this plan writes and reads
+  struct {
+    int ok;                            // 1 when this plan may be switched to TQ_LAYOUT_NIBBLE
+    int nbi, nbq;                      // 64-byte blocks of an idx row / a qjl row
+    uint32_t hi_a, hi_b, lo_a, lo_b;   // 16-bit centroid table t_i = 256 h_i + l_i as bytes: h of entries 0..3, 4..7, l alike
+    double delta;                      // c_i ~ delta * t_i
+  } nb;
   int* d_status;   // device word: set to TQ_ERR_TIMEOUT by a kernel whose bounded wait ran out
 };
 

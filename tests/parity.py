@@ -27,14 +27,17 @@ RTOL = 1e-4
 class Setup:
     """Oracle-made global parameters (Pi, S, fp32 codebook) and the matching GPU plan."""
 
-    def __init__(self, d, bits, mode, pi_seed=42, s_seed=43):
+    def __init__(self, d, bits, mode, pi_seed=42, s_seed=43, layout=None):
         self.d, self.bits, self.mode = d, bits, mode
+        self.layout = layout
         self.mse_bits = bits - 1 if mode == tq.TQ_PROD else bits
         self.Pi = orc.rotation(d, pi_seed).astype(np.float32)
         self.S = orc.projection(d, s_seed).astype(np.float32) if mode == tq.TQ_PROD else None
         self.c = orc.codebook(d, self.mse_bits).astype(np.float32)
         self.t = (0.5 * (self.c[:-1].astype(np.float64) + self.c[1:].astype(np.float64)))
         self.plan = tq.Plan(d, bits, mode, self.Pi, self.S, self.c)
+        if layout is not None:
+            self.plan.set_layout(layout)
         self.idx_rb = tq.tq_idx_row_bytes(d, self.mse_bits)
         self.qjl_rb = tq.tq_qjl_row_bytes(d)
 
@@ -85,7 +88,19 @@ def as_f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().to("cpu").to(torch.float64).numpy()
 
 
+def nibble_rows_to_coordinates(idx: np.ndarray, qjl: np.ndarray, d: int):
+    """The nibble layout read literally from its definition: nibble j of the row [idx row | qjl row] holds
+    coordinate j, index in its low three bits and the sign bit on top.  Returns (index [n, d], bit [n, d]) and
+    the nibbles beyond d (which must be zero)."""
+    row = np.concatenate([idx, qjl], axis=1)
+    nib = np.stack([row & 15, row >> 4], axis=2).reshape(row.shape[0], -1)
+    return nib[:, :d] & 7, nib[:, :d] >> 3, nib[:, d:]
+
+
 def unpack(su: Setup, idx, qjl):
+    if getattr(su, "layout", None) == tq.TQ_LAYOUT_NIBBLE:
+        i3, bit, _ = nibble_rows_to_coordinates(idx.cpu().numpy(), qjl.cpu().numpy(), su.d)
+        return i3.astype(np.uint8), bit.astype(np.int8) * 2 - 1
     idx_np = orc.unpack_bits(idx.cpu().numpy(), su.mse_bits, su.d) if su.mse_bits > 0 else \
         np.zeros((idx.shape[0], su.d), dtype=np.uint8)
     z_np = None
@@ -107,7 +122,10 @@ def check_quantize(su: Setup, X: torch.Tensor, idx, qjl, gamma, norms, unit_inpu
     Xd = as_f64(X)
     n = Xd.shape[0]
     idx_gpu, z_gpu = unpack(su, idx, qjl)
-    if su.mse_bits > 0:
+    nibble = getattr(su, "layout", None) == tq.TQ_LAYOUT_NIBBLE
+    if nibble:
+        assert not nibble_rows_to_coordinates(idx.cpu().numpy(), qjl.cpu().numpy(), su.d)[2].any(), "pad nibbles must be zero"
+    elif su.mse_bits > 0:
         check_pad_bits_zero(idx, su.mse_bits, su.d)
     nu_orc = np.sqrt(np.sum(Xd * Xd, axis=1))
     if norms is not None:
@@ -132,7 +150,8 @@ def check_quantize(su: Setup, X: torch.Tensor, idx, qjl, gamma, norms, unit_inpu
     # a flip inside the window must still land on an adjacent cell
     assert np.all(np.abs(idx_gpu.astype(int) - idx_orc.astype(int))[diff] == 1)
     if su.mode == tq.TQ_PROD:
-        check_pad_bits_zero(qjl, 1, su.d)
+        if not nibble:
+            check_pad_bits_zero(qjl, 1, su.d)
         ok_rows = ~np.any(diff & ~inside, axis=1)
         # unit_input: feed the oracle rows that it will not rescale
         Xo = U if unit_input else Xd
