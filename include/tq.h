@@ -151,6 +151,12 @@ int tq_convert_layout(const tq_plan* plan, int64_t n, uint8_t* idx, uint8_t* qjl
  * time limit so that a stalled pipeline ends as this status instead of a hung GPU. */
 int tq_plan_status(tq_plan* plan);
 
+/* Self test of that mechanism, for test suites: enqueues a one-warp kernel that waits, through the same bounded
+ * wait the tensor-core kernels use, on a barrier nobody arrives at, with a limit of `limit_cycles` SM cycles
+ * (1 .. 1e8) instead of the seconds-long production limit.  The kernel returns on its own; the next
+ * tq_plan_status(plan) must report TQ_ERR_TIMEOUT.  Nothing faults, traps or hangs. */
+int tq_selftest_wait_timeout(tq_plan* plan, long long limit_cycles, void* stream);
+
 /* Bytes of device scratch the given operation asks for (0 if none).  For TQ_OP_QUANTIZE and
  * TQ_OP_TOPK this is the preferred size; a smaller buffer is accepted down to the value returned
  * for n = 128 (QUANTIZE) resp. n = 4096 (TOPK) and means more, smaller launches (for TOPK also the
@@ -205,21 +211,39 @@ int tq_score(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ld
              float* scores, int64_t lds, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Queries prepared once and scanned many times (a search over several segments or shards of a database, a
+ * cache that grows between decoding steps): tq_query_prepare does the query-side work of tq_score -- the
+ * rotations q' = Pi q, q'' = S q and the scan's fixed-point operand -- into a caller buffer, tq_score_prepared
+ * runs only the scan over the codes.  tq_score(Q) == tq_query_prepare(Q) followed by tq_score_prepared, bit for bit.
+ *   prepared   device, 256-byte aligned, >= tq_query_bytes(plan, nq); valid for this plan, its current layout
+ *              and exactly this nq until overwritten
+ */
+size_t tq_query_bytes(const tq_plan* plan, int nq);
+int tq_query_prepare(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq,
+                     void* prepared, size_t prepared_bytes, void* stream);
+int tq_score_prepared(const tq_plan* plan, const void* prepared, int nq, int64_t n,
+                      const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms,
+                      float* scores, int64_t lds, void* stream);
+
+/*
  * tq_score without caller-provided workspace and without any allocation (the paper has no
- * counterpart: this is a packaging variant of tq_score, same arithmetic, same kernels).
+ * counterpart: this is a packaging variant of tq_score with the same arithmetic and the same scan kernels;
+ * its estimates equal tq_score's bit for bit).
  *
  * Who needs it: callers that are not allowed to obtain device memory at the time they score --
  * an inference server that gave the whole GPU to its own memory pool at start-up, a plug-in whose
  * host forbids driver allocations after initialisation, a latency-critical loop that cannot afford
  * the device-wide synchronisation cudaMalloc / cudaFree imply.  Such a caller has nowhere to take
- * the rotated-query workspace from, so the library keeps it: a fixed array of
- * TQ_STATIC_SCRATCH_BYTES that lives in the library's device image.  Every GPU that loads the
+ * the workspace from (rotated queries and the scan's query-side operand), so the library keeps it: a fixed
+ * array of TQ_STATIC_SCRATCH_BYTES that lives in the library's device image.  Every GPU that loads the
  * library holds that array until the process exits, whether or not this function is ever called.
  *
  *   arguments   as tq_score, minus workspace / workspace_bytes
- *   limit       nq * ncat * dpad * 4 <= TQ_STATIC_SCRATCH_BYTES, ncat = 1 (TQ_MSE) or 2 (TQ_PROD),
- *               dpad = d rounded up to a multiple of 8; larger requests return TQ_ERR_WORKSPACE
- *               and launch nothing (largest accepted nq: 85 at d = 1536 TQ_PROD, 256 at d = 512 TQ_PROD).
+ *   limit       rotated queries (nq * ncat * dpad * 4 bytes, ncat = 1 for TQ_MSE, 2 for TQ_PROD, dpad = d rounded
+ *               up to a multiple of 8) plus one scan operand must fit in TQ_STATIC_SCRATCH_BYTES;
+ *               tq_score_static_max_queries(plan) gives the largest accepted nq (75 at d = 1536 TQ_PROD b = 4).
+ *               Larger requests return TQ_ERR_WORKSPACE and launch nothing.  Where the many-query engine's
+ *               operand does not fit, the few-query engine runs instead (more passes, same estimates).
  *   first call  the first call on each device looks up the array's device address (with that
  *               device current) and remembers it; make that first call outside any stream capture.
  *   sharing     all calls on a device use the same array and it keeps whatever the previous call
@@ -232,6 +256,7 @@ int tq_score(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ld
 int tq_score_static(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, int64_t n,
                     const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms,
                     float* scores, int64_t lds, void* stream);
+int tq_score_static_max_queries(const tq_plan* plan);
 
 /*
  * The k vectors with the largest estimate per query (nearest-neighbour search by estimated

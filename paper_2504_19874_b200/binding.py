@@ -42,6 +42,12 @@ _SIGNATURES = {
                          c_void_p, c_int64, c_void_p, c_size_t, c_void_p]),
     "tq_score_static": (c_int, [c_void_p, c_void_p, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                                 c_void_p, c_int64, c_void_p]),
+    "tq_score_static_max_queries": (c_int, [c_void_p]),
+    "tq_query_bytes": (c_size_t, [c_void_p, c_int]),
+    "tq_query_prepare": (c_int, [c_void_p, c_void_p, c_int, c_int, c_int64, c_void_p, c_size_t, c_void_p]),
+    "tq_score_prepared": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                  c_int64, c_void_p]),
+    "tq_selftest_wait_timeout": (c_int, [c_void_p, ctypes.c_longlong, c_void_p]),
     "tq_topk": (c_int, [c_void_p, c_void_p, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                         c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "tq_select_topk": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_int, c_void_p, c_void_p, c_void_p]),
@@ -234,6 +240,31 @@ def tq_score_static(plan: Plan, Q, n: int, idx, qjl, gamma, norms, scores):
     _, lds = _rows(scores)
     _check(lib().tq_score_static(plan.handle, _dev(Q), _dtype_code(Q), nq, ldq, n, _dev(idx), _dev(qjl), _dev(gamma),
                                  _dev(norms), _dev(scores), lds, _stream()))
+
+
+def tq_score_static_max_queries(plan: Plan) -> int:
+    return lib().tq_score_static_max_queries(plan.handle)
+
+
+def tq_query_bytes(plan: Plan, nq: int) -> int:
+    return lib().tq_query_bytes(plan.handle, nq)
+
+
+def tq_query_prepare(plan: Plan, Q, prepared):
+    """Query-side work of tq_score (rotations, scan operand) into `prepared` (>= tq_query_bytes(plan, nq) bytes)."""
+    nq, ldq = _rows(Q)
+    _check(lib().tq_query_prepare(plan.handle, _dev(Q), _dtype_code(Q), nq, ldq, *_scratch_args(prepared), _stream()))
+
+
+def tq_score_prepared(plan: Plan, prepared, nq: int, n: int, idx, qjl, gamma, norms, scores):
+    _, lds = _rows(scores)
+    _check(lib().tq_score_prepared(plan.handle, _dev(prepared), nq, n, _dev(idx), _dev(qjl), _dev(gamma), _dev(norms),
+                                   _dev(scores), lds, _stream()))
+
+
+def tq_selftest_wait_timeout(plan: Plan, limit_cycles: int = 20000) -> None:
+    """Enqueues the library's bounded-wait self test; the next tq_plan_status(plan) must raise TqError(6)."""
+    _check(lib().tq_selftest_wait_timeout(plan.handle, limit_cycles, _stream()))
 
 
 def tq_topk(plan: Plan, Q, n: int, idx, qjl, gamma, norms, k: int, top_scores, top_ids, workspace):

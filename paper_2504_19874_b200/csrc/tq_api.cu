@@ -13,6 +13,7 @@
 #include "tq_scan_nib.h"
 #include "tq_scan_simt.cuh"
 #include "tq_scan_tc.h"
+#include "tq_tc.cuh"
 
 using namespace tq;
 
@@ -528,6 +529,34 @@ extern "C" int tq_convert_layout(const tq_plan* plan, int64_t n, uint8_t* idx, u
   return nscan::convert(plan, n, idx, qjl, to, static_cast<cudaStream_t>(stream), who);
 }
 
+// A one-warp kernel whose barrier nobody arrives at: the bounded wait must give up after `limit` cycles, raise the
+// CTA's abort flag and record TQ_ERR_TIMEOUT in the plan's status word.  Nothing traps, nothing spins past the limit.
+__global__ void wait_timeout_selftest_kernel(int* status, long long limit) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(&bar, 1);
+    abort_flag = 0;
+    tc::fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const bool ok = tc::mbar_wait_slow(&bar, 0u, &abort_flag, status, limit);
+    if (ok || abort_flag != 1) atomicExch(status, TQ_ERR_CUDA);   // anything but "gave up and said so" is a different error
+  }
+}
+
+extern "C" int tq_selftest_wait_timeout(tq_plan* plan, long long limit_cycles, void* stream) {
+  const char* who = "tq_selftest_wait_timeout";
+  int rc = check_plan(plan, who);
+  if (rc) return rc;
+  TQ_REQUIRE(limit_cycles >= 1 && limit_cycles <= 100000000LL, TQ_ERR_INVALID_ARG, "%s: limit outside 1..1e8 cycles", who);
+  wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(plan->d_status, limit_cycles);
+  count_launches(1);
+  TQ_CHECK_CUDA(cudaGetLastError(), who);
+  return TQ_OK;
+}
+
 extern "C" int tq_plan_status(tq_plan* plan) {
   const char* who = "tq_plan_status";
   TQ_REQUIRE(plan != nullptr, TQ_ERR_INVALID_ARG, "%s: plan is NULL", who);
@@ -536,6 +565,10 @@ extern "C" int tq_plan_status(tq_plan* plan) {
   TQ_CHECK_CUDA(cudaMemcpy(&st, plan->d_status, sizeof(int), cudaMemcpyDeviceToHost), who);
   if (st != 0) {
     cudaMemset(plan->d_status, 0, sizeof(int));
+    if (st != TQ_ERR_TIMEOUT) {
+      set_error("%s: a kernel recorded the unexpected status %d", who, st);
+      return TQ_ERR_CUDA;
+    }
     set_error("%s: a kernel gave up a bounded wait (pipeline stall); results of that call are invalid", who);
     return TQ_ERR_TIMEOUT;
   }
@@ -692,6 +725,47 @@ extern "C" int tq_dequantize(const tq_plan* plan, int64_t n, const uint8_t* idx,
   return TQ_OK;
 }
 
+// Engine for a score call whose workspace holds `avail` bytes behind the rotated queries: the preferred one, or,
+// when the many-query engine's operand does not fit, the few-query engine (same estimates, more passes).
+static bool engine_that_fits(const tq_plan* plan, int nq, size_t avail, ScanEngine* out) {
+  *out = pick_engine(plan, nq);
+  if (align_up(out->ws_bytes, 256) <= avail) return true;
+  if (!out->tc) return false;
+  *out = pick_engine(plan, std::min(nq, 6));
+  return align_up(out->ws_bytes, 256) <= avail;
+}
+
+// tq_score on a workspace that is known to be large enough: rotated queries first, then the engine's operand.
+static int score_on_workspace(const tq_plan* plan, const ScanEngine* eng, const void* Q, int q_dtype, int nq, int64_t ldq,
+                              int64_t n, const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms,
+                              float* scores, int64_t lds, void* workspace, cudaStream_t st, const char* who) {
+  int rc;
+  float* Qcat = static_cast<float*>(workspace);
+  TQ_CHECK_CUDA(prepare_queries(plan, Q, q_dtype, nq, ldq, Qcat, st), who);
+  if (plan->ms.ok) {
+    void* msw = static_cast<char*>(workspace) + qcat_bytes(plan, nq);
+    for (int q0 = 0; q0 < nq; q0 += eng->qpp) {
+      const int nqp = std::min(eng->qpp, nq - q0);
+      if ((rc = engine_prepare(*eng, Qcat, q0, nq, msw, st, who))) return rc;
+      if ((rc = engine_run(*eng, q0, nqp, n, idx, qjl, gamma, norms, scores + (int64_t)q0 * lds, lds, nullptr, nullptr, msw, st, who)))
+        return rc;
+    }
+    return TQ_OK;
+  }
+  TQ_CHECK_CUDA(score_block(plan, Qcat, nq, 0, n, idx, qjl, gamma, norms, scores, lds, st), who);
+  return TQ_OK;
+}
+
+static int check_score_args(const tq_plan* plan, const char* who, const void* Q, int q_dtype, int nq, int64_t ldq, int64_t n,
+                            const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* scores, int64_t lds) {
+  int rc;
+  if ((rc = check_rows(who, "Q", Q, q_dtype, nq, ldq, plan->d))) return rc;
+  if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
+  TQ_REQUIRE(scores != nullptr && lds >= n, TQ_ERR_INVALID_ARG, "%s: scores is NULL or lds < n", who);
+  TQ_REQUIRE(aligned(scores, 16), TQ_ERR_ALIGNMENT, "%s: scores is not 16-byte aligned", who);
+  return TQ_OK;
+}
+
 extern "C" int tq_score(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, int64_t n,
                         const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms, float* scores,
                         int64_t lds, void* workspace, size_t workspace_bytes, void* stream) {
@@ -700,29 +774,89 @@ extern "C" int tq_score(const tq_plan* plan, const void* Q, int q_dtype, int nq,
   if (rc) return rc;
   TQ_REQUIRE(n >= 0 && nq >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
   if (n == 0 || nq == 0) return TQ_OK;
-  if ((rc = check_rows(who, "Q", Q, q_dtype, nq, ldq, plan->d))) return rc;
-  if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
-  TQ_REQUIRE(scores != nullptr && lds >= n, TQ_ERR_INVALID_ARG, "%s: scores is NULL or lds < n", who);
-  TQ_REQUIRE(aligned(scores, 16), TQ_ERR_ALIGNMENT, "%s: scores is not 16-byte aligned", who);
+  if ((rc = check_score_args(plan, who, Q, q_dtype, nq, ldq, n, idx, qjl, gamma, scores, lds))) return rc;
   const size_t need = tq_workspace_bytes(plan, TQ_OP_SCORE, n, nq, 0);
   TQ_REQUIRE(workspace != nullptr && workspace_bytes >= need, TQ_ERR_WORKSPACE, "%s: workspace of %zu bytes, %zu needed",
              who, workspace_bytes, need);
   TQ_REQUIRE(aligned(workspace, 16), TQ_ERR_ALIGNMENT, "%s: workspace is not 16-byte aligned", who);
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  float* Qcat = static_cast<float*>(workspace);
-  TQ_CHECK_CUDA(prepare_queries(plan, Q, q_dtype, nq, ldq, Qcat, st), who);
+  ScanEngine eng{};
+  if (plan->ms.ok) eng = pick_engine(plan, nq);
+  return score_on_workspace(plan, &eng, Q, q_dtype, nq, ldq, n, idx, qjl, gamma, norms, scores, lds, workspace,
+                            static_cast<cudaStream_t>(stream), who);
+}
+
+// ---- prepared queries: rotation and operand set-up once, any number of scans afterwards
+// Buffer: rotated queries, then one engine workspace per pass (per group of 256 queries on the tcgen05 engine).
+static size_t prepared_slots(const ScanEngine& e, int nq) {
+  const int per = e.tc ? kGroupQueries : e.qpp;
+  return (size_t)((nq + per - 1) / per);
+}
+
+extern "C" size_t tq_query_bytes(const tq_plan* plan, int nq) {
+  if (!plan || nq <= 0) return 0;
+  size_t b = qcat_bytes(plan, nq);
   if (plan->ms.ok) {
-    void* msw = static_cast<char*>(workspace) + qcat_bytes(plan, nq);
-    const ScanEngine eng = pick_engine(plan, nq);
-    for (int q0 = 0; q0 < nq; q0 += eng.qpp) {
-      const int nqp = std::min(eng.qpp, nq - q0);
-      if ((rc = engine_prepare(eng, Qcat, q0, nq, msw, st, who))) return rc;
-      if ((rc = engine_run(eng, q0, nqp, n, idx, qjl, gamma, norms, scores + (int64_t)q0 * lds, lds, nullptr, nullptr, msw, st, who)))
-        return rc;
-    }
+    const ScanEngine e = pick_engine(plan, nq);
+    b += prepared_slots(e, nq) * align_up(e.ws_bytes, 256);
+  }
+  return b;
+}
+
+extern "C" int tq_query_prepare(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, void* prepared,
+                                size_t prepared_bytes, void* stream) {
+  const char* who = "tq_query_prepare";
+  int rc = check_plan(plan, who);
+  if (rc) return rc;
+  TQ_REQUIRE(nq >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
+  if (nq == 0) return TQ_OK;
+  if ((rc = check_rows(who, "Q", Q, q_dtype, nq, ldq, plan->d))) return rc;
+  const size_t need = tq_query_bytes(plan, nq);
+  TQ_REQUIRE(prepared != nullptr && prepared_bytes >= need, TQ_ERR_WORKSPACE, "%s: buffer of %zu bytes, %zu needed", who,
+             prepared_bytes, need);
+  TQ_REQUIRE(aligned(prepared, 256), TQ_ERR_ALIGNMENT, "%s: buffer is not 256-byte aligned", who);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* Qcat = static_cast<float*>(prepared);
+  TQ_CHECK_CUDA(prepare_queries(plan, Q, q_dtype, nq, ldq, Qcat, st), who);
+  if (!plan->ms.ok) return TQ_OK;
+  const ScanEngine eng = pick_engine(plan, nq);
+  const size_t slot = align_up(eng.ws_bytes, 256);
+  char* base = static_cast<char*>(prepared) + qcat_bytes(plan, nq);
+  const int per = eng.tc ? kGroupQueries : eng.qpp;
+  for (int q0 = 0; q0 < nq; q0 += per)
+    if ((rc = engine_prepare(eng, Qcat, q0, nq, base + (size_t)(q0 / per) * slot, st, who))) return rc;
+  return TQ_OK;
+}
+
+extern "C" int tq_score_prepared(const tq_plan* plan, const void* prepared, int nq, int64_t n, const uint8_t* idx,
+                                 const uint8_t* qjl, const float* gamma, const float* norms, float* scores, int64_t lds,
+                                 void* stream) {
+  const char* who = "tq_score_prepared";
+  int rc = check_plan(plan, who);
+  if (rc) return rc;
+  TQ_REQUIRE(n >= 0 && nq >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
+  if (n == 0 || nq == 0) return TQ_OK;
+  TQ_REQUIRE(prepared != nullptr && aligned(prepared, 256), TQ_ERR_INVALID_ARG, "%s: prepared buffer is NULL or misaligned", who);
+  if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
+  TQ_REQUIRE(scores != nullptr && lds >= n, TQ_ERR_INVALID_ARG, "%s: scores is NULL or lds < n", who);
+  TQ_REQUIRE(aligned(scores, 16), TQ_ERR_ALIGNMENT, "%s: scores is not 16-byte aligned", who);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const float* Qcat = static_cast<const float*>(prepared);
+  if (!plan->ms.ok) {
+    TQ_CHECK_CUDA(score_block(plan, Qcat, nq, 0, n, idx, qjl, gamma, norms, scores, lds, st), who);
     return TQ_OK;
   }
-  TQ_CHECK_CUDA(score_block(plan, Qcat, nq, 0, n, idx, qjl, gamma, norms, scores, lds, st), who);
+  const ScanEngine eng = pick_engine(plan, nq);
+  const size_t slot = align_up(eng.ws_bytes, 256);
+  const char* base = static_cast<const char*>(prepared) + qcat_bytes(plan, nq);
+  const int per = eng.tc ? kGroupQueries : eng.qpp;
+  for (int q0 = 0; q0 < nq; q0 += eng.qpp) {
+    const int nqp = std::min(eng.qpp, nq - q0);
+    const void* ws = base + (size_t)(q0 / per) * slot;
+    // the codes may have been written by the kernel just ahead in the stream: no early start of the scan here
+    if (eng.nib) rc = nscan::run(plan, nqp, n, idx, qjl, gamma, norms, scores + (int64_t)q0 * lds, lds, nullptr, nullptr, ws, false, st, who);
+    else rc = engine_run(eng, q0, nqp, n, idx, qjl, gamma, norms, scores + (int64_t)q0 * lds, lds, nullptr, nullptr, ws, st, who);
+    if (rc) return rc;
+  }
   return TQ_OK;
 }
 
@@ -958,6 +1092,21 @@ int static_scratch(const char* who, int device, void** out) {
 
 }  // namespace
 
+// Largest nq tq_score_static accepts for this plan (0 if even one query does not fit).
+extern "C" int tq_score_static_max_queries(const tq_plan* plan) {
+  if (!plan) return 0;
+  int lo = 0, hi = 1 << 16;
+  while (lo < hi) {   // the need grows with nq
+    const int mid = lo + (hi - lo + 1) / 2;
+    const size_t qb = qcat_bytes(plan, mid);
+    ScanEngine e{};
+    const bool ok = qb <= (size_t)TQ_STATIC_SCRATCH_BYTES &&
+                    (!plan->ms.ok || engine_that_fits(plan, mid, (size_t)TQ_STATIC_SCRATCH_BYTES - qb, &e));
+    if (ok) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
 extern "C" int tq_score_static(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, int64_t n,
                                const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms,
                                float* scores, int64_t lds, void* stream) {
@@ -966,22 +1115,19 @@ extern "C" int tq_score_static(const tq_plan* plan, const void* Q, int q_dtype, 
   if (rc) return rc;
   TQ_REQUIRE(n >= 0 && nq >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
   if (n == 0 || nq == 0) return TQ_OK;
-  if ((rc = check_rows(who, "Q", Q, q_dtype, nq, ldq, plan->d))) return rc;
-  if ((rc = check_codes(plan, who, idx, qjl, gamma))) return rc;
-  TQ_REQUIRE(scores != nullptr && lds >= n, TQ_ERR_INVALID_ARG, "%s: scores is NULL or lds < n", who);
-  TQ_REQUIRE(aligned(scores, 16), TQ_ERR_ALIGNMENT, "%s: scores is not 16-byte aligned", who);
-  const size_t need = qcat_bytes(plan, nq);
-  TQ_REQUIRE(need <= (size_t)TQ_STATIC_SCRATCH_BYTES, TQ_ERR_WORKSPACE,
-             "%s: %d queries at d=%d need %zu bytes of rotated-query scratch, the built-in array holds %u; "
-             "use tq_score with a caller workspace or fewer queries per call",
-             who, nq, plan->d, need, (unsigned)TQ_STATIC_SCRATCH_BYTES);
+  if ((rc = check_score_args(plan, who, Q, q_dtype, nq, ldq, n, idx, qjl, gamma, scores, lds))) return rc;
+  const size_t qb = qcat_bytes(plan, nq);
+  ScanEngine eng{};
+  const bool fits = qb <= (size_t)TQ_STATIC_SCRATCH_BYTES &&
+                    (!plan->ms.ok || engine_that_fits(plan, nq, (size_t)TQ_STATIC_SCRATCH_BYTES - qb, &eng));
+  TQ_REQUIRE(fits, TQ_ERR_WORKSPACE,
+             "%s: %d queries at d=%d need more scratch than the built-in array holds (%u bytes; at most %d queries "
+             "for this plan); use tq_score with a caller workspace or fewer queries per call",
+             who, nq, plan->d, (unsigned)TQ_STATIC_SCRATCH_BYTES, tq_score_static_max_queries(plan));
   void* ws = nullptr;
   if ((rc = static_scratch(who, plan->device, &ws))) return rc;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  float* Qcat = static_cast<float*>(ws);
-  // Every element of Qcat[nq, ncat*dpad] is written by prepare_queries before score_block reads
-  // it, so the previous call's leftovers never show.
-  TQ_CHECK_CUDA(prepare_queries(plan, Q, q_dtype, nq, ldq, Qcat, st), who);
-  TQ_CHECK_CUDA(score_block(plan, Qcat, nq, 0, n, idx, qjl, gamma, norms, scores, lds, st), who);
-  return TQ_OK;
+  // Every byte the kernels read from the array (rotated queries, then the scan engine's constants and operand)
+  // is written by this call before it is read, so the previous call's leftovers never show.
+  return score_on_workspace(plan, &eng, Q, q_dtype, nq, ldq, n, idx, qjl, gamma, norms, scores, lds, ws,
+                            static_cast<cudaStream_t>(stream), who);
 }

@@ -43,14 +43,15 @@ constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2-3 s of SM clock
 
 // Bounded wait.  `abort_flag` lives in shared memory; once any thread of the CTA gives up,
 // every other wait of that CTA returns false at its next check.
-static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                                   long long limit_cycles = kWaitLimitCycles) {
   const long long t0 = clock64();
   uint32_t polls = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((++polls & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit_cycles) {
         *abort_flag = 1;
         atomicExch(status, TQ_ERR_TIMEOUT);
         return false;

@@ -22,9 +22,9 @@ def _sample_rows(n, count, seed):
     return torch.unique(torch.cat([rows, extra[extra < n]])).to(DEV)
 
 
-def _check_full(name, bits, mode, n, nq, k, samples=1536):
+def _check_full(name, bits, mode, n, nq, k, samples=1536, layout=None):
     cfg = wl.CONFIGS[name]
-    su = P.Setup(cfg.d, bits, mode, cfg.pi_seed, cfg.s_seed)
+    su = P.Setup(cfg.d, bits, mode, cfg.pi_seed, cfg.s_seed, layout=layout)
     X = wl.database(cfg, n, device=DEV)
     Q = wl.queries(cfg, nq, device=DEV)
     idx, qjl, gamma, norms = su.quantize(X)
@@ -57,6 +57,10 @@ def test_c4_d1536_prod_b4_one_million():
     _check_full("c4", 4, tq.TQ_PROD, 1_000_000, 8, 100)
 
 
+def test_c4_d1536_prod_b4_one_million_nibble_layout():
+    _check_full("c4", 4, tq.TQ_PROD, 1_000_000, 8, 100, layout=tq.TQ_LAYOUT_NIBBLE)
+
+
 def test_c4_d1536_mse_b2_one_million():
     _check_full("c4", 2, tq.TQ_MSE, 1_000_000, 8, 100)
 
@@ -67,4 +71,4 @@ def test_c2_d200_prod_b3_one_million():
 
 @pytest.mark.parametrize("bits,k", [(2, 10), (4, 100)])
 def test_c5_d3072_prod(bits, k):
-    _check_full("c5", bits, tq.TQ_PROD, 400_000, 8, k, samples=768)
+    _check_full("c5", bits, tq.TQ_PROD, 1_000_000, 8, k, samples=768, layout=tq.TQ_LAYOUT_NIBBLE if bits == 4 else None)
