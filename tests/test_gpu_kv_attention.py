@@ -17,6 +17,14 @@ from tests import parity as P
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 HEAD_DIM, GROUP = 128, 64
+# Attention outputs (relative L2 error per output row) and softmax weights (relative, per weight) against the fp64
+# oracle on the same codes.  Measured worst cases at the full shape of the KV configuration (8 x 32,768 tokens):
+# outputs 2.1e-6 (separate calls), 2.1e-6 (fused), fused against separate 2.7e-6, weights 4.1e-6; the other
+# shapes and bit widths of this file 0.5e-6 .. 2.2e-6.  The bounds are about four times that: the logits are
+# fp32 sums of ~128 terms of magnitude up to ~30, i.e. ~1e-6 absolute after the 1/sqrt(128) scale, and the
+# weights and outputs inherit exactly that.
+S5_TOL = 1e-5
+S5_TOL_WEIGHTS = 2e-5
 
 
 def split_channels(Xh: torch.Tensor):
@@ -81,7 +89,9 @@ def test_kv_decode_full_shape(groups):
         # softmax weights against the oracle's, then the output rows
         p = np.exp(s / math.sqrt(HEAD_DIM) - (s / math.sqrt(HEAD_DIM)).max(axis=1, keepdims=True))
         p /= p.sum(axis=1, keepdims=True)
-        assert np.allclose(P.as_f64(W), p, rtol=2e-3, atol=1e-9)
+        wdev = np.abs(P.as_f64(W) - p) / np.maximum(p, 1e-9)
+        worst_w = max(locals().get("worst_w", 0.0), float(wdev[p > 1e-9].max()))
+        assert np.allclose(P.as_f64(W), p, rtol=S5_TOL_WEIGHTS, atol=1e-9)
         err = np.linalg.norm(P.as_f64(out) - ref, axis=1) / np.linalg.norm(ref, axis=1)
         worst = max(worst, float(err.max()))
         if h == 0:   # codes of the four groups of one head against the oracle's quantiser
@@ -90,6 +100,7 @@ def test_kv_decode_full_shape(groups):
                     st = P.check_quantize(su, Xg, *codes)
                     assert st["idx_mismatch"] == 0
     # logits carry the fp32 score error (<= 1e-4 of ||q|| nu) times 1/sqrt(128); weights and outputs inherit it
+    print(f"S5 measured: separate calls, full shape: output {worst:.3e}, weights {worst_w:.3e}")
     assert worst <= 1e-3, worst
 
 
@@ -170,7 +181,12 @@ def test_fused_decode_full_shape_against_the_separate_calls(groups):
     ref = torch.cat(outs)
     fused = _fused_layer(gK, gV, recs, Q, heads, T, 4)
     err = (fused - ref).norm(dim=1) / ref.norm(dim=1)
-    assert float(err.max()) <= 2e-4, float(err.max())
+    print(f"S5 measured: fused vs separate calls, full shape: {float(err.max()):.3e}")
+    assert float(err.max()) <= S5_TOL, float(err.max())
+    orc_ref = np.concatenate([attend_oracle(recs[h], Q[4 * h:4 * h + 4])[0] for h in range(heads)])
+    err_o = np.linalg.norm(P.as_f64(fused) - orc_ref, axis=1) / np.linalg.norm(orc_ref, axis=1)
+    print(f"S5 measured: fused vs oracle, full shape: {float(err_o.max()):.3e}")
+    assert float(err_o.max()) <= S5_TOL, float(err_o.max())
 
 
 @pytest.mark.parametrize("heads,T,qpk", [(2, 2500, 3), (1, 1024, 1), (3, 77, 4)])
@@ -186,7 +202,8 @@ def test_fused_decode_against_the_oracle(groups, heads, T, qpk):
     ref = np.concatenate(refs)
     fused = P.as_f64(_fused_layer(gK, gV, recs, Q, heads, T, qpk))
     err = np.linalg.norm(fused - ref, axis=1) / np.linalg.norm(ref, axis=1)
-    assert float(err.max()) <= 1e-3, float(err.max())
+    print(f"S5 measured: fused vs oracle heads={heads} T={T}: {float(err.max()):.3e}")
+    assert float(err.max()) <= S5_TOL, float(err.max())
 
 
 def test_fused_decode_other_bit_widths_and_argument_checks():
@@ -208,7 +225,8 @@ def test_fused_decode_other_bit_widths_and_argument_checks():
         fused = P.as_f64(_fused_layer(gK, gV, recs, Q, heads, T, qpk))
         ref = np.concatenate(refs)
         err = np.linalg.norm(fused - ref, axis=1) / np.linalg.norm(ref, axis=1)
-        assert float(err.max()) <= 1e-3, (kbits, kmode, vbits, float(err.max()))
+        print(f"S5 measured: fused vs oracle kbits={kbits} mode={kmode} vbits={vbits}: {float(err.max()):.3e}")
+        assert float(err.max()) <= S5_TOL, (kbits, kmode, vbits, float(err.max()))
     with pytest.raises(tq.TqError):     # a workspace that is too small is refused
         g = {"plan_k": gK[0].plan, "plan_v": gV[0].plan, "k_idx": recs[0]["K"][0][3][0], "k_qjl": recs[0]["K"][0][3][1],
              "k_gamma": recs[0]["K"][0][3][2], "k_norms": recs[0]["K"][0][3][3], "v_idx": recs[0]["V"][0][3][0],
@@ -274,7 +292,8 @@ def test_streaming_append_then_decode(groups):
     torch.cuda.synchronize()
     ref = np.concatenate([attend_oracle(recs[h], Q[qpk * h:qpk * h + qpk])[0] for h in range(heads)])
     err = np.linalg.norm(P.as_f64(out) - ref, axis=1) / np.linalg.norm(ref, axis=1)
-    assert float(err.max()) <= 1e-3, float(err.max())
+    print(f"S5 measured: appended cache, fused vs oracle: {float(err.max()):.3e}")
+    assert float(err.max()) <= S5_TOL, float(err.max())
     with pytest.raises(tq.TqError):
         tq.tq_kv_append(gds, heads, cap, cap, K[:, 0].contiguous(), V[:, 0].contiguous())   # position outside the cache
 
