@@ -577,14 +577,18 @@ struct Config {
 int nblocks_of(const tq_plan* plan) { return plan->nb.nbi + plan->nb.nbq; }
 
 size_t bfrag_bytes(const tq_plan* plan, bool tiled) {
-  // whole stages of four blocks, so that either stage size finds its operand
-  return (size_t)((nblocks_of(plan) + 3) / 4 * 4) * (tiled ? KPB_TILE : KPB_COL) * 32 * sizeof(uint2);
+  // whole stages of 2, 3 or 4 blocks, so that every stage size finds its operand
+  return (size_t)((nblocks_of(plan) + 11) / 12 * 12) * (tiled ? KPB_TILE : KPB_COL) * 32 * sizeof(uint2);
 }
 
-// Stages of four blocks when two of them fit beside the operand, else of two.
+// Blocks per stage: as measured at d = 1536 on 10^6 rows, the two-query shape runs best on three (or more) stages
+// of three blocks (166 us against 172 us on two stages of four: its consumers outrun a shallow pipeline), the
+// eight-query shape, whose operand leaves room for two large or four small stages, on two stages of four (244 us
+// against 251 us: fewer, longer steps).
 bool pick_config(const tq_plan* plan, bool tiled, Config* out) {
   const size_t fixed = bfrag_bytes(plan, tiled) + 1024 /*alignment*/ + 2 * MAX_STAGES * 8 + 16 + 8 * sizeof(NQConst);
-  for (int sb : {4, 2}) {
+  const int order[2][3] = {{3, 2, 4}, {4, 3, 2}};
+  for (int sb : order[tiled ? 1 : 0]) {
     const size_t stage = (size_t)sb * BLOCK_BYTES;
     if (fixed + 2 * stage > (size_t)SMEM_LIMIT) continue;
     out->sb = sb;
@@ -628,8 +632,9 @@ cudaError_t launch_t(const CUtensorMap& mi, const CUtensorMap& mq, const ScanArg
 template <int TILED, int MODE>
 cudaError_t launch_sb(int sb, const CUtensorMap& mi, const CUtensorMap& mq, const ScanArgs& args, size_t smem, bool dependent,
                       cudaStream_t st) {
-  return sb == 4 ? launch_t<TILED, MODE, 4>(mi, mq, args, smem, dependent, st)
-                 : launch_t<TILED, MODE, 2>(mi, mq, args, smem, dependent, st);
+  return sb == 4   ? launch_t<TILED, MODE, 4>(mi, mq, args, smem, dependent, st)
+         : sb == 3 ? launch_t<TILED, MODE, 3>(mi, mq, args, smem, dependent, st)
+                   : launch_t<TILED, MODE, 2>(mi, mq, args, smem, dependent, st);
 }
 
 }  // namespace
@@ -695,7 +700,7 @@ int prepare(const tq_plan* plan, const float* Qcat, int nqp, void* workspace, cu
   pa.nbi = plan->nb.nbi;
   pa.idx_rb = (int)plan->idx_row_bytes;
   pa.qjl_rb = (int)plan->qjl_row_bytes;
-  pa.nblocks = (nblocks_of(plan) + 3) / 4 * 4;   // blocks beyond the rows get a zero operand
+  pa.nblocks = (nblocks_of(plan) + 11) / 12 * 12;   // blocks beyond the rows get a zero operand
   pa.tiled = tiled ? 1 : 0;
   pa.delta = plan->nb.delta;
   pa.out = reinterpret_cast<uint2*>(static_cast<char*>(workspace) + kQConstBytes);
