@@ -1,4 +1,5 @@
 // C ABI of libtq: argument checking, plan set-up and kernel dispatch.
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <mutex>
@@ -291,13 +292,13 @@ cudaError_t launch_rotate_queries(const tq_plan* plan, const T* Q, int64_t ldq, 
   const int ncols = plan->ncat * plan->dpad;
   constexpr int smem = kRotQ * kRotChunk * (int)sizeof(float);
   // function attributes are per device: remember the devices this launcher has prepared
-  static unsigned long long attr_devices = 0;
+  static std::atomic<unsigned long long> attr_devices{0};   // written by any thread that launches
   int attr_dev = 0;
   if (cudaGetDevice(&attr_dev) != cudaSuccess) return cudaErrorInvalidDevice;
-  if (attr_dev >= 64 || !((attr_devices >> attr_dev) & 1ull)) {
+  if (attr_dev >= 64 || !((attr_devices.load(std::memory_order_relaxed) >> attr_dev) & 1ull)) {
     cudaError_t e = cudaFuncSetAttribute(rotate_queries_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    if (attr_dev < 64) attr_devices |= 1ull << attr_dev;
+    if (attr_dev < 64) attr_devices.fetch_or(1ull << attr_dev, std::memory_order_relaxed);
   }
   const dim3 grid((unsigned)((ncols + 7) / 8), (unsigned)((nq + kRotQPerBlock - 1) / kRotQPerBlock));
   rotate_queries_kernel<T><<<grid, 256, smem, st>>>(plan->dRotCat, ncols, plan->d, Q, ldq, nq, Qcat, ncols);
@@ -658,10 +659,8 @@ extern "C" int tq_quantize_prod(const tq_plan* plan, const void* X, int x_dtype,
     TQ_REQUIRE(scratch != nullptr && scratch_bytes >= least, TQ_ERR_WORKSPACE,
                "%s: scratch of %zu bytes, at least %zu needed", who, scratch_bytes, least);
     TQ_REQUIRE(aligned(scratch, 256), TQ_ERR_ALIGNMENT, "%s: scratch is not 256-byte aligned", who);
-    if ((rc = tc::quantize(plan, X, x_dtype, n, ldx, idx, qjl, gamma, norms, scratch, scratch_bytes, st, who))) return rc;
-    // the GEMM epilogues write the bit streams; the nibble layout is an in-place permutation of each row
-    if (plan->layout == TQ_LAYOUT_NIBBLE) return nscan::convert(plan, n, idx, qjl, TQ_LAYOUT_NIBBLE, st, who);
-    return TQ_OK;
+    // (the GEMM epilogues write whichever layout the plan has)
+    return tc::quantize(plan, X, x_dtype, n, ldx, idx, qjl, gamma, norms, scratch, scratch_bytes, st, who);
   }
   const size_t need = tq_workspace_bytes(plan, TQ_OP_QUANTIZE, n, 0, 0);
   TQ_REQUIRE(scratch != nullptr && scratch_bytes >= need, TQ_ERR_WORKSPACE, "%s: scratch of %zu bytes, %zu needed", who,

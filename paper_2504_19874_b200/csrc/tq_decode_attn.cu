@@ -5,7 +5,7 @@
 //
 //   prepare_kernel   per (head, group): gathers the group's channels of the head's queries and forms
 //                    q' = Pi q, q'' = S q.
-//   partial_kernel   per (head, slice of <= 1024 tokens), flash-decode style:
+//   partial_kernel   per (head, slice of 256 tokens), flash-decode style:
 //                    A) thread = token.  The MSE term sum_c q'_c c[idx_c] and the QJL term
 //                       sum_i q''_i z_i are sums of table entries: four index bits (4, 2 or 1
 //                       coordinates; one coordinate for 3-bit indices) select one float4 holding the
@@ -20,6 +20,7 @@
 // Work per token is ~50 warp instructions, i.e. CUDA-core bound at roughly 10x the time the code
 // bytes take from HBM; the unfused path (tq_score, tq_softmax, tq_wsum per head and group) is two
 // orders of magnitude slower at 32k tokens because each of its 88 launches serves one head.
+#include <atomic>
 #include <algorithm>
 #include <cfloat>
 #include <cstring>
@@ -477,7 +478,9 @@ __global__ void __launch_bounds__(MAXD) append_kernel(AppendArgs a, const T* __r
   }
   xs[j] = x;
   if (j < (int)(sizeof(words) / sizeof(words[0]))) words[j] = 0u;
-  const float nu = sqrtf(block_sum(x * x));   // the sync inside also publishes xs and words
+  float nu = sqrtf(block_sum(x * x));   // the sync inside also publishes xs and words
+  // no norms array: the row is taken as already unit-norm and quantised as it is, like tq_quantize_*
+  if ((isv ? g.v_norms : g.k_norms) == nullptr) nu = 1.f;
   const float inv = nu > 0.f ? 1.f / nu : 0.f, vcmp = nu > 0.f ? nu : 1.f;
   const float* bt = isv ? g.v_backt : g.k_backt;
   const int ncols = isv ? g.v_ncols : g.k_ncols;
@@ -522,6 +525,21 @@ size_t workspace_bytes(int ngroups, int heads, int64_t tokens, int d) {
   return (b + 255) / 256 * 256;
 }
 
+}  // namespace kvdec
+}  // namespace tq
+
+namespace tq {
+namespace kvdec {
+struct ZeroArgs {
+  const int32_t* v_channels[MAXG];
+  int ngroups, d, q_per_kv;
+};
+// Row r = h * q_per_kv + j of `out`: zeros in the columns that receive the groups' coordinates for KV head h.
+__global__ void zero_channels_kernel(ZeroArgs z, float* __restrict__ out, int64_t ldo) {
+  const int r = blockIdx.x, h = r / z.q_per_kv;
+  for (int gi = 0; gi < z.ngroups; ++gi)
+    for (int c = threadIdx.x; c < z.d; c += blockDim.x) out[(int64_t)r * ldo + z.v_channels[gi][h * z.d + c]] = 0.f;
+}
 }  // namespace kvdec
 }  // namespace tq
 
@@ -589,9 +607,13 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
     g.v_idx_soff = vbytes;
     vbytes += (SLICE * g.v_idx_rb + 15) / 16 * 16;
   }
-  if (tokens == 0) {   // no tokens: the output rows are zero
-    TQ_CHECK_CUDA(cudaMemset2DAsync(out, (size_t)ldo * sizeof(float), 0, (size_t)ngroups * d * sizeof(float),
-                                    (size_t)heads * q_per_kv, st), who);
+  if (tokens == 0) {   // no tokens: the columns named by v_channels are zero
+    ZeroArgs z;
+    for (int gi = 0; gi < ngroups; ++gi) z.v_channels[gi] = groups[gi].v_channels;
+    z.ngroups = ngroups; z.d = d; z.q_per_kv = q_per_kv;
+    zero_channels_kernel<<<heads * q_per_kv, 128, 0, st>>>(z, out, ldo);
+    TQ_CHECK_CUDA(cudaGetLastError(), who);
+    count_launches(1);
     return TQ_OK;
   }
   const int64_t nslices = (tokens + SLICE - 1) / SLICE;
@@ -625,12 +647,10 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   const size_t smem = (size_t)a.region0 * sizeof(float4) + (size_t)ngroups * SLICE * sizeof(float4) + kbytes + vbytes +
                       MAXG * 16 * sizeof(float) + (NT / 32 + 1) * MAXQ * sizeof(float);
   TQ_REQUIRE(smem <= 220 * 1024, TQ_ERR_UNSUPPORTED, "%s: %zu bytes of shared memory needed (too many wide groups)", who, smem);
-  static size_t smem_set[16] = {0};
-  if (dev < 16 && smem > smem_set[dev]) {
+  static std::atomic<size_t> smem_set[16];   // zero-initialised; written by any thread that launches
+  if (dev >= 16 || smem > smem_set[dev].load(std::memory_order_relaxed)) {
     TQ_CHECK_CUDA(cudaFuncSetAttribute(partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), who);
-    smem_set[dev] = smem;
-  } else if (dev >= 16) {
-    TQ_CHECK_CUDA(cudaFuncSetAttribute(partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), who);
+    if (dev < 16) smem_set[dev].store(smem, std::memory_order_relaxed);
   }
   partial_kernel<<<(unsigned)(heads * nslices), NT, smem, st>>>(a);
   TQ_CHECK_CUDA(cudaGetLastError(), who);
@@ -681,6 +701,11 @@ extern "C" int tq_kv_append(const tq_kv_group* groups, int ngroups, int heads, i
     g.k_ncols = s.plan_k->ncat * s.plan_k->dpad; g.v_ncols = s.plan_v->ncat * s.plan_v->dpad;
   }
   a.ngroups = ngroups; a.heads = heads; a.d = d; a.head_stride = head_stride; a.position = position;
+  int dev = -1;
+  TQ_CHECK_CUDA(cudaGetDevice(&dev), who);
+  for (int gi = 0; gi < ngroups; ++gi)
+    TQ_REQUIRE(groups[gi].plan_k->device == dev && groups[gi].plan_v->device == dev, TQ_ERR_INVALID_ARG,
+               "%s: group %d: the plans belong to another device than the current one (%d)", who, gi, dev);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid((unsigned)(heads * ngroups), 2);
   if (kv_dtype == TQ_F32)

@@ -7,6 +7,7 @@
 // accumulation (3 MMA passes).  The dropped terms are ~2^-17 relative per product, i.e.
 // ~1e-7 on a rotated coordinate of a unit vector at d = 1536 -- far inside the 1e-5 window in
 // which a nearest-centroid decision may legitimately differ from exact arithmetic.
+#include <atomic>
 #include <algorithm>
 #include <mutex>
 
@@ -45,8 +46,24 @@ struct GemmArgs {
   float* gpart;          // MODE 1: [EPS * tiles_n][Mpad] partial sums of e^2 (one per epilogue warp's columns)
   int64_t Mpad;
   const float* nu;       // MODE 1: per-row norm (row with nu == 0 has residual 0); nullable
+  // TQ_LAYOUT_NIBBLE (BITS = 3 with MODE 1, and MODE 2): the codes of 32 coordinates are four words of the combined
+  // row [idx row | qjl row], nibble = index | sign << 3.  MODE 1 writes them with the sign bits clear, MODE 2 ORs
+  // the sign bits in.
+  int nibble;
+  uint8_t* nib_idx;      // idx rows (stride nib_idx_rb) and qjl rows (stride nib_qjl_rb) of this block of rows
+  uint8_t* nib_qjl;
+  size_t nib_idx_rb, nib_qjl_rb;
   int* status;
 };
+
+// Bit i of the low byte of x at bit 4 i + 3.
+__device__ __forceinline__ uint32_t spread_to_nibble_tops(uint32_t x) {
+  x &= 0xffu;
+  x = (x | (x << 12)) & 0x000f000fu;
+  x = (x | (x << 6)) & 0x03030303u;
+  x = (x | (x << 3)) & 0x11111111u;
+  return x << 3;
+}
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -161,7 +178,7 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------ epilogue (8 warps: 4 TMEM lane groups x 2 column halves)
+    // ------------------------------------------------------------ epilogue (4 x EPS warps: 4 TMEM lane groups x EPS column parts)
     const int lg = warp & 3;   // TMEM lane group this warp may read
     const int half = (warp - 2) >> 2;   // which part (of EPS) of the tile's columns this warp takes
     bool ok = true;
@@ -194,12 +211,27 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
             word |= (bit ? 1u : 0u) << i;
           }
           const size_t w = (size_t)(col0 >> 5);
-          if (row_ok && w < row_words) out_row[w] = word;
+          if (a.nibble) {
+            const size_t off = 16 * w;   // the group's four words of the combined row
+            if (row_ok && off < a.nib_idx_rb + a.nib_qjl_rb) {
+              uint4* dst = reinterpret_cast<uint4*>(off < a.nib_idx_rb ? a.nib_idx + (size_t)row * a.nib_idx_rb + off
+                                                                       : a.nib_qjl + (size_t)row * a.nib_qjl_rb + (off - a.nib_idx_rb));
+              uint4 cur = *dst;   // written by the rotate launch of the same block of rows
+              cur.x |= spread_to_nibble_tops(word);
+              cur.y |= spread_to_nibble_tops(word >> 8);
+              cur.z |= spread_to_nibble_tops(word >> 16);
+              cur.w |= spread_to_nibble_tops(word >> 24);
+              *dst = cur;
+            }
+          } else if (row_ok && w < row_words) {
+            out_row[w] = word;
+          }
         } else {
           constexpr int NB = (1 << BITS) - 1;
           unsigned long long bitbuf = 0;
           int nb = 0, nw = 0;
           uint32_t words[BITS > 0 ? BITS : 1];
+          uint32_t nibw[4] = {0u, 0u, 0u, 0u};
           uint32_t e1[16], e2[16];
 #pragma unroll
           for (int i2 = 0; i2 < 16; ++i2) {
@@ -213,6 +245,7 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
 #pragma unroll
               for (int tix = 0; tix < NB; ++tix) code += (y > a.cb.t[tix]) ? 1 : 0;
               if (!col_ok) code = 0;
+              if (BITS == 3 && MODE == 1) nibw[i >> 3] |= (uint32_t)code << (4 * (i & 7));
               if (BITS > 0) {
                 bitbuf |= (unsigned long long)code << nb;
                 nb += BITS;
@@ -234,7 +267,14 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
               e2[i2] = pack_bf16x2(elo[0], elo[1]);
             }
           }
-          if (BITS > 0 && row_ok) {
+          if (BITS == 3 && MODE == 1 && a.nibble) {
+            const size_t off = 16 * (size_t)(col0 >> 5);
+            if (row_ok && off < a.nib_idx_rb + a.nib_qjl_rb) {
+              uint4* dst = reinterpret_cast<uint4*>(off < a.nib_idx_rb ? a.nib_idx + (size_t)row * a.nib_idx_rb + off
+                                                                       : a.nib_qjl + (size_t)row * a.nib_qjl_rb + (off - a.nib_idx_rb));
+              *dst = make_uint4(nibw[0], nibw[1], nibw[2], nibw[3]);
+            }
+          } else if (BITS > 0 && row_ok) {
             const size_t w0 = (size_t)(col0 >> 5) * BITS;
 #pragma unroll
             for (int q = 0; q < BITS; ++q)
@@ -259,7 +299,14 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
       if (lane == 0) mbar_arrive(&tempty[acc]);
       if (MODE == 1 && row_ok) a.gpart[(int64_t)(EPS * tn + half) * a.Mpad + row] = gsum;
       // pad words past the last tile's columns (rows whose stride exceeds the tiles' coverage)
-      if (tn == a.tiles_n - 1 && half == EPS - 1 && row_ok) {
+      if (a.nibble && tn == a.tiles_n - 1 && half == EPS - 1 && row_ok) {
+        if (MODE == 1) {   // words of the combined row that no group of 32 coordinates owns
+          const size_t wi = a.nib_idx_rb / 4, wq = a.nib_qjl_rb / 4;
+          for (size_t w = (size_t)((a.N + 31) >> 5) * 4; w < wi + wq; ++w)
+            (w < wi ? reinterpret_cast<uint32_t*>(a.nib_idx + (size_t)row * a.nib_idx_rb)[w]
+                    : reinterpret_cast<uint32_t*>(a.nib_qjl + (size_t)row * a.nib_qjl_rb)[w - wi]) = 0u;
+        }
+      } else if (tn == a.tiles_n - 1 && half == EPS - 1 && row_ok) {
         constexpr int kBitsPerCoord = (MODE == 2) ? 1 : BITS;
         if (kBitsPerCoord > 0) {
           const size_t covered = (size_t)((a.N + 31) >> 5) * kBitsPerCoord;
@@ -390,11 +437,13 @@ bool make_byte_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t r
 }
 
 int sm_count() {
-  static int sms = 0;
+  static std::atomic<int> cached{0};   // all devices of a process are taken to be alike
+  int sms = cached.load(std::memory_order_relaxed);
   if (sms == 0) {
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cached.store(sms, std::memory_order_relaxed);
   }
   return sms;
 }
@@ -406,13 +455,13 @@ cudaError_t launch_gemm_t(const CUtensorMap& a1, const CUtensorMap& a2, const CU
                           const GemmArgs& args, cudaStream_t st) {
   auto kern = quantize_gemm_kernel<BN, MODE, BITS>;
   // function attributes are per device: remember the devices this launcher has prepared
-  static unsigned long long attr_devices = 0;
+  static std::atomic<unsigned long long> attr_devices{0};   // written by any thread that launches
   int attr_dev = 0;
   if (cudaGetDevice(&attr_dev) != cudaSuccess) return cudaErrorInvalidDevice;
-  if (attr_dev >= 64 || !((attr_devices >> attr_dev) & 1ull)) {
+  if (attr_dev >= 64 || !((attr_devices.load(std::memory_order_relaxed) >> attr_dev) & 1ull)) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes);
     if (e != cudaSuccess) return e;
-    if (attr_dev < 64) attr_devices |= 1ull << attr_dev;
+    if (attr_dev < 64) attr_devices.fetch_or(1ull << attr_dev, std::memory_order_relaxed);
   }
   const int64_t tiles = (int64_t)args.tiles_m * args.tiles_n;
   const int grid = (int)std::min<int64_t>(tiles, sm_count());
@@ -545,6 +594,11 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     g.gpart = gpart;
     g.Mpad = R;
     g.nu = nu_out;
+    g.nibble = (plan->layout == TQ_LAYOUT_NIBBLE) ? 1 : 0;
+    g.nib_idx = idx ? idx + (size_t)r0 * plan->idx_row_bytes : nullptr;
+    g.nib_qjl = qjl ? qjl + (size_t)r0 * plan->qjl_row_bytes : nullptr;
+    g.nib_idx_rb = plan->idx_row_bytes;
+    g.nib_qjl_rb = plan->qjl_row_bytes;
     g.status = plan->d_status;
     // 2. y = Pi u, idx (+ residual limbs and partial norms)
     if (!prod) {

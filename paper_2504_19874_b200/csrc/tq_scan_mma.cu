@@ -27,6 +27,7 @@
 // shared memory.  The epilogue recombines the digit columns exactly (64-bit integer), applies gamma, nu and
 // the per-query constants in fp32 and either stores dense scores or appends (score, id) pairs that pass a
 // per-query threshold to a candidate list (top-k).
+#include <atomic>
 #include <algorithm>
 #include <cmath>
 
@@ -762,13 +763,13 @@ template <int BM, bool PROD, int NW, int MT, int NT, int MODE>
 cudaError_t launch_t(const CUtensorMap& mi, const CUtensorMap& mq, const ScanArgs& args, size_t smem, cudaStream_t st) {
   auto kern = scan_mma_kernel<BM, PROD, NW, MT, NT, MODE>;
   // function attributes are per device: the largest size set so far, per device
-  static size_t attr[64] = {0};
+  static std::atomic<size_t> attr[64];   // zero-initialised; written by any thread that launches
   int attr_dev = 0;
   if (cudaGetDevice(&attr_dev) != cudaSuccess) return cudaErrorInvalidDevice;
-  if (attr_dev >= 64 || smem > attr[attr_dev]) {
+  if (attr_dev >= 64 || smem > attr[attr_dev].load(std::memory_order_relaxed)) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    if (attr_dev < 64) attr[attr_dev] = smem;
+    if (attr_dev < 64) attr[attr_dev].store(smem, std::memory_order_relaxed);
   }
   const int grid = (int)std::min<int64_t>(args.ntiles, tc::sm_count());
   kern<<<grid, 32 * (NW + 1), smem, st>>>(mi, mq, args);

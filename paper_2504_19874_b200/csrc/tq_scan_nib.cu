@@ -503,9 +503,8 @@ scan_nib_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
 }
 
 // ------------------------------------------------------------------ layout conversion
-// One CTA per group of rows: the rows' coordinates are unpacked to one byte each (index | sign << 3) in shared
-// memory, then every thread assembles 32-bit words of the target layout.  In place: a row is read completely
-// before any of it is written.
+// One warp per row, one lane per group of 32 coordinates (three idx words + one qjl word <-> four words of the
+// combined nibble row).  In place: a warp holds its whole row in registers before it writes any of it.
 struct ConvArgs {
   int64_t n;
   uint8_t* idx;
@@ -513,57 +512,84 @@ struct ConvArgs {
   int d, idx_rb, qjl_rb, to_nibble;
 };
 
-constexpr int CONV_ROWS = 4;
+constexpr int CONV_MAX_GROUPS_PER_LANE = TQ_MAX_D / 32 / 32;   // 8
 
 __global__ void __launch_bounds__(256) convert_kernel(ConvArgs a) {
-  extern __shared__ unsigned char cs[];   // [CONV_ROWS][dround] unpacked coordinates, dround = 2 (idx_rb + qjl_rb)
-  const int dround = 2 * (a.idx_rb + a.qjl_rb);
-  const int64_t r0 = (int64_t)blockIdx.x * CONV_ROWS;
-  const int nrows = (int)min((int64_t)CONV_ROWS, a.n - r0);
-  for (int e = threadIdx.x; e < nrows * dround; e += blockDim.x) {
-    const int r = e / dround, j = e % dround;
-    const uint8_t* ri = a.idx + (size_t)(r0 + r) * a.idx_rb;
-    const uint8_t* rq = a.qjl + (size_t)(r0 + r) * a.qjl_rb;
-    unsigned v = 0;
-    if (j < a.d) {
-      if (a.to_nibble) {   // source: bit streams
-        const int bp = 3 * j, b0 = bp >> 3, sh = bp & 7;
-        unsigned x = ri[b0];
-        if (sh > 5) x |= (unsigned)ri[b0 + 1] << 8;
-        v = ((x >> sh) & 7u) | (((rq[j >> 3] >> (j & 7)) & 1u) << 3);
-      } else {             // source: nibbles
-        const int byte = j >> 1;
-        const unsigned x = byte < a.idx_rb ? ri[byte] : rq[byte - a.idx_rb];
-        v = (x >> (4 * (j & 1))) & 15u;
-      }
-    }
-    cs[e] = (unsigned char)v;
-  }
-  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= a.n) return;
+  uint32_t* ri = reinterpret_cast<uint32_t*>(a.idx + (size_t)row * a.idx_rb);
+  uint32_t* rq = reinterpret_cast<uint32_t*>(a.qjl + (size_t)row * a.qjl_rb);
   const int wi = a.idx_rb / 4, wq = a.qjl_rb / 4;
-  for (int e = threadIdx.x; e < nrows * (wi + wq); e += blockDim.x) {
-    const int r = e / (wi + wq), wd = e % (wi + wq);
-    const unsigned char* c = cs + r * dround;
-    uint32_t out = 0;
-    if (a.to_nibble) {
-      const int j0 = 8 * wd;   // word wd of the combined row
+  const int ngroups = (a.d + 31) / 32;
+  // word w of the combined row [idx row | qjl row]
+  auto comb = [&](int w) -> uint32_t* { return w < wi ? ri + w : rq + (w - wi); };
+  uint32_t in[CONV_MAX_GROUPS_PER_LANE][4];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) out |= (uint32_t)c[j0 + i] << (4 * i);
-    } else if (wd < wi) {
-#pragma unroll 4
-      for (int b = 0; b < 32; ++b) {
-        const int bp = 32 * wd + b, j = bp / 3;
-        if (j < a.d) out |= (uint32_t)((c[j] >> (bp - 3 * j)) & 1u) << b;
-      }
+  for (int t = 0; t < CONV_MAX_GROUPS_PER_LANE; ++t) {
+    const int g = lane + 32 * t;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) in[t][i] = 0u;
+    if (g >= ngroups) continue;
+    if (a.to_nibble) {
+#pragma unroll
+      for (int i = 0; i < 3; ++i)
+        if (3 * g + i < wi) in[t][i] = ri[3 * g + i];
+      if (g < wq) in[t][3] = rq[g];
     } else {
-      const int j0 = 32 * (wd - wi);
-#pragma unroll 4
-      for (int b = 0; b < 32; ++b)
-        if (j0 + b < a.d) out |= (uint32_t)((c[j0 + b] >> 3) & 1u) << b;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (4 * g + i < wi + wq) in[t][i] = *comb(4 * g + i);
     }
-    uint32_t* dst = wd < wi ? reinterpret_cast<uint32_t*>(a.idx + (size_t)(r0 + r) * a.idx_rb) + wd
-                            : reinterpret_cast<uint32_t*>(a.qjl + (size_t)(r0 + r) * a.qjl_rb) + (wd - wi);
-    *dst = out;
+  }
+  __syncwarp();
+#pragma unroll
+  for (int t = 0; t < CONV_MAX_GROUPS_PER_LANE; ++t) {
+    const int g = lane + 32 * t;
+    if (g >= ngroups) continue;
+    const int valid = min(32, a.d - 32 * g);   // coordinates of this group that exist
+    uint32_t out[4] = {0u, 0u, 0u, 0u};
+    if (a.to_nibble) {
+      const unsigned long long lo = (unsigned long long)in[t][0] | ((unsigned long long)in[t][1] << 32);
+      const uint32_t hi = in[t][2], z = in[t][3];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) {
+        const int bp = 3 * c;
+        uint32_t f;
+        if (bp + 3 <= 64) f = (uint32_t)(lo >> bp) & 7u;
+        else if (bp >= 64) f = (hi >> (bp - 64)) & 7u;
+        else f = ((uint32_t)(lo >> bp) | (hi << (64 - bp))) & 7u;
+        const uint32_t nib = c < valid ? (f | (((z >> c) & 1u) << 3)) : 0u;
+        out[c >> 3] |= nib << (4 * (c & 7));
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (4 * g + i < wi + wq) *comb(4 * g + i) = out[i];
+    } else {
+      unsigned long long lo = 0ull;
+      uint32_t hi = 0u, z = 0u;
+#pragma unroll
+      for (int c = 0; c < 32; ++c) {
+        const uint32_t nib = c < valid ? (in[t][c >> 3] >> (4 * (c & 7))) & 15u : 0u;
+        const int bp = 3 * c;
+        const unsigned long long f = nib & 7u;
+        if (bp < 64) lo |= f << bp;
+        if (bp + 3 > 64) hi |= bp >= 64 ? (uint32_t)f << (bp - 64) : (uint32_t)(f >> (64 - bp));
+        z |= (nib >> 3) << c;
+      }
+      out[0] = (uint32_t)lo; out[1] = (uint32_t)(lo >> 32); out[2] = hi;
+#pragma unroll
+      for (int i = 0; i < 3; ++i)
+        if (3 * g + i < wi) ri[3 * g + i] = out[i];
+      if (g < wq) rq[g] = z;
+    }
+  }
+  // words that no group owns (row padding) are zero in either layout
+  if (a.to_nibble) {
+    for (int w = 4 * ngroups + lane; w < wi + wq; w += 32) *comb(w) = 0u;
+  } else {
+    for (int w = 3 * ngroups + lane; w < wi; w += 32) ri[w] = 0u;
+    for (int w = ngroups + lane; w < wq; w += 32) rq[w] = 0u;
   }
 }
 
@@ -766,10 +792,7 @@ int convert(const tq_plan* plan, int64_t n, uint8_t* idx, uint8_t* qjl, int to_l
   a.idx_rb = (int)plan->idx_row_bytes;
   a.qjl_rb = (int)plan->qjl_row_bytes;
   a.to_nibble = to_layout == TQ_LAYOUT_NIBBLE ? 1 : 0;
-  const size_t smem = (size_t)CONV_ROWS * 2 * (a.idx_rb + a.qjl_rb);
-  cudaError_t e = cudaFuncSetAttribute(convert_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  TQ_CHECK_CUDA(e, who);
-  convert_kernel<<<(unsigned)((n + CONV_ROWS - 1) / CONV_ROWS), 256, smem, st>>>(a);
+  convert_kernel<<<(unsigned)((n + 7) / 8), 256, 0, st>>>(a);
   count_launches(1);
   TQ_CHECK_CUDA(cudaGetLastError(), who);
   return TQ_OK;

@@ -34,6 +34,7 @@
 // barrier (one commit per issuer).  Ring positions and phases are masks and shifts of 32-bit counters: the
 // single-lane roles run dependent instruction chains, where 64-bit division costs real time.  All waits
 // are bounded.
+#include <atomic>
 #include <algorithm>
 #include <cmath>
 
@@ -631,13 +632,13 @@ cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& ms, const CUtenso
                      const ScanArgs& args, cudaStream_t st) {
   auto kern = scan_tc_kernel<BM, MODE>;
   // function attributes are per device: remember the devices this launcher has prepared
-  static unsigned long long attr_devices = 0;
+  static std::atomic<unsigned long long> attr_devices{0};   // written by any thread that launches
   int attr_dev = 0;
   if (cudaGetDevice(&attr_dev) != cudaSuccess) return cudaErrorInvalidDevice;
-  if (attr_dev >= 64 || !((attr_devices >> attr_dev) & 1ull)) {
+  if (attr_dev >= 64 || !((attr_devices.load(std::memory_order_relaxed) >> attr_dev) & 1ull)) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    if (attr_dev < 64) attr_devices |= 1ull << attr_dev;
+    if (attr_dev < 64) attr_devices.fetch_or(1ull << attr_dev, std::memory_order_relaxed);
   }
   const int grid = (int)std::min<int64_t>(args.npairs, tc::sm_count());
   kern<<<grid, NTHREADS, kSmemBytes, st>>>(ma, ms, pa, ps, args);

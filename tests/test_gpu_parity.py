@@ -93,7 +93,7 @@ def test_small_scratch_forces_several_blocks_of_rows():
         for u, v in zip(full, part):
             assert (u is None and v is None) or torch.equal(u, v)
         P.check_quantize(su, X, *part)
-        # room for a second set of operand limbs: blocks overlap on the plan's second stream
+        # a scratch between the minimum and the preferred size: more, smaller launches, same codes
         dpad = (cfg.d + 7) // 8 * 8
         piped = su.quantize(X, scratch_bytes=small + 256 * dpad * 4)
         for u, v in zip(full, piped):
