@@ -108,7 +108,7 @@ constexpr int kGroupQueries = tscan::kQueriesPerPass * tscan::kPassesPerGroup;
 struct ScanEngine {
   const tq_plan* plan;
   bool tc;
-  bool nib;                 // table-lookup scan of the nibble layout (2 or 8 queries per pass)
+  bool nib;                 // register-fed table-lookup scan of the nibble layout (2 or 8 queries per pass)
   int qpp;                  // queries per pass
   int64_t dense_rows_pref;  // rows of the dense score buffer that keep the rescue pass to a few launches
   size_t ws_bytes;          // engine workspace (constants + B operand)
@@ -118,10 +118,15 @@ ScanEngine pick_engine(const tq_plan* plan, int nq) {
   ScanEngine e;
   e.plan = plan;
   e.nib = plan->layout == TQ_LAYOUT_NIBBLE;
-  e.tc = !e.nib && nq >= 7 && tscan::available(plan);
-  e.qpp = e.nib ? nscan::queries_per_pass(plan, nq) : e.tc ? tscan::kQueriesPerPass : mscan::queries_per_pass(plan, nq);
+  // nibble layout (measured at n = 10^6): at d = 1536 a tcgen05 pass costs 0.53 ms against 0.28 ms per pass of the
+  // eight-query register-fed shape, so it wins from 15 queries on; where that shape does not fit shared memory
+  // (d = 3072: 0.84 ms against 0.35 ms per two-query pass) from five queries on
+  const int tc_from = !e.nib ? 7 : nscan::queries_per_pass(plan, 8) == 8 ? 15 : 5;
+  e.tc = nq >= tc_from && tscan::available(plan);
+  e.nib = e.nib && !e.tc;
+  e.qpp = e.tc ? tscan::kQueriesPerPass : e.nib ? nscan::queries_per_pass(plan, nq) : mscan::queries_per_pass(plan, nq);
   e.dense_rows_pref = e.tc ? (1 << 18) : (1 << 20);
-  e.ws_bytes = e.nib ? nscan::workspace_bytes(plan) : e.tc ? tscan::workspace_bytes(plan) : mscan::workspace_bytes(plan);
+  e.ws_bytes = e.tc ? tscan::workspace_bytes(plan) : e.nib ? nscan::workspace_bytes(plan) : mscan::workspace_bytes(plan);
   return e;
 }
 

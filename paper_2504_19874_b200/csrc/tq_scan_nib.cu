@@ -27,6 +27,7 @@
 #include <algorithm>
 #include <cmath>
 
+#include "tq_nib_common.cuh"
 #include "tq_quantize_tc.h"
 #include "tq_scan_nib.h"
 #include "tq_tc.cuh"
@@ -44,28 +45,13 @@ constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr int KPB_COL = 12, KPB_TILE = 28;  // operand elements (uint2) per lane and 64-byte block (two word pairs)
 constexpr size_t kQConstBytes = 256;
 
-struct NQConst {
-  float sa;   // mse term   = T  * sa
-  float ss;   // qjl term   = TQ * ss + cs
-  float cs;
-  int pad;
-};
+using NQConst = nib::QConst;
+using QScale = nib::QScale;
 
-// Coordinate whose nibble is nibble `nib` (0..7) of code word `wd` (0..3) that quad thread t4 holds of block b,
-// or -1 when that nibble lies in the zero fill.  Blocks are the 64-byte pieces of the sequence
-// [idx row | qjl row]; thread t4 owns bytes 16 t4 .. 16 t4 + 15 of a block.
-__host__ __device__ inline int coord_of(int nbi, int idx_rb, int qjl_rb, int d, int b, int t4, int wd, int nib) {
-  int coord;
-  if (b < nbi) {
-    const int byte = 64 * b + 16 * t4 + 4 * wd + (nib >> 1);
-    if (byte >= idx_rb) return -1;
-    coord = 2 * byte + (nib & 1);
-  } else {
-    const int byte = 64 * (b - nbi) + 16 * t4 + 4 * wd + (nib >> 1);
-    if (byte >= qjl_rb) return -1;
-    coord = 2 * idx_rb + 2 * byte + (nib & 1);
-  }
-  return coord < d ? coord : -1;
+// Coordinate whose nibble is nibble `nib` (0..7) of code word `wd` (0..3) that quad thread t4 holds of block b
+// (thread t4 owns bytes 16 t4 .. 16 t4 + 15 of a block), or -1 when that nibble lies in the zero fill.
+__host__ __device__ inline int coord_of(int nbi, int idx_rb, int qjl_rb, int d, int b, int t4, int wd, int nibble) {
+  return nib::coord_of_block(nbi, idx_rb, qjl_rb, d, b, 32 * t4 + 8 * wd + nibble);
 }
 
 // ------------------------------------------------------------------ query-side operand
@@ -78,25 +64,6 @@ struct PrepArgs {
   double delta;
   uint2* out;          // [nblocks][KPB][32], k-steps 2j and 2j + 1 of a lane side by side
 };
-
-struct QScale {
-  int fh;      // Wh = round(q' 2^fh)
-  double sq;   // J = round(q'' sq)
-};
-
-__device__ __forceinline__ double pow2_of(int e) {
-  if (e < -1000 || e > 1000) return ldexp(1.0, e);
-  return __hiloint2double((e + 1023) << 20, 0);
-}
-
-__device__ __forceinline__ int digit_of(long long J, int limb) {
-  int dg = 0;
-  for (int l = 0; l <= limb; ++l) {
-    dg = (int)(((J + 128) & 255) - 128);
-    J = (J - dg) >> 8;
-  }
-  return dg;
-}
 
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start while its
 // predecessor in the stream still runs; it must pass this wait before touching anything the predecessor
@@ -125,25 +92,9 @@ __device__ void query_scales(const PrepArgs& a, QScale* sc /* shared, [8] */) {
       sm2 += __shfl_xor_sync(0xffffffffu, sm2, o);
     }
     if (lane == 0) {
-      QScale s;
-      // |v| < 2^e  ->  |v| 2^(22 - e) < 2^22: Wh in three signed digits, Wl = Wh / 256 in two
-      s.fh = 0;
-      if (mx1 > 0.f && isfinite(mx1)) {
-        int e;
-        frexpf(mx1, &e);
-        s.fh = 22 - e;
-      }
-      // J in two signed digits (|J| <= 127 * 257): the scale need not be a power of two, so all of that range is used
-      s.sq = (mx2 > 0.f && isfinite(mx2)) ? 32639.0 / (double)mx2 : 1.0;
+      const QScale s = nib::make_scale(mx1, mx2);
       sc[warp] = s;
-      if (blockIdx.x == 0) {
-        NQConst c;
-        c.sa = (float)(a.delta * ldexp(1.0, 8 - s.fh));
-        c.ss = (float)(1.0 / (64.0 * s.sq));   // sum_i 2 q''_i z_i = (16 TQ3 + TQ7) / (64 sq)
-        c.cs = (float)(-sm2);
-        c.pad = 0;
-        a.qc[warp] = c;
-      }
+      if (blockIdx.x == 0) a.qc[warp] = nib::make_const(s, a.delta, sm2);
     }
   }
   __syncthreads();
@@ -193,8 +144,6 @@ __global__ void __launch_bounds__(256) nprep_kernel(PrepArgs a) {
   if (ql < a.nq_pass) {
     const float* q = a.Qcat + (int64_t)ql * a.ldq;
     const QScale qs = sc[ql];
-    const double scale = type == 0 ? pow2_of(qs.fh) : type == 1 ? pow2_of(qs.fh - 8) : qs.sq;
-    const double bound = type == 0 ? 4194304.0 : type == 1 ? 16384.0 : 32639.0;
 #pragma unroll
     for (int half = 0; half < 2; ++half)
 #pragma unroll
@@ -209,9 +158,8 @@ __global__ void __launch_bounds__(256) nprep_kernel(PrepArgs a) {
         }
         const int coord = coord_of(a.nbi, a.idx_rb, a.qjl_rb, a.d, b, t4, wd, nib);
         if (coord < 0) continue;
-        double J = rint((double)q[(type < 2 ? 0 : a.dpad) + coord] * scale);
-        if (!(fabs(J) <= bound)) J = 0.0;   // non-finite query entries contribute nothing
-        regs[half] |= (uint32_t)(digit_of((long long)J, digit) & 255) << (8 * i);
+        const long long J = nib::weight(qs, type < 2 ? type : 2, q[(type < 2 ? 0 : a.dpad) + coord]);
+        regs[half] |= (uint32_t)(nib::digit_of(J, digit) & 255) << (8 * i);
       }
   }
   a.out[((size_t)b * KPB + (ks & ~1)) * 32 + lane * 2 + (ks & 1)] = make_uint2(regs[0], regs[1]);

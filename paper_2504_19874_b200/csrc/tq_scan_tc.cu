@@ -38,6 +38,7 @@
 #include <algorithm>
 #include <cmath>
 
+#include "tq_nib_common.cuh"
 #include "tq_quantize_tc.h"
 #include "tq_scan_tc.h"
 #include "tq_tc.cuh"
@@ -76,6 +77,9 @@ struct Geo {
   int bm, d, dpad;
   int widx, wq;    // 32-bit words per idx / qjl row
   int kba, kbs;    // k-blocks of the MSE part and of the QJL part
+  // TQ_LAYOUT_NIBBLE: every 64-byte block of the combined row [idx row | qjl row] gives three k-blocks in turn --
+  // the h bytes (signed A), the l bytes, the sign bits -- of its 128 coordinates; kba holds their total, kbs = 0
+  int nib, nbi, nblk, idx_rb, qjl_rb;
 };
 
 __host__ __device__ inline int div_up(int a, int b) { return (a + b - 1) / b; }
@@ -91,6 +95,15 @@ Geo make_geo(const tq_plan* plan) {
   g.wq = (plan->mode == TQ_PROD) ? (int)(plan->qjl_row_bytes / 4) : 0;
   g.kba = g.bm == 0 ? 0 : g.bm == 3 ? div_up(g.widx, 3) : g.bm == 4 ? div_up(g.widx, 2) : div_up(g.widx, 4);
   g.kbs = div_up(g.wq, 4);
+  g.nib = plan->layout == TQ_LAYOUT_NIBBLE ? 1 : 0;
+  g.nbi = plan->nb.nbi;
+  g.nblk = plan->nb.nbi + plan->nb.nbq;
+  g.idx_rb = (int)plan->idx_row_bytes;
+  g.qjl_rb = (int)plan->qjl_row_bytes;
+  if (g.nib) {
+    g.kba = 3 * g.nblk;
+    g.kbs = 0;
+  }
   return g;
 }
 
@@ -127,8 +140,41 @@ struct StatArgs {
   int64_t ldq;
   int d, dpad, prod;
   double amax, csum;
+  int nib;          // nibble layout: the scales and constants of the table-lookup form
+  double delta;
   QConst* out;
 };
+
+// Nibble layout: one warp per query, the same reductions in the same order as the register-fed engine's
+// (lane-strided maxima in fp32, the sum of q'' in fp64 folded by xor shuffles).
+__global__ void __launch_bounds__(32) tstats_nib_kernel(StatArgs a) {
+  const int lane = threadIdx.x;
+  const float* q = a.Qcat + (int64_t)blockIdx.x * a.ldq;
+  float mx1 = 0.f, mx2 = 0.f;
+  double sm2 = 0.0;
+  for (int j = lane; j < a.d; j += 32) {
+    mx1 = fmaxf(mx1, fabsf(q[j]));
+    const float u = q[a.dpad + j];
+    mx2 = fmaxf(mx2, fabsf(u));
+    sm2 += (double)u;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+    mx2 = fmaxf(mx2, __shfl_xor_sync(0xffffffffu, mx2, o));
+    sm2 += __shfl_xor_sync(0xffffffffu, sm2, o);
+  }
+  if (lane == 0) {
+    const nib::QScale s = nib::make_scale(mx1, mx2);
+    const nib::QConst n = nib::make_const(s, a.delta, sm2);
+    QConst c;
+    c.sa = n.sa; c.ca = 0.f; c.ss = n.ss; c.cs = n.cs;
+    c.fa = s.fh; c.fs = 0;
+    // the real scale of the sign-bit weights travels in the two spare words
+    c.pad[0] = __double2loint(s.sq); c.pad[1] = __double2hiint(s.sq);
+    a.out[blockIdx.x] = c;
+  }
+}
 
 __global__ void __launch_bounds__(256) tstats_kernel(StatArgs a) {
   __shared__ double red[4][8];
@@ -243,9 +289,52 @@ __global__ void __launch_bounds__(256) tbprep_kernel(BPrepArgs a, int part, int 
   *reinterpret_cast<uint4*>(dst + 16) = make_uint4(out[4], out[5], out[6], out[7]);
 }
 
+// Nibble layout: one B matrix Bn[pass*96 + n][3 nblk * 128]; k-block 3 b + type of block b.  K-byte kappa of an h or l
+// k-block <-> coordinate kappa of the block; of a sign k-block: register kappa / 4 = 2 word + parity, byte i = kappa % 4
+// <-> coordinate 8 word + 2 i + parity (low nibbles, parity 0, have the value 8 and carry 16 J; high nibbles 128 and J).
+__global__ void __launch_bounds__(256) tbprep_nib_kernel(BPrepArgs a, int rows) {
+  const int nkb = a.g.kba;
+  const int64_t total = (int64_t)rows * nkb * 4;
+  const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (tid >= total) return;
+  const int wl = (int)(tid & 3);
+  const int kb = (int)((tid >> 2) % nkb);
+  const int row = (int)((tid >> 2) / nkb);      // pass * 96 + n
+  const int ql = (row / NCOL) * kQueriesPerPass + (row % NCOL) % kQueriesPerPass, limb = (row % NCOL) / kQueriesPerPass;
+  const int b = kb / 3, type = kb % 3;
+  uint32_t out[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+  if (ql < a.nqg) {
+    const float* q = a.Qcat + (int64_t)ql * a.ldq;
+    const QConst c = a.qc[ql];
+    nib::QScale sc;
+    sc.fh = c.fa;
+    sc.sq = __hiloint2double(c.pad[1], c.pad[0]);
+    for (int r = 0; r < 8; ++r)
+      for (int i = 0; i < 4; ++i) {
+        const int kappa = 32 * wl + 4 * r + i;
+        int cib, mul = 1;
+        if (type < 2) {
+          cib = kappa;
+        } else {
+          const int reg = kappa >> 2;
+          cib = 8 * (reg >> 1) + 2 * i + (reg & 1);
+          mul = (reg & 1) ? 1 : 16;
+        }
+        const int coord = nib::coord_of_block(a.g.nbi, a.g.idx_rb, a.g.qjl_rb, a.g.d, b, cib);
+        if (coord < 0) continue;
+        const long long J = mul * nib::weight(sc, type, q[(type < 2 ? 0 : a.g.dpad) + coord]);
+        out[r] |= (uint32_t)(nib::digit_of(J, limb) & 255) << (8 * i);
+      }
+  }
+  uint8_t* dst = a.Ba + (size_t)row * nkb * KB_BYTES + (size_t)kb * KB_BYTES + wl * 32;
+  *reinterpret_cast<uint4*>(dst) = make_uint4(out[0], out[1], out[2], out[3]);
+  *reinterpret_cast<uint4*>(dst + 16) = make_uint4(out[4], out[5], out[6], out[7]);
+}
+
 // ------------------------------------------------------------------ scan kernel
 struct ScanArgs {
   int64_t n, npairs;
+  uint32_t hi_a, hi_b, lo_a, lo_b;   // nibble layout: the 16-bit centroid table as bytes (h of entries 0..3, 4..7; l alike)
   Geo g;
   int pass, nqp;
   const QConst* qc;        // constants of this pass's queries
@@ -277,11 +366,16 @@ __device__ __forceinline__ void umma_i8_ts(uint32_t tmem_d, uint32_t tmem_a, uin
       : "memory");
 }
 // kind::i8: D = s32, A = unsigned 8-bit, B = signed 8-bit, both K-major.
-__host__ __device__ constexpr uint32_t idesc_i8(int M, int N) {
-  return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+__host__ __device__ constexpr uint32_t idesc_i8(int M, int N, bool a_signed = false) {
+  return (2u << 4) | ((a_signed ? 1u : 0u) << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
 }
 
-template <int BM, int MODE>
+template <int BM, int MODE, bool NIB = false>
 __global__ void __launch_bounds__(NTHREADS, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__ CUtensorMap tmBs,
                const __grid_constant__ CUtensorMap tmPa, const __grid_constant__ CUtensorMap tmPs, ScanArgs a) {
@@ -354,12 +448,18 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
         for (int f = 0; f < nkb_total; ++f, ++kc) {
           const bool part_s = f >= a.g.kba;
           const int kb = part_s ? f - a.g.kba : f;
-          if ((kb & 3) == 0) {   // the packed rows of the pair for the next four k-blocks
+          if (NIB ? (kb % 3 == 0) : ((kb & 3) == 0)) {   // the packed rows of the pair for the next group of k-blocks
             if (!(ok = tc::mbar_wait(&pempty[pstage], pphase ^ 1u, abort_flag, a.status))) break;
-            const int gb = part_s ? 64 : group_bytes(BM);
+            const int gb = (part_s || NIB) ? 64 : group_bytes(BM);
             tc::mbar_arrive_expect_tx(&pfull[pstage], (uint32_t)(2 * TILE * gb));
-            tc::tma_load_2d(pring + pstage * PTILE_BYTES, part_s ? &tmPs : &tmPa, &pfull[pstage], (kb >> 2) * gb,
-                            (int)(pair * (2 * TILE)));
+            if (NIB) {   // block kb / 3 of the combined row: from the idx rows, then from the qjl rows
+              const int b = kb / 3;
+              tc::tma_load_2d(pring + pstage * PTILE_BYTES, b < a.g.nbi ? &tmPa : &tmPs, &pfull[pstage],
+                              64 * (b < a.g.nbi ? b : b - a.g.nbi), (int)(pair * (2 * TILE)));
+            } else {
+              tc::tma_load_2d(pring + pstage * PTILE_BYTES, part_s ? &tmPs : &tmPa, &pfull[pstage], (kb >> 2) * gb,
+                              (int)(pair * (2 * TILE)));
+            }
             if (++pstage == P_STAGES) {
               pstage = 0;
               pphase ^= 1u;
@@ -401,7 +501,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
           if (!(ok = tc::mbar_wait(&bfull[bstage], (kc / B_STAGES) & 1u, abort_flag, a.status))) break;
           if (!(ok = tc::mbar_wait(&afull[stage], (kc / A_SLOTS) & 1u, abort_flag, a.status))) break;
           tc::tc_fence_after();
-          const bool part_s = f >= a.g.kba;
+          // nibble layout: k-blocks of h bytes (signed A), l bytes and sign bits in turn; the sign bits have the
+          // second accumulator
+          const int kind = NIB ? f % 3 : 0;
+          const bool part_s = NIB ? kind == 2 : f >= a.g.kba;
+          const uint32_t idesc_f = (NIB && kind == 0) ? idesc_i8(TILE, NCOL, true) : idesc;
           const uint64_t bdesc = bdesc0 + (uint64_t)(bstage * (BTILE_BYTES >> 4));
 #pragma unroll
           for (int t = 0; t < 2; ++t) {
@@ -409,7 +513,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
             const uint32_t d_tmem = tmem_base + (uint32_t)(t * D_COLS + (part_s ? NCOL : 0));
 #pragma unroll
             for (int step = 0; step < 4; ++step)   // 32 K-bytes per MMA: 8 TMEM columns of A, +32 bytes inside B's swizzled row
-              umma_i8_ts(d_tmem, a_tmem + 8 * step, bdesc + 2 * step, idesc, 1u);
+              umma_i8_ts(d_tmem, a_tmem + 8 * step, bdesc + 2 * step, idesc_f, 1u);
           }
           tc::umma_commit(&kdone[bstage]);   // A slot and B stage reusable once these MMAs have read them
         }
@@ -435,7 +539,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
     };
     auto load_gm = [&](int64_t pr) -> float {
       const int64_t rw = pr * (2 * TILE) + t * TILE + r;
-      return (pr < a.npairs && rw < a.n && a.g.kbs > 0) ? a.coef * __ldg(a.gamma + rw) : 0.f;
+      return (pr < a.npairs && rw < a.n && (a.g.kbs > 0 || NIB)) ? a.coef * __ldg(a.gamma + rw) : 0.f;
     };
     float nu_next = load_nu(blockIdx.x), gm_next = load_gm(blockIdx.x);
     for (int64_t pair = blockIdx.x; pair < a.npairs && ok; pair += gridDim.x, ++it) {
@@ -450,6 +554,23 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
 #pragma unroll
       for (int c = 0; c < D_COLS; c += 16) tc::tmem_fill16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(t * D_COLS + c), 0u);
 
+      // stores one k-block's 32 A registers of this row into the current A slot and announces it
+      auto store_a = [&](const uint32_t (&v)[32]) -> bool {
+        // A slot kt % 2 was last read by the MMAs of k-block kt - 2: completion number (kt - 2) / B_STAGES of its barrier
+        if (kt >= A_SLOTS) {
+          const uint32_t kp = kt - A_SLOTS;
+          if (!tc::mbar_wait(&kdone[kp & (B_STAGES - 1)], (kp / B_STAGES) & 1u, abort_flag, a.status)) return false;
+        }
+        tc::tc_fence_after();
+        tc::tmem_st32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(A_COL0 + t * (A_SLOTS * 32) + stage * 32), v);
+        tc::tmem_st_wait();
+        tc::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&afull[stage]);
+        if (++stage == A_SLOTS) stage = 0;
+        ++kt;
+        return true;
+      };
       // expands one k-block's words into the row's 128 bytes of the A tile of the current stage
       auto emit = [&](uint32_t (&w)[4], int f) -> bool {
         if (f >= nkb_total) return true;
@@ -477,20 +598,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
 #pragma unroll
           for (int e2 = 0; e2 < 4; ++e2) v[4 * c + e2] = x & (0x01010101u << (k0 + e2));
         }
-        // A slot kt % 2 was last read by the MMAs of k-block kt - 2: completion number (kt - 2) / B_STAGES of its barrier
-        if (kt >= A_SLOTS) {
-          const uint32_t kp = kt - A_SLOTS;
-          if (!tc::mbar_wait(&kdone[kp & (B_STAGES - 1)], (kp / B_STAGES) & 1u, abort_flag, a.status)) return false;
-        }
-        tc::tc_fence_after();
-        tc::tmem_st32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(A_COL0 + t * (A_SLOTS * 32) + stage * 32), v);
-        tc::tmem_st_wait();
-        tc::tc_fence_before();
-        __syncwarp();
-        if (lane == 0) tc::mbar_arrive(&afull[stage]);
-        if (++stage == A_SLOTS) stage = 0;
-        ++kt;
-        return true;
+        return store_a(v);
       };
       // groups of four k-blocks: the pair's packed rows arrive by TMA ([256 rows x group bytes], swizzled so that
       // row-per-thread 16-byte reads are conflict-free); the thread copies its row's bytes to registers, frees the
@@ -498,7 +606,48 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
       const int prow = t * TILE + r;   // row inside the pair
       int pstage = pstage_keep;
       uint32_t pphase = pphase_keep;
-      for (int f0 = 0; f0 < nkb_total && ok; f0 += 4) {
+      if (NIB) {
+        // nibble layout: a group is one 64-byte block of the combined row = 16 code words = 128 coordinates, expanded
+        // into three k-blocks: h bytes and l bytes by byte permutes with the masked word as selector, sign bits by masks
+        for (int f0 = 0; f0 < nkb_total && ok; f0 += 3) {
+          if (!(ok = tc::mbar_wait(&pfull[pstage], pphase, abort_flag, a.status))) break;
+          const unsigned char* ps = pring + pstage * PTILE_BYTES;
+          uint32_t x[16];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {   // 64 bytes per row, 64-byte swizzle: chunk c at c ^ ((row >> 1) & 3)
+            const uint4 v4 = *reinterpret_cast<const uint4*>(ps + prow * 64 + ((j ^ ((prow >> 1) & 3)) << 4));
+            x[4 * j] = v4.x; x[4 * j + 1] = v4.y; x[4 * j + 2] = v4.z; x[4 * j + 3] = v4.w;
+          }
+          __syncwarp();
+          if (lane == 0) tc::mbar_arrive(&pempty[pstage]);
+          if (++pstage == P_STAGES) {
+            pstage = 0;
+            pphase ^= 1u;
+          }
+          uint32_t v[32];
+#pragma unroll
+          for (int wd = 0; wd < 16; ++wd) {
+            const uint32_t sl = x[wd] & 0x77777777u;
+            v[2 * wd] = prmt(a.hi_a, a.hi_b, sl);
+            v[2 * wd + 1] = prmt(a.hi_a, a.hi_b, sl >> 16);
+          }
+          ok = ok && store_a(v);
+#pragma unroll
+          for (int wd = 0; wd < 16; ++wd) {
+            const uint32_t sl = x[wd] & 0x77777777u;
+            v[2 * wd] = prmt(a.lo_a, a.lo_b, sl);
+            v[2 * wd + 1] = prmt(a.lo_a, a.lo_b, sl >> 16);
+          }
+          ok = ok && store_a(v);
+#pragma unroll
+          for (int wd = 0; wd < 16; ++wd) {
+            v[2 * wd] = x[wd] & 0x08080808u;
+            v[2 * wd + 1] = x[wd] & 0x80808080u;
+          }
+          ok = ok && store_a(v);
+        }
+      }
+      for (int f0 = 0; !NIB && f0 < nkb_total && ok; f0 += 4) {
         // a part boundary inside a group cannot happen: each part starts a new group
         const bool part_s = f0 >= a.g.kba;
         if (!(ok = tc::mbar_wait(&pfull[pstage], pphase, abort_flag, a.status))) break;
@@ -557,7 +706,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
 #pragma unroll
         for (int l = 0; l < LIMBS; ++l) {
           if (a.g.kba > 0) tc::tmem_ld16(taddr + l * 32 + h * 16, va[l]);
-          if (a.g.kbs > 0) tc::tmem_ld16(taddr + NCOL + l * 32 + h * 16, vs[l]);
+          if (a.g.kbs > 0 || NIB) tc::tmem_ld16(taddr + NCOL + l * 32 + h * 16, vs[l]);
         }
         tc::tmem_ld_wait();
 #pragma unroll
@@ -571,7 +720,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
             const long long T = ((long long)(int)va[2][qq] * 256 + (int)va[1][qq]) * 256 + (int)va[0][qq];
             av = fmaf((float)T, c.sa, c.ca);
           }
-          if (a.g.kbs > 0) {
+          if (a.g.kbs > 0 || NIB) {
             const long long T = ((long long)(int)vs[2][qq] * 256 + (int)vs[1][qq]) * 256 + (int)vs[0][qq];
             sv = fmaf((float)T, c.ss, c.cs);
           }
@@ -627,10 +776,10 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
 constexpr size_t kSmemUsed = B_STAGES * BTILE_BYTES + P_STAGES * PTILE_BYTES + 1024 + 512 + kQueriesPerPass * (sizeof(QConst) + sizeof(float) + sizeof(int) + LBUF * sizeof(uint2));
 constexpr size_t kSmemBytes = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;
 
-template <int BM, int MODE>
+template <int BM, int MODE, bool NIB = false>
 cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
                      const ScanArgs& args, cudaStream_t st) {
-  auto kern = scan_tc_kernel<BM, MODE>;
+  auto kern = scan_tc_kernel<BM, MODE, NIB>;
   // function attributes are per device: remember the devices this launcher has prepared
   static std::atomic<unsigned long long> attr_devices{0};   // written by any thread that launches
   int attr_dev = 0;
@@ -649,6 +798,7 @@ cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& ms, const CUtenso
 template <int MODE>
 cudaError_t launch_bm(int bm, const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
                       const ScanArgs& args, cudaStream_t st) {
+  if (args.g.nib) return launch_t<3, MODE, true>(ma, ms, pa, ps, args, st);
   switch (bm) {
     case 0: return launch_t<0, MODE>(ma, ms, pa, ps, args, st);
     case 1: return launch_t<1, MODE>(ma, ms, pa, ps, args, st);
@@ -686,8 +836,11 @@ int prepare_group(const tq_plan* plan, const float* Qcat, int nqg, void* workspa
   sa.prod = plan->mode == TQ_PROD ? 1 : 0;
   sa.amax = plan->ms.amax;
   sa.csum = plan->ms.csum;
+  sa.nib = g.nib;
+  sa.delta = plan->nb.delta;
   sa.out = qc;
-  tstats_kernel<<<nqg, 256, 0, st>>>(sa);
+  if (g.nib) tstats_nib_kernel<<<nqg, 32, 0, st>>>(sa);
+  else tstats_kernel<<<nqg, 256, 0, st>>>(sa);
   count_launches(1);
   TQ_CHECK_CUDA(cudaGetLastError(), who);
   BPrepArgs ba;
@@ -701,6 +854,13 @@ int prepare_group(const tq_plan* plan, const float* Qcat, int nqg, void* workspa
   ba.Bs = Bs;
   const int passes = (nqg + kQueriesPerPass - 1) / kQueriesPerPass;
   const int rows = passes * NCOL;
+  if (g.nib) {
+    const int64_t total = (int64_t)rows * g.kba * 4;
+    tbprep_nib_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(ba, rows);
+    count_launches(1);
+    TQ_CHECK_CUDA(cudaGetLastError(), who);
+    return TQ_OK;
+  }
   for (int part = 0; part < 2; ++part) {
     const int nkb = part ? g.kbs : g.kba;
     if (nkb == 0) continue;
@@ -731,19 +891,24 @@ int run_pass(const tq_plan* plan, int pass, int nqp, int64_t n, const uint8_t* i
   if (g.kbs == 0) ms = ma;
   // packed rows: boxes of [256 rows x group bytes]; 64- and 32-byte boxes are swizzled (row-per-thread reads)
   CUtensorMap pa, ps;
-  const int gb = group_bytes(g.bm);
-  if (g.kba > 0)
+  const int gb = g.nib ? 64 : group_bytes(g.bm);
+  if (g.nib) {
+    TQ_REQUIRE(tc::make_byte_map(&pa, idx, (uint64_t)n, plan->idx_row_bytes, plan->idx_row_bytes, 64, 2 * TILE, 64) &&
+                   tc::make_byte_map(&ps, qjl, (uint64_t)n, plan->qjl_row_bytes, plan->qjl_row_bytes, 64, 2 * TILE, 64),
+               TQ_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (code rows)", who);
+  } else if (g.kba > 0)
     TQ_REQUIRE(tc::make_byte_map(&pa, idx, (uint64_t)n, plan->idx_row_bytes, plan->idx_row_bytes, gb, 2 * TILE,
                                  gb == 64 ? 64 : gb == 32 ? 32 : 0),
                TQ_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (idx rows)", who);
-  if (g.kbs > 0)
+  if (!g.nib && g.kbs > 0)
     TQ_REQUIRE(tc::make_byte_map(&ps, qjl, (uint64_t)n, plan->qjl_row_bytes, plan->qjl_row_bytes, 64, 2 * TILE, 64), TQ_ERR_CUDA,
                "%s: cuTensorMapEncodeTiled failed (qjl rows)", who);
-  if (g.kba == 0) pa = ps;
-  if (g.kbs == 0) ps = pa;
+  if (!g.nib && g.kba == 0) pa = ps;
+  if (!g.nib && g.kbs == 0) ps = pa;
   ScanArgs a;
   a.n = n;
   a.npairs = (n + 2 * TILE - 1) / (2 * TILE);
+  a.hi_a = plan->nb.hi_a; a.hi_b = plan->nb.hi_b; a.lo_a = plan->nb.lo_a; a.lo_b = plan->nb.lo_b;
   a.g = g;
   a.pass = pass;
   a.nqp = nqp;

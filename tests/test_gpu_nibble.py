@@ -57,8 +57,8 @@ def test_layout_is_refused_where_it_does_not_exist():
 
 
 @pytest.mark.parametrize("d", [128, 200, 520, 1536, 3072])
-@pytest.mark.parametrize("nq", [1, 2, 3, 8, 11])
-def test_scores_both_operand_shapes(d, nq):
+@pytest.mark.parametrize("nq", [1, 2, 3, 8, 11, 37])
+def test_scores_every_engine_and_operand_shape(d, nq):
     su = P.Setup(d, 4, tq.TQ_PROD, layout=NIB)
     n = 300 if d >= 1536 else 777
     X, Q = _data(d, n, nq, 1000 * d + nq)
@@ -66,9 +66,12 @@ def test_scores_both_operand_shapes(d, nq):
     sc = su.score(Q, n, *codes)
     P.check_scores(su, sc, Q, *codes)
     assert torch.equal(sc, su.score(Q, n, *codes))
-    # a query's estimate does not depend on which other queries share its pass, nor on the operand shape
+    # a query's estimate does not depend on which other queries share its pass, nor on the operand shape or engine
+    # (two-query and eight-query register-fed shapes, tcgen05 with 32 queries per pass)
     one = su.score(Q[nq - 1:nq].contiguous(), n, *codes)
     assert torch.equal(one[0], sc[nq - 1])
+    if nq > 8:
+        assert torch.equal(su.score(Q[:8].contiguous(), n, *codes), sc[:8])
 
 
 def test_measured_error_of_both_engines():
@@ -107,7 +110,7 @@ def test_topk_flows():
     d = 264
     su = P.Setup(d, 4, tq.TQ_PROD, layout=NIB)
     n, k = 70001, 100
-    for nq in (2, 6, 19):
+    for nq in (2, 6, 19, 40):
         X, Q = _data(d, n, nq, 99 + nq)
         codes = su.quantize(X)
         sc = su.score(Q, n, *codes)
