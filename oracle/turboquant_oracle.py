@@ -17,7 +17,9 @@ Pins (see tests/test_oracle_pins.py): closed-form b=1 centroid, the large-d
 centroids the paper prints for b=1,2, the distortion values of Theorems 1
 and 2 and both pairs of bounds, Pi Pi^T = I, brute-force argmin on tiny d,
 Monte-Carlo unbiasedness of the prod estimator, the 2/pi bias of the mse
-estimator at b=1, the index entropy at b=4.
+estimator at b=1, the index entropy at b=4; the entropy coder of the indices:
+dyadic probabilities, the worked example of RFC 1951 3.2.2, Kraft equality,
+optimality against brute force, a hand-computed row stream, round trips.
 `attend` (softmax-weighted sum over dequantised values) has no value in the
 paper to pin against beyond its textbook softmax definition: parity unpinned.
 `select_outlier_channels` is a harness rule the paper does not define:
@@ -297,3 +299,76 @@ def select_outlier_channels(X, count: int) -> np.ndarray:
     energy = np.sum(X * X, axis=0)
     order = np.lexsort((np.arange(energy.size), -energy))
     return np.sort(order[:count])
+
+
+# --------------------------------------------------------------------------
+# Entropy coding of the indices (Section 3.1, "entropy encoding codebook
+# pointers"): the index of a coordinate takes value l with probability p_l (the
+# mass of the l-th cell), so a lossless prefix code brings the average bit width
+# from b down towards the entropy of {p_l} (about 3.8 bits at b = 4).  The
+# paper names no particular code; this is a Huffman code over the 2^b values
+# (optimal among prefix codes), written out as the textbook algorithm, with the
+# code words assigned canonically from the lengths as in RFC 1951, 3.2.2.
+# Row format (the library's, stated in its header): every vector is coded on
+# its own; bit p of the row stream is bit (p & 7) of byte (p >> 3), code words
+# follow one another without gaps, each written from its most significant bit.
+# --------------------------------------------------------------------------
+def huffman_lengths(p) -> np.ndarray:
+    """Code length per symbol of a Huffman code for probabilities p (all > 0): repeatedly merge the two least
+    probable nodes; among equally probable nodes the one created earlier (leaves in symbol order first) goes first."""
+    p = [float(v) for v in p]
+    n = len(p)
+    if n == 1:
+        return np.array([0], dtype=np.uint8)
+    nodes = [(p[s], s, (s,)) for s in range(n)]           # (probability, creation order, symbols below)
+    depth = [0] * n
+    created = n
+    while len(nodes) > 1:
+        nodes.sort(key=lambda t: (t[0], t[1]))
+        a, b = nodes[0], nodes[1]
+        for s in a[2] + b[2]:
+            depth[s] += 1
+        nodes = nodes[2:] + [(a[0] + b[0], created, a[2] + b[2])]
+        created += 1
+    return np.array(depth, dtype=np.uint8)
+
+
+def canonical_codes(lengths) -> np.ndarray:
+    """Code word (as an integer, most significant bit first) per symbol from the lengths: symbols sorted by
+    (length, symbol) receive consecutive values, shifted left whenever the length grows (RFC 1951, 3.2.2)."""
+    lengths = [int(v) for v in lengths]
+    codes = [0] * len(lengths)
+    code, prev = 0, 0
+    for length, s in sorted((l, s) for s, l in enumerate(lengths) if l > 0):
+        code <<= length - prev
+        codes[s] = code
+        code += 1
+        prev = length
+    return np.array(codes, dtype=np.uint32)
+
+
+def entropy_encode_row(symbols, lengths, codes):
+    """(bytes, number of bits) of one row's code stream."""
+    bits = []
+    for s in symbols:
+        l, c = int(lengths[s]), int(codes[s])
+        bits.extend((c >> (l - 1 - i)) & 1 for i in range(l))
+    out = np.zeros((len(bits) + 7) // 8, dtype=np.uint8)
+    for pos, b in enumerate(bits):
+        out[pos >> 3] |= b << (pos & 7)
+    return out, len(bits)
+
+
+def entropy_decode_row(stream, count, lengths, codes) -> np.ndarray:
+    """`count` symbols read back from a row stream, one bit at a time (prefix property)."""
+    table = {(int(lengths[s]), int(codes[s])): s for s in range(len(lengths))}
+    out = np.zeros(count, dtype=np.uint8)
+    pos = 0
+    for j in range(count):
+        l, c = 0, 0
+        while (l, c) not in table:
+            c = (c << 1) | ((int(stream[pos >> 3]) >> (pos & 7)) & 1)
+            l += 1
+            pos += 1
+        out[j] = table[(l, c)]
+    return out

@@ -425,3 +425,60 @@ def test_outlier_channel_rule():
     X = np.ones((10, 6)); X[:, 4] = 3; X[:, 1] = 2; X[:, 5] = 2
     assert orc.select_outlier_channels(X, 2).tolist() == [1, 4]
     assert orc.select_outlier_channels(X, 3).tolist() == [1, 4, 5]
+
+
+# ------------------------------------------------------------------ entropy coding of the indices
+def test_huffman_on_dyadic_probabilities_has_the_textbook_lengths():
+    # p = 2^-len exactly: the optimal code assigns exactly -log2 p bits
+    assert orc.huffman_lengths([0.5, 0.25, 0.125, 0.125]).tolist() == [1, 2, 3, 3]
+    assert orc.huffman_lengths([0.125, 0.5, 0.125, 0.25]).tolist() == [3, 1, 3, 2]
+    assert orc.huffman_lengths([0.25] * 4).tolist() == [2, 2, 2, 2]
+
+
+def test_canonical_codes_follow_the_published_worked_example():
+    # RFC 1951, section 3.2.2: symbols A..H with lengths (3, 3, 3, 3, 3, 2, 4, 4)
+    codes = orc.canonical_codes([3, 3, 3, 3, 3, 2, 4, 4])
+    assert codes.tolist() == [0b010, 0b011, 0b100, 0b101, 0b110, 0b00, 0b1110, 0b1111]
+
+
+@pytest.mark.parametrize("d,b", [(1536, 4), (1536, 3), (200, 2), (64, 3)])
+def test_huffman_code_of_the_index_distribution(d, b):
+    c = orc.codebook(d, b)
+    p = orc.index_probabilities(d, c)
+    lengths = orc.huffman_lengths(p)
+    assert sum(2.0 ** -int(l) for l in lengths) == 1.0                      # Kraft equality: a complete prefix code
+    entropy = float(-(p * np.log2(p)).sum())
+    avg = float((p * lengths).sum())
+    assert entropy <= avg < entropy + 1.0                                     # optimal prefix code
+    order = np.argsort(-p, kind="stable")
+    assert np.all(np.diff(lengths[order].astype(int)) >= 0)                   # a likelier index never has the longer code
+    # no other length assignment satisfying Kraft does better (all assignments with lengths <= 8 at b <= 2)
+    if b <= 2:
+        import itertools
+        best = min(float((p * np.array(ls)).sum()) for ls in itertools.product(range(1, 6), repeat=1 << b)
+                   if sum(2.0 ** -l for l in ls) <= 1.0)
+        assert abs(best - avg) < 1e-12
+    if (d, b) == (1536, 4):
+        # Section 3.1: the entropy is about 3.8 bits at b = 4 and coding saves about 5 % of the bit width
+        assert abs(entropy - 3.8) < 0.05 and 0.03 < (4.0 - avg) / 4.0 < 0.07
+
+
+def test_entropy_row_stream_worked_example_and_round_trip():
+    lengths = np.array([2, 1, 3, 3], dtype=np.uint8)
+    codes = orc.canonical_codes(lengths)
+    assert codes.tolist() == [0b10, 0b0, 0b110, 0b111]
+    # symbols 1, 0, 3, 2, 1 -> bits 0 | 1 0 | 1 1 1 | 1 1 0 | 0, stream position p = bit (p & 7) of byte (p >> 3):
+    # byte 0 holds 0,1,0,1,1,1,1,1 from its least significant bit = 2 + 8 + 16 + 32 + 64 + 128 = 250; byte 1 holds 0,0
+    stream, nbits = orc.entropy_encode_row([1, 0, 3, 2, 1], lengths, codes)
+    assert nbits == 10
+    assert stream.tolist() == [250, 0]
+    assert orc.entropy_decode_row(stream, 5, lengths, codes).tolist() == [1, 0, 3, 2, 1]
+    rng = np.random.default_rng(0)
+    c = orc.codebook(256, 4)
+    p = orc.index_probabilities(256, c)
+    ln = orc.huffman_lengths(p)
+    cd = orc.canonical_codes(ln)
+    sym = rng.choice(16, size=500, p=p / p.sum())
+    st, nb = orc.entropy_encode_row(sym, ln, cd)
+    assert nb == int(ln[sym].sum())
+    assert np.array_equal(orc.entropy_decode_row(st, 500, ln, cd), sym)
