@@ -363,6 +363,36 @@ int tq_attend_decode(const tq_kv_group* groups, int ngroups, int heads, int64_t 
 int tq_kv_append(const tq_kv_group* groups, int ngroups, int heads, int64_t head_stride, int64_t position,
                  const void* K, const void* V, int kv_dtype, int64_t ldk, int64_t ldv, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Entropy coding of the indices (Section 3.1, the paragraph on entropy encoding the codebook pointers): index
+ * value l occurs with probability p_l, the mass of the l-th cell under the density of Lemma 1, so a lossless
+ * prefix code stores the indices in about the entropy of {p_l} instead of b bits per coordinate (3.8 bits at
+ * b = 4).  The paper leaves the code open; here it is a Huffman code given by its lengths, with code words assigned
+ * canonically (symbols sorted by (length, symbol) take consecutive values, shifted left when the length grows).
+ * Every vector is coded on its own.  Row stream: bit p is bit (p & 7) of byte (p >> 3); code words follow one
+ * another without gaps, each from its most significant bit; a row occupies a whole number of 32-bit words.
+ * Storage / transfer format only: the scans read the fixed-width rows (tq_entropy_unpack restores them exactly).
+ * Plans with TQ_LAYOUT_CANONICAL and b_m >= 1.
+ */
+/* Huffman code lengths (1..15 in general; the coder accepts up to 12) for the 2^bits index values of the given
+ * codebook in dimension d.  Host only.  centroids: host, 2^bits ascending; lengths: host out, 2^bits bytes. */
+int tq_entropy_lengths(int d, int bits, const float* centroids, uint8_t* lengths);
+/* Bytes of device workspace tq_entropy_measure needs for n rows. */
+size_t tq_entropy_workspace_bytes(int64_t n);
+/* Byte offset of every row's stream: row_offsets[i] for i < n, and row_offsets[n] = total bytes of the packed
+ * array (read it back to size the output of tq_entropy_pack).
+ *   lengths  host, 2^b_m code lengths (from tq_entropy_lengths or the caller's own; must satisfy Kraft's inequality)
+ *   idx      device, n canonical rows;  row_offsets device out, n + 1 values;  workspace device, 256-byte aligned */
+int tq_entropy_measure(const tq_plan* plan, const uint8_t* lengths, int64_t n, const uint8_t* idx,
+                       uint64_t* row_offsets, void* workspace, size_t workspace_bytes, void* stream);
+/* Writes the rows' streams at their offsets.  out: device, 4-byte aligned, out_bytes >= row_offsets[n]; if it is
+ * smaller the rows that do not fit are skipped and the next tq_plan_status(plan) reports an error. */
+int tq_entropy_pack(const tq_plan* plan, const uint8_t* lengths, int64_t n, const uint8_t* idx,
+                    const uint64_t* row_offsets, uint8_t* out, size_t out_bytes, void* stream);
+/* The inverse: n canonical idx rows (pad bits zero) from the packed streams. */
+int tq_entropy_unpack(const tq_plan* plan, const uint8_t* lengths, int64_t n, const uint8_t* packed,
+                      const uint64_t* row_offsets, uint8_t* idx, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

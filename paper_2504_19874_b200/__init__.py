@@ -9,6 +9,6 @@ from .binding import (  # noqa: F401
     TQ_ORTHOGONAL, TQ_PROD, Plan, TqError, lib, tq_codebook, tq_dequantize, tq_idx_row_bytes, tq_launch_count, tq_plan_status, tq_qjl_row_bytes,
     tq_quantize_mse, tq_quantize_prod, tq_rotation, tq_score, tq_score_static, tq_select_topk, tq_softmax, tq_topk, TQ_STATIC_SCRATCH_BYTES, tq_workspace_bytes, tq_wsum,
     TQ_LAYOUT_CANONICAL, TQ_LAYOUT_NIBBLE, tq_convert_layout, tq_query_bytes, tq_query_prepare, tq_score_prepared,
-    tq_score_static_max_queries, tq_selftest_wait_timeout,
+    tq_score_static_max_queries, tq_selftest_wait_timeout, tq_entropy_lengths, tq_entropy_pack, tq_entropy_unpack,
     KvGroup, tq_attend_decode, tq_attend_decode_workspace_bytes, tq_kv_append,
 )

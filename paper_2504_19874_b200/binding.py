@@ -48,6 +48,11 @@ _SIGNATURES = {
     "tq_score_prepared": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                   c_int64, c_void_p]),
     "tq_selftest_wait_timeout": (c_int, [c_void_p, ctypes.c_longlong, c_void_p]),
+    "tq_entropy_lengths": (c_int, [c_int, c_int, _F, c_void_p]),
+    "tq_entropy_workspace_bytes": (c_size_t, [c_int64]),
+    "tq_entropy_measure": (c_int, [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "tq_entropy_pack": (c_int, [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "tq_entropy_unpack": (c_int, [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]),
     "tq_topk": (c_int, [c_void_p, c_void_p, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                         c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "tq_select_topk": (c_int, [c_void_p, c_void_p, c_int, c_int64, c_int64, c_int, c_void_p, c_void_p, c_void_p]),
@@ -326,6 +331,34 @@ def tq_kv_append(groups, heads: int, head_stride: int, position: int, K, V):
         raise ValueError("K and V must have one dtype")
     _check(lib().tq_kv_append(ctypes.cast(arr, c_void_p), len(groups), heads, head_stride, position, _dev(K), _dev(V),
                               _dtype_code(K), ldk, ldv, _stream()))
+
+
+def tq_entropy_lengths(d: int, bits: int, centroids) -> np.ndarray:
+    """Huffman code lengths of the 2^bits index values for the given codebook (uint8 array)."""
+    cent = np.ascontiguousarray(centroids, dtype=np.float32)
+    out = np.zeros(1 << bits, dtype=np.uint8)
+    _check(lib().tq_entropy_lengths(d, bits, _fptr(cent), out.ctypes.data_as(c_void_p)))
+    return out
+
+
+def tq_entropy_pack(plan: Plan, lengths, n: int, idx):
+    """(packed uint8 tensor, row_offsets int64 tensor of n + 1 byte offsets): the entropy-coded index rows."""
+    ln = np.ascontiguousarray(lengths, dtype=np.uint8)
+    lp = ln.ctypes.data_as(c_void_p)
+    dev = idx.device
+    offsets = torch.empty(n + 1, dtype=torch.int64, device=dev)
+    ws = torch.empty(max(lib().tq_entropy_workspace_bytes(n), 256), dtype=torch.uint8, device=dev)
+    _check(lib().tq_entropy_measure(plan.handle, lp, n, _dev(idx), _dev(offsets), *_scratch_args(ws), _stream()))
+    total = int(offsets[n].item())
+    out = torch.empty(max(total, 4), dtype=torch.uint8, device=dev)
+    _check(lib().tq_entropy_pack(plan.handle, lp, n, _dev(idx), _dev(offsets), _dev(out), total, _stream()))
+    return out[:total], offsets
+
+
+def tq_entropy_unpack(plan: Plan, lengths, n: int, packed, offsets, idx_out):
+    ln = np.ascontiguousarray(lengths, dtype=np.uint8)
+    _check(lib().tq_entropy_unpack(plan.handle, ln.ctypes.data_as(c_void_p), n, _dev(packed), _dev(offsets), _dev(idx_out),
+                                   _stream()))
 
 
 def tq_select_topk(cand_scores, cand_ids, k: int, top_scores, top_ids):

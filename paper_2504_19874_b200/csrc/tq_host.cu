@@ -123,6 +123,31 @@ int lloyd_max(int d, int bits, double* c_out) {
   return TQ_ERR_NOT_CONVERGED;
 }
 
+// p_l = mass of the l-th cell (boundaries halfway between neighbouring centroids) under the density of Lemma 1:
+// the probability of index value l (entropy-coding paragraph of Section 3.1).
+int cell_masses(int d, int levels, const float* centroids, double* p_out) {
+  static const GaussLegendre gl;
+  const double expo = d - 2.0;
+  std::vector<double> t(levels + 1);
+  t[0] = -M_PI / 2;
+  t[levels] = M_PI / 2;
+  for (int i = 1; i < levels; ++i) {
+    const double b = 0.5 * ((double)centroids[i - 1] + (double)centroids[i]);
+    if (!(b > -1.0 && b < 1.0) || !(centroids[i] > centroids[i - 1])) {
+      set_error("cell_masses: centroids must be strictly ascending inside (-1, 1)");
+      return TQ_ERR_INVALID_ARG;
+    }
+    t[i] = std::asin(b);
+  }
+  double tot = 0.0;
+  for (int i = 0; i < levels; ++i) {
+    p_out[i] = cos_power_integral(t[i], t[i + 1], expo, gl);
+    tot += p_out[i];
+  }
+  for (int i = 0; i < levels; ++i) p_out[i] /= tot;
+  return TQ_OK;
+}
+
 // ---------------------------------------------------------------------------------------
 // Counter-based Gaussian draws (documented in tq.h so that anyone can reproduce a matrix).
 // ---------------------------------------------------------------------------------------
