@@ -262,6 +262,13 @@ scan_nib_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
   }
   __syncthreads();
 
+  // This CTA's contiguous range of rows: the 16-row units are dealt evenly, so that every CTA ends with the same
+  // fraction of a tile instead of some running a whole tile more than the others (10^6 rows on 148 CTAs: 26.4
+  // tiles each instead of 26 or 27: measured 1.3 % faster with two queries, 2.3 % with eight).  Rows of a last, partial tile beyond the range belong to the next CTA.
+  const int64_t units = (a.n + 15) / 16;
+  const int64_t row_begin = 16 * (units * blockIdx.x / gridDim.x);
+  const int64_t row_end = min(a.n, 16 * (units * (blockIdx.x + 1) / gridDim.x));
+
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
     // The codes are inputs of the call: their copies start at once, also while the kernel that builds the
@@ -270,8 +277,8 @@ scan_nib_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int64_t tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x) {
-        const int y = (int)(tile * VT);
+      for (int64_t rt = row_begin; rt < row_end && ok; rt += VT) {
+        const int y = (int)rt;
         for (int s = 0; s < a.nsteps; ++s) {
           if (!(ok = tc::mbar_wait(&empty[stage], phase ^ 1u, abort_flag, a.status))) break;
           unsigned char* sb = stage_base + (size_t)stage * STAGE_BYTES;
@@ -318,7 +325,8 @@ scan_nib_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
   int stage = 0;
   uint32_t phase = 0;
   bool ok = true;
-  for (int64_t tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x) {
+  for (int64_t rt = row_begin; rt < row_end && ok; rt += VT) {
+    const bool active = rt + cw * 16 < row_end;   // a warp without rows in a partial tile only keeps the pipeline's pace
     int accT[NT_T][4], accQ3[NT_Q][4], accQ7[NT_Q][4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -331,28 +339,31 @@ scan_nib_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
     float nu_pre[2], gm_pre[2];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      const int64_t row = tile * VT + cw * 16 + g + 8 * h;
-      nu_pre[h] = (row < a.n && a.norms != nullptr) ? ldg_now(a.norms + row) : 1.f;
-      gm_pre[h] = (row < a.n) ? ldg_now(a.gamma + row) : 0.f;
+      const int64_t row = rt + cw * 16 + g + 8 * h;
+      nu_pre[h] = (row < row_end && a.norms != nullptr) ? ldg_now(a.norms + row) : 1.f;
+      gm_pre[h] = (row < row_end) ? ldg_now(a.gamma + row) : 0.f;
     }
 
     for (int s = 0; s < a.nsteps; ++s) {
       if (!(ok = tc::mbar_wait(&full[stage], phase, abort_flag, a.status))) break;
       const unsigned char* sb = stage_base + (size_t)stage * STAGE_BYTES + lane_off;
       uint32_t w[2][4 * SB];
+      if (active) {
 #pragma unroll
-      for (int u = 0; u < SB; ++u)
+        for (int u = 0; u < SB; ++u)
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const uint4 v = *reinterpret_cast<const uint4*>(sb + u * BLOCK_BYTES + h * 512);
-          w[h][4 * u] = v.x; w[h][4 * u + 1] = v.y; w[h][4 * u + 2] = v.z; w[h][4 * u + 3] = v.w;
-        }
+          for (int h = 0; h < 2; ++h) {
+            const uint4 v = *reinterpret_cast<const uint4*>(sb + u * BLOCK_BYTES + h * 512);
+            w[h][4 * u] = v.x; w[h][4 * u + 1] = v.y; w[h][4 * u + 2] = v.z; w[h][4 * u + 3] = v.w;
+          }
+      }
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(&empty[stage]);   // the stage now lives in registers
       if (++stage == a.stages) {
         stage = 0;
         phase ^= 1u;
       }
+      if (!active) continue;
       // blocks of the last step that do not exist hold stale bytes; their operand is zero
       const uint4* Bb = reinterpret_cast<const uint4*>(Bs + (size_t)s * (SB * KPB) * 32) + lane;
 #pragma unroll
@@ -399,13 +410,14 @@ scan_nib_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
     if (!ok) break;
 
     // ---------------------------------------------------------------- epilogue
-    const int64_t row0 = tile * VT + cw * 16;
+    if (!active) continue;
+    const int64_t row0 = rt + cw * 16;
     auto finish = [&](long long T, long long TQ, int ql, int64_t row, float nu, float gamma) {
       const NQConst c = qcs[ql];
       const float av = __fmul_rn((float)T, c.sa);
       const float sv = fmaf((float)TQ, c.ss, c.cs);
       const float est = __fmul_rn(nu, fmaf(__fmul_rn(a.coef, gamma), sv, av));
-      if (row < a.n && ql < a.nq_pass) {
+      if (row < row_end && ql < a.nq_pass) {
         if (MODE == 0) {
           a.scores[(int64_t)ql * a.lds + row] = est;
         } else if (est >= __ldg(a.tau + ql)) {
