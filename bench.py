@@ -390,16 +390,7 @@ def run_b200(args):
             ms_q = time_call(lambda: tq.tq_quantize_prod(plan_c, Xc, ci, cq, cg, cn, cs), f"{cname}b{cbits}:quantize", min_ms=0.0, max_reps=2)
             del Xc, cs
             bpv = plan_c.idx_row_bytes + plan_c.qjl_row_bytes + 8
-            # d = 3072 in the nibble layout: the eight-query operand does not fit shared memory, so the many-query
-            # search of that configuration runs on the canonical layout (tcgen05 engine) after an in-place conversion
-            legs = scan_legs(plan_c, f"{cname}b{cbits}", nn, (ci, cq, cg, cn), Qc, ck, few=(1, 8),
-                             many=None if (nibble and dd > 2048) else 10_000, bytes_per_vec=bpv)
-            if nibble and dd > 2048:
-                tq.tq_convert_layout(plan_c, nn, ci, cq, tq.TQ_LAYOUT_NIBBLE, tq.TQ_LAYOUT_CANONICAL)
-                plan_c.set_layout(tq.TQ_LAYOUT_CANONICAL)
-                legs.update({"many_queries": scan_legs(plan_c, f"{cname}b{cbits}can", nn, (ci, cq, cg, cn), Qc, ck, few=(),
-                                                       many=10_000, bytes_per_vec=bpv)["many_queries"]})
-                legs["many_queries"]["layout"] = "canonical"
+            legs = scan_legs(plan_c, f"{cname}b{cbits}", nn, (ci, cq, cg, cn), Qc, ck, few=(1, 8), many=10_000, bytes_per_vec=bpv)
             other.append({"workload": f"{cname}: d={dd}, TurboQuant_prod b={cbits}, n={nn}, top-{ck}",
                           "layout": "nibble" if nibble else "canonical",
                           "quantize_ms": ms_q, "quantize_vectors_per_s": nn / (ms_q * 1e-3),

@@ -48,7 +48,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    link = [nvcc, "-shared", "-o", LIB] + objs + ["-lgomp"]
+    link = [nvcc, "-shared", "-o", LIB] + objs + ["-lgomp", "-ldl"]
     subprocess.run(link, check=True)
     return LIB
 

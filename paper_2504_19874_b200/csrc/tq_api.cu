@@ -404,6 +404,7 @@ cudaError_t score_block(const tq_plan* plan, const float* Qcat, int nq, int64_t 
 extern "C" int tq_plan_create(int d, int bits, int mode, const float* Pi, const float* S, const float* centroids,
                               tq_plan** out) {
   const char* who = "tq_plan_create";
+  TQ_RANGE(who);
   TQ_REQUIRE(out != nullptr, TQ_ERR_INVALID_ARG, "%s: out is NULL", who);
   *out = nullptr;
   TQ_REQUIRE(mode == TQ_MSE || mode == TQ_PROD, TQ_ERR_INVALID_ARG, "%s: unknown mode %d", who, mode);
@@ -523,6 +524,7 @@ extern "C" int tq_plan_layout(const tq_plan* plan) { return plan ? plan->layout 
 
 extern "C" int tq_convert_layout(const tq_plan* plan, int64_t n, uint8_t* idx, uint8_t* qjl, int from, int to, void* stream) {
   const char* who = "tq_convert_layout";
+  TQ_RANGE(who);
   int rc = check_plan(plan, who);
   if (rc) return rc;
   TQ_REQUIRE(n >= 0, TQ_ERR_INVALID_ARG, "%s: n is negative", who);
@@ -554,6 +556,7 @@ __global__ void wait_timeout_selftest_kernel(int* status, long long limit) {
 
 extern "C" int tq_selftest_wait_timeout(tq_plan* plan, long long limit_cycles, void* stream) {
   const char* who = "tq_selftest_wait_timeout";
+  TQ_RANGE(who);
   int rc = check_plan(plan, who);
   if (rc) return rc;
   TQ_REQUIRE(limit_cycles >= 1 && limit_cycles <= 100000000LL, TQ_ERR_INVALID_ARG, "%s: limit outside 1..1e8 cycles", who);
@@ -565,6 +568,7 @@ extern "C" int tq_selftest_wait_timeout(tq_plan* plan, long long limit_cycles, v
 
 extern "C" int tq_plan_status(tq_plan* plan) {
   const char* who = "tq_plan_status";
+  TQ_RANGE(who);
   TQ_REQUIRE(plan != nullptr, TQ_ERR_INVALID_ARG, "%s: plan is NULL", who);
   TQ_CHECK_CUDA(cudaDeviceSynchronize(), who);
   int st = 0;
@@ -623,6 +627,7 @@ extern "C" size_t tq_workspace_bytes(const tq_plan* plan, int op, int64_t n, int
 extern "C" int tq_quantize_mse(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t ldx, uint8_t* idx,
                                float* norms, void* scratch, size_t scratch_bytes, void* stream) {
   const char* who = "tq_quantize_mse";
+  TQ_RANGE(who);
   int rc = check_plan(plan, who);
   if (rc) return rc;
   TQ_REQUIRE(plan->mode == TQ_MSE, TQ_ERR_INVALID_ARG, "%s: plan was created for TQ_PROD", who);
@@ -650,6 +655,7 @@ extern "C" int tq_quantize_prod(const tq_plan* plan, const void* X, int x_dtype,
                                 uint8_t* qjl, float* gamma, float* norms, void* scratch, size_t scratch_bytes,
                                 void* stream) {
   const char* who = "tq_quantize_prod";
+  TQ_RANGE(who);
   int rc = check_plan(plan, who);
   if (rc) return rc;
   TQ_REQUIRE(plan->mode == TQ_PROD, TQ_ERR_INVALID_ARG, "%s: plan was created for TQ_MSE", who);
@@ -712,6 +718,7 @@ extern "C" int tq_quantize_prod(const tq_plan* plan, const void* X, int x_dtype,
 extern "C" int tq_dequantize(const tq_plan* plan, int64_t n, const uint8_t* idx, const uint8_t* qjl, const float* gamma,
                              const float* norms, float* Xhat, int64_t ldxh, void* stream) {
   const char* who = "tq_dequantize";
+  TQ_RANGE(who);
   int rc = check_plan(plan, who);
   if (rc) return rc;
   TQ_REQUIRE(n >= 0, TQ_ERR_INVALID_ARG, "%s: n is negative", who);
@@ -774,6 +781,7 @@ extern "C" int tq_score(const tq_plan* plan, const void* Q, int q_dtype, int nq,
                         const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms, float* scores,
                         int64_t lds, void* workspace, size_t workspace_bytes, void* stream) {
   const char* who = "tq_score";
+  TQ_RANGE(who);
   int rc = check_plan(plan, who);
   if (rc) return rc;
   TQ_REQUIRE(n >= 0 && nq >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
@@ -809,6 +817,7 @@ extern "C" size_t tq_query_bytes(const tq_plan* plan, int nq) {
 extern "C" int tq_query_prepare(const tq_plan* plan, const void* Q, int q_dtype, int nq, int64_t ldq, void* prepared,
                                 size_t prepared_bytes, void* stream) {
   const char* who = "tq_query_prepare";
+  TQ_RANGE(who);
   int rc = check_plan(plan, who);
   if (rc) return rc;
   TQ_REQUIRE(nq >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
@@ -835,6 +844,7 @@ extern "C" int tq_score_prepared(const tq_plan* plan, const void* prepared, int 
                                  const uint8_t* qjl, const float* gamma, const float* norms, float* scores, int64_t lds,
                                  void* stream) {
   const char* who = "tq_score_prepared";
+  TQ_RANGE(who);
   int rc = check_plan(plan, who);
   if (rc) return rc;
   TQ_REQUIRE(n >= 0 && nq >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
@@ -925,6 +935,7 @@ extern "C" int tq_topk(const tq_plan* plan, const void* Q, int q_dtype, int nq, 
                        const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms, int k,
                        float* top_scores, int32_t* top_ids, void* workspace, size_t workspace_bytes, void* stream) {
   const char* who = "tq_topk";
+  TQ_RANGE(who);
   int rc = check_plan(plan, who);
   if (rc) return rc;
   TQ_REQUIRE(n >= 0 && nq >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
@@ -974,6 +985,7 @@ extern "C" int tq_wsum(const tq_plan* plan, const float* W, int nw, int64_t ldw,
                        const uint8_t* qjl, const float* gamma, const float* norms, float* out, int64_t ldo,
                        void* workspace, size_t workspace_bytes, void* stream) {
   const char* who = "tq_wsum";
+  TQ_RANGE(who);
   int rc = check_plan(plan, who);
   if (rc) return rc;
   TQ_REQUIRE(n >= 0 && nw >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
@@ -1042,6 +1054,7 @@ extern "C" int tq_wsum(const tq_plan* plan, const float* W, int nw, int64_t ldw,
 extern "C" int tq_select_topk(const float* cand_scores, const int32_t* cand_ids, int nq, int64_t m, int64_t ld, int k,
                               float* top_scores, int32_t* top_ids, void* stream) {
   const char* who = "tq_select_topk";
+  TQ_RANGE(who);
   TQ_REQUIRE(nq >= 0 && m >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
   TQ_REQUIRE(k >= 1 && k <= TQ_MAX_K, TQ_ERR_UNSUPPORTED, "%s: k=%d outside 1..%d", who, k, TQ_MAX_K);
   TQ_REQUIRE(m <= 0x7fffffffLL && ld <= 0x7fffffffLL, TQ_ERR_UNSUPPORTED, "%s: m / ld too large", who);
@@ -1057,6 +1070,7 @@ extern "C" int tq_select_topk(const float* cand_scores, const int32_t* cand_ids,
 extern "C" int tq_softmax(const float* s1, const float* s2, int nw, int64_t n, int64_t lds, float scale, float* W,
                           int64_t ldw, void* stream) {
   const char* who = "tq_softmax";
+  TQ_RANGE(who);
   TQ_REQUIRE(nw >= 0 && n >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
   if (nw == 0 || n == 0) return TQ_OK;
   TQ_REQUIRE(s1 != nullptr && W != nullptr, TQ_ERR_INVALID_ARG, "%s: s1 / W is NULL", who);
@@ -1115,6 +1129,7 @@ extern "C" int tq_score_static(const tq_plan* plan, const void* Q, int q_dtype, 
                                const uint8_t* idx, const uint8_t* qjl, const float* gamma, const float* norms,
                                float* scores, int64_t lds, void* stream) {
   const char* who = "tq_score_static";
+  TQ_RANGE(who);
   int rc = check_plan(plan, who);   // also makes sure the plan's device is the current one
   if (rc) return rc;
   TQ_REQUIRE(n >= 0 && nq >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);

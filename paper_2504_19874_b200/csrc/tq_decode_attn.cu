@@ -554,6 +554,7 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   using namespace tq;
   using namespace tq::kvdec;
   const char* who = "tq_attend_decode";
+  TQ_RANGE(who);
   TQ_REQUIRE(groups != nullptr && ngroups >= 1 && ngroups <= MAXG, TQ_ERR_INVALID_ARG, "%s: 1..%d channel groups", who, MAXG);
   TQ_REQUIRE(heads >= 0 && tokens >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
   TQ_REQUIRE(head_stride >= tokens, TQ_ERR_INVALID_ARG, "%s: head_stride %lld is smaller than tokens %lld", who,
@@ -665,6 +666,7 @@ extern "C" int tq_kv_append(const tq_kv_group* groups, int ngroups, int heads, i
   using namespace tq;
   using namespace tq::kvdec;
   const char* who = "tq_kv_append";
+  TQ_RANGE(who);
   TQ_REQUIRE(groups != nullptr && ngroups >= 1 && ngroups <= MAXG, TQ_ERR_INVALID_ARG, "%s: 1..%d channel groups", who, MAXG);
   TQ_REQUIRE(heads >= 0, TQ_ERR_INVALID_ARG, "%s: negative size", who);
   TQ_REQUIRE(position >= 0 && position < head_stride, TQ_ERR_INVALID_ARG, "%s: position %lld outside [0, head_stride %lld)", who,

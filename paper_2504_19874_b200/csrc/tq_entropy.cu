@@ -275,6 +275,7 @@ extern "C" size_t tq_entropy_workspace_bytes(int64_t n) { return n > 0 ? (size_t
 extern "C" int tq_entropy_measure(const tq_plan* plan, const uint8_t* lengths, int64_t n, const uint8_t* idx, uint64_t* row_offsets,
                                   void* workspace, size_t workspace_bytes, void* stream) {
   const char* who = "tq_entropy_measure";
+  TQ_RANGE(who);
   int rc = entropy::check(plan, who, lengths, n);
   if (rc) return rc;
   TQ_REQUIRE(row_offsets != nullptr && (n == 0 || idx != nullptr), TQ_ERR_INVALID_ARG, "%s: NULL argument", who);
@@ -298,6 +299,7 @@ extern "C" int tq_entropy_measure(const tq_plan* plan, const uint8_t* lengths, i
 extern "C" int tq_entropy_pack(const tq_plan* plan, const uint8_t* lengths, int64_t n, const uint8_t* idx, const uint64_t* row_offsets,
                                uint8_t* out, size_t out_bytes, void* stream) {
   const char* who = "tq_entropy_pack";
+  TQ_RANGE(who);
   int rc = entropy::check(plan, who, lengths, n);
   if (rc) return rc;
   if (n == 0) return TQ_OK;
@@ -317,6 +319,7 @@ extern "C" int tq_entropy_pack(const tq_plan* plan, const uint8_t* lengths, int6
 extern "C" int tq_entropy_unpack(const tq_plan* plan, const uint8_t* lengths, int64_t n, const uint8_t* packed,
                                  const uint64_t* row_offsets, uint8_t* idx, void* stream) {
   const char* who = "tq_entropy_unpack";
+  TQ_RANGE(who);
   int rc = entropy::check(plan, who, lengths, n);
   if (rc) return rc;
   if (n == 0) return TQ_OK;

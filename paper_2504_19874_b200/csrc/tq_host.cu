@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -15,6 +16,14 @@ static thread_local char g_err[512] = "";
 
 static std::atomic<unsigned long long> g_launches{0};
 void count_launches(int k) { g_launches.fetch_add((unsigned long long)k, std::memory_order_relaxed); }
+
+bool log_enabled() {
+  static const bool on = [] {
+    const char* v = std::getenv("TQ_LOG");
+    return v != nullptr && v[0] != '\0' && !(v[0] == '0' && v[1] == '\0');
+  }();
+  return on;
+}
 
 void set_error(const char* fmt, ...) {
   va_list ap;

@@ -4,6 +4,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <cstdarg>
 #include <cstdint>
@@ -16,6 +17,21 @@ namespace tq {
 void set_error(const char* fmt, ...);
 void count_launches(int k);   // kernels enqueued by this library (diagnostic counter)
 int lloyd_max(int d, int bits, double* c_out);
+
+// Every API call that enqueues device work opens an NVTX range with its own name (visible in Nsight Systems /
+// Compute timelines; a no-op without a profiler attached) and, when the environment variable TQ_LOG is set to a
+// non-empty value other than 0, writes one line to stderr.
+bool log_enabled();
+struct CallRange {
+  explicit CallRange(const char* name) {
+    nvtxRangePushA(name);
+    if (log_enabled()) std::fprintf(stderr, "[tq] %s\n", name);
+  }
+  ~CallRange() { nvtxRangePop(); }
+  CallRange(const CallRange&) = delete;
+  CallRange& operator=(const CallRange&) = delete;
+};
+#define TQ_RANGE(name) tq::CallRange tq_call_range_(name)
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 inline int64_t round_up64(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
