@@ -23,7 +23,8 @@ constexpr int BM = 128;          // rows of X per tile = TMEM lanes
 constexpr int BK = 64;           // bf16 elements per 128-byte swizzled row
 constexpr int UMMA_K = 16;
 constexpr int EPS = 4;           // epilogue warps per TMEM lane group: each takes 1/EPS of the tile's columns
-constexpr int NTHREADS = 32 * (2 + 4 * EPS);   // warp 0: TMA, warp 1: MMA + TMEM owner, then the epilogue warps
+constexpr int NSPLIT = 2;        // warps that prepare the next block's operand limbs beside the GEMM (see SplitTask)
+constexpr int NTHREADS = 32 * (2 + 4 * EPS + NSPLIT);   // warp 0: TMA, warp 1: MMA + TMEM owner, the epilogue warps, the split warps
 
 template <int BN>
 struct Cfg {
@@ -50,6 +51,18 @@ struct GemmArgs {
   // row [idx row | qjl row], nibble = index | sign << 3.  MODE 1 writes them with the sign bits clear, MODE 2 ORs
   // the sign bits in.
   int nibble;
+  // Operand preparation of the NEXT block of rows (nu = ||x||, u = x / nu, bf16 limbs of u), done by NSPLIT spare
+  // warps of every CTA while this launch's GEMM runs: the GEMM is bound by the tensor pipe and shared memory, the
+  // preparation by HBM and a little issue bandwidth, so it hides completely.  Only the project launch (MODE 2)
+  // carries one: its own A operand is the residual, so the limb buffers of X are free to be rewritten.
+  struct SplitTask {
+    const void* X;       // first row of the next block
+    int64_t ldx, rows;   // rows == 0: nothing to do
+    int d, dpad, is_f32, normalize;
+    __nv_bfloat16* L1;
+    __nv_bfloat16* L2;
+    float* norms;        // nullable
+  } split;
   uint8_t* nib_idx;      // idx rows (stride nib_idx_rb) and qjl rows (stride nib_qjl_rb) of this block of rows
   uint8_t* nib_qjl;
   size_t nib_idx_rb, nib_qjl_rb;
@@ -68,6 +81,107 @@ __device__ __forceinline__ uint32_t spread_to_nibble_tops(uint32_t x) {
 __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// One warp per row: nu = ||x|| (optional), u = x / nu, u = hi + lo in bf16.  Rows warp, warp + nwarps, ...
+template <typename T, bool NORMALIZE>
+__device__ __forceinline__ void split_rows(const T* __restrict__ X, int64_t ldx, int64_t n, int d, int dpad,
+                                           __nv_bfloat16* __restrict__ L1, __nv_bfloat16* __restrict__ L2,
+                                           float* __restrict__ norms, int64_t warp, int64_t nwarps, int lane) {
+  // fp32 rows, 16-byte aligned: segments of 2048 elements held in registers (16 x 16 bytes per lane, all loads in
+  // flight at once); a row of one segment is read once, longer rows a second time (from L2) after the norm is known
+  if constexpr (sizeof(T) == 4) {
+    if ((d & 3) == 0 && (ldx & 3) == 0 && (reinterpret_cast<uintptr_t>(X) & 15) == 0 && dpad == d) {
+      const int nseg = (d + 2047) / 2048;
+      for (int64_t r = warp; r < n; r += nwarps) {
+        const float4* row4 = reinterpret_cast<const float4*>(X + r * ldx);
+        float4 v[16];
+        auto load_seg = [&](int seg) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int c = seg * 512 + lane + 32 * i;
+            v[i] = (4 * c < d) ? __ldg(row4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        };
+        float inv = 1.f;
+        load_seg(0);
+        if (NORMALIZE) {
+          float s = 0.f;
+          for (int seg = 0; seg < nseg; ++seg) {
+            if (seg > 0) load_seg(seg);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) s = fmaf(v[i].x, v[i].x, fmaf(v[i].y, v[i].y, fmaf(v[i].z, v[i].z, fmaf(v[i].w, v[i].w, s))));
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+          const float nu = sqrtf(s);
+          inv = (nu > 0.f) ? 1.f / nu : 0.f;
+          if (lane == 0 && norms != nullptr) norms[r] = nu;
+        }
+        for (int seg = 0; seg < nseg; ++seg) {
+          if (nseg > 1 && (seg > 0 || NORMALIZE)) load_seg(seg);   // registers hold the last segment read
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int c = seg * 512 + lane + 32 * i;
+            if (4 * c >= d) continue;
+            const float u0 = v[i].x * inv, u1 = v[i].y * inv, u2 = v[i].z * inv, u3 = v[i].w * inv;
+            const float h0 = __bfloat162float(__float2bfloat16_rn(u0)), h1 = __bfloat162float(__float2bfloat16_rn(u1));
+            const float h2 = __bfloat162float(__float2bfloat16_rn(u2)), h3 = __bfloat162float(__float2bfloat16_rn(u3));
+            *reinterpret_cast<uint2*>(L1 + r * dpad + 4 * c) = make_uint2(pack_bf16x2(h0, h1), pack_bf16x2(h2, h3));
+            *reinterpret_cast<uint2*>(L2 + r * dpad + 4 * c) = make_uint2(pack_bf16x2(u0 - h0, u1 - h1), pack_bf16x2(u2 - h2, u3 - h3));
+          }
+        }
+      }
+      return;
+    }
+  }
+  for (int64_t r = warp; r < n; r += nwarps) {
+    const T* row = X + r * ldx;
+    float inv = 1.f;
+    if (NORMALIZE) {
+      float s = 0.f;
+      for (int j = lane; j < d; j += 32) {
+        float v;
+        if constexpr (sizeof(T) == 4) v = row[j]; else v = __bfloat162float(row[j]);
+        s = fmaf(v, v, s);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      const float nu = sqrtf(s);
+      inv = (nu > 0.f) ? 1.f / nu : 0.f;
+      if (lane == 0 && norms != nullptr) norms[r] = nu;
+    }
+    for (int j0 = lane * 8; j0 < dpad; j0 += 256) {
+      uint32_t h[4], l[4];
+#pragma unroll
+      for (int p = 0; p < 4; ++p) {
+        float u[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int j = j0 + 2 * p + q;
+          float v = 0.f;
+          if (j < d) {
+            if constexpr (sizeof(T) == 4) v = row[j]; else v = __bfloat162float(row[j]);
+          }
+          u[q] = v * inv;
+        }
+        const float h0 = __bfloat162float(__float2bfloat16_rn(u[0]));
+        const float h1 = __bfloat162float(__float2bfloat16_rn(u[1]));
+        h[p] = pack_bf16x2(h0, h1);
+        l[p] = pack_bf16x2(u[0] - h0, u[1] - h1);
+      }
+      *reinterpret_cast<uint4*>(L1 + r * dpad + j0) = make_uint4(h[0], h[1], h[2], h[3]);
+      *reinterpret_cast<uint4*>(L2 + r * dpad + j0) = make_uint4(l[0], l[1], l[2], l[3]);
+    }
+  }
+}
+
+template <typename T, bool NORMALIZE>
+__global__ void __launch_bounds__(256) split_rows_kernel(const T* __restrict__ X, int64_t ldx, int64_t n, int d, int dpad,
+                                                         __nv_bfloat16* __restrict__ L1, __nv_bfloat16* __restrict__ L2,
+                                                         float* __restrict__ norms) {
+  split_rows<T, NORMALIZE>(X, ldx, n, d, dpad, L1, L2, norms, (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5),
+                           (int64_t)gridDim.x * (blockDim.x >> 5), threadIdx.x & 31);
 }
 
 // MODE 0: idx.  MODE 1: idx + residual limbs + partial ||e||^2.  MODE 2: sign bits.
@@ -177,6 +291,21 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
       }
     }
     __syncwarp();
+  } else if (warp >= 2 + 4 * EPS) {
+    // ------------------------------------------------------------ operand limbs of the next block of rows
+    const GemmArgs::SplitTask& t = a.split;
+    if (t.rows > 0) {
+      const int64_t sw = (int64_t)blockIdx.x * NSPLIT + (warp - 2 - 4 * EPS), nsw = (int64_t)gridDim.x * NSPLIT;
+      if (t.is_f32) {
+        const float* X = static_cast<const float*>(t.X);
+        if (t.normalize) split_rows<float, true>(X, t.ldx, t.rows, t.d, t.dpad, t.L1, t.L2, t.norms, sw, nsw, lane);
+        else split_rows<float, false>(X, t.ldx, t.rows, t.d, t.dpad, t.L1, t.L2, t.norms, sw, nsw, lane);
+      } else {
+        const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(t.X);
+        if (t.normalize) split_rows<__nv_bfloat16, true>(X, t.ldx, t.rows, t.d, t.dpad, t.L1, t.L2, t.norms, sw, nsw, lane);
+        else split_rows<__nv_bfloat16, false>(X, t.ldx, t.rows, t.d, t.dpad, t.L1, t.L2, t.norms, sw, nsw, lane);
+      }
+    }
   } else {
     // ------------------------------------------------------------ epilogue (4 x EPS warps: 4 TMEM lane groups x EPS column parts)
     const int lg = warp & 3;   // TMEM lane group this warp may read
@@ -325,55 +454,6 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
 }
 
 // ---------------------------------------------------------------- operand splitting
-// One warp per row: nu = ||x|| (optional), u = x / nu, u = hi + lo in bf16.
-template <typename T, bool NORMALIZE>
-__global__ void __launch_bounds__(256) split_rows_kernel(const T* __restrict__ X, int64_t ldx, int64_t n, int d, int dpad,
-                                                         __nv_bfloat16* __restrict__ L1, __nv_bfloat16* __restrict__ L2,
-                                                         float* __restrict__ norms) {
-  const int lane = threadIdx.x & 31;
-  const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
-  for (int64_t r = warp; r < n; r += nwarps) {
-    const T* row = X + r * ldx;
-    float inv = 1.f;
-    if (NORMALIZE) {
-      float s = 0.f;
-      for (int j = lane; j < d; j += 32) {
-        float v;
-        if constexpr (sizeof(T) == 4) v = row[j]; else v = __bfloat162float(row[j]);
-        s = fmaf(v, v, s);
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      const float nu = sqrtf(s);
-      inv = (nu > 0.f) ? 1.f / nu : 0.f;
-      if (lane == 0 && norms != nullptr) norms[r] = nu;
-    }
-    for (int j0 = lane * 8; j0 < dpad; j0 += 256) {
-      uint32_t h[4], l[4];
-#pragma unroll
-      for (int p = 0; p < 4; ++p) {
-        float u[2];
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-          const int j = j0 + 2 * p + q;
-          float v = 0.f;
-          if (j < d) {
-            if constexpr (sizeof(T) == 4) v = row[j]; else v = __bfloat162float(row[j]);
-          }
-          u[q] = v * inv;
-        }
-        const float h0 = __bfloat162float(__float2bfloat16_rn(u[0]));
-        const float h1 = __bfloat162float(__float2bfloat16_rn(u[1]));
-        h[p] = pack_bf16x2(h0, h1);
-        l[p] = pack_bf16x2(u[0] - h0, u[1] - h1);
-      }
-      *reinterpret_cast<uint4*>(L1 + r * dpad + j0) = make_uint4(h[0], h[1], h[2], h[3]);
-      *reinterpret_cast<uint4*>(L2 + r * dpad + j0) = make_uint4(l[0], l[1], l[2], l[3]);
-    }
-  }
-}
-
 // gamma = sqrt(sum over column tiles of the partial sums), in tile order (deterministic).
 __global__ void gamma_finish_kernel(const float* __restrict__ gpart, int64_t Mpad, int tiles_n, int64_t rows,
                                     float* __restrict__ gamma) {
@@ -537,24 +617,34 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
   int64_t R = (int64_t)(scratch_bytes / per_row) / BM * BM;
   R = std::min<int64_t>(R, round_up64(n, BM));
   TQ_REQUIRE(R >= BM, TQ_ERR_WORKSPACE, "%s: scratch of %zu bytes cannot hold one block of %d rows", who, scratch_bytes, BM);
-  // carve the scratch (every part is a multiple of 256 bytes because R is a multiple of 128)
+  // The operand limbs of block i + 1 are prepared by spare warps of a GEMM launch of block i.  TQ_PROD: the project
+  // launch (its A operand is the residual, the limbs of X are free by then), one set of limb buffers.  TQ_MSE: the
+  // rotate launch itself, so the scratch is used as two half-size sets written and read in turn (when the data
+  // spans more than one block and each half still holds a tile).
+  const bool pingpong = !prod && n > R / 2 / BM * BM && R / 2 >= BM;
+  const int64_t Rbuf = R;   // rows the carved buffers hold in all
+  if (pingpong) R = R / 2 / BM * BM;
+  // carve the scratch (every part is a multiple of 256 bytes because Rbuf is a multiple of 128)
   char* p = static_cast<char*>(scratch);
-  __nv_bfloat16* XL1 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
-  __nv_bfloat16* XL2 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
+  __nv_bfloat16* XL1 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)Rbuf * dpad * 2;
+  __nv_bfloat16* XL2 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)Rbuf * dpad * 2;
   __nv_bfloat16 *EL1 = nullptr, *EL2 = nullptr;
   float* gpart = nullptr;
   if (prod) {
-    EL1 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
-    EL2 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)R * dpad * 2;
-    gpart = reinterpret_cast<float*>(p); p += (size_t)R * tiles_n * 4 * EPS;
+    EL1 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)Rbuf * dpad * 2;
+    EL2 = reinterpret_cast<__nv_bfloat16*>(p); p += (size_t)Rbuf * dpad * 2;
+    gpart = reinterpret_cast<float*>(p); p += (size_t)Rbuf * tiles_n * 4 * EPS;
   }
+  // limb buffers of block number b
+  auto limbs1 = [&](int64_t b) { return XL1 + (pingpong && (b & 1) ? (size_t)R * dpad : 0); };
+  auto limbs2 = [&](int64_t b) { return XL2 + (pingpong && (b & 1) ? (size_t)R * dpad : 0); };
   const size_t xsz = (x_dtype == TQ_F32) ? 4 : 2;
   auto launch_split = [&](int64_t r0, cudaStream_t s) -> cudaError_t {
     const int64_t rows = std::min(R, n - r0);
     const void* Xc = static_cast<const char*>(X) + (size_t)r0 * ldx * xsz;
     float* nu_out = norms ? norms + r0 : nullptr;
     const int blocks = (int)std::min<int64_t>((rows + 7) / 8, (int64_t)sm_count() * 8);
-    __nv_bfloat16 *L1 = XL1, *L2 = XL2;
+    __nv_bfloat16 *L1 = limbs1(r0 / R), *L2 = limbs2(r0 / R);
     if (norms) {
       if (x_dtype == TQ_F32)
         split_rows_kernel<float, true><<<blocks, 256, 0, s>>>(static_cast<const float*>(Xc), ldx, rows, d, dpad, L1, L2, nu_out);
@@ -572,9 +662,22 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
   for (int64_t r0 = 0; r0 < n; r0 += R) {
     const int64_t rows = std::min(R, n - r0);
     float* nu_out = norms ? norms + r0 : nullptr;
-    // 1. nu, u = x / nu, bf16 limbs of u
-    TQ_CHECK_CUDA(launch_split(r0, st), who);
-    __nv_bfloat16 *XLc1 = XL1, *XLc2 = XL2;
+    // 1. nu, u = x / nu, bf16 limbs of u: by a launch of its own for the first block (and for TQ_MSE plans), by the
+    //    spare warps of the previous block's project launch otherwise
+    if (r0 == 0 || (!prod && !pingpong)) TQ_CHECK_CUDA(launch_split(r0, st), who);
+    __nv_bfloat16 *XLc1 = limbs1(r0 / R), *XLc2 = limbs2(r0 / R);
+    auto next_block_task = [&](GemmArgs& ga) {
+      ga.split.X = static_cast<const char*>(X) + (size_t)(r0 + R) * ldx * xsz;
+      ga.split.ldx = ldx;
+      ga.split.rows = std::min(R, n - (r0 + R));
+      ga.split.d = d;
+      ga.split.dpad = dpad;
+      ga.split.is_f32 = x_dtype == TQ_F32 ? 1 : 0;
+      ga.split.normalize = norms ? 1 : 0;
+      ga.split.L1 = limbs1(r0 / R + 1);
+      ga.split.L2 = limbs2(r0 / R + 1);
+      ga.split.norms = norms ? norms + r0 + R : nullptr;
+    };
 
     CUtensorMap mA1, mA2;
     TQ_REQUIRE(make_map(&mA1, XLc1, rows, d, dpad, BM) && make_map(&mA2, XLc2, rows, d, dpad, BM), TQ_ERR_CUDA,
@@ -594,6 +697,7 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     g.gpart = gpart;
     g.Mpad = R;
     g.nu = nu_out;
+    g.split.rows = 0;
     g.nibble = (plan->layout == TQ_LAYOUT_NIBBLE) ? 1 : 0;
     g.nib_idx = idx ? idx + (size_t)r0 * plan->idx_row_bytes : nullptr;
     g.nib_qjl = qjl ? qjl + (size_t)r0 * plan->qjl_row_bytes : nullptr;
@@ -602,6 +706,7 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     g.status = plan->d_status;
     // 2. y = Pi u, idx (+ residual limbs and partial norms)
     if (!prod) {
+      if (pingpong && r0 + R < n) next_block_task(g);
       TQ_CHECK_CUDA(launch_gemm<0>(bn, plan->mse_bits, mA1, mA2, plan->pi_limbs.map_hi, plan->pi_limbs.map_lo, g, st), who);
       continue;
     }
@@ -616,6 +721,7 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
                "%s: cuTensorMapEncodeTiled failed", who);
     g.out = qjl + (size_t)r0 * plan->qjl_row_bytes;
     g.out_rb = plan->qjl_row_bytes;
+    if (r0 + R < n) next_block_task(g);   // the limbs of X are free by now
     TQ_CHECK_CUDA(launch_gemm<2>(bn, 1, mE1, mE2, plan->sp_limbs.map_hi, plan->sp_limbs.map_lo, g, st), who);
   }
   return TQ_OK;
