@@ -502,7 +502,9 @@ def run_b200(args):
                 "frac": achieved_tf / peaks["bf16_tflops_sustained"],
                 "frac_of_three_pass_bound": 3.0 * achieved_tf / peaks["bf16_tflops_sustained"],
                 "traffic": QUANTIZE_TRAFFIC_PER_98304_ROWS if d == 1536 else None,
-                "traffic_source": "ncu capture of one rotate + one project launch of 98,304 rows (profile summary, not measured in this run)",
+                "traffic_source": "ncu capture of one rotate + one project launch of 98,304 rows (profile summary, not measured in this run); "
+                                  "the project launch also prepares the operand limbs of the next block of rows (reads its fp32 input, "
+                                  "writes two bf16 limbs): captured with a 32,768-row next block, that part scaled to 98,304 rows",
                 "algorithmic_bytes_per_launch": algo_bytes_row * rows_per_launch,
                 "peak_source": f"bf16 sustained, of {peaks['source']}",
                 "note": "achieved = algorithmic flops 4 n d^2 of the step / CUDA-event time of the quantise phase "
@@ -517,7 +519,7 @@ def run_b200(args):
                      "frac_nq8": few[8]["scan_prepared_frac_hbm"] if 8 in few else None,
                      "frac_nq8_whole_call": few[8]["score_call_frac_hbm"] if 8 in few else None,
                      "traffic": SCAN_TRAFFIC_PER_VECTOR * n,
-                     "traffic_source": "ncu capture at n = 262,144 (203.5 MB read + 4.2 MB written), scaled by n",
+                     "traffic_source": "ncu capture at n = 262,144 (205.9 MB read + 5.0 MB written), scaled by n",
                      "peak_source": f"copy bandwidth, of {peaks['source']}",
                      "note": "achieved = algorithmic code bytes (idx + qjl + gamma + nu = 776 B per vector) of one pass / "
                              "CUDA-event time of tq_score_prepared (the scan kernel alone; queries prepared once by "
@@ -548,8 +550,10 @@ def run_b200(args):
 
 
 # DRAM bytes of the dominant kernels from ncu captures (one launch each; see the summaries under profiles/)
-QUANTIZE_TRAFFIC_PER_98304_ROWS = 1303.8e6 + 633.4e6
-SCAN_TRAFFIC_PER_VECTOR = (203.5e6 + 4.2e6) / 262144
+# rotate launch (651.2 MB read + 666.4 MB written) + project launch (925.8 + 271.3 MB, of which 201.3 + 201.3 MB are the
+# limbs of a 32,768-row next block) + the same limb traffic for the other 65,536 rows of a full next block
+QUANTIZE_TRAFFIC_PER_98304_ROWS = (651.2e6 + 666.4e6) + (925.8e6 + 271.3e6) + 2 * 2 * 201.3e6
+SCAN_TRAFFIC_PER_VECTOR = (205.9e6 + 5.0e6) / 262144
 
 
 def kv_decode_legs(tq, wl, dev, peaks, time_call):
