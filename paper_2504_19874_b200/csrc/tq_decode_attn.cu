@@ -376,56 +376,99 @@ __global__ void __launch_bounds__(NT) partial_kernel(Args a) {
   }
 }
 
+#include "tq_decode_mma.cuh"
+
 // ------------------------------------------------------------------ merge of the slices + inverse rotation
+// One CTA per (head, group), all queries of the head at once: slice weights exp(m_s - M) / L, the weighted sum of the
+// slices' partial value sums (float4 = the four queries of a coordinate), then x~ = Pi_V^T y' scattered to the group's
+// channels.  Every sum runs in a fixed order.
 __global__ void __launch_bounds__(256) merge_kernel(Args a, float* __restrict__ out, int64_t ldo) {
-  __shared__ float yp[2][MAXG * MAXD];
-  __shared__ float wsl[64];
-  __shared__ float stat[2];
-  const int h = blockIdx.x / a.qpk, j = blockIdx.x % a.qpk;
-  const int ncoord = a.ngroups * a.d, d = a.d;
-  const float* ml = a.part_ml + (size_t)h * a.nslices * 2 * MAXQ;
-  if (threadIdx.x < 32) {   // global maximum and sum: lanes take slices in turn, combined in a fixed order
-    const int lane = threadIdx.x;
-    float M = -FLT_MAX;
-    for (int s = lane; s < a.nslices; s += 32) M = fmaxf(M, ml[s * 2 * MAXQ + j]);
+  __shared__ float4 wsl[256];
+  __shared__ float4 yp[256];
+  __shared__ float ys[MAXQ][MAXD];
+  __shared__ float redm[8][MAXQ];
+  __shared__ double redl[8][MAXQ];
+  __shared__ float stat[2][MAXQ];
+  const int h = blockIdx.x / a.ngroups, gi = blockIdx.x % a.ngroups;
+  const int ncoord = a.ngroups * a.d, d = a.d, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const GroupDev& g = a.g[gi];
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // the slices' partial results come from the kernel before
+  const float4* ml4 = reinterpret_cast<const float4*>(a.part_ml + (size_t)h * a.nslices * 2 * MAXQ);   // [slice][max, sum]
+  {   // global maximum and sum per query
+    float M[MAXQ] = {-FLT_MAX, -FLT_MAX, -FLT_MAX, -FLT_MAX};
+    for (int s = tid; s < a.nslices; s += 256) {
+      const float4 m = ml4[2 * s];
+      M[0] = fmaxf(M[0], m.x); M[1] = fmaxf(M[1], m.y); M[2] = fmaxf(M[2], m.z); M[3] = fmaxf(M[3], m.w);
+    }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    double L = 0.0;
-    for (int s = lane; s < a.nslices; s += 32) L += (double)ml[s * 2 * MAXQ + MAXQ + j] * (double)expf(ml[s * 2 * MAXQ + j] - M);
+    for (int j = 0; j < MAXQ; ++j) {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
-    if (lane == 0) {
-      stat[0] = M;
-      stat[1] = (float)(1.0 / L);
+      for (int o = 16; o > 0; o >>= 1) M[j] = fmaxf(M[j], __shfl_xor_sync(0xffffffffu, M[j], o));
+      if (lane == 0) redm[warp][j] = M[j];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < MAXQ; ++j) {
+      M[j] = redm[0][j];
+      for (int w = 1; w < 8; ++w) M[j] = fmaxf(M[j], redm[w][j]);
+    }
+    double L[MAXQ] = {0.0, 0.0, 0.0, 0.0};
+    for (int s = tid; s < a.nslices; s += 256) {
+      const float4 m = ml4[2 * s], l = ml4[2 * s + 1];
+      L[0] += (double)l.x * (double)expf(m.x - M[0]); L[1] += (double)l.y * (double)expf(m.y - M[1]);
+      L[2] += (double)l.z * (double)expf(m.z - M[2]); L[3] += (double)l.w * (double)expf(m.w - M[3]);
+    }
+#pragma unroll
+    for (int j = 0; j < MAXQ; ++j) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) L[j] += __shfl_xor_sync(0xffffffffu, L[j], o);
+      if (lane == 0) redl[warp][j] = L[j];
+    }
+    __syncthreads();
+    if (tid < MAXQ) {
+      double Ls = 0.0;
+      for (int w = 0; w < 8; ++w) Ls += redl[w][tid];
+      stat[0][tid] = M[tid];
+      stat[1][tid] = (float)(1.0 / Ls);
+    }
+    __syncthreads();
+  }
+  const float4 Mv = make_float4(stat[0][0], stat[0][1], stat[0][2], stat[0][3]);
+  const float4 inv = make_float4(stat[1][0], stat[1][1], stat[1][2], stat[1][3]);
+  // thread = (coordinate c of the group, slice phase ph)
+  const int nph = 256 / d, c = tid % d, ph = tid / d;
+  const float4* acc4 = reinterpret_cast<const float4*>(a.part_acc) + (size_t)h * a.nslices * ncoord + gi * d + c;
+  float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s0 = 0; s0 < a.nslices; s0 += 256) {
+    const int ns = min(256, a.nslices - s0);
+    __syncthreads();
+    if (tid < ns) {
+      const float4 m = ml4[2 * (s0 + tid)];
+      wsl[tid] = make_float4(expf(m.x - Mv.x) * inv.x, expf(m.y - Mv.y) * inv.y, expf(m.z - Mv.z) * inv.z, expf(m.w - Mv.w) * inv.w);
+    }
+    __syncthreads();
+    if (ph < nph) {
+#pragma unroll 8
+      for (int s = ph; s < ns; s += nph) {
+        const float4 v = acc4[(size_t)(s0 + s) * ncoord], w = wsl[s];
+        y.x = fmaf(w.x, v.x, y.x); y.y = fmaf(w.y, v.y, y.y); y.z = fmaf(w.z, v.z, y.z); y.w = fmaf(w.w, v.w, y.w);
+      }
     }
   }
+  yp[tid] = y;
   __syncthreads();
-  const float M = stat[0], inv = stat[1];
-  const float* acc = a.part_acc + (size_t)h * a.nslices * ncoord * MAXQ;
-  const int half = threadIdx.x >> 7, t = threadIdx.x & 127;   // each half of the CTA adds every other slice
-  for (int oc = t; oc < ncoord; oc += 128) yp[half][oc] = 0.f;
-  for (int s0 = 0; s0 < a.nslices; s0 += 64) {   // slice weights in chunks of 64
-    const int ns = min(64, a.nslices - s0);
-    __syncthreads();
-    if ((int)threadIdx.x < ns) wsl[threadIdx.x] = expf(ml[(s0 + threadIdx.x) * 2 * MAXQ + j] - M) * inv;
-    __syncthreads();
-    for (int oc = t; oc < ncoord; oc += 128) {
-      float v = yp[half][oc];
-#pragma unroll 16
-      for (int s = half; s < ns; s += 2) v = fmaf(wsl[s], acc[((size_t)(s0 + s) * ncoord + oc) * MAXQ + j], v);
-      yp[half][oc] = v;
-    }
+  if (tid < d) {
+    float4 sum = yp[tid];
+    for (int p = 1; p < nph; ++p) add4(sum, yp[p * d + tid]);
+    ys[0][tid] = sum.x; ys[1][tid] = sum.y; ys[2][tid] = sum.z; ys[3][tid] = sum.w;
   }
   __syncthreads();
-  for (int oc = threadIdx.x; oc < ncoord; oc += blockDim.x) yp[0][oc] += yp[1][oc];
-  __syncthreads();
-  // x~_k = sum_c Pi[c][k] y'_c per group, scattered to the group's channels of this head
-  for (int ok = threadIdx.x; ok < ncoord; ok += blockDim.x) {
-    const int gi = ok / d, k = ok % d;
-    const GroupDev& g = a.g[gi];
+  // x~_k = sum_c Pi[c][k] y'_c, scattered to the group's channels of this head
+  for (int it = tid; it < d * a.qpk; it += 256) {
+    const int k = it % d, j = it / d;
     float v = 0.f;
 #pragma unroll 16
-    for (int c = 0; c < d; ++c) v = fmaf(g.v_pi[(size_t)c * d + k], yp[0][gi * d + c], v);
+    for (int cc = 0; cc < d; ++cc) v = fmaf(g.v_pi[(size_t)cc * d + k], ys[j][cc], v);
     out[(int64_t)(h * a.qpk + j) * ldo + g.v_channels[h * d + k]] = v;
   }
 }
@@ -516,15 +559,113 @@ __global__ void __launch_bounds__(MAXD) append_kernel(AppendArgs a, const T* __r
   }
 }
 
+// B fragments of the tensor path: at most 8 plane words and one sign word per 32 coordinates and group
+size_t bfrag_bytes(int ngroups, int heads, int d) { return (size_t)heads * ngroups * (d / 32) * 9 * 32 * sizeof(uint4); }
+
 size_t workspace_bytes(int ngroups, int heads, int64_t tokens, int d) {
   const int64_t nslices = std::max<int64_t>(1, (tokens + SLICE - 1) / SLICE);
   size_t b = (size_t)heads * ngroups * MAXQ * 2 * MAXD * sizeof(float);
   b += (size_t)heads * nslices * 2 * MAXQ * sizeof(float);
   b = (b + 255) / 256 * 256;
   b += (size_t)heads * nslices * ngroups * d * MAXQ * sizeof(float);
+  b = (b + 255) / 256 * 256;
+  b += bfrag_bytes(ngroups, heads, d);
+  b += (size_t)heads * ngroups * MAXQ * 2 * sizeof(KConst);
   return (b + 255) / 256 * 256;
 }
 
+
+// Launch with the programmatic-stream-serialisation attribute.
+template <typename... KArgs, typename... LArgs>
+cudaError_t launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, LArgs... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, args...);
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+// Walsh coefficients of an antisymmetric codebook of 2^bits entries (see tq_decode_mma.cuh); false if it is not one.
+bool walsh_coefficients(const float* c, int bits, float* alpha) {
+  for (int i = 0; i < 8; ++i) alpha[i] = 0.f;
+  if (bits == 0) return true;
+  const int n = 1 << bits;
+  for (int i = 0; i < n / 2; ++i)
+    if (c[i] != -c[n - 1 - i]) return false;
+  auto coef = [&](unsigned subset) {
+    double s = 0.0;
+    for (int idx = 0; idx < n; ++idx) {
+      int sign = 1;
+      for (int i = 0; i < bits; ++i)
+        if (((subset >> i) & 1u) && !((idx >> i) & 1)) sign = -sign;
+      s += sign * (double)c[idx];
+    }
+    return (float)(s / n);
+  };
+  for (int o = 0; o < bits; ++o) alpha[o] = coef(1u << o);
+  if (bits == 3) alpha[3] = coef(7u);
+  if (bits == 4)
+    for (int o = 0; o < 4; ++o) alpha[4 + o] = coef(15u & ~(1u << o));
+  return true;
+}
+
+int piece_bytes(const void* base, int row_stride, int row_bytes, int dst_off_bytes) {
+  const uintptr_t x = reinterpret_cast<uintptr_t>(base) | (uintptr_t)row_stride | (uintptr_t)row_bytes | (uintptr_t)dst_off_bytes;
+  return (x & 15) == 0 ? 16 : (x & 7) == 0 ? 8 : 4;
+}
+
+// Layout of the tensor path for this call; false if it cannot run (codebook shape, shared memory).
+bool plan_mma(int ngroups, int d, const Args& a, char* workspace, size_t off, int heads, MmaArgs* out, size_t* smem_out) {
+  MmaArgs& ma = *out;
+  std::memset(&ma, 0, sizeof(ma));
+  int kw = 0, vw = 0;
+  for (int gi = 0; gi < ngroups; ++gi) {
+    const GroupDev& g = a.g[gi];
+    MmaGroup& m = ma.m[gi];
+    if (!walsh_coefficients(g.k_cent, g.k_bits, m.k_alpha) || !walsh_coefficients(g.v_cent, g.v_bits, m.v_alpha)) return false;
+    m.k_w0 = kw;
+    m.k_mse_nw = plane_words(d, g.k_bits);
+    m.k_raw_nw = raw_words(d, g.k_bits);
+    m.k_qjl_nw = g.k_prod ? d / 32 : 0;
+    if (g.k_bits > 0 && g.k_idx_rb < 4 * m.k_raw_nw) return false;
+    if (g.k_prod && g.k_qjl_rb < 4 * m.k_qjl_nw) return false;
+    m.k_piece_idx = piece_bytes(g.k_idx, g.k_idx_rb, 4 * m.k_raw_nw, 4 * m.k_w0);
+    m.k_piece_qjl = piece_bytes(g.k_qjl, g.k_qjl_rb, 4 * m.k_qjl_nw, 4 * (m.k_w0 + m.k_mse_nw));
+    kw += m.k_mse_nw + m.k_qjl_nw;
+    m.v_w0 = vw;
+    m.v_nw = plane_words(d, g.v_bits);
+    m.v_raw_nw = raw_words(d, g.v_bits);
+    if (g.v_idx_rb < 4 * m.v_raw_nw) return false;
+    m.v_pos0 = 32 * vw;
+    vw += m.v_nw;
+  }
+  if (kw == 0) return false;
+  int ks = (kw + 3) / 4 * 4;
+  if ((ks / 4) % 2 == 0) ks += 4;
+  ma.kw = kw; ma.kstride = ks;
+  ma.vw = vw;
+  ma.qstride16 = vw | 1;
+  ma.vpos = 32 * vw;
+  ma.dstride = (ma.vpos + 8 * ngroups + 31) / 32 * 32 + 8;
+  ma.region0 = (int)std::max<size_t>((size_t)4 * SLICE * ma.kstride + (size_t)16 * kw * 32 + (size_t)2 * ngroups * SLICE * 4,
+                                     (size_t)16 * ma.dstride * 4);
+  ma.region0 = (ma.region0 + 15) / 16 * 16;
+  const size_t smem = (size_t)ma.region0 + (size_t)16 * (SLICE / 4) * ma.qstride16 + (size_t)ngroups * 16 * WT_STRIDE +
+                      (size_t)ngroups * SLICE * 4 + (size_t)ngroups * MAXQ * 2 * sizeof(KConst) + 2 * (NT / 32) * MAXQ * 4 + MAXG * 4;
+  if (smem > 200 * 1024) return false;
+  if ((size_t)kw * 32 * sizeof(uint4) * heads > bfrag_bytes(ngroups, heads, d)) return false;
+  ma.bfrag = reinterpret_cast<uint4*>(workspace + off);
+  ma.kconst = reinterpret_cast<KConst*>(workspace + off + bfrag_bytes(ngroups, heads, d));
+  *smem_out = smem;
+  return true;
+}
 }  // namespace kvdec
 }  // namespace tq
 
@@ -635,11 +776,34 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   off += (size_t)heads * nslices * 2 * MAXQ * sizeof(float);
   off = (off + 255) / 256 * 256;
   a.part_acc = reinterpret_cast<float*>(w + off);
+  off += (size_t)heads * nslices * ngroups * d * MAXQ * sizeof(float);
+  off = (off + 255) / 256 * 256;
 
   int dev = 0;
   TQ_CHECK_CUDA(cudaGetDevice(&dev), who);
   TQ_REQUIRE(dev == groups[0].plan_k->device, TQ_ERR_INVALID_ARG, "%s: the plans belong to device %d, current device is %d", who,
              groups[0].plan_k->device, dev);
+  // ---- the tensor path: antisymmetric codebooks (every Lloyd-Max codebook of the library is) and a slice that fits
+  //      in shared memory; otherwise the table-lookup kernel
+  MmaArgs ma;
+  size_t mma_smem = 0;
+  if (plan_mma(ngroups, d, a, static_cast<char*>(workspace), off, heads, &ma, &mma_smem)) {
+    if (q_dtype == TQ_F32)
+      prepare_mma_kernel<float><<<heads * ngroups, 256, 0, st>>>(a, ma, static_cast<const float*>(Q), ldq);
+    else
+      prepare_mma_kernel<__nv_bfloat16><<<heads * ngroups, 256, 0, st>>>(a, ma, static_cast<const __nv_bfloat16*>(Q), ldq);
+    TQ_CHECK_CUDA(cudaGetLastError(), who);
+    static std::atomic<size_t> mma_smem_set[16];
+    if (dev >= 16 || mma_smem > mma_smem_set[dev].load(std::memory_order_relaxed)) {
+      TQ_CHECK_CUDA(cudaFuncSetAttribute(partial_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_smem), who);
+      if (dev < 16) mma_smem_set[dev].store(mma_smem, std::memory_order_relaxed);
+    }
+    // both successors may be scheduled while their predecessor drains; each orders itself with griddepcontrol.wait
+    TQ_CHECK_CUDA(launch_after(partial_mma_kernel, dim3((unsigned)(heads * nslices)), dim3(NT), mma_smem, st, a, ma), who);
+    TQ_CHECK_CUDA(launch_after(merge_kernel, dim3((unsigned)(heads * ngroups)), dim3(256), 0, st, a, out, ldo), who);
+    count_launches(3);
+    return TQ_OK;
+  }
   if (q_dtype == TQ_F32)
     prepare_kernel<float><<<heads * ngroups, 128, 0, st>>>(a, static_cast<const float*>(Q), ldq);
   else
@@ -655,7 +819,7 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   }
   partial_kernel<<<(unsigned)(heads * nslices), NT, smem, st>>>(a);
   TQ_CHECK_CUDA(cudaGetLastError(), who);
-  merge_kernel<<<heads * q_per_kv, 256, 0, st>>>(a, out, ldo);
+  merge_kernel<<<heads * ngroups, 256, 0, st>>>(a, out, ldo);
   TQ_CHECK_CUDA(cudaGetLastError(), who);
   count_launches(3);
   return TQ_OK;

@@ -1,0 +1,538 @@
+// Decode attention over a compressed KV cache on the integer tensor path (mma.sync.m16n8k32, u8 x s8 / u8 x u8 -> s32).
+// Included by tq_decode_attn.cu inside namespace tq::kvdec, after Args and GroupDev.
+//
+// Bit-plane form.  A Lloyd-Max codebook of the even coordinate density (Section 3.1) is antisymmetric, i.e. an odd
+// function of the index bits: c[idx] = sum_T alpha_T s_T over the subsets T of odd size, s_T = prod_{i in T} (2 bit_i - 1)
+// = 2 parity_T - 1.  A code row therefore becomes a row of "plane bits" (the index bits themselves, plus for 3-bit
+// indices the parity of the three bits, for 4-bit indices the four 3-subset parities) and
+//     sum_c q_c c[idx_c]          = sum_pos alpha(pos) q_{c(pos)} (2 bit(pos) - 1)      (Section 3.2 estimator, MSE term)
+//     sum_t w_t c[idx_{t,c}]      = sum_{pos in c} alpha(pos) sum_t w_t (2 bit_t(pos) - 1)   (value sums, Section 4.3)
+// are 0/1 matrices times fixed-point integer matrices.  `word & (0x01010101 << k)` turns plane bits k, k + 8, k + 16,
+// k + 24 of a word into the four bytes (0 or 2^k) of an operand register; the factor 2^k is divided out of the other
+// operand (scores) or of the result (value sums, exactly).  int32 accumulation is exact, so neither term depends on the
+// order of the tokens or on which warp took which tile.
+//
+//   prepare_mma_kernel   per (head, group): q' = Pi q, q'' = S q of the head's queries, then the B operand of the scores
+//                        (four balanced radix-256 digits of round(2 alpha q 2^f / 2^k) per plane bit and query) and the
+//                        per-query constants.
+//   partial_mma_kernel   per (head, slice of 256 tokens):
+//                        0) code rows -> shared memory (cp.async): key planes as [token][word], value planes as
+//                           [4 tokens][word][token of the four], then transposed in place to [4 tokens][word][byte]
+//                           so that a register holds one byte of four consecutive tokens; derived planes, scalars
+//                        A) scores: A = plane bits of 16 tokens, B = query digits (columns = 4 queries x 4 digits)
+//                        B) slice maximum, p = exp(logit - max), sum of p; w = p nu^V as three u8 digits per (group,
+//                           query, token)
+//                        C) value sums: A = weight digits (rows = 4 queries x 4 digit slots, K = tokens), B = value
+//                           plane bits (columns = plane bits) and one column of ones (sum_t w); per digit 2 X - sum_t w
+//                           is a small exact integer; the plane bits of a coordinate are added in a fixed order
+//   merge_kernel         combines the slices.
+
+struct MmaGroup {
+  int k_w0, k_mse_nw, k_raw_nw, k_qjl_nw;   // K plane row: words [k_w0, +k_mse_nw) MSE planes (first k_raw_nw raw), then k_qjl_nw sign words
+  int v_w0, v_nw, v_raw_nw;                 // V plane row
+  int k_piece_idx, k_piece_qjl;             // bytes per cp.async piece (4, 8 or 16)
+  int v_pos0;                               // first plane-bit position of the group among all V positions
+  float k_alpha[8], v_alpha[8];             // Walsh coefficients: single bits o = 0..3, then (b = 3) the parity of all
+                                            // three bits at [3], (b = 4) the parity of the bits other than o at [4 + o]
+};
+
+struct KConst {
+  int wd[4];        // per balanced digit: sum over the plane bits of 2^k digit(pos), k = pos % 8
+  float scale;      // 2^-(f + 1)
+  float pad[3];
+};
+
+struct MmaArgs {
+  MmaGroup m[MAXG];
+  int kw, kstride;        // words per K plane row, padded row stride (words, 4 * odd)
+  int vw;                 // words per V plane row
+  int qstride16;          // 16-byte units between consecutive token quads of the value planes (odd, >= vw)
+  int vpos;               // plane-bit positions of all groups' values = 32 * vw
+  int dstride;            // ints between digit rows of the value sums (>= vpos + 8 * ngroups, = 8 mod 32)
+  int region0;            // bytes of the region that holds what the scores need, later the value sums
+  uint4* bfrag;           // [heads][kw][32]  B fragments of the scores
+  KConst* kconst;         // [heads][ngroups][MAXQ][2]  constants of the MSE and sign terms
+};
+
+constexpr int WT_STRIDE = SLICE + 16;   // bytes between digit rows of the weights (bank-conflict-free fragment loads)
+constexpr int MAXPW = 9 * (MAXD / 32);  // plane words of one group's keys: at most 8 per 32 coordinates + the sign word
+
+__device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_u8u8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t prmt_b(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+// 2^e as a float, e in [-126, 127]
+__device__ __forceinline__ float pow2f(int e) { return __int_as_float((e + 127) << 23); }
+
+// Words of the plane row of a d-coordinate code row with `bits` index bits per coordinate.
+__host__ __device__ inline int plane_words(int d, int bits) {
+  return bits == 0 ? 0 : bits <= 2 ? d * bits / 32 : bits == 3 ? d * 4 / 32 : d * 8 / 32;
+}
+__host__ __device__ inline int raw_words(int d, int bits) { return d * bits / 32; }
+
+// Plane-bit position -> coordinate and Walsh coefficient.
+__device__ __forceinline__ void plane_pos(int d, int bits, int pos, const float* __restrict__ alpha, int& c, float& a) {
+  if (bits == 1) {
+    c = pos; a = alpha[0];
+  } else if (bits == 2) {
+    c = pos >> 1; a = alpha[pos & 1];
+  } else if (bits == 3) {
+    if (pos < 3 * d) {
+      c = pos / 3; a = alpha[pos % 3];
+    } else {   // parity word j, bit p: taken from word 3 j + p % 3 of the stream, same bit
+      const int q = pos - 3 * d, j = q >> 5, p = q & 31;
+      c = (96 * j + 32 * (p % 3) + p) / 3; a = alpha[3];
+    }
+  } else {
+    if (pos < 4 * d) {
+      c = pos >> 2; a = alpha[pos & 3];
+    } else {
+      const int q = pos - 4 * d;
+      c = q >> 2; a = alpha[4 + (q & 3)];
+    }
+  }
+}
+
+// Derived plane words of one code row (thread-local): word i of the row is row[i * STRIDE]; the raw words are followed
+// by room for the derived ones.
+template <int STRIDE>
+__device__ __forceinline__ void derive_planes(uint32_t* row, int d, int bits) {
+  if (bits == 3) {
+    const int nw = 3 * d / 32;
+    for (int j = 0; j < nw / 3; ++j) {
+      uint32_t z = 0u;
+#pragma unroll
+      for (int r = 0; r < 3; ++r) {
+        const int i = 3 * j + r;
+        const uint32_t x = row[i * STRIDE], nx = i + 1 < nw ? row[(i + 1) * STRIDE] : 0u;
+        const uint32_t y = x ^ __funnelshift_r(x, nx, 1) ^ __funnelshift_r(x, nx, 2);
+        z |= y & (0x49249249u << r);   // bits p with p % 3 == r
+      }
+      row[(nw + j) * STRIDE] = z;
+    }
+  } else if (bits == 4) {
+    const int nw = d / 8;
+    for (int i = 0; i < nw; ++i) {
+      const uint32_t x = row[i * STRIDE];
+      const uint32_t t = (x ^ (x >> 1) ^ (x >> 2) ^ (x >> 3)) & 0x11111111u;   // parity of each nibble
+      row[(nw + i) * STRIDE] = x ^ (t * 15u);                                  // bit o: parity of the other three bits
+    }
+  }
+}
+
+// ------------------------------------------------------------------ query preparation for the tensor path
+template <typename T>
+__global__ void __launch_bounds__(256) prepare_mma_kernel(Args a, MmaArgs ma, const T* __restrict__ Q, int64_t ldq) {
+  __shared__ float qs[MAXQ][MAXD];
+  __shared__ float qr[MAXQ][2 * MAXD];           // q' then q''
+  __shared__ int wmax[2][MAXQ];                  // bit patterns of the largest |weight| per term and query
+  __shared__ int wdsum[2][MAXQ][4];
+  __shared__ uint32_t wdig[MAXPW * 32][MAXQ];    // the four digit bytes of every (plane bit, query)
+  const int h = blockIdx.x / a.ngroups, gi = blockIdx.x % a.ngroups;
+  const GroupDev& g = a.g[gi];
+  const MmaGroup& m = ma.m[gi];
+  const int d = a.d, tid = threadIdx.x;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the slices' code rows may start to travel
+  for (int e = tid; e < MAXQ * d; e += blockDim.x) {
+    const int j = e / d, c = e % d;
+    float v = 0.f;
+    if (j < a.qpk) v = (float)Q[(int64_t)(h * a.qpk + j) * ldq + g.k_channels[h * d + c]];
+    qs[j][c] = v;
+  }
+  if (tid < 2 * MAXQ) wmax[tid / MAXQ][tid % MAXQ] = 0;
+  if (tid < 2 * MAXQ * 4) (&wdsum[0][0][0])[tid] = 0;
+  __syncthreads();
+  const int nrows = (g.k_prod ? 2 : 1) * g.k_dpad;
+  for (int o = tid; o < 2 * MAXD; o += blockDim.x) {
+    const int half = o / MAXD, r = o % MAXD;
+    float acc[MAXQ] = {0.f, 0.f, 0.f, 0.f};
+    if (r < d && (half == 0 || g.k_prod)) {
+      const float* col = g.k_backt + half * g.k_dpad + r;
+#pragma unroll 32
+      for (int c = 0; c < d; ++c) {   // independent loads: unrolled deep, the kernel is latency-bound
+        const float mm = __ldg(col + (size_t)c * nrows);
+#pragma unroll
+        for (int j = 0; j < MAXQ; ++j) acc[j] = fmaf(mm, qs[j][c], acc[j]);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < MAXQ; ++j) qr[j][o] = acc[j];
+  }
+  __syncthreads();
+
+  // weight of plane bit `pos` (group-local: MSE planes, then sign bits) for query j: 2 alpha q'_c, 2 q''_i
+  const int npos_mse = 32 * m.k_mse_nw, npos = npos_mse + 32 * m.k_qjl_nw;
+  auto weight = [&](int pos, int j) -> float {
+    if (pos < npos_mse) {
+      int c; float al;
+      plane_pos(d, g.k_bits, pos, m.k_alpha, c, al);
+      return 2.f * al * qr[j][c];
+    }
+    return 2.f * qr[j][MAXD + pos - npos_mse];
+  };
+  for (int it = tid; it < npos * MAXQ; it += blockDim.x) {
+    const int pos = it >> 2, j = it & 3;
+    atomicMax(&wmax[pos < npos_mse ? 0 : 1][j], __float_as_int(fabsf(weight(pos, j))));
+  }
+  __syncthreads();
+  // exponent f with |w| 2^f < 2^30 (clamped: weights below 2^-90 of the scale do not matter)
+  auto fexp = [&](int term, int j) -> int {
+    const int bits = wmax[term][j];
+    if (bits == 0) return 0;
+    const int e = ((bits >> 23) & 255) - 126;   // |w| < 2^e
+    return max(-90, min(110, 30 - e));
+  };
+  for (int it = tid; it < npos * MAXQ; it += blockDim.x) {
+    const int pos = it >> 2, j = it & 3, term = pos < npos_mse ? 0 : 1, k = pos & 7;
+    int W = __float2int_rn(weight(pos, j) * pow2f(fexp(term, j) - k));
+    uint32_t packed = 0u;
+#pragma unroll
+    for (int dg = 0; dg < 4; ++dg) {   // balanced radix-256 digits, the top one takes what is left
+      const int lo = dg == 3 ? W : ((W + 128) & 255) - 128;
+      W = (W - lo) >> 8;
+      packed |= (uint32_t)(lo & 255) << (8 * dg);
+      atomicAdd(&wdsum[term][j][dg], lo * (1 << k));
+    }
+    wdig[pos][j] = packed;
+  }
+  __syncthreads();
+  // B fragments: word w, lane (n, kq): registers (tile 0, K half 0), (tile 0, half 1), (tile 1, half 0), (tile 1, half 1);
+  // byte i of K half r: plane bit 32 w + 8 i + kq + 4 r; column n of tile tt: query n / 2, digit 2 tt + (n & 1)
+  uint4* bf = ma.bfrag + ((size_t)h * ma.kw + m.k_w0) * 32;
+  for (int it = tid; it < (npos >> 5) * 32; it += blockDim.x) {
+    const int w = it >> 5, lane = it & 31, n = lane >> 2, kq = lane & 3, j = n >> 1;
+    uint32_t reg[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int r = 0; r < 2; ++r)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t pk = wdig[32 * w + 8 * i + kq + 4 * r][j] >> (8 * (n & 1));
+        reg[r] |= (pk & 255u) << (8 * i);
+        reg[2 + r] |= ((pk >> 16) & 255u) << (8 * i);
+      }
+    bf[(size_t)w * 32 + lane] = make_uint4(reg[0], reg[1], reg[2], reg[3]);
+  }
+  if (tid < 2 * MAXQ) {
+    const int term = tid / MAXQ, j = tid % MAXQ;
+    KConst c;
+#pragma unroll
+    for (int dg = 0; dg < 4; ++dg) c.wd[dg] = wdsum[term][j][dg];
+    c.scale = pow2f(-(fexp(term, j) + 1));
+    c.pad[0] = c.pad[1] = c.pad[2] = 0.f;
+    ma.kconst[((size_t)(h * a.ngroups + gi) * MAXQ + j) * 2 + term] = c;
+  }
+}
+
+// ------------------------------------------------------------------ per-slice scores, weights, value sums
+template <int BYTES>
+__device__ __forceinline__ void cp_async_piece(uint32_t dst, const void* src) {
+  if (BYTES == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+  else if (BYTES == 8) asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+  else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+
+// The first `nb` bytes of this thread's code row to its plane row in shared memory, in pieces of `piece` bytes.
+__device__ __forceinline__ void stage_row(uint32_t dst, const unsigned char* src, int nb, int piece) {
+  if (piece == 16) {
+    for (int o = 0; o < nb; o += 16) cp_async_piece<16>(dst + o, src + o);
+  } else if (piece == 8) {
+    for (int o = 0; o < nb; o += 8) cp_async_piece<8>(dst + o, src + o);
+  } else {
+    for (int o = 0; o < nb; o += 4) cp_async_piece<4>(dst + o, src + o);
+  }
+}
+
+__global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int ng = a.ngroups, d = a.d;
+  // region 0: what the scores need (key planes, B fragments, key scalars); later the digit rows of the value sums
+  uint32_t* krow = reinterpret_cast<uint32_t*>(smem_raw);                        // [SLICE][kstride]
+  uint4* bs = reinterpret_cast<uint4*>(krow + SLICE * ma.kstride);               // [kw][32]
+  float* knu = reinterpret_cast<float*>(bs + ma.kw * 32);                        // [ng][SLICE]
+  float* kgm = knu + ng * SLICE;                                                 // [ng][SLICE]
+  int* dbuf = reinterpret_cast<int*>(smem_raw);                                  // [16][dstride]
+  uint32_t* vq = reinterpret_cast<uint32_t*>(smem_raw + ma.region0);             // [SLICE / 4][qstride16][4]
+  unsigned char* wt = reinterpret_cast<unsigned char*>(vq + (SLICE / 4) * ma.qstride16 * 4);   // [ng][16][WT_STRIDE]
+  float* vnu = reinterpret_cast<float*>(wt + ng * 16 * WT_STRIDE);               // [ng][SLICE]
+  KConst* kc = reinterpret_cast<KConst*>(vnu + ng * SLICE);                      // [ng][MAXQ][2]
+  float* red = reinterpret_cast<float*>(kc + ng * MAXQ * 2);                     // [2][NT / 32][MAXQ]
+  int* vmax = reinterpret_cast<int*>(red + 2 * (NT / 32) * MAXQ);                // [MAXG] bit patterns of max nu^V
+
+  const int h = blockIdx.x / a.nslices, sl = blockIdx.x % a.nslices;
+  const int64_t t0 = (int64_t)sl * SLICE;
+  const int ntok = (int)min((int64_t)SLICE, a.tokens - t0);
+  const int64_t row0 = (int64_t)h * a.head_stride + t0;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g8 = lane >> 2, kq = lane & 3;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  // ---- 0) thread = token: its code rows and scalars travel to shared memory (inputs of the call: before the
+  //         dependency wait).  Word w of the token's value planes goes to [token / 4][w][token % 4].
+  uint32_t* vmine = vq + (tid >> 2) * ma.qstride16 * 4 + (tid & 3);   // this token's word 0; words are 4 apart
+  if (tid < ntok) {
+    const int64_t row = row0 + tid;
+    const uint32_t kdst = (uint32_t)__cvta_generic_to_shared(krow + tid * ma.kstride);
+    const uint32_t vdst = (uint32_t)__cvta_generic_to_shared(vmine);
+    for (int gi = 0; gi < ng; ++gi) {
+      const GroupDev& g = a.g[gi];
+      const MmaGroup& m = ma.m[gi];
+      if (g.k_bits > 0) stage_row(kdst + 4 * m.k_w0, g.k_idx + (size_t)row * g.k_idx_rb, 4 * m.k_raw_nw, m.k_piece_idx);
+      if (g.k_prod) stage_row(kdst + 4 * (m.k_w0 + m.k_mse_nw), g.k_qjl + (size_t)row * g.k_qjl_rb, 4 * m.k_qjl_nw, m.k_piece_qjl);
+      const unsigned char* vsrc = g.v_idx + (size_t)row * g.v_idx_rb;
+      for (int w = 0; w < m.v_raw_nw; ++w) cp_async_piece<4>(vdst + 16 * (m.v_w0 + w), vsrc + 4 * w);
+      if (g.k_norms) cp_async_piece<4>((uint32_t)__cvta_generic_to_shared(knu + gi * SLICE + tid), g.k_norms + row);
+      if (g.k_prod) cp_async_piece<4>((uint32_t)__cvta_generic_to_shared(kgm + gi * SLICE + tid), g.k_gamma + row);
+      if (g.v_norms) cp_async_piece<4>((uint32_t)__cvta_generic_to_shared(vnu + gi * SLICE + tid), g.v_norms + row);
+    }
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  if (tid < MAXG) vmax[tid] = 0;
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // the query-side operand is the previous kernel's output
+  {
+    const uint4* src = ma.bfrag + (size_t)h * ma.kw * 32;
+    for (int i = tid; i < ma.kw * 32; i += NT) bs[i] = __ldg(src + i);
+    const uint4* cs = reinterpret_cast<const uint4*>(ma.kconst + (size_t)h * ng * MAXQ * 2);
+    for (int i = tid; i < ng * MAXQ * 2 * 2; i += NT) reinterpret_cast<uint4*>(kc)[i] = __ldg(cs + i);
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+
+  // ---- derived planes, defaults of absent scalars, largest value norm of the slice (thread = token)
+  for (int gi = 0; gi < ng; ++gi) {
+    const GroupDev& g = a.g[gi];
+    const MmaGroup& m = ma.m[gi];
+    float vm = 0.f;
+    if (tid < ntok) {
+      if (g.k_bits >= 3) derive_planes<1>(krow + tid * ma.kstride + m.k_w0, d, g.k_bits);
+      if (g.v_bits >= 3) derive_planes<4>(vmine + 4 * m.v_w0, d, g.v_bits);
+      if (!g.k_norms) knu[gi * SLICE + tid] = 1.f;
+      if (!g.k_prod) kgm[gi * SLICE + tid] = 0.f;
+      if (!g.v_norms) vnu[gi * SLICE + tid] = 1.f;
+      vm = vnu[gi * SLICE + tid];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xffffffffu, vm, o));
+    if (lane == 0) atomicMax(&vmax[gi], __float_as_int(fmaxf(vm, 0.f)));
+  }
+  __syncthreads();
+
+  // ---- value planes transposed in place: (quad, word) holds the word of the quad's four tokens; afterwards
+  //      register s = byte s of that word for the four tokens
+  {
+    uint4* vq4 = reinterpret_cast<uint4*>(vq);
+    const int wl = tid & 7;
+    for (int qd = tid >> 3; qd < SLICE / 4; qd += NT / 8)
+      for (int w = wl; w < ma.vw; w += 8) {
+        uint4* p = vq4 + qd * ma.qstride16 + w;
+        const uint4 x = *p;
+        const uint32_t lo01 = prmt_b(x.x, x.y, 0x5140u), lo23 = prmt_b(x.z, x.w, 0x5140u);
+        const uint32_t hi01 = prmt_b(x.x, x.y, 0x7362u), hi23 = prmt_b(x.z, x.w, 0x7362u);
+        *p = make_uint4(prmt_b(lo01, lo23, 0x5410u), prmt_b(lo01, lo23, 0x7632u), prmt_b(hi01, hi23, 0x5410u),
+                        prmt_b(hi01, hi23, 0x7632u));
+      }
+  }
+
+  // ---- A) scores.  Thread (g8, kq) of a warp: tokens g8 and g8 + 8 of the warp's 16-token tile, query kq.
+  constexpr int MT = SLICE / 16 / (NT / 32);   // tiles per warp
+  const uint32_t m0 = 0x01010101u << kq, m1 = m0 << 4;
+  float logit[MT][2];
+#pragma unroll
+  for (int i = 0; i < MT; ++i) {
+    const int tb = 16 * (warp + (NT / 32) * i);
+    float score[2] = {0.f, 0.f};
+    for (int gi = 0; gi < ng; ++gi) {
+      const MmaGroup& m = ma.m[gi];
+      const uint32_t* r0 = krow + (tb + g8) * ma.kstride + m.k_w0;
+      const uint32_t* r1 = r0 + 8 * ma.kstride;
+      const uint4* bb = bs + m.k_w0 * 32 + lane;
+      float term[2][2];   // [mse, sign][row]
+#pragma unroll
+      for (int tm = 0; tm < 2; ++tm) {
+        const int w_lo = tm == 0 ? 0 : m.k_mse_nw, w_hi = tm == 0 ? m.k_mse_nw : m.k_mse_nw + m.k_qjl_nw;
+        int acc[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+        for (int w = w_lo; w < w_hi; ++w) {
+          const uint32_t x0 = r0[w], x1 = r1[w];
+          const uint4 b = bb[w * 32];
+          mma_u8s8(acc[0], x0 & m0, x1 & m0, x0 & m1, x1 & m1, b.x, b.y);
+          mma_u8s8(acc[1], x0 & m0, x1 & m0, x0 & m1, x1 & m1, b.z, b.w);
+        }
+        // sum_pos W (2 bit - 1), digit by digit (each difference is a small exact integer), then Horner in fp32
+        const KConst c = kc[(gi * MAXQ + kq) * 2 + tm];
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          const float d0 = (float)(2 * acc[0][2 * hh] - c.wd[0]), d1 = (float)(2 * acc[0][2 * hh + 1] - c.wd[1]);
+          const float d2 = (float)(2 * acc[1][2 * hh] - c.wd[2]), d3 = (float)(2 * acc[1][2 * hh + 1] - c.wd[3]);
+          term[tm][hh] = fmaf(256.f, fmaf(256.f, fmaf(256.f, d3, d2), d1), d0) * c.scale;
+        }
+      }
+      const float coef = a.g[gi].coef;
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const int t = tb + g8 + 8 * hh;
+        score[hh] += knu[gi * SLICE + t] * fmaf(coef * kgm[gi * SLICE + t], term[1][hh], term[0][hh]);
+      }
+    }
+    logit[i][0] = a.scale * score[0];
+    logit[i][1] = a.scale * score[1];
+  }
+
+  // ---- B) slice maximum per query, exponentials, their sum (fixed order), weight digits (three per weight)
+  {
+    float mx = -FLT_MAX;
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh)
+        if (16 * (warp + (NT / 32) * i) + g8 + 8 * hh < ntok) mx = fmaxf(mx, logit[i][hh]);
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (g8 == 0) red[warp * MAXQ + kq] = mx;
+  }
+  __syncthreads();
+  float smax = red[kq];
+#pragma unroll
+  for (int w = 1; w < NT / 32; ++w) smax = fmaxf(smax, red[w * MAXQ + kq]);
+  float sg[MAXG];   // nu^V < 2^e and p <= 1: w 2^(24 - e) < 2^24
+#pragma unroll
+  for (int gi = 0; gi < MAXG; ++gi) {
+    const int bits = gi < ng ? vmax[gi] : 0;
+    sg[gi] = bits > 0 ? pow2f(max(-126, min(127, 24 - (((bits >> 23) & 255) - 126)))) : 1.f;
+  }
+  {
+    float psum = 0.f;
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const int t = 16 * (warp + (NT / 32) * i) + g8 + 8 * hh;
+        const bool live = t < ntok && kq < a.qpk;
+        const float p = live ? expf(logit[i][hh] - smax) : 0.f;
+        psum += p;
+#pragma unroll
+        for (int gi = 0; gi < MAXG; ++gi)
+          if (gi < ng) {
+            const uint32_t W = live ? min(__float2uint_rn(p * vnu[gi * SLICE + t] * sg[gi]), 0xffffffu) : 0u;
+            unsigned char* col = wt + (gi * 16 + 4 * kq) * WT_STRIDE + t;
+            col[0] = (unsigned char)W;
+            col[WT_STRIDE] = (unsigned char)(W >> 8);
+            col[2 * WT_STRIDE] = (unsigned char)(W >> 16);
+          }
+      }
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) psum += __shfl_xor_sync(0xffffffffu, psum, o);
+    if (g8 == 0) red[(NT / 32) * MAXQ + warp * MAXQ + kq] = psum;
+  }
+  __syncthreads();   // the weights are complete; region 0 is dead
+  if (tid < MAXQ) {
+    float* ml = a.part_ml + (size_t)(h * a.nslices + sl) * 2 * MAXQ;
+    float s = 0.f, m = red[tid];
+    for (int w = 0; w < NT / 32; ++w) {
+      s += red[(NT / 32) * MAXQ + w * MAXQ + tid];
+      m = fmaxf(m, red[w * MAXQ + tid]);
+    }
+    ml[tid] = m;
+    ml[MAXQ + tid] = s;
+  }
+
+  // ---- C) value sums.  Rows of A: weight digit dg of query j at row 4 j + dg (row 4 j + 3 is not used); K = the
+  //         slice's tokens; columns of B: plane bits.  A unit = half a plane word (two 8-column tiles); the units of
+  //         a group are dealt to the warps; warp gi % 8 also takes the group's column of ones (sum_t w).
+  constexpr int CH = 3;   // units in flight per warp
+  const int nks = (ntok + 31) / 32;
+  const uint32_t mn = 0x01010101u << g8;
+  const uint4* vq4 = reinterpret_cast<const uint4*>(vq);
+  for (int gi = 0; gi < ng; ++gi) {
+    const MmaGroup& m = ma.m[gi];
+    const int U = 2 * m.v_nw;
+    const int ub = U * warp / (NT / 32), ue = U * (warp + 1) / (NT / 32);
+    const unsigned char* wr0 = wt + (gi * 16 + g8) * WT_STRIDE + 4 * kq;
+    const bool ones = warp == (gi & (NT / 32 - 1));
+    for (int u0 = ub; u0 < ue || (ones && u0 == ub); u0 += CH) {
+      int acc[CH][2][4], acc1[4] = {0, 0, 0, 0};
+#pragma unroll
+      for (int uu = 0; uu < CH; ++uu)
+#pragma unroll
+        for (int tt = 0; tt < 2; ++tt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[uu][tt][e] = 0;
+      const bool with_ones = ones && u0 == ub;
+      for (int ks = 0; ks < nks; ++ks) {
+        const unsigned char* wr = wr0 + 32 * ks;
+        const uint32_t a0 = *reinterpret_cast<const uint32_t*>(wr), a1 = *reinterpret_cast<const uint32_t*>(wr + 8 * WT_STRIDE);
+        const uint32_t a2 = *reinterpret_cast<const uint32_t*>(wr + 16), a3 = *reinterpret_cast<const uint32_t*>(wr + 8 * WT_STRIDE + 16);
+        const uint4* q0 = vq4 + (8 * ks + kq) * ma.qstride16 + m.v_w0;
+        const uint4* q1 = q0 + 4 * ma.qstride16;
+        if (with_ones) mma_u8u8(acc1, a0, a1, a2, a3, 0x01010101u, 0x01010101u);
+#pragma unroll
+        for (int uu = 0; uu < CH; ++uu) {
+          const int u = u0 + uu;
+          if (u < ue) {
+            const uint2 b0 = reinterpret_cast<const uint2*>(q0 + (u >> 1))[u & 1];
+            const uint2 b1 = reinterpret_cast<const uint2*>(q1 + (u >> 1))[u & 1];
+            mma_u8u8(acc[uu][0], a0, a1, a2, a3, b0.x & mn, b1.x & mn);
+            mma_u8u8(acc[uu][1], a0, a1, a2, a3, b0.y & mn, b1.y & mn);
+          }
+        }
+      }
+      // digit rows g8 and g8 + 8, columns 2 kq and 2 kq + 1 of each tile
+      if (with_ones) {
+        int* dd = dbuf + g8 * ma.dstride + ma.vpos + 8 * gi + 2 * kq;
+        *reinterpret_cast<int2*>(dd) = make_int2(acc1[0], acc1[1]);
+        *reinterpret_cast<int2*>(dd + 8 * ma.dstride) = make_int2(acc1[2], acc1[3]);
+      }
+#pragma unroll
+      for (int uu = 0; uu < CH; ++uu) {
+        const int u = u0 + uu;
+        if (u < ue) {
+#pragma unroll
+          for (int tt = 0; tt < 2; ++tt) {
+            int* dd = dbuf + g8 * ma.dstride + m.v_pos0 + 32 * (u >> 1) + 8 * (2 * (u & 1) + tt) + 2 * kq;
+            *reinterpret_cast<int2*>(dd) = make_int2(acc[uu][tt][0], acc[uu][tt][1]);
+            *reinterpret_cast<int2*>(dd + 8 * ma.dstride) = make_int2(acc[uu][tt][2], acc[uu][tt][3]);
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- item = (coordinate, query): per digit 2 X - sum_t w is a small exact integer (column pos carries the factor
+  //      2^(pos % 8)); Horner over the digits in fp32; the coordinate's plane bits added in a fixed order
+  const int ncoord = ng * d;
+  float* out = a.part_acc + (size_t)(h * a.nslices + sl) * ncoord * MAXQ;
+  for (int it = tid; it < ncoord * MAXQ; it += NT) {
+    const int oc = it >> 2, j = it & 3, gi = oc / d, c = oc - gi * d, bits = a.g[gi].v_bits;
+    const MmaGroup& m = ma.m[gi];
+    const int* dj = dbuf + 4 * j * ma.dstride;
+    const int oc0 = ma.vpos + 8 * gi;
+    const int o0 = dj[oc0], o1 = dj[ma.dstride + oc0], o2 = dj[2 * ma.dstride + oc0];
+    auto plane = [&](int pos, float alpha) -> float {
+      const int col = m.v_pos0 + pos, sh = pos & 7;
+      const float e0 = (float)(2 * (dj[col] >> sh) - o0), e1 = (float)(2 * (dj[ma.dstride + col] >> sh) - o1);
+      const float e2 = (float)(2 * (dj[2 * ma.dstride + col] >> sh) - o2);
+      return alpha * fmaf(256.f, fmaf(256.f, e2, e1), e0);
+    };
+    float s = 0.f;
+    if (bits <= 2) {
+      for (int o = 0; o < bits; ++o) s += plane(bits * c + o, m.v_alpha[o]);
+    } else if (bits == 3) {
+      for (int o = 0; o < 3; ++o) s += plane(3 * c + o, m.v_alpha[o]);
+      const int sp = 3 * c;
+      s += plane(3 * d + 32 * ((sp >> 5) / 3) + (sp & 31), m.v_alpha[3]);
+    } else {
+      for (int o = 0; o < 4; ++o) s += plane(4 * c + o, m.v_alpha[o]);
+      for (int o = 0; o < 4; ++o) s += plane(4 * d + 4 * c + o, m.v_alpha[4 + o]);
+    }
+    out[it] = s / sg[gi];
+  }
+}
