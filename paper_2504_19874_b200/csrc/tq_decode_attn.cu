@@ -381,22 +381,33 @@ __global__ void __launch_bounds__(NT) partial_kernel(Args a) {
 // ------------------------------------------------------------------ merge of the slices + inverse rotation
 // One CTA per (head, group), all queries of the head at once: slice weights exp(m_s - M) / L, the weighted sum of the
 // slices' partial value sums (float4 = the four queries of a coordinate), then x~ = Pi_V^T y' scattered to the group's
-// channels.  Every sum runs in a fixed order.
-__global__ void __launch_bounds__(256) merge_kernel(Args a, float* __restrict__ out, int64_t ldo) {
-  __shared__ float4 wsl[256];
-  __shared__ float4 yp[256];
+// channels.  Every sum runs in a fixed order.  The kernel is a chain of memory latencies, so Pi_V (an input of the
+// call) is fetched into shared memory before the wait for the kernel ahead, and the threads are many enough that
+// every load of a step is in flight at once.
+constexpr int MERGE_NT = 512;
+__global__ void __launch_bounds__(MERGE_NT) merge_kernel(Args a, float* __restrict__ out, int64_t ldo) {
+  extern __shared__ __align__(16) float pis[];   // [d][d] Pi_V
+  __shared__ float4 wsl[MERGE_NT];
+  __shared__ float4 yp[MERGE_NT];
   __shared__ float ys[MAXQ][MAXD];
-  __shared__ float redm[8][MAXQ];
-  __shared__ double redl[8][MAXQ];
+  __shared__ float redm[MERGE_NT / 32][MAXQ];
+  __shared__ double redl[MERGE_NT / 32][MAXQ];
   __shared__ float stat[2][MAXQ];
+  __shared__ int chan[MAXD];
   const int h = blockIdx.x / a.ngroups, gi = blockIdx.x % a.ngroups;
   const int ncoord = a.ngroups * a.d, d = a.d, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const GroupDev& g = a.g[gi];
+  {
+    const float4* src = reinterpret_cast<const float4*>(g.v_pi);
+    float4* dst = reinterpret_cast<float4*>(pis);
+    for (int i = tid; i < d * d / 4; i += MERGE_NT) dst[i] = __ldg(src + i);
+    if (tid < d) chan[tid] = g.v_channels[h * d + tid];
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");   // the slices' partial results come from the kernel before
   const float4* ml4 = reinterpret_cast<const float4*>(a.part_ml + (size_t)h * a.nslices * 2 * MAXQ);   // [slice][max, sum]
   {   // global maximum and sum per query
     float M[MAXQ] = {-FLT_MAX, -FLT_MAX, -FLT_MAX, -FLT_MAX};
-    for (int s = tid; s < a.nslices; s += 256) {
+    for (int s = tid; s < a.nslices; s += MERGE_NT) {
       const float4 m = ml4[2 * s];
       M[0] = fmaxf(M[0], m.x); M[1] = fmaxf(M[1], m.y); M[2] = fmaxf(M[2], m.z); M[3] = fmaxf(M[3], m.w);
     }
@@ -410,10 +421,10 @@ __global__ void __launch_bounds__(256) merge_kernel(Args a, float* __restrict__ 
 #pragma unroll
     for (int j = 0; j < MAXQ; ++j) {
       M[j] = redm[0][j];
-      for (int w = 1; w < 8; ++w) M[j] = fmaxf(M[j], redm[w][j]);
+      for (int w = 1; w < MERGE_NT / 32; ++w) M[j] = fmaxf(M[j], redm[w][j]);
     }
     double L[MAXQ] = {0.0, 0.0, 0.0, 0.0};
-    for (int s = tid; s < a.nslices; s += 256) {
+    for (int s = tid; s < a.nslices; s += MERGE_NT) {
       const float4 m = ml4[2 * s], l = ml4[2 * s + 1];
       L[0] += (double)l.x * (double)expf(m.x - M[0]); L[1] += (double)l.y * (double)expf(m.y - M[1]);
       L[2] += (double)l.z * (double)expf(m.z - M[2]); L[3] += (double)l.w * (double)expf(m.w - M[3]);
@@ -427,7 +438,7 @@ __global__ void __launch_bounds__(256) merge_kernel(Args a, float* __restrict__ 
     __syncthreads();
     if (tid < MAXQ) {
       double Ls = 0.0;
-      for (int w = 0; w < 8; ++w) Ls += redl[w][tid];
+      for (int w = 0; w < MERGE_NT / 32; ++w) Ls += redl[w][tid];
       stat[0][tid] = M[tid];
       stat[1][tid] = (float)(1.0 / Ls);
     }
@@ -436,11 +447,11 @@ __global__ void __launch_bounds__(256) merge_kernel(Args a, float* __restrict__ 
   const float4 Mv = make_float4(stat[0][0], stat[0][1], stat[0][2], stat[0][3]);
   const float4 inv = make_float4(stat[1][0], stat[1][1], stat[1][2], stat[1][3]);
   // thread = (coordinate c of the group, slice phase ph)
-  const int nph = 256 / d, c = tid % d, ph = tid / d;
+  const int nph = MERGE_NT / d, c = tid % d, ph = tid / d;
   const float4* acc4 = reinterpret_cast<const float4*>(a.part_acc) + (size_t)h * a.nslices * ncoord + gi * d + c;
   float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s0 = 0; s0 < a.nslices; s0 += 256) {
-    const int ns = min(256, a.nslices - s0);
+  for (int s0 = 0; s0 < a.nslices; s0 += MERGE_NT) {
+    const int ns = min(MERGE_NT, a.nslices - s0);
     __syncthreads();
     if (tid < ns) {
       const float4 m = ml4[2 * (s0 + tid)];
@@ -464,12 +475,12 @@ __global__ void __launch_bounds__(256) merge_kernel(Args a, float* __restrict__ 
   }
   __syncthreads();
   // x~_k = sum_c Pi[c][k] y'_c, scattered to the group's channels of this head
-  for (int it = tid; it < d * a.qpk; it += 256) {
+  for (int it = tid; it < d * a.qpk; it += MERGE_NT) {
     const int k = it % d, j = it / d;
     float v = 0.f;
-#pragma unroll 16
-    for (int cc = 0; cc < d; ++cc) v = fmaf(g.v_pi[(size_t)cc * d + k], ys[j][cc], v);
-    out[(int64_t)(h * a.qpk + j) * ldo + g.v_channels[h * d + k]] = v;
+#pragma unroll 8
+    for (int cc = 0; cc < d; ++cc) v = fmaf(pis[cc * d + k], ys[j][cc], v);
+    out[(int64_t)(h * a.qpk + j) * ldo + chan[k]] = v;
   }
 }
 
@@ -783,6 +794,12 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   TQ_CHECK_CUDA(cudaGetDevice(&dev), who);
   TQ_REQUIRE(dev == groups[0].plan_k->device, TQ_ERR_INVALID_ARG, "%s: the plans belong to device %d, current device is %d", who,
              groups[0].plan_k->device, dev);
+  const size_t merge_smem = (size_t)d * d * sizeof(float);
+  static std::atomic<size_t> merge_smem_set[16];
+  if (dev >= 16 || merge_smem > merge_smem_set[dev].load(std::memory_order_relaxed)) {
+    TQ_CHECK_CUDA(cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)merge_smem), who);
+    if (dev < 16) merge_smem_set[dev].store(merge_smem, std::memory_order_relaxed);
+  }
   // ---- the tensor path: antisymmetric codebooks (every Lloyd-Max codebook of the library is) and a slice that fits
   //      in shared memory; otherwise the table-lookup kernel
   MmaArgs ma;
@@ -796,11 +813,13 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
     static std::atomic<size_t> mma_smem_set[16];
     if (dev >= 16 || mma_smem > mma_smem_set[dev].load(std::memory_order_relaxed)) {
       TQ_CHECK_CUDA(cudaFuncSetAttribute(partial_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_smem), who);
+      // several CTAs per SM hide the latencies of the kernel's short phases: ask for the largest shared-memory carve-out
+      TQ_CHECK_CUDA(cudaFuncSetAttribute(partial_mma_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared), who);
       if (dev < 16) mma_smem_set[dev].store(mma_smem, std::memory_order_relaxed);
     }
     // both successors may be scheduled while their predecessor drains; each orders itself with griddepcontrol.wait
     TQ_CHECK_CUDA(launch_after(partial_mma_kernel, dim3((unsigned)(heads * nslices)), dim3(NT), mma_smem, st, a, ma), who);
-    TQ_CHECK_CUDA(launch_after(merge_kernel, dim3((unsigned)(heads * ngroups)), dim3(256), 0, st, a, out, ldo), who);
+    TQ_CHECK_CUDA(launch_after(merge_kernel, dim3((unsigned)(heads * ngroups)), dim3(MERGE_NT), merge_smem, st, a, out, ldo), who);
     count_launches(3);
     return TQ_OK;
   }
@@ -819,7 +838,7 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   }
   partial_kernel<<<(unsigned)(heads * nslices), NT, smem, st>>>(a);
   TQ_CHECK_CUDA(cudaGetLastError(), who);
-  merge_kernel<<<heads * ngroups, 256, 0, st>>>(a, out, ldo);
+  merge_kernel<<<heads * ngroups, MERGE_NT, merge_smem, st>>>(a, out, ldo);
   TQ_CHECK_CUDA(cudaGetLastError(), who);
   count_launches(3);
   return TQ_OK;

@@ -181,56 +181,80 @@ __global__ void __launch_bounds__(256) prepare_mma_kernel(Args a, MmaArgs ma, co
     }
     return 2.f * qr[j][MAXD + pos - npos_mse];
   };
-  for (int it = tid; it < npos * MAXQ; it += blockDim.x) {
-    const int pos = it >> 2, j = it & 3;
-    atomicMax(&wmax[pos < npos_mse ? 0 : 1][j], __float_as_int(fabsf(weight(pos, j))));
+  // (item = tid + 256 i: a thread keeps its query j = tid % 4; lanes of equal j are combined before the atomics)
+  const int j = tid & 3;
+  {
+    float mx[2] = {0.f, 0.f};
+    for (int pos = tid >> 2; pos < npos; pos += blockDim.x / 4) {
+      const float w = fabsf(weight(pos, j));
+      if (pos < npos_mse) mx[0] = fmaxf(mx[0], w); else mx[1] = fmaxf(mx[1], w);
+    }
+#pragma unroll
+    for (int term = 0; term < 2; ++term) {
+#pragma unroll
+      for (int o = 4; o < 32; o <<= 1) mx[term] = fmaxf(mx[term], __shfl_xor_sync(0xffffffffu, mx[term], o));
+      if ((tid & 31) < 4) atomicMax(&wmax[term][j], __float_as_int(mx[term]));
+    }
   }
   __syncthreads();
   // exponent f with |w| 2^f < 2^30 (clamped: weights below 2^-90 of the scale do not matter)
-  auto fexp = [&](int term, int j) -> int {
-    const int bits = wmax[term][j];
+  auto fexp = [&](int term, int jj) -> int {
+    const int bits = wmax[term][jj];
     if (bits == 0) return 0;
     const int e = ((bits >> 23) & 255) - 126;   // |w| < 2^e
     return max(-90, min(110, 30 - e));
   };
-  for (int it = tid; it < npos * MAXQ; it += blockDim.x) {
-    const int pos = it >> 2, j = it & 3, term = pos < npos_mse ? 0 : 1, k = pos & 7;
-    int W = __float2int_rn(weight(pos, j) * pow2f(fexp(term, j) - k));
-    uint32_t packed = 0u;
+  {
+    const int fe[2] = {fexp(0, j), fexp(1, j)};
+    int sums[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+    for (int pos = tid >> 2; pos < npos; pos += blockDim.x / 4) {
+      const int term = pos < npos_mse ? 0 : 1, k = pos & 7;
+      int W = __float2int_rn(weight(pos, j) * pow2f(fe[term] - k));
+      uint32_t packed = 0u;
 #pragma unroll
-    for (int dg = 0; dg < 4; ++dg) {   // balanced radix-256 digits, the top one takes what is left
-      const int lo = dg == 3 ? W : ((W + 128) & 255) - 128;
-      W = (W - lo) >> 8;
-      packed |= (uint32_t)(lo & 255) << (8 * dg);
-      atomicAdd(&wdsum[term][j][dg], lo * (1 << k));
+      for (int dg = 0; dg < 4; ++dg) {   // balanced radix-256 digits, the top one takes what is left
+        const int lo = dg == 3 ? W : ((W + 128) & 255) - 128;
+        W = (W - lo) >> 8;
+        packed |= (uint32_t)(lo & 255) << (8 * dg);
+        if (term == 0) sums[0][dg] += lo * (1 << k); else sums[1][dg] += lo * (1 << k);
+      }
+      wdig[pos][j] = packed;
     }
-    wdig[pos][j] = packed;
+#pragma unroll
+    for (int term = 0; term < 2; ++term)
+#pragma unroll
+      for (int dg = 0; dg < 4; ++dg) {
+        int v = sums[term][dg];
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if ((tid & 31) < 4) atomicAdd(&wdsum[term][j][dg], v);
+      }
   }
   __syncthreads();
   // B fragments: word w, lane (n, kq): registers (tile 0, K half 0), (tile 0, half 1), (tile 1, half 0), (tile 1, half 1);
   // byte i of K half r: plane bit 32 w + 8 i + kq + 4 r; column n of tile tt: query n / 2, digit 2 tt + (n & 1)
   uint4* bf = ma.bfrag + ((size_t)h * ma.kw + m.k_w0) * 32;
   for (int it = tid; it < (npos >> 5) * 32; it += blockDim.x) {
-    const int w = it >> 5, lane = it & 31, n = lane >> 2, kq = lane & 3, j = n >> 1;
+    const int w = it >> 5, lane = it & 31, n = lane >> 2, kq = lane & 3, jq = n >> 1;
     uint32_t reg[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
     for (int r = 0; r < 2; ++r)
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint32_t pk = wdig[32 * w + 8 * i + kq + 4 * r][j] >> (8 * (n & 1));
+        const uint32_t pk = wdig[32 * w + 8 * i + kq + 4 * r][jq] >> (8 * (n & 1));
         reg[r] |= (pk & 255u) << (8 * i);
         reg[2 + r] |= ((pk >> 16) & 255u) << (8 * i);
       }
     bf[(size_t)w * 32 + lane] = make_uint4(reg[0], reg[1], reg[2], reg[3]);
   }
   if (tid < 2 * MAXQ) {
-    const int term = tid / MAXQ, j = tid % MAXQ;
+    const int term = tid / MAXQ, jc = tid % MAXQ;
     KConst c;
 #pragma unroll
-    for (int dg = 0; dg < 4; ++dg) c.wd[dg] = wdsum[term][j][dg];
-    c.scale = pow2f(-(fexp(term, j) + 1));
+    for (int dg = 0; dg < 4; ++dg) c.wd[dg] = wdsum[term][jc][dg];
+    c.scale = pow2f(-(fexp(term, jc) + 1));
     c.pad[0] = c.pad[1] = c.pad[2] = 0.f;
-    ma.kconst[((size_t)(h * a.ngroups + gi) * MAXQ + j) * 2 + term] = c;
+    ma.kconst[((size_t)(h * a.ngroups + gi) * MAXQ + jc) * 2 + term] = c;
   }
 }
 
@@ -307,40 +331,61 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
   asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
 
-  // ---- derived planes, defaults of absent scalars, largest value norm of the slice (thread = token)
-  for (int gi = 0; gi < ng; ++gi) {
-    const GroupDev& g = a.g[gi];
-    const MmaGroup& m = ma.m[gi];
-    float vm = 0.f;
-    if (tid < ntok) {
-      if (g.k_bits >= 3) derive_planes<1>(krow + tid * ma.kstride + m.k_w0, d, g.k_bits);
-      if (g.v_bits >= 3) derive_planes<4>(vmine + 4 * m.v_w0, d, g.v_bits);
-      if (!g.k_norms) knu[gi * SLICE + tid] = 1.f;
-      if (!g.k_prod) kgm[gi * SLICE + tid] = 0.f;
-      if (!g.v_norms) vnu[gi * SLICE + tid] = 1.f;
-      vm = vnu[gi * SLICE + tid];
-    }
+  // ---- thread = token: derived planes, defaults of absent scalars, largest value norm of the slice; then the value
+  //      planes are transposed in place: the four lanes of a token quad hold word w of their tokens and exchange
+  //      bytes, so that lane s ends with byte s of the four tokens and stores it where it read its own word
+  {
+    const uint32_t sel1 = (lane & 1) ? 0x3715u : 0x6240u, sel2 = (lane & 2) ? 0x3276u : 0x5410u;
+    auto transpose_store = [&](uint32_t* slot, uint32_t x) {
+      const uint32_t u = prmt_b(x, __shfl_xor_sync(0xffffffffu, x, 1), sel1);
+      *slot = prmt_b(u, __shfl_xor_sync(0xffffffffu, u, 2), sel2);
+    };
+    const bool live = tid < ntok;
+    for (int gi = 0; gi < ng; ++gi) {
+      const GroupDev& g = a.g[gi];
+      const MmaGroup& m = ma.m[gi];
+      float vm = 0.f;
+      if (live) {
+        if (g.k_bits >= 3) derive_planes<1>(krow + tid * ma.kstride + m.k_w0, d, g.k_bits);
+        if (!g.k_norms) knu[gi * SLICE + tid] = 1.f;
+        if (!g.k_prod) kgm[gi * SLICE + tid] = 0.f;
+        if (!g.v_norms) vnu[gi * SLICE + tid] = 1.f;
+        vm = fmaxf(vnu[gi * SLICE + tid], 0.f);
+      }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xffffffffu, vm, o));
-    if (lane == 0) atomicMax(&vmax[gi], __float_as_int(fmaxf(vm, 0.f)));
+      for (int o = 16; o > 0; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xffffffffu, vm, o));
+      if (lane == 0) atomicMax(&vmax[gi], __float_as_int(vm));
+      uint32_t* v0 = vmine + 4 * m.v_w0;
+      if (g.v_bits <= 2) {
+        for (int w = 0; w < m.v_raw_nw; ++w) transpose_store(v0 + 4 * w, live ? v0[4 * w] : 0u);
+      } else if (g.v_bits == 3) {
+        const int nw = m.v_raw_nw;
+        for (int j = 0; j < nw / 3; ++j) {
+          uint32_t x[4];
+#pragma unroll
+          for (int r = 0; r < 4; ++r) x[r] = (live && 3 * j + r < nw) ? v0[4 * (3 * j + r)] : 0u;
+          uint32_t z = 0u;
+#pragma unroll
+          for (int r = 0; r < 3; ++r) {
+            const uint32_t y = x[r] ^ __funnelshift_r(x[r], x[r + 1], 1) ^ __funnelshift_r(x[r], x[r + 1], 2);
+            z |= y & (0x49249249u << r);
+          }
+#pragma unroll
+          for (int r = 0; r < 3; ++r) transpose_store(v0 + 4 * (3 * j + r), x[r]);   // a lane reads and writes its own slot only
+          transpose_store(v0 + 4 * (nw + j), z);
+        }
+      } else {
+        const int nw = m.v_raw_nw;
+        for (int w = 0; w < nw; ++w) {
+          const uint32_t x = live ? v0[4 * w] : 0u;
+          const uint32_t t = (x ^ (x >> 1) ^ (x >> 2) ^ (x >> 3)) & 0x11111111u;
+          transpose_store(v0 + 4 * w, x);
+          transpose_store(v0 + 4 * (nw + w), x ^ (t * 15u));
+        }
+      }
+    }
   }
   __syncthreads();
-
-  // ---- value planes transposed in place: (quad, word) holds the word of the quad's four tokens; afterwards
-  //      register s = byte s of that word for the four tokens
-  {
-    uint4* vq4 = reinterpret_cast<uint4*>(vq);
-    const int wl = tid & 7;
-    for (int qd = tid >> 3; qd < SLICE / 4; qd += NT / 8)
-      for (int w = wl; w < ma.vw; w += 8) {
-        uint4* p = vq4 + qd * ma.qstride16 + w;
-        const uint4 x = *p;
-        const uint32_t lo01 = prmt_b(x.x, x.y, 0x5140u), lo23 = prmt_b(x.z, x.w, 0x5140u);
-        const uint32_t hi01 = prmt_b(x.x, x.y, 0x7362u), hi23 = prmt_b(x.z, x.w, 0x7362u);
-        *p = make_uint4(prmt_b(lo01, lo23, 0x5410u), prmt_b(lo01, lo23, 0x7632u), prmt_b(hi01, hi23, 0x5410u),
-                        prmt_b(hi01, hi23, 0x7632u));
-      }
-  }
 
   // ---- A) scores.  Thread (g8, kq) of a warp: tokens g8 and g8 + 8 of the warp's 16-token tile, query kq.
   constexpr int MT = SLICE / 16 / (NT / 32);   // tiles per warp
@@ -448,7 +493,7 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
   //         slice's tokens; columns of B: plane bits.  A unit = half a plane word (two 8-column tiles); the units of
   //         a group are dealt to the warps; warp gi % 8 also takes the group's column of ones (sum_t w).
   constexpr int CH = 3;   // units in flight per warp
-  const int nks = (ntok + 31) / 32;
+  constexpr int NKS = SLICE / 32;   // all of them: the weights of absent tokens are zero
   const uint32_t mn = 0x01010101u << g8;
   const uint4* vq4 = reinterpret_cast<const uint4*>(vq);
   for (int gi = 0; gi < ng; ++gi) {
@@ -466,7 +511,8 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
 #pragma unroll
           for (int e = 0; e < 4; ++e) acc[uu][tt][e] = 0;
       const bool with_ones = ones && u0 == ub;
-      for (int ks = 0; ks < nks; ++ks) {
+#pragma unroll
+      for (int ks = 0; ks < NKS; ++ks) {
         const unsigned char* wr = wr0 + 32 * ks;
         const uint32_t a0 = *reinterpret_cast<const uint32_t*>(wr), a1 = *reinterpret_cast<const uint32_t*>(wr + 8 * WT_STRIDE);
         const uint32_t a2 = *reinterpret_cast<const uint32_t*>(wr + 16), a3 = *reinterpret_cast<const uint32_t*>(wr + 8 * WT_STRIDE + 16);
@@ -510,29 +556,32 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
   //      2^(pos % 8)); Horner over the digits in fp32; the coordinate's plane bits added in a fixed order
   const int ncoord = ng * d;
   float* out = a.part_acc + (size_t)(h * a.nslices + sl) * ncoord * MAXQ;
-  for (int it = tid; it < ncoord * MAXQ; it += NT) {
-    const int oc = it >> 2, j = it & 3, gi = oc / d, c = oc - gi * d, bits = a.g[gi].v_bits;
+  for (int gi = 0; gi < ng; ++gi) {
     const MmaGroup& m = ma.m[gi];
-    const int* dj = dbuf + 4 * j * ma.dstride;
-    const int oc0 = ma.vpos + 8 * gi;
-    const int o0 = dj[oc0], o1 = dj[ma.dstride + oc0], o2 = dj[2 * ma.dstride + oc0];
-    auto plane = [&](int pos, float alpha) -> float {
-      const int col = m.v_pos0 + pos, sh = pos & 7;
-      const float e0 = (float)(2 * (dj[col] >> sh) - o0), e1 = (float)(2 * (dj[ma.dstride + col] >> sh) - o1);
-      const float e2 = (float)(2 * (dj[2 * ma.dstride + col] >> sh) - o2);
-      return alpha * fmaf(256.f, fmaf(256.f, e2, e1), e0);
-    };
-    float s = 0.f;
-    if (bits <= 2) {
-      for (int o = 0; o < bits; ++o) s += plane(bits * c + o, m.v_alpha[o]);
-    } else if (bits == 3) {
-      for (int o = 0; o < 3; ++o) s += plane(3 * c + o, m.v_alpha[o]);
-      const int sp = 3 * c;
-      s += plane(3 * d + 32 * ((sp >> 5) / 3) + (sp & 31), m.v_alpha[3]);
-    } else {
-      for (int o = 0; o < 4; ++o) s += plane(4 * c + o, m.v_alpha[o]);
-      for (int o = 0; o < 4; ++o) s += plane(4 * d + 4 * c + o, m.v_alpha[4 + o]);
+    const int bits = a.g[gi].v_bits, oc0 = ma.vpos + 8 * gi;
+    const float rs = 1.f / sg[gi];
+    for (int it = tid; it < d * MAXQ; it += NT) {
+      const int c = it >> 2, j = it & 3;
+      const int* dj = dbuf + 4 * j * ma.dstride;
+      const int o0 = dj[oc0], o1 = dj[ma.dstride + oc0], o2 = dj[2 * ma.dstride + oc0];
+      auto plane = [&](int pos, float alpha) -> float {
+        const int col = m.v_pos0 + pos, sh = pos & 7;
+        const float e0 = (float)(2 * (dj[col] >> sh) - o0), e1 = (float)(2 * (dj[ma.dstride + col] >> sh) - o1);
+        const float e2 = (float)(2 * (dj[2 * ma.dstride + col] >> sh) - o2);
+        return alpha * fmaf(256.f, fmaf(256.f, e2, e1), e0);
+      };
+      float s = 0.f;
+      if (bits <= 2) {
+        for (int o = 0; o < bits; ++o) s += plane(bits * c + o, m.v_alpha[o]);
+      } else if (bits == 3) {
+        for (int o = 0; o < 3; ++o) s += plane(3 * c + o, m.v_alpha[o]);
+        const int sp = 3 * c;
+        s += plane(3 * d + 32 * ((sp >> 5) / 3) + (sp & 31), m.v_alpha[3]);
+      } else {
+        for (int o = 0; o < 4; ++o) s += plane(4 * c + o, m.v_alpha[o]);
+        for (int o = 0; o < 4; ++o) s += plane(4 * d + 4 * c + o, m.v_alpha[4 + o]);
+      }
+      out[gi * d * MAXQ + it] = s * rs;
     }
-    out[it] = s / sg[gi];
   }
 }
