@@ -627,16 +627,16 @@ bool walsh_coefficients(const float* c, int bits, float* alpha) {
   return true;
 }
 
-int piece_bytes(const void* base, int row_stride, int row_bytes, int dst_off_bytes) {
-  const uintptr_t x = reinterpret_cast<uintptr_t>(base) | (uintptr_t)row_stride | (uintptr_t)row_bytes | (uintptr_t)dst_off_bytes;
-  return (x & 15) == 0 ? 16 : (x & 7) == 0 ? 8 : 4;
-}
-
 // Layout of the tensor path for this call; false if it cannot run (codebook shape, shared memory).
 bool plan_mma(int ngroups, int d, const Args& a, char* workspace, size_t off, int heads, MmaArgs* out, size_t* smem_out) {
   MmaArgs& ma = *out;
   std::memset(&ma, 0, sizeof(ma));
-  int kw = 0, vw = 0;
+  int kw = 0, vw = 0, r0 = 0;
+  auto take = [&](int bytes) {
+    const int at = r0;
+    r0 += (bytes + 15) / 16 * 16;
+    return at;
+  };
   for (int gi = 0; gi < ngroups; ++gi) {
     const GroupDev& g = a.g[gi];
     MmaGroup& m = ma.m[gi];
@@ -647,28 +647,33 @@ bool plan_mma(int ngroups, int d, const Args& a, char* workspace, size_t off, in
     m.k_qjl_nw = g.k_prod ? d / 32 : 0;
     if (g.k_bits > 0 && g.k_idx_rb < 4 * m.k_raw_nw) return false;
     if (g.k_prod && g.k_qjl_rb < 4 * m.k_qjl_nw) return false;
-    m.k_piece_idx = piece_bytes(g.k_idx, g.k_idx_rb, 4 * m.k_raw_nw, 4 * m.k_w0);
-    m.k_piece_qjl = piece_bytes(g.k_qjl, g.k_qjl_rb, 4 * m.k_qjl_nw, 4 * (m.k_w0 + m.k_mse_nw));
+    m.k_idx_rb = g.k_bits > 0 ? g.k_idx_rb : 0;
+    m.k_qjl_rb = g.k_prod ? g.k_qjl_rb : 0;
+    m.k_der_rb = 4 * (m.k_mse_nw - m.k_raw_nw);
+    m.k_idx_off = take(SLICE * m.k_idx_rb);
+    m.k_qjl_off = take(SLICE * m.k_qjl_rb);
+    m.k_der_off = take(SLICE * m.k_der_rb);
     kw += m.k_mse_nw + m.k_qjl_nw;
     m.v_w0 = vw;
     m.v_nw = plane_words(d, g.v_bits);
     m.v_raw_nw = raw_words(d, g.v_bits);
     if (g.v_idx_rb < 4 * m.v_raw_nw) return false;
+    m.v_rb = g.v_idx_rb;
+    m.v_raw_off = take(SLICE * m.v_rb);
     m.v_pos0 = 32 * vw;
     vw += m.v_nw;
   }
   if (kw == 0) return false;
-  int ks = (kw + 3) / 4 * 4;
-  if ((ks / 4) % 2 == 0) ks += 4;
-  ma.kw = kw; ma.kstride = ks;
+  ma.kw = kw;
   ma.vw = vw;
   ma.qstride16 = vw | 1;
   ma.vpos = 32 * vw;
   ma.dstride = (ma.vpos + 8 * ngroups + 31) / 32 * 32 + 8;
-  ma.region0 = (int)std::max<size_t>((size_t)4 * SLICE * ma.kstride + (size_t)16 * kw * 32 + (size_t)2 * ngroups * SLICE * 4,
-                                     (size_t)16 * ma.dstride * 4);
+  ma.bs_off = take(16 * kw * 32);
+  ma.knu_off = take(2 * ngroups * SLICE * 4);
+  ma.region0 = std::max(r0, WT_ROWS * ma.dstride * 4);
   ma.region0 = (ma.region0 + 15) / 16 * 16;
-  const size_t smem = (size_t)ma.region0 + (size_t)16 * (SLICE / 4) * ma.qstride16 + (size_t)ngroups * 16 * WT_STRIDE +
+  const size_t smem = (size_t)ma.region0 + (size_t)16 * (SLICE / 4) * ma.qstride16 + (size_t)ngroups * WT_ROWS * WT_STRIDE +
                       (size_t)ngroups * SLICE * 4 + (size_t)ngroups * MAXQ * 2 * sizeof(KConst) + 2 * (NT / 32) * MAXQ * 4 + MAXG * 4;
   if (smem > 200 * 1024) return false;
   if ((size_t)kw * 32 * sizeof(uint4) * heads > bfrag_bytes(ngroups, heads, d)) return false;

@@ -28,9 +28,12 @@
 //   merge_kernel         combines the slices.
 
 struct MmaGroup {
-  int k_w0, k_mse_nw, k_raw_nw, k_qjl_nw;   // K plane row: words [k_w0, +k_mse_nw) MSE planes (first k_raw_nw raw), then k_qjl_nw sign words
-  int v_w0, v_nw, v_raw_nw;                 // V plane row
-  int k_piece_idx, k_piece_qjl;             // bytes per cp.async piece (4, 8 or 16)
+  int k_w0;                                 // first B-fragment word (k-step) of the group: MSE planes, then sign words
+  int k_mse_nw, k_raw_nw, k_qjl_nw;         // words of the MSE planes (the first k_raw_nw are the index bits themselves), sign words
+  int k_idx_off, k_qjl_off, k_der_off;      // byte offsets in region 0: staged index rows, sign rows, derived plane words
+  int k_idx_rb, k_qjl_rb, k_der_rb;         // bytes per staged row / per token of derived words
+  int v_w0, v_nw, v_raw_nw;                 // words of the value planes in a token quad's row of the transposed planes
+  int v_raw_off, v_rb;                      // staged value rows
   int v_pos0;                               // first plane-bit position of the group among all V positions
   float k_alpha[8], v_alpha[8];             // Walsh coefficients: single bits o = 0..3, then (b = 3) the parity of all
                                             // three bits at [3], (b = 4) the parity of the bits other than o at [4 + o]
@@ -44,18 +47,40 @@ struct KConst {
 
 struct MmaArgs {
   MmaGroup m[MAXG];
-  int kw, kstride;        // words per K plane row, padded row stride (words, 4 * odd)
-  int vw;                 // words per V plane row
+  int kw;                 // B-fragment words of all groups
+  int vw;                 // words per token of the value planes
   int qstride16;          // 16-byte units between consecutive token quads of the value planes (odd, >= vw)
   int vpos;               // plane-bit positions of all groups' values = 32 * vw
   int dstride;            // ints between digit rows of the value sums (>= vpos + 8 * ngroups, = 8 mod 32)
+  int bs_off, knu_off;    // byte offsets in region 0 of the B fragments and of the key scalars (nu, then gamma)
   int region0;            // bytes of the region that holds what the scores need, later the value sums
   uint4* bfrag;           // [heads][kw][32]  B fragments of the scores
   KConst* kconst;         // [heads][ngroups][MAXQ][2]  constants of the MSE and sign terms
 };
 
 constexpr int WT_STRIDE = SLICE + 16;   // bytes between digit rows of the weights (bank-conflict-free fragment loads)
+constexpr int WT_ROWS = 12;             // rows 3 j + dg: three digits of four queries
 constexpr int MAXPW = 9 * (MAXD / 32);  // plane words of one group's keys: at most 8 per 32 coordinates + the sign word
+
+// shared-memory accesses by 32-bit address (the hot loops keep their address arithmetic in 32 bits)
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts64(uint32_t a, int x, int y) {
+  asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(a), "r"(x), "r"(y) : "memory");
+}
 
 __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
   asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -104,10 +129,9 @@ __device__ __forceinline__ void plane_pos(int d, int bits, int pos, const float*
   }
 }
 
-// Derived plane words of one code row (thread-local): word i of the row is row[i * STRIDE]; the raw words are followed
-// by room for the derived ones.
-template <int STRIDE>
-__device__ __forceinline__ void derive_planes(uint32_t* row, int d, int bits) {
+// Derived plane words of one code row: from its raw index words to `der` (3-bit indices: one parity word per three
+// raw words; 4-bit indices: one word of 3-subset parities per raw word).
+__device__ __forceinline__ void derive_planes(const uint32_t* raw, uint32_t* der, int d, int bits) {
   if (bits == 3) {
     const int nw = 3 * d / 32;
     for (int j = 0; j < nw / 3; ++j) {
@@ -115,18 +139,18 @@ __device__ __forceinline__ void derive_planes(uint32_t* row, int d, int bits) {
 #pragma unroll
       for (int r = 0; r < 3; ++r) {
         const int i = 3 * j + r;
-        const uint32_t x = row[i * STRIDE], nx = i + 1 < nw ? row[(i + 1) * STRIDE] : 0u;
+        const uint32_t x = raw[i], nx = i + 1 < nw ? raw[i + 1] : 0u;
         const uint32_t y = x ^ __funnelshift_r(x, nx, 1) ^ __funnelshift_r(x, nx, 2);
         z |= y & (0x49249249u << r);   // bits p with p % 3 == r
       }
-      row[(nw + j) * STRIDE] = z;
+      der[j] = z;
     }
   } else if (bits == 4) {
     const int nw = d / 8;
     for (int i = 0; i < nw; ++i) {
-      const uint32_t x = row[i * STRIDE];
+      const uint32_t x = raw[i];
       const uint32_t t = (x ^ (x >> 1) ^ (x >> 2) ^ (x >> 3)) & 0x11111111u;   // parity of each nibble
-      row[(nw + i) * STRIDE] = x ^ (t * 15u);                                  // bit o: parity of the other three bits
+      der[i] = x ^ (t * 15u);                                                  // bit o: parity of the other three bits
     }
   }
 }
@@ -259,39 +283,35 @@ __global__ void __launch_bounds__(256) prepare_mma_kernel(Args a, MmaArgs ma, co
 }
 
 // ------------------------------------------------------------------ per-slice scores, weights, value sums
-template <int BYTES>
-__device__ __forceinline__ void cp_async_piece(uint32_t dst, const void* src) {
-  if (BYTES == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-  else if (BYTES == 8) asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
-  else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
-}
-
-// The first `nb` bytes of this thread's code row to its plane row in shared memory, in pieces of `piece` bytes.
-__device__ __forceinline__ void stage_row(uint32_t dst, const unsigned char* src, int nb, int piece) {
-  if (piece == 16) {
-    for (int o = 0; o < nb; o += 16) cp_async_piece<16>(dst + o, src + o);
-  } else if (piece == 8) {
-    for (int o = 0; o < nb; o += 8) cp_async_piece<8>(dst + o, src + o);
-  } else {
-    for (int o = 0; o < nb; o += 4) cp_async_piece<4>(dst + o, src + o);
+// Scores of two 16-token tiles against `nw` plane words: rows r0 (tile 0, token g8), r0 + skip8 (token g8 + 8),
+// r1, r1 + skip8 (tile 1); bfr = this lane's B fragment of the first word, 512 bytes per word.
+__device__ __forceinline__ void score_words(int (&acc)[2][2][4], uint32_t r0, uint32_t r1, uint32_t skip8, int nw, uint32_t bfr,
+                                            uint32_t m0, uint32_t m1) {
+#pragma unroll 2
+  for (int w = 0; w < nw; ++w) {
+    const uint32_t x0 = lds32(r0 + 4 * w), x1 = lds32(r0 + skip8 + 4 * w);
+    const uint32_t y0 = lds32(r1 + 4 * w), y1 = lds32(r1 + skip8 + 4 * w);
+    const uint4 b = lds128(bfr + 512 * w);
+    mma_u8s8(acc[0][0], x0 & m0, x1 & m0, x0 & m1, x1 & m1, b.x, b.y);
+    mma_u8s8(acc[0][1], x0 & m0, x1 & m0, x0 & m1, x1 & m1, b.z, b.w);
+    mma_u8s8(acc[1][0], y0 & m0, y1 & m0, y0 & m1, y1 & m1, b.x, b.y);
+    mma_u8s8(acc[1][1], y0 & m0, y1 & m0, y0 & m1, y1 & m1, b.z, b.w);
   }
 }
 
-__global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
+__global__ void __launch_bounds__(NT, 4) partial_mma_kernel(Args a, MmaArgs ma) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int ng = a.ngroups, d = a.d;
-  // region 0: what the scores need (key planes, B fragments, key scalars); later the digit rows of the value sums
-  uint32_t* krow = reinterpret_cast<uint32_t*>(smem_raw);                        // [SLICE][kstride]
-  uint4* bs = reinterpret_cast<uint4*>(krow + SLICE * ma.kstride);               // [kw][32]
-  float* knu = reinterpret_cast<float*>(bs + ma.kw * 32);                        // [ng][SLICE]
+  // region 0: what the scores need (staged code rows, B fragments, key scalars); later the digit rows of the value sums
+  float* knu = reinterpret_cast<float*>(smem_raw + ma.knu_off);                  // [ng][SLICE]
   float* kgm = knu + ng * SLICE;                                                 // [ng][SLICE]
-  int* dbuf = reinterpret_cast<int*>(smem_raw);                                  // [16][dstride]
   uint32_t* vq = reinterpret_cast<uint32_t*>(smem_raw + ma.region0);             // [SLICE / 4][qstride16][4]
-  unsigned char* wt = reinterpret_cast<unsigned char*>(vq + (SLICE / 4) * ma.qstride16 * 4);   // [ng][16][WT_STRIDE]
-  float* vnu = reinterpret_cast<float*>(wt + ng * 16 * WT_STRIDE);               // [ng][SLICE]
+  unsigned char* wt = reinterpret_cast<unsigned char*>(vq + (SLICE / 4) * ma.qstride16 * 4);   // [ng][WT_ROWS][WT_STRIDE]
+  float* vnu = reinterpret_cast<float*>(wt + ng * WT_ROWS * WT_STRIDE);          // [ng][SLICE]
   KConst* kc = reinterpret_cast<KConst*>(vnu + ng * SLICE);                      // [ng][MAXQ][2]
   float* red = reinterpret_cast<float*>(kc + ng * MAXQ * 2);                     // [2][NT / 32][MAXQ]
   int* vmax = reinterpret_cast<int*>(red + 2 * (NT / 32) * MAXQ);                // [MAXG] bit patterns of max nu^V
+  const uint32_t s_base = (uint32_t)__cvta_generic_to_shared(smem_raw);
 
   const int h = blockIdx.x / a.nslices, sl = blockIdx.x % a.nslices;
   const int64_t t0 = (int64_t)sl * SLICE;
@@ -300,30 +320,26 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g8 = lane >> 2, kq = lane & 3;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  // ---- 0) thread = token: its code rows and scalars travel to shared memory (inputs of the call: before the
-  //         dependency wait).  Word w of the token's value planes goes to [token / 4][w][token % 4].
-  uint32_t* vmine = vq + (tid >> 2) * ma.qstride16 * 4 + (tid & 3);   // this token's word 0; words are 4 apart
-  if (tid < ntok) {
-    const int64_t row = row0 + tid;
-    const uint32_t kdst = (uint32_t)__cvta_generic_to_shared(krow + tid * ma.kstride);
-    const uint32_t vdst = (uint32_t)__cvta_generic_to_shared(vmine);
-    for (int gi = 0; gi < ng; ++gi) {
-      const GroupDev& g = a.g[gi];
-      const MmaGroup& m = ma.m[gi];
-      if (g.k_bits > 0) stage_row(kdst + 4 * m.k_w0, g.k_idx + (size_t)row * g.k_idx_rb, 4 * m.k_raw_nw, m.k_piece_idx);
-      if (g.k_prod) stage_row(kdst + 4 * (m.k_w0 + m.k_mse_nw), g.k_qjl + (size_t)row * g.k_qjl_rb, 4 * m.k_qjl_nw, m.k_piece_qjl);
-      const unsigned char* vsrc = g.v_idx + (size_t)row * g.v_idx_rb;
-      for (int w = 0; w < m.v_raw_nw; ++w) cp_async_piece<4>(vdst + 16 * (m.v_w0 + w), vsrc + 4 * w);
-      if (g.k_norms) cp_async_piece<4>((uint32_t)__cvta_generic_to_shared(knu + gi * SLICE + tid), g.k_norms + row);
-      if (g.k_prod) cp_async_piece<4>((uint32_t)__cvta_generic_to_shared(kgm + gi * SLICE + tid), g.k_gamma + row);
-      if (g.v_norms) cp_async_piece<4>((uint32_t)__cvta_generic_to_shared(vnu + gi * SLICE + tid), g.v_norms + row);
+  // ---- 0) the slice's code rows and scalars are contiguous in global memory: flat copies to shared memory (inputs of
+  //         the call: before the dependency wait)
+  for (int gi = 0; gi < ng; ++gi) {
+    const GroupDev& g = a.g[gi];
+    const MmaGroup& m = ma.m[gi];
+    if (g.k_bits > 0) stage_rows(smem_raw + m.k_idx_off, g.k_idx + (size_t)row0 * g.k_idx_rb, ntok * g.k_idx_rb);
+    if (g.k_prod) {
+      stage_rows(smem_raw + m.k_qjl_off, g.k_qjl + (size_t)row0 * g.k_qjl_rb, ntok * g.k_qjl_rb);
+      stage_rows(reinterpret_cast<unsigned char*>(kgm + gi * SLICE), reinterpret_cast<const unsigned char*>(g.k_gamma + row0), ntok * 4);
     }
+    stage_rows(smem_raw + m.v_raw_off, g.v_idx + (size_t)row0 * g.v_idx_rb, ntok * g.v_idx_rb);
+    if (g.k_norms) stage_rows(reinterpret_cast<unsigned char*>(knu + gi * SLICE), reinterpret_cast<const unsigned char*>(g.k_norms + row0), ntok * 4);
+    if (g.v_norms) stage_rows(reinterpret_cast<unsigned char*>(vnu + gi * SLICE), reinterpret_cast<const unsigned char*>(g.v_norms + row0), ntok * 4);
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
   if (tid < MAXG) vmax[tid] = 0;
   asm volatile("griddepcontrol.wait;" ::: "memory");   // the query-side operand is the previous kernel's output
   {
     const uint4* src = ma.bfrag + (size_t)h * ma.kw * 32;
+    uint4* bs = reinterpret_cast<uint4*>(smem_raw + ma.bs_off);
     for (int i = tid; i < ma.kw * 32; i += NT) bs[i] = __ldg(src + i);
     const uint4* cs = reinterpret_cast<const uint4*>(ma.kconst + (size_t)h * ng * MAXQ * 2);
     for (int i = tid; i < ng * MAXQ * 2 * 2; i += NT) reinterpret_cast<uint4*>(kc)[i] = __ldg(cs + i);
@@ -331,11 +347,12 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
   asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
 
-  // ---- thread = token: derived planes, defaults of absent scalars, largest value norm of the slice; then the value
-  //      planes are transposed in place: the four lanes of a token quad hold word w of their tokens and exchange
-  //      bytes, so that lane s ends with byte s of the four tokens and stores it where it read its own word
+  // ---- thread = token: derived planes, defaults of absent scalars, largest value norm of the slice; the value
+  //      planes go to [token quad][word][byte]: the four lanes of a quad hold word w of their tokens and exchange
+  //      bytes, so that lane s ends with byte s of the four tokens
   {
     const uint32_t sel1 = (lane & 1) ? 0x3715u : 0x6240u, sel2 = (lane & 2) ? 0x3276u : 0x5410u;
+    uint32_t* vslot = vq + (tid >> 2) * ma.qstride16 * 4 + (tid & 3);   // [quad][word 0][lane of the quad]; words are 4 apart
     auto transpose_store = [&](uint32_t* slot, uint32_t x) {
       const uint32_t u = prmt_b(x, __shfl_xor_sync(0xffffffffu, x, 1), sel1);
       *slot = prmt_b(u, __shfl_xor_sync(0xffffffffu, u, 2), sel2);
@@ -346,7 +363,9 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
       const MmaGroup& m = ma.m[gi];
       float vm = 0.f;
       if (live) {
-        if (g.k_bits >= 3) derive_planes<1>(krow + tid * ma.kstride + m.k_w0, d, g.k_bits);
+        if (g.k_bits >= 3)
+          derive_planes(reinterpret_cast<const uint32_t*>(smem_raw + m.k_idx_off + tid * m.k_idx_rb),
+                        reinterpret_cast<uint32_t*>(smem_raw + m.k_der_off + tid * m.k_der_rb), d, g.k_bits);
         if (!g.k_norms) knu[gi * SLICE + tid] = 1.f;
         if (!g.k_prod) kgm[gi * SLICE + tid] = 0.f;
         if (!g.v_norms) vnu[gi * SLICE + tid] = 1.f;
@@ -355,29 +374,28 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xffffffffu, vm, o));
       if (lane == 0) atomicMax(&vmax[gi], __float_as_int(vm));
-      uint32_t* v0 = vmine + 4 * m.v_w0;
+      const uint32_t* rv = reinterpret_cast<const uint32_t*>(smem_raw + m.v_raw_off + tid * m.v_rb);
+      uint32_t* v0 = vslot + 4 * m.v_w0;
+      const int nw = m.v_raw_nw;
       if (g.v_bits <= 2) {
-        for (int w = 0; w < m.v_raw_nw; ++w) transpose_store(v0 + 4 * w, live ? v0[4 * w] : 0u);
+        for (int w = 0; w < nw; ++w) transpose_store(v0 + 4 * w, live ? rv[w] : 0u);
       } else if (g.v_bits == 3) {
-        const int nw = m.v_raw_nw;
         for (int j = 0; j < nw / 3; ++j) {
           uint32_t x[4];
 #pragma unroll
-          for (int r = 0; r < 4; ++r) x[r] = (live && 3 * j + r < nw) ? v0[4 * (3 * j + r)] : 0u;
+          for (int r = 0; r < 4; ++r) x[r] = (live && 3 * j + r < nw) ? rv[3 * j + r] : 0u;
           uint32_t z = 0u;
 #pragma unroll
           for (int r = 0; r < 3; ++r) {
             const uint32_t y = x[r] ^ __funnelshift_r(x[r], x[r + 1], 1) ^ __funnelshift_r(x[r], x[r + 1], 2);
             z |= y & (0x49249249u << r);
+            transpose_store(v0 + 4 * (3 * j + r), x[r]);
           }
-#pragma unroll
-          for (int r = 0; r < 3; ++r) transpose_store(v0 + 4 * (3 * j + r), x[r]);   // a lane reads and writes its own slot only
           transpose_store(v0 + 4 * (nw + j), z);
         }
       } else {
-        const int nw = m.v_raw_nw;
         for (int w = 0; w < nw; ++w) {
-          const uint32_t x = live ? v0[4 * w] : 0u;
+          const uint32_t x = live ? rv[w] : 0u;
           const uint32_t t = (x ^ (x >> 1) ^ (x >> 2) ^ (x >> 3)) & 0x11111111u;
           transpose_store(v0 + 4 * w, x);
           transpose_store(v0 + 4 * (nw + w), x ^ (t * 15u));
@@ -387,48 +405,62 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
   }
   __syncthreads();
 
-  // ---- A) scores.  Thread (g8, kq) of a warp: tokens g8 and g8 + 8 of the warp's 16-token tile, query kq.
-  constexpr int MT = SLICE / 16 / (NT / 32);   // tiles per warp
+  // ---- A) scores.  Thread (g8, kq) of a warp: tokens g8 and g8 + 8 of the warp's two 16-token tiles, query kq.
+  constexpr int MT = SLICE / 16 / (NT / 32);
+  static_assert(MT == 2, "two tiles per warp");
   const uint32_t m0 = 0x01010101u << kq, m1 = m0 << 4;
+  const int tok0 = 16 * warp + g8, tok1 = 16 * (warp + NT / 32) + g8;   // rows g8 of the two tiles
   float logit[MT][2];
-#pragma unroll
-  for (int i = 0; i < MT; ++i) {
-    const int tb = 16 * (warp + (NT / 32) * i);
-    float score[2] = {0.f, 0.f};
+  {
+    float score[MT][2] = {{0.f, 0.f}, {0.f, 0.f}};
     for (int gi = 0; gi < ng; ++gi) {
       const MmaGroup& m = ma.m[gi];
-      const uint32_t* r0 = krow + (tb + g8) * ma.kstride + m.k_w0;
-      const uint32_t* r1 = r0 + 8 * ma.kstride;
-      const uint4* bb = bs + m.k_w0 * 32 + lane;
-      float term[2][2];   // [mse, sign][row]
+      const uint32_t bfr = s_base + ma.bs_off + (m.k_w0 * 32 + lane) * 16;
+      float term[2][MT][2];   // [mse, sign][tile][row]
 #pragma unroll
       for (int tm = 0; tm < 2; ++tm) {
-        const int w_lo = tm == 0 ? 0 : m.k_mse_nw, w_hi = tm == 0 ? m.k_mse_nw : m.k_mse_nw + m.k_qjl_nw;
-        int acc[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
-        for (int w = w_lo; w < w_hi; ++w) {
-          const uint32_t x0 = r0[w], x1 = r1[w];
-          const uint4 b = bb[w * 32];
-          mma_u8s8(acc[0], x0 & m0, x1 & m0, x0 & m1, x1 & m1, b.x, b.y);
-          mma_u8s8(acc[1], x0 & m0, x1 & m0, x0 & m1, x1 & m1, b.z, b.w);
+        int acc[MT][2][4];
+#pragma unroll
+        for (int i = 0; i < MT; ++i)
+#pragma unroll
+          for (int tt = 0; tt < 2; ++tt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[i][tt][e] = 0;
+        if (tm == 0) {
+          score_words(acc, s_base + m.k_idx_off + tok0 * m.k_idx_rb, s_base + m.k_idx_off + tok1 * m.k_idx_rb, 8 * m.k_idx_rb,
+                      m.k_raw_nw, bfr, m0, m1);
+          if (m.k_mse_nw > m.k_raw_nw)
+            score_words(acc, s_base + m.k_der_off + tok0 * m.k_der_rb, s_base + m.k_der_off + tok1 * m.k_der_rb, 8 * m.k_der_rb,
+                        m.k_mse_nw - m.k_raw_nw, bfr + 512 * m.k_raw_nw, m0, m1);
+        } else {
+          score_words(acc, s_base + m.k_qjl_off + tok0 * m.k_qjl_rb, s_base + m.k_qjl_off + tok1 * m.k_qjl_rb, 8 * m.k_qjl_rb,
+                      m.k_qjl_nw, bfr + 512 * m.k_mse_nw, m0, m1);
         }
         // sum_pos W (2 bit - 1), digit by digit (each difference is a small exact integer), then Horner in fp32
         const KConst c = kc[(gi * MAXQ + kq) * 2 + tm];
 #pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-          const float d0 = (float)(2 * acc[0][2 * hh] - c.wd[0]), d1 = (float)(2 * acc[0][2 * hh + 1] - c.wd[1]);
-          const float d2 = (float)(2 * acc[1][2 * hh] - c.wd[2]), d3 = (float)(2 * acc[1][2 * hh + 1] - c.wd[3]);
-          term[tm][hh] = fmaf(256.f, fmaf(256.f, fmaf(256.f, d3, d2), d1), d0) * c.scale;
-        }
+        for (int i = 0; i < MT; ++i)
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            const float d0 = (float)(2 * acc[i][0][2 * hh] - c.wd[0]), d1 = (float)(2 * acc[i][0][2 * hh + 1] - c.wd[1]);
+            const float d2 = (float)(2 * acc[i][1][2 * hh] - c.wd[2]), d3 = (float)(2 * acc[i][1][2 * hh + 1] - c.wd[3]);
+            term[tm][i][hh] = fmaf(256.f, fmaf(256.f, fmaf(256.f, d3, d2), d1), d0) * c.scale;
+          }
       }
       const float coef = a.g[gi].coef;
 #pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        const int t = tb + g8 + 8 * hh;
-        score[hh] += knu[gi * SLICE + t] * fmaf(coef * kgm[gi * SLICE + t], term[1][hh], term[0][hh]);
-      }
+      for (int i = 0; i < MT; ++i)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          const int t = (i == 0 ? tok0 : tok1) + 8 * hh;
+          score[i][hh] += knu[gi * SLICE + t] * fmaf(coef * kgm[gi * SLICE + t], term[1][i][hh], term[0][i][hh]);
+        }
     }
-    logit[i][0] = a.scale * score[0];
-    logit[i][1] = a.scale * score[1];
+#pragma unroll
+    for (int i = 0; i < MT; ++i) {
+      logit[i][0] = a.scale * score[i][0];
+      logit[i][1] = a.scale * score[i][1];
+    }
   }
 
   // ---- B) slice maximum per query, exponentials, their sum (fixed order), weight digits (three per weight)
@@ -438,7 +470,7 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
     for (int i = 0; i < MT; ++i)
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh)
-        if (16 * (warp + (NT / 32) * i) + g8 + 8 * hh < ntok) mx = fmaxf(mx, logit[i][hh]);
+        if ((i == 0 ? tok0 : tok1) + 8 * hh < ntok) mx = fmaxf(mx, logit[i][hh]);
 #pragma unroll
     for (int o = 4; o < 32; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if (g8 == 0) red[warp * MAXQ + kq] = mx;
@@ -459,7 +491,7 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
     for (int i = 0; i < MT; ++i)
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh) {
-        const int t = 16 * (warp + (NT / 32) * i) + g8 + 8 * hh;
+        const int t = (i == 0 ? tok0 : tok1) + 8 * hh;
         const bool live = t < ntok && kq < a.qpk;
         const float p = live ? expf(logit[i][hh] - smax) : 0.f;
         psum += p;
@@ -467,7 +499,7 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
         for (int gi = 0; gi < MAXG; ++gi)
           if (gi < ng) {
             const uint32_t W = live ? min(__float2uint_rn(p * vnu[gi * SLICE + t] * sg[gi]), 0xffffffu) : 0u;
-            unsigned char* col = wt + (gi * 16 + 4 * kq) * WT_STRIDE + t;
+            unsigned char* col = wt + (gi * WT_ROWS + 3 * kq) * WT_STRIDE + t;
             col[0] = (unsigned char)W;
             col[WT_STRIDE] = (unsigned char)(W >> 8);
             col[2 * WT_STRIDE] = (unsigned char)(W >> 16);
@@ -489,71 +521,73 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
     ml[MAXQ + tid] = s;
   }
 
-  // ---- C) value sums.  Rows of A: weight digit dg of query j at row 4 j + dg (row 4 j + 3 is not used); K = the
-  //         slice's tokens; columns of B: plane bits.  A unit = half a plane word (two 8-column tiles); the units of
-  //         a group are dealt to the warps; warp gi % 8 also takes the group's column of ones (sum_t w).
-  constexpr int CH = 3;   // units in flight per warp
-  constexpr int NKS = SLICE / 32;   // all of them: the weights of absent tokens are zero
+  // ---- C) value sums.  Rows of A: weight digit dg of query j at row 3 j + dg (rows 12..15 of the tile carry nothing);
+  //         K = the slice's tokens (all eight k-steps: the weights of absent tokens are zero); columns of B: plane bits.
+  //         A unit = half a plane word (two 8-column tiles); the units of a group are dealt to the warps; warp gi % 8
+  //         also takes the group's column of ones (sum_t w).
+  constexpr int CH = 3;              // units in flight per warp
+  constexpr int NKS = SLICE / 32;
   const uint32_t mn = 0x01010101u << g8;
-  const uint4* vq4 = reinterpret_cast<const uint4*>(vq);
+  const uint32_t qrow = 16u * ma.qstride16;                          // bytes per token quad
+  const uint32_t vq_s = (uint32_t)__cvta_generic_to_shared(vq) + kq * qrow;
+  const uint32_t wt_s = (uint32_t)__cvta_generic_to_shared(wt) + 4 * kq;
+  const int row_hi = min(g8 + 8, WT_ROWS - 1);                       // rows 12..15: any row, the results are not stored
+  const uint32_t db_s = s_base + (g8 * ma.dstride + 2 * kq) * 4;     // digit row g8, columns 2 kq, 2 kq + 1
   for (int gi = 0; gi < ng; ++gi) {
     const MmaGroup& m = ma.m[gi];
     const int U = 2 * m.v_nw;
     const int ub = U * warp / (NT / 32), ue = U * (warp + 1) / (NT / 32);
-    const unsigned char* wr0 = wt + (gi * 16 + g8) * WT_STRIDE + 4 * kq;
+    const uint32_t wa_lo = wt_s + (gi * WT_ROWS + g8) * WT_STRIDE, wa_hi = wt_s + (gi * WT_ROWS + row_hi) * WT_STRIDE;
     const bool ones = warp == (gi & (NT / 32 - 1));
     for (int u0 = ub; u0 < ue || (ones && u0 == ub); u0 += CH) {
       int acc[CH][2][4], acc1[4] = {0, 0, 0, 0};
+      uint32_t boff[CH];
 #pragma unroll
-      for (int uu = 0; uu < CH; ++uu)
+      for (int uu = 0; uu < CH; ++uu) {
+        boff[uu] = vq_s + (m.v_w0 + ((u0 + uu) >> 1)) * 16 + ((u0 + uu) & 1) * 8;
 #pragma unroll
         for (int tt = 0; tt < 2; ++tt)
 #pragma unroll
           for (int e = 0; e < 4; ++e) acc[uu][tt][e] = 0;
+      }
       const bool with_ones = ones && u0 == ub;
 #pragma unroll
       for (int ks = 0; ks < NKS; ++ks) {
-        const unsigned char* wr = wr0 + 32 * ks;
-        const uint32_t a0 = *reinterpret_cast<const uint32_t*>(wr), a1 = *reinterpret_cast<const uint32_t*>(wr + 8 * WT_STRIDE);
-        const uint32_t a2 = *reinterpret_cast<const uint32_t*>(wr + 16), a3 = *reinterpret_cast<const uint32_t*>(wr + 8 * WT_STRIDE + 16);
-        const uint4* q0 = vq4 + (8 * ks + kq) * ma.qstride16 + m.v_w0;
-        const uint4* q1 = q0 + 4 * ma.qstride16;
+        const uint32_t a0 = lds32(wa_lo + 32 * ks), a1 = lds32(wa_hi + 32 * ks);
+        const uint32_t a2 = lds32(wa_lo + 32 * ks + 16), a3 = lds32(wa_hi + 32 * ks + 16);
         if (with_ones) mma_u8u8(acc1, a0, a1, a2, a3, 0x01010101u, 0x01010101u);
 #pragma unroll
-        for (int uu = 0; uu < CH; ++uu) {
-          const int u = u0 + uu;
-          if (u < ue) {
-            const uint2 b0 = reinterpret_cast<const uint2*>(q0 + (u >> 1))[u & 1];
-            const uint2 b1 = reinterpret_cast<const uint2*>(q1 + (u >> 1))[u & 1];
+        for (int uu = 0; uu < CH; ++uu)
+          if (u0 + uu < ue) {
+            const uint2 b0 = lds64(boff[uu] + (8 * ks) * qrow), b1 = lds64(boff[uu] + (8 * ks + 4) * qrow);
             mma_u8u8(acc[uu][0], a0, a1, a2, a3, b0.x & mn, b1.x & mn);
             mma_u8u8(acc[uu][1], a0, a1, a2, a3, b0.y & mn, b1.y & mn);
           }
-        }
       }
-      // digit rows g8 and g8 + 8, columns 2 kq and 2 kq + 1 of each tile
+      // digit rows g8 and (for g8 < 4) g8 + 8, columns 2 kq and 2 kq + 1 of each tile
       if (with_ones) {
-        int* dd = dbuf + g8 * ma.dstride + ma.vpos + 8 * gi + 2 * kq;
-        *reinterpret_cast<int2*>(dd) = make_int2(acc1[0], acc1[1]);
-        *reinterpret_cast<int2*>(dd + 8 * ma.dstride) = make_int2(acc1[2], acc1[3]);
+        const uint32_t dd = db_s + (ma.vpos + 8 * gi) * 4;
+        sts64(dd, acc1[0], acc1[1]);
+        if (g8 < 4) sts64(dd + 32 * ma.dstride, acc1[2], acc1[3]);
       }
 #pragma unroll
-      for (int uu = 0; uu < CH; ++uu) {
-        const int u = u0 + uu;
-        if (u < ue) {
+      for (int uu = 0; uu < CH; ++uu)
+        if (u0 + uu < ue) {
+          const int u = u0 + uu;
 #pragma unroll
           for (int tt = 0; tt < 2; ++tt) {
-            int* dd = dbuf + g8 * ma.dstride + m.v_pos0 + 32 * (u >> 1) + 8 * (2 * (u & 1) + tt) + 2 * kq;
-            *reinterpret_cast<int2*>(dd) = make_int2(acc[uu][tt][0], acc[uu][tt][1]);
-            *reinterpret_cast<int2*>(dd + 8 * ma.dstride) = make_int2(acc[uu][tt][2], acc[uu][tt][3]);
+            const uint32_t dd = db_s + (m.v_pos0 + 32 * (u >> 1) + 8 * (2 * (u & 1) + tt)) * 4;
+            sts64(dd, acc[uu][tt][0], acc[uu][tt][1]);
+            if (g8 < 4) sts64(dd + 32 * ma.dstride, acc[uu][tt][2], acc[uu][tt][3]);
           }
         }
-      }
     }
   }
   __syncthreads();
 
   // ---- item = (coordinate, query): per digit 2 X - sum_t w is a small exact integer (column pos carries the factor
   //      2^(pos % 8)); Horner over the digits in fp32; the coordinate's plane bits added in a fixed order
+  const int* dbuf = reinterpret_cast<const int*>(smem_raw);   // [WT_ROWS][dstride]
   const int ncoord = ng * d;
   float* out = a.part_acc + (size_t)(h * a.nslices + sl) * ncoord * MAXQ;
   for (int gi = 0; gi < ng; ++gi) {
@@ -562,7 +596,7 @@ __global__ void __launch_bounds__(NT) partial_mma_kernel(Args a, MmaArgs ma) {
     const float rs = 1.f / sg[gi];
     for (int it = tid; it < d * MAXQ; it += NT) {
       const int c = it >> 2, j = it & 3;
-      const int* dj = dbuf + 4 * j * ma.dstride;
+      const int* dj = dbuf + 3 * j * ma.dstride;
       const int o0 = dj[oc0], o1 = dj[ma.dstride + oc0], o2 = dj[2 * ma.dstride + oc0];
       auto plane = [&](int pos, float alpha) -> float {
         const int col = m.v_pos0 + pos, sh = pos & 7;
