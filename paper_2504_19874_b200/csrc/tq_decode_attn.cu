@@ -671,8 +671,27 @@ bool plan_mma(int ngroups, int d, const Args& a, char* workspace, size_t off, in
   ma.dstride = (ma.vpos + 8 * ngroups + 31) / 32 * 32 + 8;
   ma.bs_off = take(16 * kw * 32);
   ma.knu_off = take(2 * ngroups * SLICE * 4);
+  const int vnu_off_rel = 16 * (SLICE / 4) * ma.qstride16 + ngroups * WT_ROWS * WT_STRIDE;   // behind region 0
   ma.region0 = std::max(r0, WT_ROWS * ma.dstride * 4);
   ma.region0 = (ma.region0 + 15) / 16 * 16;
+  for (int gi = 0; gi < ngroups; ++gi) {   // the copies of the slice's rows and scalars
+    const GroupDev& g = a.g[gi];
+    const MmaGroup& m = ma.m[gi];
+    auto add = [&](const void* src, int rb, int dst_off) {
+      CopyJob& j = ma.job[ma.njobs++];
+      j.src = static_cast<const unsigned char*>(src);
+      j.row_bytes = rb;
+      j.dst_off = dst_off;
+    };
+    add(g.v_idx, g.v_idx_rb, m.v_raw_off);
+    if (g.k_bits > 0) add(g.k_idx, g.k_idx_rb, m.k_idx_off);
+    if (g.k_prod) {
+      add(g.k_qjl, g.k_qjl_rb, m.k_qjl_off);
+      add(g.k_gamma, 4, ma.knu_off + (ngroups + gi) * SLICE * 4);
+    }
+    if (g.k_norms) add(g.k_norms, 4, ma.knu_off + gi * SLICE * 4);
+    if (g.v_norms) add(g.v_norms, 4, ma.region0 + vnu_off_rel + gi * SLICE * 4);
+  }
   const size_t smem = (size_t)ma.region0 + (size_t)16 * (SLICE / 4) * ma.qstride16 + (size_t)ngroups * WT_ROWS * WT_STRIDE +
                       (size_t)ngroups * SLICE * 4 + (size_t)ngroups * MAXQ * 2 * sizeof(KConst) + 2 * (NT / 32) * MAXQ * 4 + MAXG * 4;
   if (smem > 200 * 1024) return false;

@@ -45,8 +45,16 @@ struct KConst {
   float pad[3];
 };
 
+struct CopyJob {
+  const unsigned char* src;   // first row of head 0
+  int row_bytes;              // bytes per token in global memory
+  int dst_off;                // byte offset in shared memory
+};
+
 struct MmaArgs {
   MmaGroup m[MAXG];
+  CopyJob job[6 * MAXG];  // the slice's code rows and per-token scalars: one contiguous run of global memory each
+  int njobs;
   int kw;                 // B-fragment words of all groups
   int vw;                 // words per token of the value planes
   int qstride16;          // 16-byte units between consecutive token quads of the value planes (odd, >= vw)
@@ -283,6 +291,12 @@ __global__ void __launch_bounds__(256) prepare_mma_kernel(Args a, MmaArgs ma, co
 }
 
 // ------------------------------------------------------------------ per-slice scores, weights, value sums
+template <int BYTES>
+__device__ __forceinline__ void cp_async_piece(uint32_t dst, const void* src) {
+  if (BYTES == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+  else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+
 // Scores of two 16-token tiles against `nw` plane words: rows r0 (tile 0, token g8), r0 + skip8 (token g8 + 8),
 // r1, r1 + skip8 (tile 1); bfr = this lane's B fragment of the first word, 512 bytes per word.
 __device__ __forceinline__ void score_words(int (&acc)[2][2][4], uint32_t r0, uint32_t r1, uint32_t skip8, int nw, uint32_t bfr,
@@ -320,19 +334,19 @@ __global__ void __launch_bounds__(NT, 4) partial_mma_kernel(Args a, MmaArgs ma) 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g8 = lane >> 2, kq = lane & 3;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  // ---- 0) the slice's code rows and scalars are contiguous in global memory: flat copies to shared memory (inputs of
-  //         the call: before the dependency wait)
-  for (int gi = 0; gi < ng; ++gi) {
-    const GroupDev& g = a.g[gi];
-    const MmaGroup& m = ma.m[gi];
-    if (g.k_bits > 0) stage_rows(smem_raw + m.k_idx_off, g.k_idx + (size_t)row0 * g.k_idx_rb, ntok * g.k_idx_rb);
-    if (g.k_prod) {
-      stage_rows(smem_raw + m.k_qjl_off, g.k_qjl + (size_t)row0 * g.k_qjl_rb, ntok * g.k_qjl_rb);
-      stage_rows(reinterpret_cast<unsigned char*>(kgm + gi * SLICE), reinterpret_cast<const unsigned char*>(g.k_gamma + row0), ntok * 4);
+  // ---- 0) the slice's code rows and scalars are contiguous in global memory: one flat copy each, dealt to the warps
+  //         (inputs of the call: before the dependency wait)
+  for (int jb = warp; jb < ma.njobs; jb += NT / 32) {
+    const CopyJob job = ma.job[jb];
+    const unsigned char* src = job.src + (size_t)row0 * job.row_bytes;
+    const uint32_t dst = s_base + job.dst_off;
+    const int bytes = ntok * job.row_bytes;
+    int done = 0;
+    if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+      done = bytes & ~15;
+      for (int i = lane * 16; i < done; i += 32 * 16) cp_async_piece<16>(dst + i, src + i);
     }
-    stage_rows(smem_raw + m.v_raw_off, g.v_idx + (size_t)row0 * g.v_idx_rb, ntok * g.v_idx_rb);
-    if (g.k_norms) stage_rows(reinterpret_cast<unsigned char*>(knu + gi * SLICE), reinterpret_cast<const unsigned char*>(g.k_norms + row0), ntok * 4);
-    if (g.v_norms) stage_rows(reinterpret_cast<unsigned char*>(vnu + gi * SLICE), reinterpret_cast<const unsigned char*>(g.v_norms + row0), ntok * 4);
+    for (int i = done + lane * 4; i < bytes; i += 32 * 4) cp_async_piece<4>(dst + i, src + i);
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
   if (tid < MAXG) vmax[tid] = 0;
@@ -528,7 +542,7 @@ __global__ void __launch_bounds__(NT, 4) partial_mma_kernel(Args a, MmaArgs ma) 
   constexpr int CH = 3;              // units in flight per warp
   constexpr int NKS = SLICE / 32;
   const uint32_t mn = 0x01010101u << g8;
-  const uint32_t qrow = 16u * ma.qstride16;                          // bytes per token quad
+  const uint32_t qrow = 16u * ma.qstride16, qrow4 = 4 * qrow, qrow8 = 8 * qrow;   // bytes per token quad
   const uint32_t vq_s = (uint32_t)__cvta_generic_to_shared(vq) + kq * qrow;
   const uint32_t wt_s = (uint32_t)__cvta_generic_to_shared(wt) + 4 * kq;
   const int row_hi = min(g8 + 8, WT_ROWS - 1);                       // rows 12..15: any row, the results are not stored
@@ -544,7 +558,7 @@ __global__ void __launch_bounds__(NT, 4) partial_mma_kernel(Args a, MmaArgs ma) 
       uint32_t boff[CH];
 #pragma unroll
       for (int uu = 0; uu < CH; ++uu) {
-        boff[uu] = vq_s + (m.v_w0 + ((u0 + uu) >> 1)) * 16 + ((u0 + uu) & 1) * 8;
+        boff[uu] = vq_s + (m.v_w0 + ((u0 + uu) >> 1)) * 16 + ((u0 + uu) & 1) * 8;   // advanced by 8 token quads per k-step
 #pragma unroll
         for (int tt = 0; tt < 2; ++tt)
 #pragma unroll
@@ -559,7 +573,8 @@ __global__ void __launch_bounds__(NT, 4) partial_mma_kernel(Args a, MmaArgs ma) 
 #pragma unroll
         for (int uu = 0; uu < CH; ++uu)
           if (u0 + uu < ue) {
-            const uint2 b0 = lds64(boff[uu] + (8 * ks) * qrow), b1 = lds64(boff[uu] + (8 * ks + 4) * qrow);
+            const uint2 b0 = lds64(boff[uu]), b1 = lds64(boff[uu] + qrow4);
+            boff[uu] += qrow8;
             mma_u8u8(acc[uu][0], a0, a1, a2, a3, b0.x & mn, b1.x & mn);
             mma_u8u8(acc[uu][1], a0, a1, a2, a3, b0.y & mn, b1.y & mn);
           }
