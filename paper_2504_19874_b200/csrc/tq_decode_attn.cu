@@ -397,6 +397,7 @@ __global__ void __launch_bounds__(MERGE_NT) merge_kernel(Args a, float* __restri
   const int h = blockIdx.x / a.ngroups, gi = blockIdx.x % a.ngroups;
   const int ncoord = a.ngroups * a.d, d = a.d, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const GroupDev& g = a.g[gi];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   {
     const float4* src = reinterpret_cast<const float4*>(g.v_pi);
     float4* dst = reinterpret_cast<float4*>(pis);
@@ -829,11 +830,14 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   MmaArgs ma;
   size_t mma_smem = 0;
   if (plan_mma(ngroups, d, a, static_cast<char*>(workspace), off, heads, &ma, &mma_smem)) {
+    // all three launches may be scheduled while their predecessor in the stream drains; each orders itself with
+    // griddepcontrol.wait before it reads or writes global memory that another kernel touches
     if (q_dtype == TQ_F32)
-      prepare_mma_kernel<float><<<heads * ngroups, 256, 0, st>>>(a, ma, static_cast<const float*>(Q), ldq);
+      TQ_CHECK_CUDA(launch_after(prepare_mma_kernel<float>, dim3((unsigned)(heads * ngroups)), dim3(256), 0, st, a, ma,
+                                 static_cast<const float*>(Q), ldq), who);
     else
-      prepare_mma_kernel<__nv_bfloat16><<<heads * ngroups, 256, 0, st>>>(a, ma, static_cast<const __nv_bfloat16*>(Q), ldq);
-    TQ_CHECK_CUDA(cudaGetLastError(), who);
+      TQ_CHECK_CUDA(launch_after(prepare_mma_kernel<__nv_bfloat16>, dim3((unsigned)(heads * ngroups)), dim3(256), 0, st, a, ma,
+                                 static_cast<const __nv_bfloat16*>(Q), ldq), who);
     static std::atomic<size_t> mma_smem_set[16];
     if (dev >= 16 || mma_smem > mma_smem_set[dev].load(std::memory_order_relaxed)) {
       TQ_CHECK_CUDA(cudaFuncSetAttribute(partial_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_smem), who);
@@ -841,7 +845,6 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
       TQ_CHECK_CUDA(cudaFuncSetAttribute(partial_mma_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared), who);
       if (dev < 16) mma_smem_set[dev].store(mma_smem, std::memory_order_relaxed);
     }
-    // both successors may be scheduled while their predecessor drains; each orders itself with griddepcontrol.wait
     TQ_CHECK_CUDA(launch_after(partial_mma_kernel, dim3((unsigned)(heads * nslices)), dim3(NT), mma_smem, st, a, ma), who);
     TQ_CHECK_CUDA(launch_after(merge_kernel, dim3((unsigned)(heads * ngroups)), dim3(MERGE_NT), merge_smem, st, a, out, ldo), who);
     count_launches(3);

@@ -176,6 +176,8 @@ __global__ void __launch_bounds__(256) prepare_mma_kernel(Args a, MmaArgs ma, co
   const MmaGroup& m = ma.m[gi];
   const int d = a.d, tid = threadIdx.x;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the slices' code rows may start to travel
+  // this kernel may itself have been scheduled while the kernel ahead in the stream drains (it may produce Q)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   for (int e = tid; e < MAXQ * d; e += blockDim.x) {
     const int j = e / d, c = e % d;
     float v = 0.f;
@@ -311,6 +313,45 @@ __device__ __forceinline__ void score_words(int (&acc)[2][2][4], uint32_t r0, ui
     mma_u8s8(acc[1][0], y0 & m0, y1 & m0, y0 & m1, y1 & m1, b.x, b.y);
     mma_u8s8(acc[1][1], y0 & m0, y1 & m0, y0 & m1, y1 & m1, b.z, b.w);
   }
+}
+
+// Value sums of N units (half plane words) of one group over all k-steps of the slice; digit rows to shared memory.
+// wa_lo / wa_hi: this lane's weight rows g8 and g8 + 8 (K offset 4 kq applied); b0[u]: this lane's first token quad of
+// unit u; dd[u]: where the unit's first tile goes in digit row g8 (columns 2 kq, 2 kq + 1).
+template <int N>
+__device__ __forceinline__ void vsum_chunk(uint32_t wa_lo, uint32_t wa_hi, const uint32_t (&b0)[3], const uint32_t (&dd)[3],
+                                           uint32_t qrow4, uint32_t mn, bool hi_rows, uint32_t hi_skip, bool with_ones, uint32_t dd_ones) {
+  constexpr int NKS = SLICE / 32;
+  int acc[N > 0 ? N : 1][2][4], acc1[4] = {0, 0, 0, 0};
+#pragma unroll
+  for (int u = 0; u < N; ++u)
+#pragma unroll
+    for (int tt = 0; tt < 2; ++tt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[u][tt][e] = 0;
+#pragma unroll
+  for (int ks = 0; ks < NKS; ++ks) {
+    const uint32_t a0 = lds32(wa_lo + 32 * ks), a1 = lds32(wa_hi + 32 * ks);
+    const uint32_t a2 = lds32(wa_lo + 32 * ks + 16), a3 = lds32(wa_hi + 32 * ks + 16);
+    if (with_ones) mma_u8u8(acc1, a0, a1, a2, a3, 0x01010101u, 0x01010101u);
+#pragma unroll
+    for (int u = 0; u < N; ++u) {
+      const uint2 x0 = lds64(b0[u] + 2 * ks * qrow4), x1 = lds64(b0[u] + (2 * ks + 1) * qrow4);
+      mma_u8u8(acc[u][0], a0, a1, a2, a3, x0.x & mn, x1.x & mn);
+      mma_u8u8(acc[u][1], a0, a1, a2, a3, x0.y & mn, x1.y & mn);
+    }
+  }
+  if (with_ones) {
+    sts64(dd_ones, acc1[0], acc1[1]);
+    if (hi_rows) sts64(dd_ones + hi_skip, acc1[2], acc1[3]);
+  }
+#pragma unroll
+  for (int u = 0; u < N; ++u)
+#pragma unroll
+    for (int tt = 0; tt < 2; ++tt) {
+      sts64(dd[u] + 32 * tt, acc[u][tt][0], acc[u][tt][1]);
+      if (hi_rows) sts64(dd[u] + 32 * tt + hi_skip, acc[u][tt][2], acc[u][tt][3]);
+    }
 }
 
 __global__ void __launch_bounds__(NT, 4) partial_mma_kernel(Args a, MmaArgs ma) {
@@ -539,10 +580,8 @@ __global__ void __launch_bounds__(NT, 4) partial_mma_kernel(Args a, MmaArgs ma) 
   //         K = the slice's tokens (all eight k-steps: the weights of absent tokens are zero); columns of B: plane bits.
   //         A unit = half a plane word (two 8-column tiles); the units of a group are dealt to the warps; warp gi % 8
   //         also takes the group's column of ones (sum_t w).
-  constexpr int CH = 3;              // units in flight per warp
-  constexpr int NKS = SLICE / 32;
   const uint32_t mn = 0x01010101u << g8;
-  const uint32_t qrow = 16u * ma.qstride16, qrow4 = 4 * qrow, qrow8 = 8 * qrow;   // bytes per token quad
+  const uint32_t qrow = 16u * ma.qstride16;                          // bytes per token quad
   const uint32_t vq_s = (uint32_t)__cvta_generic_to_shared(vq) + kq * qrow;
   const uint32_t wt_s = (uint32_t)__cvta_generic_to_shared(wt) + 4 * kq;
   const int row_hi = min(g8 + 8, WT_ROWS - 1);                       // rows 12..15: any row, the results are not stored
@@ -553,49 +592,21 @@ __global__ void __launch_bounds__(NT, 4) partial_mma_kernel(Args a, MmaArgs ma) 
     const int ub = U * warp / (NT / 32), ue = U * (warp + 1) / (NT / 32);
     const uint32_t wa_lo = wt_s + (gi * WT_ROWS + g8) * WT_STRIDE, wa_hi = wt_s + (gi * WT_ROWS + row_hi) * WT_STRIDE;
     const bool ones = warp == (gi & (NT / 32 - 1));
-    for (int u0 = ub; u0 < ue || (ones && u0 == ub); u0 += CH) {
-      int acc[CH][2][4], acc1[4] = {0, 0, 0, 0};
-      uint32_t boff[CH];
+    for (int u0 = ub; u0 < ue || (ones && u0 == ub); u0 += 3) {
+      uint32_t b0[3], dd[3];
 #pragma unroll
-      for (int uu = 0; uu < CH; ++uu) {
-        boff[uu] = vq_s + (m.v_w0 + ((u0 + uu) >> 1)) * 16 + ((u0 + uu) & 1) * 8;   // advanced by 8 token quads per k-step
-#pragma unroll
-        for (int tt = 0; tt < 2; ++tt)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) acc[uu][tt][e] = 0;
+      for (int uu = 0; uu < 3; ++uu) {
+        const int u = u0 + uu;
+        b0[uu] = vq_s + (m.v_w0 + (u >> 1)) * 16 + (u & 1) * 8;
+        dd[uu] = db_s + (m.v_pos0 + 16 * u) * 4;
       }
       const bool with_ones = ones && u0 == ub;
-#pragma unroll
-      for (int ks = 0; ks < NKS; ++ks) {
-        const uint32_t a0 = lds32(wa_lo + 32 * ks), a1 = lds32(wa_hi + 32 * ks);
-        const uint32_t a2 = lds32(wa_lo + 32 * ks + 16), a3 = lds32(wa_hi + 32 * ks + 16);
-        if (with_ones) mma_u8u8(acc1, a0, a1, a2, a3, 0x01010101u, 0x01010101u);
-#pragma unroll
-        for (int uu = 0; uu < CH; ++uu)
-          if (u0 + uu < ue) {
-            const uint2 b0 = lds64(boff[uu]), b1 = lds64(boff[uu] + qrow4);
-            boff[uu] += qrow8;
-            mma_u8u8(acc[uu][0], a0, a1, a2, a3, b0.x & mn, b1.x & mn);
-            mma_u8u8(acc[uu][1], a0, a1, a2, a3, b0.y & mn, b1.y & mn);
-          }
-      }
-      // digit rows g8 and (for g8 < 4) g8 + 8, columns 2 kq and 2 kq + 1 of each tile
-      if (with_ones) {
-        const uint32_t dd = db_s + (ma.vpos + 8 * gi) * 4;
-        sts64(dd, acc1[0], acc1[1]);
-        if (g8 < 4) sts64(dd + 32 * ma.dstride, acc1[2], acc1[3]);
-      }
-#pragma unroll
-      for (int uu = 0; uu < CH; ++uu)
-        if (u0 + uu < ue) {
-          const int u = u0 + uu;
-#pragma unroll
-          for (int tt = 0; tt < 2; ++tt) {
-            const uint32_t dd = db_s + (m.v_pos0 + 32 * (u >> 1) + 8 * (2 * (u & 1) + tt)) * 4;
-            sts64(dd, acc[uu][tt][0], acc[uu][tt][1]);
-            if (g8 < 4) sts64(dd + 32 * ma.dstride, acc[uu][tt][2], acc[uu][tt][3]);
-          }
-        }
+      const uint32_t dd_ones = db_s + (ma.vpos + 8 * gi) * 4;
+      const int n = min(3, ue - u0);
+      if (n == 3) vsum_chunk<3>(wa_lo, wa_hi, b0, dd, 4 * qrow, mn, g8 < 4, 32 * ma.dstride, with_ones, dd_ones);
+      else if (n == 2) vsum_chunk<2>(wa_lo, wa_hi, b0, dd, 4 * qrow, mn, g8 < 4, 32 * ma.dstride, with_ones, dd_ones);
+      else if (n == 1) vsum_chunk<1>(wa_lo, wa_hi, b0, dd, 4 * qrow, mn, g8 < 4, 32 * ma.dstride, with_ones, dd_ones);
+      else vsum_chunk<0>(wa_lo, wa_hi, b0, dd, 4 * qrow, mn, g8 < 4, 32 * ma.dstride, with_ones, dd_ones);
     }
   }
   __syncthreads();
