@@ -1,7 +1,10 @@
-// Decode attention over a compressed KV cache in two launches (plus a small query-preparation
-// launch): scores of the Section 3.2 estimator on the packed K codes, softmax over the tokens, and
-// the weighted sum of the dequantised V vectors taken in the code domain (Section 4.3 use of the
-// quantisers), for all KV heads and channel groups of a layer at once.
+// Decode attention over a compressed KV cache in three launches: scores of the Section 3.2 estimator on the packed K
+// codes, softmax over the tokens, and the weighted sum of the dequantised V vectors taken in the code domain
+// (Section 4.3 use of the quantisers), for all KV heads and channel groups of a layer at once.
+//
+// Two sets of kernels.  Antisymmetric codebooks (every Lloyd-Max codebook of the even coordinate density) take the
+// integer tensor path of tq_decode_mma.cuh: prepare_mma_kernel, partial_mma_kernel.  Any other codebook takes the
+// table-lookup kernels of this file:
 //
 //   prepare_kernel   per (head, group): gathers the group's channels of the head's queries and forms
 //                    q' = Pi q, q'' = S q.
@@ -14,12 +17,14 @@
 //                    B) slice maximum, p = exp(logit - max), sum of p.
 //                    C) thread = output coordinate: acc[c] = sum_t p_t nu^V_t c_V[idx^V_{t,c}], walked
 //                       in a fixed order, so results do not depend on timing.
-//   merge_kernel     per (head, query): combines the slices (max / sum rescaling), divides by the sum and
+//
+// Both are followed by
+//   merge_kernel     per (head, group): combines the slices (max / sum rescaling), divides by the sum and
 //                    applies x~ = Pi_V^T y' per group, scattering to the group's channels.
 //
-// Work per token is ~50 warp instructions, i.e. CUDA-core bound at roughly 10x the time the code
-// bytes take from HBM; the unfused path (tq_score, tq_softmax, tq_wsum per head and group) is two
-// orders of magnitude slower at 32k tokens because each of its 88 launches serves one head.
+// The table-lookup kernel spends ~120 warp instructions per token and head on CUDA cores; the unfused path (tq_score,
+// tq_softmax, tq_wsum per head and group) is two orders of magnitude slower at 32k tokens because each of its 88
+// launches serves one head.
 #include <atomic>
 #include <algorithm>
 #include <cfloat>

@@ -27,13 +27,13 @@ RTOL = 1e-4
 class Setup:
     """Oracle-made global parameters (Pi, S, fp32 codebook) and the matching GPU plan."""
 
-    def __init__(self, d, bits, mode, pi_seed=42, s_seed=43, layout=None):
+    def __init__(self, d, bits, mode, pi_seed=42, s_seed=43, layout=None, centroids=None):
         self.d, self.bits, self.mode = d, bits, mode
         self.layout = layout
         self.mse_bits = bits - 1 if mode == tq.TQ_PROD else bits
         self.Pi = orc.rotation(d, pi_seed).astype(np.float32)
         self.S = orc.projection(d, s_seed).astype(np.float32) if mode == tq.TQ_PROD else None
-        self.c = orc.codebook(d, self.mse_bits).astype(np.float32)
+        self.c = (orc.codebook(d, self.mse_bits) if centroids is None else np.asarray(centroids)).astype(np.float32)
         self.t = (0.5 * (self.c[:-1].astype(np.float64) + self.c[1:].astype(np.float64)))
         self.plan = tq.Plan(d, bits, mode, self.Pi, self.S, self.c)
         if layout is not None:

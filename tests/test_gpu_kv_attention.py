@@ -206,6 +206,31 @@ def test_fused_decode_against_the_oracle(groups, heads, T, qpk):
     assert float(err.max()) <= S5_TOL, float(err.max())
 
 
+def test_fused_decode_with_codebooks_that_are_not_antisymmetric():
+    """The tensor-core kernels expand an antisymmetric codebook over the index bits; any other codebook (the API
+    accepts what the caller passes) takes the table-lookup kernel.  Same check against the oracle."""
+    def skewed(bits):
+        c = orc.codebook(GROUP, bits).copy()
+        c[0] *= 1.05
+        c[-1] *= 0.97
+        return c
+    gK = (P.Setup(GROUP, 3, tq.TQ_PROD, 72, 73, centroids=skewed(2)), P.Setup(GROUP, 2, tq.TQ_PROD, 74, 75, centroids=skewed(1)))
+    gV = (P.Setup(GROUP, 3, tq.TQ_MSE, 76, 77, centroids=skewed(3)), P.Setup(GROUP, 2, tq.TQ_MSE, 78, 79, centroids=skewed(2)))
+    heads, T, qpk = 2, 1300, 4
+    K, V, Q = wl.kv_cache(heads=heads, tokens=T, q_per_kv=qpk, seed=17, device=DEV)
+    recs, refs = [], []
+    for h in range(heads):
+        Qh = Q[qpk * h:qpk * h + qpk]
+        _, _, rec = attend_gpu(gK, gV, K[h], V[h], Qh)
+        recs.append(rec)
+        refs.append(attend_oracle(rec, Qh)[0])
+    ref = np.concatenate(refs)
+    fused = P.as_f64(_fused_layer(gK, gV, recs, Q, heads, T, qpk))
+    err = np.linalg.norm(fused - ref, axis=1) / np.linalg.norm(ref, axis=1)
+    print(f"S5 measured: fused (table-lookup kernel) vs oracle: {float(err.max()):.3e}")
+    assert float(err.max()) <= S5_TOL, float(err.max())
+
+
 def test_fused_decode_other_bit_widths_and_argument_checks():
     # one group of 128 channels: keys TurboQuant_mse 4-bit (no QJL part), values 4-bit; then keys prod 4-bit (3-bit indices)
     for kbits, kmode, vbits in ((4, tq.TQ_MSE, 4), (4, tq.TQ_PROD, 1), (1, tq.TQ_PROD, 2), (2, tq.TQ_MSE, 3)):
