@@ -375,8 +375,9 @@ __global__ void __launch_bounds__(NT, 4) partial_mma_kernel(Args a, MmaArgs ma) 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g8 = lane >> 2, kq = lane & 3;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  // ---- 0) the slice's code rows and scalars are contiguous in global memory: one flat copy each, dealt to the warps
-  //         (inputs of the call: before the dependency wait)
+  // ---- 0) the slice's code rows and scalars are contiguous in global memory: one flat copy each, dealt to the warps.
+  //         They are inputs of the call; the wait for the kernel ahead (the query-side operand) comes only after the
+  //         value planes are in place, so that the first wave of CTAs works while that kernel runs.
   for (int jb = warp; jb < ma.njobs; jb += NT / 32) {
     const CopyJob job = ma.job[jb];
     const unsigned char* src = job.src + (size_t)row0 * job.row_bytes;
@@ -391,14 +392,6 @@ __global__ void __launch_bounds__(NT, 4) partial_mma_kernel(Args a, MmaArgs ma) 
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
   if (tid < MAXG) vmax[tid] = 0;
-  asm volatile("griddepcontrol.wait;" ::: "memory");   // the query-side operand is the previous kernel's output
-  {
-    const uint4* src = ma.bfrag + (size_t)h * ma.kw * 32;
-    uint4* bs = reinterpret_cast<uint4*>(smem_raw + ma.bs_off);
-    for (int i = tid; i < ma.kw * 32; i += NT) bs[i] = __ldg(src + i);
-    const uint4* cs = reinterpret_cast<const uint4*>(ma.kconst + (size_t)h * ng * MAXQ * 2);
-    for (int i = tid; i < ng * MAXQ * 2 * 2; i += NT) reinterpret_cast<uint4*>(kc)[i] = __ldg(cs + i);
-  }
   asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
 
@@ -457,6 +450,14 @@ __global__ void __launch_bounds__(NT, 4) partial_mma_kernel(Args a, MmaArgs ma) 
         }
       }
     }
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // the query-side operand is the previous kernel's output
+  {
+    const uint4* src = ma.bfrag + (size_t)h * ma.kw * 32;
+    uint4* bs = reinterpret_cast<uint4*>(smem_raw + ma.bs_off);
+    for (int i = tid; i < ma.kw * 32; i += NT) bs[i] = __ldg(src + i);
+    const uint4* cs = reinterpret_cast<const uint4*>(ma.kconst + (size_t)h * ng * MAXQ * 2);
+    for (int i = tid; i < ng * MAXQ * 2 * 2; i += NT) reinterpret_cast<uint4*>(kc)[i] = __ldg(cs + i);
   }
   __syncthreads();
 
