@@ -206,6 +206,66 @@ def test_fused_decode_against_the_oracle(groups, heads, T, qpk):
     assert float(err.max()) <= S5_TOL, float(err.max())
 
 
+@pytest.mark.parametrize("d,specs,unit_norm", [
+    (32, [(4, tq.TQ_PROD, 4), (3, tq.TQ_MSE, 1), (1, tq.TQ_PROD, 2), (2, tq.TQ_PROD, 3)], False),   # four groups of 32 channels
+    (96, [(3, tq.TQ_PROD, 3)], False),                                                                # one group of 96
+    (64, [(4, tq.TQ_PROD, 4), (3, tq.TQ_PROD, 3)], False),                                            # the 3.5-bit split
+    (64, [(3, tq.TQ_PROD, 3), (2, tq.TQ_PROD, 2)], True),                                             # rows of unit norm, no norm arrays
+])
+def test_fused_decode_group_shapes(d, specs, unit_norm):
+    """Group counts, group widths, bit widths and quantiser kinds other than the configuration's, fp32 queries,
+    a head stride larger than the token count and a ragged last slice.  specs: (key bits, key quantiser, value bits)."""
+    ng, heads, T, qpk, cap = len(specs), 3, 777, 3, 801
+    hd = ng * d
+    gK = [P.Setup(d, kb, km, 90 + 2 * i, 91 + 2 * i) for i, (kb, km, vb) in enumerate(specs)]
+    gV = [P.Setup(d, vb, tq.TQ_MSE, 70 + 2 * i, 71 + 2 * i) for i, (kb, km, vb) in enumerate(specs)]
+    g = torch.Generator(device="cpu").manual_seed(1000 + d + ng)
+    K = torch.randn((heads, T, hd), generator=g).to(DEV)
+    V = torch.randn((heads, T, hd), generator=g).to(DEV)
+    Q = torch.randn((heads * qpk, hd), generator=g).to(DEV)
+    perm = [torch.randperm(hd, generator=g).to(DEV) for _ in range(heads)]      # arbitrary channel lists
+    gds, Khat, Vhat = [], np.zeros((heads, T, hd)), np.zeros((heads, T, hd))
+    for gi in range(ng):
+        suk, suv = gK[gi], gV[gi]
+        gd = {"plan_k": suk.plan, "plan_v": suv.plan,
+              "k_idx": torch.zeros((heads * cap, max(suk.idx_rb, 1)), dtype=torch.uint8, device=DEV),
+              "k_qjl": torch.zeros((heads * cap, suk.qjl_rb), dtype=torch.uint8, device=DEV) if suk.mode == tq.TQ_PROD else None,
+              "k_gamma": torch.zeros(heads * cap, device=DEV) if suk.mode == tq.TQ_PROD else None,
+              "k_norms": None if unit_norm else torch.zeros(heads * cap, device=DEV),
+              "v_idx": torch.zeros((heads * cap, suv.idx_rb), dtype=torch.uint8, device=DEV),
+              "v_norms": None if unit_norm else torch.zeros(heads * cap, device=DEV),
+              "k_channels": torch.stack([perm[h][gi * d:(gi + 1) * d] for h in range(heads)]).to(torch.int32).contiguous(),
+              "v_channels": torch.stack([perm[h][gi * d:(gi + 1) * d] for h in range(heads)]).to(torch.int32).contiguous()}
+        if suk.mse_bits == 0:
+            gd["k_idx"] = None
+        for h in range(heads):
+            ch = perm[h][gi * d:(gi + 1) * d]
+            Xk, Xv = K[h][:, ch].contiguous(), V[h][:, ch].contiguous()
+            if unit_norm:
+                Xk, Xv = Xk / Xk.norm(dim=1, keepdim=True), Xv / Xv.norm(dim=1, keepdim=True)
+            ck, cv = suk.quantize(Xk, with_norms=not unit_norm), suv.quantize(Xv, with_norms=not unit_norm)
+            r = slice(h * cap, h * cap + T)
+            if gd["k_idx"] is not None:
+                gd["k_idx"][r] = ck[0]
+            if suk.mode == tq.TQ_PROD:
+                gd["k_qjl"][r], gd["k_gamma"][r] = ck[1], ck[2]
+            gd["v_idx"][r] = cv[0]
+            if not unit_norm:
+                gd["k_norms"][r], gd["v_norms"][r] = ck[3], cv[3]
+            Khat[h][:, ch.cpu().numpy()] = P.oracle_dequant(suk, *ck)
+            Vhat[h][:, ch.cpu().numpy()] = P.oracle_dequant(suv, *cv)
+        gds.append(gd)
+    ws = torch.empty(tq.tq_attend_decode_workspace_bytes(ng, heads, T, d), dtype=torch.uint8, device=DEV)
+    out = torch.full((heads * qpk, hd), float("nan"), device=DEV)
+    scale = 1.0 / math.sqrt(hd)
+    tq.tq_attend_decode(gds, heads, T, qpk, Q, scale, out, ws, head_stride=cap)
+    torch.cuda.synchronize()
+    ref = np.concatenate([orc.attend(orc.score(P.as_f64(Q[qpk * h:qpk * h + qpk]), Khat[h]), Vhat[h], scale) for h in range(heads)])
+    err = np.linalg.norm(P.as_f64(out) - ref, axis=1) / np.linalg.norm(ref, axis=1)
+    print(f"S5 measured: fused vs oracle d={d} groups={specs} unit_norm={unit_norm}: {float(err.max()):.3e}")
+    assert float(err.max()) <= S5_TOL, float(err.max())
+
+
 def test_fused_decode_with_codebooks_that_are_not_antisymmetric():
     """The tensor-core kernels expand an antisymmetric codebook over the index bits; any other codebook (the API
     accepts what the caller passes) takes the table-lookup kernel.  Same check against the oracle."""
