@@ -621,7 +621,11 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
   // launch (its A operand is the residual, the limbs of X are free by then), one set of limb buffers.  TQ_MSE: the
   // rotate launch itself, so the scratch is used as two half-size sets written and read in turn (when the data
   // spans more than one block and each half still holds a tile).
-  const bool pingpong = !prod && n > R / 2 / BM * BM && R / 2 >= BM;
+  // Two warps per CTA keep up only while the GEMM gives them time: its work per row grows with d^2, theirs with d.
+  // Measured per 10^6 rows: d = 1536 gains 4 % (TQ_PROD) and 11 % (TQ_MSE), d = 3072 2 %; at d = 1024 the spare warps
+  // already lose (12.3 against 11.3 ms, TQ_MSE 6.9 against 5.6), at d = 200 they are the critical path (2.9 against 1.9 ms).
+  const bool overlap = d >= 1536;
+  const bool pingpong = overlap && !prod && n > R / 2 / BM * BM && R / 2 >= BM;
   const int64_t Rbuf = R;   // rows the carved buffers hold in all
   if (pingpong) R = R / 2 / BM * BM;
   // carve the scratch (every part is a multiple of 256 bytes because Rbuf is a multiple of 128)
@@ -664,7 +668,7 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     float* nu_out = norms ? norms + r0 : nullptr;
     // 1. nu, u = x / nu, bf16 limbs of u: by a launch of its own for the first block (and for TQ_MSE plans), by the
     //    spare warps of the previous block's project launch otherwise
-    if (r0 == 0 || (!prod && !pingpong)) TQ_CHECK_CUDA(launch_split(r0, st), who);
+    if (r0 == 0 || !overlap || (!prod && !pingpong)) TQ_CHECK_CUDA(launch_split(r0, st), who);
     __nv_bfloat16 *XLc1 = limbs1(r0 / R), *XLc2 = limbs2(r0 / R);
     auto next_block_task = [&](GemmArgs& ga) {
       ga.split.X = static_cast<const char*>(X) + (size_t)(r0 + R) * ldx * xsz;
@@ -721,7 +725,7 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
                "%s: cuTensorMapEncodeTiled failed", who);
     g.out = qjl + (size_t)r0 * plan->qjl_row_bytes;
     g.out_rb = plan->qjl_row_bytes;
-    if (r0 + R < n) next_block_task(g);   // the limbs of X are free by now
+    if (overlap && r0 + R < n) next_block_task(g);   // the limbs of X are free by now
     TQ_CHECK_CUDA(launch_gemm<2>(bn, 1, mE1, mE2, plan->sp_limbs.map_hi, plan->sp_limbs.map_lo, g, st), who);
   }
   return TQ_OK;
