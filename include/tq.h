@@ -336,7 +336,7 @@ typedef struct tq_kv_group {
   const int32_t* v_channels;  /* [heads, d] column of out that receives coordinate c of this group */
 } tq_kv_group;
 
-/* Bytes of workspace tq_attend_decode needs (rotated queries + per-slice partial results). */
+/* Bytes of workspace tq_attend_decode needs (query-side operands + per-slice partial results). */
 size_t tq_attend_decode_workspace_bytes(int ngroups, int heads, int64_t tokens, int d);
 
 /*   groups     host array of ngroups (1..TQ_MAX_KV_GROUPS) descriptors
@@ -345,6 +345,12 @@ size_t tq_attend_decode_workspace_bytes(int ngroups, int heads, int64_t tokens, 
  *   out        device fp32, [heads*q_per_kv rows, row stride ldo]; only the columns named by v_channels are written
  *   workspace  device, 256-byte aligned, >= tq_attend_decode_workspace_bytes(...)
  * tokens == 0 writes zeros to those columns.  Results do not depend on timing (fixed reduction orders).
+ * Three launches: query preparation, one CTA per (head, slice of 256 tokens), merge of the slices.  Codebooks that are
+ * antisymmetric (c[i] = -c[last - i], as every codebook of tq_codebook is) run on the integer tensor path (scores of
+ * the Section 3.2 estimator and the value sums as bit-plane MMAs with exact int32 accumulation); any other codebook
+ * runs on table-lookup CUDA-core kernels with the same results up to fp32 rounding.  The launches are programmatic
+ * dependents: the first may be scheduled while the kernel ahead of it in the stream drains and waits for it before
+ * it reads Q, so ordering against earlier work in the stream is what it would be for plain launches.
  * Errors: TQ_ERR_INVALID_ARG / _UNSUPPORTED / _ALIGNMENT / _WORKSPACE / _CUDA as for the other calls.
  */
 int tq_attend_decode(const tq_kv_group* groups, int ngroups, int heads, int64_t tokens, int64_t head_stride, int q_per_kv,
