@@ -50,6 +50,8 @@ struct MatrixLimbs {
   __nv_bfloat16* lo;
   alignas(64) CUtensorMap map_hi;
   alignas(64) CUtensorMap map_lo;
+  alignas(64) CUtensorMap map_hi_half;   // boxes of half as many rows: what one CTA of a pair loads
+  alignas(64) CUtensorMap map_lo_half;
 };
 
 }  // namespace tq

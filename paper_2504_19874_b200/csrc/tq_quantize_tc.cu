@@ -8,6 +8,7 @@
 // ~1e-7 on a rotated coordinate of a unit vector at d = 1536 -- far inside the 1e-5 window in
 // which a nearest-centroid decision may legitimately differ from exact arithmetic.
 #include <atomic>
+#include <cstdlib>
 #include <algorithm>
 #include <mutex>
 
@@ -26,10 +27,15 @@ constexpr int EPS = 4;           // epilogue warps per TMEM lane group: each tak
 constexpr int NSPLIT = 2;        // warps that prepare the next block's operand limbs beside the GEMM (see SplitTask)
 constexpr int NTHREADS = 32 * (2 + 4 * EPS + NSPLIT);   // warp 0: TMA, warp 1: MMA + TMEM owner, the epilogue warps, the split warps
 
-template <int BN>
+// CTAS = 2: two CTAs of a cluster share one 256-row tile (tcgen05 cta_group::2).  Each loads its own 128 rows of A and
+// its own half of B's rows, so a k-block costs each SM 64 KB of shared-memory writes instead of 96 and its MMAs read
+// half of B from the partner: the shared-memory bandwidth that caps the one-CTA kernel (158 bytes per clock wanted,
+// 128 available) drops to 104.
+template <int BN, int CTAS>
 struct Cfg {
-  static constexpr int kStageBytes = 2 * BM * BK * 2 + 2 * BN * BK * 2;   // A hi/lo + B hi/lo
-  static constexpr int kStages = (BN == 256) ? 2 : (BN == 128 ? 3 : 4);
+  static constexpr int kBRows = BN / CTAS;                                  // rows of B this CTA loads
+  static constexpr int kStageBytes = 2 * BM * BK * 2 + 2 * kBRows * BK * 2; // A hi/lo + B hi/lo
+  static constexpr int kStages = CTAS == 2 ? 3 : ((BN == 256) ? 2 : (BN == 128 ? 3 : 4));
   static constexpr int kTmemCols = 2 * BN;                                  // two accumulators
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
@@ -185,11 +191,13 @@ __global__ void __launch_bounds__(256) split_rows_kernel(const T* __restrict__ X
 }
 
 // MODE 0: idx.  MODE 1: idx + residual limbs + partial ||e||^2.  MODE 2: sign bits.
-template <int BN, int MODE, int BITS>
+template <int BN, int MODE, int BITS, int CTAS>
 __global__ void __launch_bounds__(NTHREADS, 1)
 quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2,
                      const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmArgs a) {
-  using C = Cfg<BN>;
+  using C = Cfg<BN, CTAS>;
+  const int rank = CTAS == 2 ? (int)cluster_ctarank() : 0;   // CTA of the pair; rank 0 issues the MMAs
+  const int64_t unit = blockIdx.x / CTAS, nunits = gridDim.x / CTAS;   // a unit = one CTA or one pair
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kStages * C::kStageBytes);
@@ -211,7 +219,7 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&tfull[i], 1);
-      mbar_init(&tempty[i], 4 * EPS);
+      mbar_init(&tempty[i], 4 * EPS * CTAS);   // the leader's: the epilogue warps of both CTAs arrive
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -220,9 +228,13 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
     tma_prefetch_desc(&tmB1);
     tma_prefetch_desc(&tmB2);
   }
-  if (warp == 1) tmem_alloc(tmem_slot, C::kTmemCols);
+  if (warp == 1) {
+    if (CTAS == 2) tmem_alloc_pair(tmem_slot, C::kTmemCols);
+    else tmem_alloc(tmem_slot, C::kTmemCols);
+  }
   tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) cluster_sync();   // the partner's barriers exist before anything arrives on them
+  else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -232,16 +244,25 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        const int m0 = (int)(t / a.tiles_n) * BM, n0 = (int)(t % a.tiles_n) * BN;
+      for (int64_t t = unit; t < num_tiles && ok; t += nunits) {
+        const int m0 = ((int)(t / a.tiles_n) * CTAS + rank) * BM, n0 = (int)(t % a.tiles_n) * BN + rank * C::kBRows;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!(ok = mbar_wait(&empty[stage], phase ^ 1u, abort_flag, a.status))) break;
           unsigned char* sa = smem + stage * C::kStageBytes;
-          mbar_arrive_expect_tx(&full[stage], C::kStageBytes);
-          tma_load_2d(sa, &tmA1, &full[stage], kb * BK, m0);
-          tma_load_2d(sa + BM * BK * 2, &tmA2, &full[stage], kb * BK, m0);
-          tma_load_2d(sa + 2 * BM * BK * 2, &tmB1, &full[stage], kb * BK, n0);
-          tma_load_2d(sa + 2 * BM * BK * 2 + BN * BK * 2, &tmB2, &full[stage], kb * BK, n0);
+          if (CTAS == 2) {
+            // both CTAs' bytes are counted on the leader's barrier, which the leader arms for both
+            if (rank == 0) mbar_arrive_expect_tx(&full[stage], 2 * C::kStageBytes);
+            tma_load_2d_pair(sa, &tmA1, &full[stage], kb * BK, m0);
+            tma_load_2d_pair(sa + BM * BK * 2, &tmA2, &full[stage], kb * BK, m0);
+            tma_load_2d_pair(sa + 2 * BM * BK * 2, &tmB1, &full[stage], kb * BK, n0);
+            tma_load_2d_pair(sa + 2 * BM * BK * 2 + C::kBRows * BK * 2, &tmB2, &full[stage], kb * BK, n0);
+          } else {
+            mbar_arrive_expect_tx(&full[stage], C::kStageBytes);
+            tma_load_2d(sa, &tmA1, &full[stage], kb * BK, m0);
+            tma_load_2d(sa + BM * BK * 2, &tmA2, &full[stage], kb * BK, m0);
+            tma_load_2d(sa + 2 * BM * BK * 2, &tmB1, &full[stage], kb * BK, n0);
+            tma_load_2d(sa + 2 * BM * BK * 2 + BN * BK * 2, &tmB2, &full[stage], kb * BK, n0);
+          }
           if (++stage == C::kStages) {
             stage = 0;
             phase ^= 1u;
@@ -256,13 +277,13 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc_bf16(BM, BN);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = instr_desc_bf16(BM * CTAS, BN);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       int64_t it = 0;
-      for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+      for (int64_t t = unit; t < num_tiles && ok; t += nunits, ++it) {
         const uint32_t acc = (uint32_t)(it & 1), acc_phase = (uint32_t)((it >> 1) & 1);
         if (!(ok = mbar_wait(&tempty[acc], acc_phase ^ 1u, abort_flag, a.status))) break;
         tc_fence_after();
@@ -273,21 +294,32 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
           const uint32_t sa = smem_u32(smem + stage * C::kStageBytes);
           const uint64_t a1 = smem_desc_sw128(sa), a2 = smem_desc_sw128(sa + BM * BK * 2);
           const uint64_t b1 = smem_desc_sw128(sa + 2 * BM * BK * 2);
-          const uint64_t b2 = smem_desc_sw128(sa + 2 * BM * BK * 2 + BN * BK * 2);
+          const uint64_t b2 = smem_desc_sw128(sa + 2 * BM * BK * 2 + C::kBRows * BK * 2);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             const uint64_t off = (uint64_t)((k * UMMA_K * 2) >> 4);   // 32 bytes per K step
-            umma_bf16(d_tmem, a1 + off, b2 + off, idesc, (kb | k) != 0 ? 1u : 0u);   // hi * lo
-            umma_bf16(d_tmem, a2 + off, b1 + off, idesc, 1u);                        // lo * hi
-            umma_bf16(d_tmem, a1 + off, b1 + off, idesc, 1u);                        // hi * hi
+            if (CTAS == 2) {
+              umma_bf16_pair(d_tmem, a1 + off, b2 + off, idesc, (kb | k) != 0 ? 1u : 0u);   // hi * lo
+              umma_bf16_pair(d_tmem, a2 + off, b1 + off, idesc, 1u);                        // lo * hi
+              umma_bf16_pair(d_tmem, a1 + off, b1 + off, idesc, 1u);                        // hi * hi
+            } else {
+              umma_bf16(d_tmem, a1 + off, b2 + off, idesc, (kb | k) != 0 ? 1u : 0u);
+              umma_bf16(d_tmem, a2 + off, b1 + off, idesc, 1u);
+              umma_bf16(d_tmem, a1 + off, b1 + off, idesc, 1u);
+            }
           }
-          umma_commit(&empty[stage]);   // frees the stage once these MMAs have read it
+          // frees the stage (in both CTAs of a pair) once these MMAs have read it
+          if (CTAS == 2) umma_commit_pair(&empty[stage]);
+          else umma_commit(&empty[stage]);
           if (++stage == C::kStages) {
             stage = 0;
             phase ^= 1u;
           }
         }
-        if (ok) umma_commit(&tfull[acc]);
+        if (ok) {
+          if (CTAS == 2) umma_commit_pair(&tfull[acc]);
+          else umma_commit(&tfull[acc]);
+        }
       }
     }
     __syncwarp();
@@ -312,10 +344,10 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
     const int half = (warp - 2) >> 2;   // which part (of EPS) of the tile's columns this warp takes
     bool ok = true;
     int64_t it = 0;
-    for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+    for (int64_t t = unit; t < num_tiles && ok; t += nunits, ++it) {
       const uint32_t acc = (uint32_t)(it & 1), acc_phase = (uint32_t)((it >> 1) & 1);
       const int tm = (int)(t / a.tiles_n), tn = (int)(t % a.tiles_n);
-      const int64_t row = (int64_t)tm * BM + lg * 32 + lane;
+      const int64_t row = (int64_t)(tm * CTAS + rank) * BM + lg * 32 + lane;
       const int n0 = tn * BN;
       if (!(ok = mbar_wait(&tfull[acc], acc_phase, abort_flag, a.status))) break;
       tc_fence_after();
@@ -425,7 +457,10 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
       // accumulator fully read: hand the TMEM buffer back to the MMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&tempty[acc]);
+      if (lane == 0) {
+        if (CTAS == 2) mbar_arrive_leader(&tempty[acc]);
+        else mbar_arrive(&tempty[acc]);
+      }
       if (MODE == 1 && row_ok) a.gpart[(int64_t)(EPS * tn + half) * a.Mpad + row] = gsum;
       // pad words past the last tile's columns (rows whose stride exceeds the tiles' coverage)
       if (a.nibble && tn == a.tiles_n - 1 && half == EPS - 1 && row_ok) {
@@ -446,10 +481,12 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
   }
 
   tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) cluster_sync();   // neither CTA leaves while the partner may still arrive on its barriers or read its rows
+  else __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, C::kTmemCols);
+    if (CTAS == 2) tmem_dealloc_pair(tmem_base, C::kTmemCols);
+    else tmem_dealloc(tmem_base, C::kTmemCols);
   }
 }
 
@@ -530,47 +567,66 @@ int sm_count() {
 
 namespace {
 
-template <int BN, int MODE, int BITS>
+template <int BN, int MODE, int BITS, int CTAS>
 cudaError_t launch_gemm_t(const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b1, const CUtensorMap& b2,
                           const GemmArgs& args, cudaStream_t st) {
-  auto kern = quantize_gemm_kernel<BN, MODE, BITS>;
+  auto kern = quantize_gemm_kernel<BN, MODE, BITS, CTAS>;
+  using C = Cfg<BN, CTAS>;
   // function attributes are per device: remember the devices this launcher has prepared
   static std::atomic<unsigned long long> attr_devices{0};   // written by any thread that launches
   int attr_dev = 0;
   if (cudaGetDevice(&attr_dev) != cudaSuccess) return cudaErrorInvalidDevice;
   if (attr_dev >= 64 || !((attr_devices.load(std::memory_order_relaxed) >> attr_dev) & 1ull)) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     if (e != cudaSuccess) return e;
     if (attr_dev < 64) attr_devices.fetch_or(1ull << attr_dev, std::memory_order_relaxed);
   }
-  const int64_t tiles = (int64_t)args.tiles_m * args.tiles_n;
-  const int grid = (int)std::min<int64_t>(tiles, sm_count());
-  kern<<<grid, NTHREADS, Cfg<BN>::kSmemBytes, st>>>(a1, a2, b1, b2, args);
+  const int64_t tiles = (int64_t)args.tiles_m * args.tiles_n;   // tiles_m counts rows of BM * CTAS
+  const int units = (int)std::min<int64_t>(tiles, sm_count() / CTAS);
   count_launches(1);
-  return cudaGetLastError();
+  if (CTAS == 1) {
+    kern<<<units, NTHREADS, C::kSmemBytes, st>>>(a1, a2, b1, b2, args);
+    return cudaGetLastError();
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(units * CTAS));
+  cfg.blockDim = dim3(NTHREADS);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTAS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, a1, a2, b1, b2, args);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-template <int BN, int MODE>
+template <int BN, int MODE, int CTAS>
 cudaError_t launch_gemm_bits(int bits, const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b1,
                              const CUtensorMap& b2, const GemmArgs& args, cudaStream_t st) {
   if constexpr (MODE == 2) {
-    return launch_gemm_t<BN, 2, 1>(a1, a2, b1, b2, args, st);
+    return launch_gemm_t<BN, 2, 1, CTAS>(a1, a2, b1, b2, args, st);
   } else {
     switch (bits) {
-      case 0: return launch_gemm_t<BN, MODE, 0>(a1, a2, b1, b2, args, st);
-      case 1: return launch_gemm_t<BN, MODE, 1>(a1, a2, b1, b2, args, st);
-      case 2: return launch_gemm_t<BN, MODE, 2>(a1, a2, b1, b2, args, st);
-      case 3: return launch_gemm_t<BN, MODE, 3>(a1, a2, b1, b2, args, st);
-      default: return launch_gemm_t<BN, MODE, 4>(a1, a2, b1, b2, args, st);
+      case 0: return launch_gemm_t<BN, MODE, 0, CTAS>(a1, a2, b1, b2, args, st);
+      case 1: return launch_gemm_t<BN, MODE, 1, CTAS>(a1, a2, b1, b2, args, st);
+      case 2: return launch_gemm_t<BN, MODE, 2, CTAS>(a1, a2, b1, b2, args, st);
+      case 3: return launch_gemm_t<BN, MODE, 3, CTAS>(a1, a2, b1, b2, args, st);
+      default: return launch_gemm_t<BN, MODE, 4, CTAS>(a1, a2, b1, b2, args, st);
     }
   }
 }
 
+// ctas = 2: CTA pairs (only with 256-column tiles); b1, b2 are then the maps with half-height boxes.
 template <int MODE>
-cudaError_t launch_gemm(int bn, int bits, const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b1,
+cudaError_t launch_gemm(int bn, int ctas, int bits, const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b1,
                         const CUtensorMap& b2, const GemmArgs& args, cudaStream_t st) {
-  if (bn == 256) return launch_gemm_bits<256, MODE>(bits, a1, a2, b1, b2, args, st);
-  return launch_gemm_bits<128, MODE>(bits, a1, a2, b1, b2, args, st);
+  if (bn == 256 && ctas == 2) return launch_gemm_bits<256, MODE, 2>(bits, a1, a2, b1, b2, args, st);
+  if (bn == 256) return launch_gemm_bits<256, MODE, 1>(bits, a1, a2, b1, b2, args, st);
+  return launch_gemm_bits<128, MODE, 1>(bits, a1, a2, b1, b2, args, st);
 }
 
 }  // namespace
@@ -590,7 +646,8 @@ cudaError_t build_matrix_limbs(const float* dM, int rows, int d, int dpad, int b
   split_rows_kernel<float, false><<<blocks, 256>>>(dM, d, rows, d, dpad, out->hi, out->lo, nullptr);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  if (!make_map(&out->map_hi, out->hi, rows, d, dpad, bn) || !make_map(&out->map_lo, out->lo, rows, d, dpad, bn))
+  if (!make_map(&out->map_hi, out->hi, rows, d, dpad, bn) || !make_map(&out->map_lo, out->lo, rows, d, dpad, bn) ||
+      !make_map(&out->map_hi_half, out->hi, rows, d, dpad, bn / 2) || !make_map(&out->map_lo_half, out->lo, rows, d, dpad, bn / 2))
     return cudaErrorInvalidValue;
   return cudaSuccess;
 }
@@ -599,6 +656,15 @@ void free_matrix_limbs(MatrixLimbs* m) {
   cudaFree(m->hi);
   cudaFree(m->lo);
   m->hi = m->lo = nullptr;
+}
+
+// CTA pairs can be switched off (TQ_GEMM_PAIRS=0) to compare the two kernels on one machine.
+bool pair_tiles_enabled() {
+  static const bool on = [] {
+    const char* e = std::getenv("TQ_GEMM_PAIRS");
+    return e == nullptr || e[0] != '0';
+  }();
+  return on;
 }
 
 size_t scratch_bytes_per_row(const tq_plan* plan) {
@@ -690,7 +756,9 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     g.M = rows;
     g.N = d;
     g.K = d;
-    g.tiles_m = (int)((rows + BM - 1) / BM);
+    // CTA pairs on 256-row tiles where the tile is 256 columns wide and the block has rows for every pair
+    const int ctas = (bn == 256 && pair_tiles_enabled() && rows >= (int64_t)BM * sm_count()) ? 2 : 1;
+    g.tiles_m = (int)((rows + BM * ctas - 1) / (BM * ctas));
     g.tiles_n = tiles_n;
     g.cb = plan->cb;
     g.out = idx ? idx + (size_t)r0 * plan->idx_row_bytes : nullptr;
@@ -711,10 +779,12 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     // 2. y = Pi u, idx (+ residual limbs and partial norms)
     if (!prod) {
       if (pingpong && r0 + R < n) next_block_task(g);
-      TQ_CHECK_CUDA(launch_gemm<0>(bn, plan->mse_bits, mA1, mA2, plan->pi_limbs.map_hi, plan->pi_limbs.map_lo, g, st), who);
+      TQ_CHECK_CUDA(launch_gemm<0>(bn, ctas, plan->mse_bits, mA1, mA2, ctas == 2 ? plan->pi_limbs.map_hi_half : plan->pi_limbs.map_hi,
+                                   ctas == 2 ? plan->pi_limbs.map_lo_half : plan->pi_limbs.map_lo, g, st), who);
       continue;
     }
-    TQ_CHECK_CUDA(launch_gemm<1>(bn, plan->mse_bits, mA1, mA2, plan->pi_limbs.map_hi, plan->pi_limbs.map_lo, g, st), who);
+    TQ_CHECK_CUDA(launch_gemm<1>(bn, ctas, plan->mse_bits, mA1, mA2, ctas == 2 ? plan->pi_limbs.map_hi_half : plan->pi_limbs.map_hi,
+                                 ctas == 2 ? plan->pi_limbs.map_lo_half : plan->pi_limbs.map_lo, g, st), who);
     // 3. gamma = ||e||
     gamma_finish_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(gpart, R, EPS * tiles_n, rows, gamma + r0);
     count_launches(1);
@@ -726,7 +796,8 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     g.out = qjl + (size_t)r0 * plan->qjl_row_bytes;
     g.out_rb = plan->qjl_row_bytes;
     if (overlap && r0 + R < n) next_block_task(g);   // the limbs of X are free by now
-    TQ_CHECK_CUDA(launch_gemm<2>(bn, 1, mE1, mE2, plan->sp_limbs.map_hi, plan->sp_limbs.map_lo, g, st), who);
+    TQ_CHECK_CUDA(launch_gemm<2>(bn, ctas, 1, mE1, mE2, ctas == 2 ? plan->sp_limbs.map_hi_half : plan->sp_limbs.map_hi,
+                                 ctas == 2 ? plan->sp_limbs.map_lo_half : plan->sp_limbs.map_lo, g, st), who);
   }
   return TQ_OK;
 }
