@@ -497,14 +497,13 @@ def run_b200(args):
     rows_per_launch = min(n, scratch_bytes // max(per_row, 1) // 128 * 128)
     launches_per_step = math.ceil(n / max(rows_per_launch, 1))
     algo_bytes_row = 4 * d + plan.idx_row_bytes + plan.qjl_row_bytes + 8
-    roofline = {"bound": "tensor", "kernel": f"tc::quantize_gemm_kernel (Y = U Pi^T and Z = E S'^T, one launch of each per {rows_per_launch} rows)",
+    roofline = {"bound": "tensor", "kernel": f"tc::quantize_gemm_kernel on CTA pairs (Y = U Pi^T and Z = E S'^T, one launch of each per {rows_per_launch} rows)",
                 "achieved": achieved_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                 "frac": achieved_tf / peaks["bf16_tflops_sustained"],
                 "frac_of_three_pass_bound": 3.0 * achieved_tf / peaks["bf16_tflops_sustained"],
                 "traffic": QUANTIZE_TRAFFIC_PER_98304_ROWS if d == 1536 else None,
-                "traffic_source": "ncu capture of one rotate + one project launch of 98,304 rows (profile summary, not measured in this run); "
-                                  "the project launch also prepares the operand limbs of the next block of rows (reads its fp32 input, "
-                                  "writes two bf16 limbs): captured with a 32,768-row next block, that part scaled to 98,304 rows",
+                "traffic_source": "ncu capture of one rotate + one project launch of 98,304 rows (profile summary, not measured in this run) "
+                                  "plus the bytes the split_rows launch of the block moves by definition",
                 "algorithmic_bytes_per_launch": algo_bytes_row * rows_per_launch,
                 "peak_source": f"bf16 sustained, of {peaks['source']}",
                 "note": "achieved = algorithmic flops 4 n d^2 of the step / CUDA-event time of the quantise phase "
@@ -550,9 +549,9 @@ def run_b200(args):
 
 
 # DRAM bytes of the dominant kernels from ncu captures (one launch each; see the summaries under profiles/)
-# rotate launch (651.2 MB read + 666.4 MB written) + project launch (925.8 + 271.3 MB, of which 201.3 + 201.3 MB are the
-# limbs of a 32,768-row next block) + the same limb traffic for the other 65,536 rows of a full next block
-QUANTIZE_TRAFFIC_PER_98304_ROWS = (651.2e6 + 666.4e6) + (925.8e6 + 271.3e6) + 2 * 2 * 201.3e6
+# rotate launch (692.5 MB read + 671.4 MB written) + project launch (690.4 + 72.1 MB) of the CTA-pair GEMM, from ncu;
+# + the split_rows launch of the block (reads 98,304 x 6144 B, writes two bf16 limbs of the same size: 604 + 604 MB)
+QUANTIZE_TRAFFIC_PER_98304_ROWS = (692.5e6 + 671.4e6) + (690.4e6 + 72.1e6) + 2 * 604.0e6
 SCAN_TRAFFIC_PER_VECTOR = (205.9e6 + 5.0e6) / 262144
 
 

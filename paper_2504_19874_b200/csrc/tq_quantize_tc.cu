@@ -688,9 +688,10 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
   // rotate launch itself, so the scratch is used as two half-size sets written and read in turn (when the data
   // spans more than one block and each half still holds a tile).
   // Two warps per CTA keep up only while the GEMM gives them time: its work per row grows with d^2, theirs with d.
-  // Measured per 10^6 rows: d = 1536 gains 4 % (TQ_PROD) and 11 % (TQ_MSE), d = 3072 2 %; at d = 1024 the spare warps
-  // already lose (12.3 against 11.3 ms, TQ_MSE 6.9 against 5.6), at d = 200 they are the critical path (2.9 against 1.9 ms).
-  const bool overlap = d >= 1536;
+  // Measured per 10^6 rows with the CTA-pair GEMMs: TQ_MSE d = 1536 10.1 ms with them against 10.6 without; TQ_PROD
+  // loses (d = 1536: 22.1 against 21.5 ms, d = 3072 alike), so its project launch carries no such task any more; at
+  // d = 1024 and below the spare warps are the critical path for both.
+  const bool overlap = !prod && d >= 1536;
   const bool pingpong = overlap && !prod && n > R / 2 / BM * BM && R / 2 >= BM;
   const int64_t Rbuf = R;   // rows the carved buffers hold in all
   if (pingpong) R = R / 2 / BM * BM;
