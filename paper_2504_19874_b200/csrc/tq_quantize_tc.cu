@@ -757,8 +757,8 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     g.M = rows;
     g.N = d;
     g.K = d;
-    // CTA pairs on 256-row tiles where the tile is 256 columns wide and the block has rows for every pair
-    const int ctas = (bn == 256 && pair_tiles_enabled() && rows >= (int64_t)BM * sm_count()) ? 2 : 1;
+    // CTA pairs on 256-row tiles where the tile is 256 columns wide and the block has more rows than one CTA's tile
+    const int ctas = (bn == 256 && pair_tiles_enabled() && rows > BM) ? 2 : 1;
     g.tiles_m = (int)((rows + BM * ctas - 1) / (BM * ctas));
     g.tiles_n = tiles_n;
     g.cb = plan->cb;
