@@ -7,6 +7,9 @@
 // accumulation (3 MMA passes).  The dropped terms are ~2^-17 relative per product, i.e.
 // ~1e-7 on a rotated coordinate of a unit vector at d = 1536 -- far inside the 1e-5 window in
 // which a nearest-centroid decision may legitimately differ from exact arithmetic.
+//
+// Two forms of the GEMM kernel: one CTA per 128 x 256 tile, and (the usual one at d > 128) a pair of CTAs of one
+// cluster per 256 x 256 tile (tcgen05 cta_group::2), which halves what every SM reads of B from shared memory.
 #include <atomic>
 #include <cstdlib>
 #include <algorithm>
