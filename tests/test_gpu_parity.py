@@ -81,6 +81,46 @@ def test_embedding_configs_subset(name, bits, mode, n):
     assert stats["idx_mismatch"] == 0
 
 
+_ONE_CTA_CHILD = r"""
+import sys, torch
+sys.path.insert(0, sys.argv[1])
+import paper_2504_19874_b200 as tq
+import tq_workloads as wl
+from tests import parity as P
+blob = torch.load(sys.argv[2])
+cfg = wl.CONFIGS["c4"]
+for (bits, mode), want in zip(((4, tq.TQ_PROD), (2, tq.TQ_MSE)), blob["codes"]):
+    su = P.Setup(cfg.d, bits, mode, cfg.pi_seed, cfg.s_seed)
+    X = blob["X"].cuda()
+    got = su.quantize(X)
+    P.check_quantize(su, X, *got)
+    for u, v in zip(got, want):
+        assert (u is None and v is None) or torch.equal(u.cpu(), v), "the two GEMM kernels disagree"
+print("one-CTA kernel ok")
+"""
+
+
+def test_one_cta_gemm_kernel_gives_the_same_codes(tmp_path):
+    """Blocks of more than 128 rows run the quantiser's GEMMs on CTA pairs; TQ_GEMM_PAIRS=0 (read once per process)
+    keeps the one-CTA kernel.  Same operands, same order of accumulation: the codes must be bit-identical, and the
+    child checks them against the oracle as well."""
+    import os
+    import subprocess
+    import sys
+    cfg = wl.CONFIGS["c4"]
+    X = wl.database(cfg, 1500, device=DEV)
+    codes = []
+    for bits, mode in ((4, tq.TQ_PROD), (2, tq.TQ_MSE)):
+        su = P.Setup(cfg.d, bits, mode, cfg.pi_seed, cfg.s_seed)
+        codes.append(tuple(None if t is None else t.cpu() for t in su.quantize(X)))
+    blob = tmp_path / "pair_codes.pt"
+    torch.save({"X": X.cpu(), "codes": codes}, blob)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, TQ_GEMM_PAIRS="0")
+    r = subprocess.run([sys.executable, "-c", _ONE_CTA_CHILD, root, str(blob)], env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "one-CTA kernel ok" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
+
+
 def test_small_scratch_forces_several_blocks_of_rows():
     cfg = wl.CONFIGS["c2"]
     for bits, mode in ((3, tq.TQ_PROD), (2, tq.TQ_MSE)):
