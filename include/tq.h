@@ -59,7 +59,8 @@ enum {
   TQ_ERR_CUDA = 4,          /* a CUDA runtime call failed (message has the CUDA error)       */
   TQ_ERR_NOT_CONVERGED = 5, /* Lloyd-Max iteration did not converge                          */
   TQ_ERR_TIMEOUT = 6,       /* a bounded device-side wait ran out                            */
-  TQ_ERR_WORKSPACE = 7      /* scratch / workspace smaller than tq_workspace_bytes says      */
+  TQ_ERR_WORKSPACE = 7,     /* scratch / workspace smaller than tq_workspace_bytes says      */
+  TQ_ERR_BOUNDS = 8         /* a TQ_DEBUG build of the library found an index outside its array */
 };
 enum { TQ_MSE = 0, TQ_PROD = 1 };              /* plan mode                                   */
 enum { TQ_F32 = 0, TQ_BF16 = 1 };              /* element type of X / Q                       */
@@ -148,7 +149,10 @@ int tq_convert_layout(const tq_plan* plan, int64_t n, uint8_t* idx, uint8_t* qjl
 /* Synchronises the device and reports whether any kernel launched for this plan since the
  * last call gave up one of its bounded device-side waits (TQ_ERR_TIMEOUT; the outputs of that
  * call are then invalid).  Every producer/consumer wait inside the tensor-core kernels has a
- * time limit so that a stalled pipeline ends as this status instead of a hung GPU. */
+ * time limit so that a stalled pipeline ends as this status instead of a hung GPU.
+ * A library built with -DTQ_DEBUG (`python -m paper_2504_19874_b200.build --debug`, libtq_debug.so) also checks the
+ * row, column and slot indices of its kernels' global stores and of the caller's channel lists on the device: an
+ * index outside its array is not stored through; TQ_ERR_BOUNDS is recorded and reported here. */
 int tq_plan_status(tq_plan* plan);
 
 /* Self test of that mechanism, for test suites: enqueues a one-warp kernel that waits, through the same bounded

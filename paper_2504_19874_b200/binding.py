@@ -14,7 +14,9 @@ TQ_LAYOUT_CANONICAL, TQ_LAYOUT_NIBBLE = 0, 1
 TQ_OP_QUANTIZE, TQ_OP_SCORE, TQ_OP_TOPK, TQ_OP_WSUM, TQ_OP_DEQUANTIZE = 0, 1, 2, 3, 4
 TQ_STATIC_SCRATCH_BYTES = 1 << 20
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libtq.so")
+# TQ_LIB_VARIANT=debug loads libtq_debug.so, the build with device-side index checks (build.py --debug)
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)),
+                         "libtq_debug.so" if os.environ.get("TQ_LIB_VARIANT") == "debug" else "libtq.so")
 _lib = None
 
 c_void_p, c_int, c_int64, c_size_t, c_u64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t, ctypes.c_uint64

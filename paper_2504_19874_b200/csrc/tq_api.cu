@@ -575,6 +575,10 @@ extern "C" int tq_plan_status(tq_plan* plan) {
   TQ_CHECK_CUDA(cudaMemcpy(&st, plan->d_status, sizeof(int), cudaMemcpyDeviceToHost), who);
   if (st != 0) {
     cudaMemset(plan->d_status, 0, sizeof(int));
+    if (st == TQ_ERR_BOUNDS) {
+      set_error("%s: a device-side index check of the TQ_DEBUG build failed (the access was skipped)", who);
+      return TQ_ERR_BOUNDS;
+    }
     if (st != TQ_ERR_TIMEOUT) {
       set_error("%s: a kernel recorded the unexpected status %d", who, st);
       return TQ_ERR_CUDA;

@@ -74,6 +74,8 @@ struct Args {
   int lut_float4;   // float4 entries of all tables
   int vunits, region0;   // units of all groups; float4 entries of the first shared-memory region
   int kbuf_bytes, vbuf_bytes;   // shared-memory room for the slice's K and V code rows
+  int* status;      // the plans' device status word (bounded waits; index checks of the TQ_DEBUG build)
+  int64_t ldq_dbg, ldo_dbg;   // row lengths of Q and out that a channel index must stay inside
 };
 
 __host__ __device__ inline int mse_lookups(int d, int bits) {   // table rows of the MSE term
@@ -93,7 +95,7 @@ __global__ void __launch_bounds__(128) prepare_kernel(Args a, const T* __restric
     float v = 0.f;
     if (j < a.qpk) {
       const int ch = g.k_channels[h * d + c];
-      v = (float)Q[(int64_t)(h * a.qpk + j) * ldq + ch];
+      if (TQ_DEVICE_CHECK(ch >= 0 && ch < a.ldq_dbg, a.status)) v = (float)Q[(int64_t)(h * a.qpk + j) * ldq + ch];
     }
     qs[j][c] = v;
   }
@@ -486,7 +488,7 @@ __global__ void __launch_bounds__(MERGE_NT) merge_kernel(Args a, float* __restri
     float v = 0.f;
 #pragma unroll 8
     for (int cc = 0; cc < d; ++cc) v = fmaf(pis[cc * d + k], ys[j][cc], v);
-    out[(int64_t)(h * a.qpk + j) * ldo + chan[k]] = v;
+    if (TQ_DEVICE_CHECK(chan[k] >= 0 && chan[k] < a.ldo_dbg, a.status)) out[(int64_t)(h * a.qpk + j) * ldo + chan[k]] = v;
   }
 }
 
@@ -808,6 +810,7 @@ extern "C" int tq_attend_decode(const tq_kv_group* groups, int ngroups, int head
   a.ngroups = ngroups; a.heads = heads; a.qpk = q_per_kv; a.d = d; a.nslices = (int)nslices;
   a.tokens = tokens; a.head_stride = head_stride; a.scale = scale; a.lut_float4 = lut;
   a.kbuf_bytes = kbytes; a.vbuf_bytes = vbytes;
+  a.status = groups[0].plan_k->d_status; a.ldq_dbg = ldq; a.ldo_dbg = ldo;
   a.vunits = vunits;
   a.region0 = std::max(lut + SLICE, std::max(1, NT / vunits) * ngroups * d);
   char* w = static_cast<char*>(workspace);

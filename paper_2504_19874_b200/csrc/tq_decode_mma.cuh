@@ -181,7 +181,10 @@ __global__ void __launch_bounds__(256) prepare_mma_kernel(Args a, MmaArgs ma, co
   for (int e = tid; e < MAXQ * d; e += blockDim.x) {
     const int j = e / d, c = e % d;
     float v = 0.f;
-    if (j < a.qpk) v = (float)Q[(int64_t)(h * a.qpk + j) * ldq + g.k_channels[h * d + c]];
+    if (j < a.qpk) {
+      const int ch = g.k_channels[h * d + c];
+      if (TQ_DEVICE_CHECK(ch >= 0 && ch < a.ldq_dbg, a.status)) v = (float)Q[(int64_t)(h * a.qpk + j) * ldq + ch];
+    }
     qs[j][c] = v;
   }
   if (tid < 2 * MAXQ) wmax[tid / MAXQ][tid % MAXQ] = 0;
@@ -642,7 +645,7 @@ __global__ void __launch_bounds__(NT, 4) partial_mma_kernel(Args a, MmaArgs ma) 
         for (int o = 0; o < 4; ++o) s += plane(4 * c + o, m.v_alpha[o]);
         for (int o = 0; o < 4; ++o) s += plane(4 * d + 4 * c + o, m.v_alpha[4 + o]);
       }
-      out[gi * d * MAXQ + it] = s * rs;
+      if (TQ_DEVICE_CHECK(h < a.heads && sl < a.nslices && gi * d * MAXQ + it < ncoord * MAXQ, a.status)) out[gi * d * MAXQ + it] = s * rs;
     }
   }
 }

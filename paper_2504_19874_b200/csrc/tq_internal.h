@@ -45,6 +45,21 @@ struct Codebook {
 
 // A d x d fp32 matrix split into two bf16 limbs (M = hi + lo + O(2^-17)), rows padded to dpad,
 // with the TMA descriptors the tensor-core GEMM uses for it as the B operand.
+// Device-side index checks of the TQ_DEBUG build: `if (TQ_DEVICE_CHECK(row < n, status)) out[row] = v;`.  In a release
+// build the condition is not evaluated.  A failed check records TQ_ERR_BOUNDS in the plan's status word (reported by
+// tq_plan_status) and the access is skipped.
+#ifdef __CUDACC__
+#ifdef TQ_DEBUG
+__device__ __forceinline__ bool device_check_failed(int* status) {
+  if (status != nullptr) atomicExch(status, TQ_ERR_BOUNDS);
+  return false;
+}
+#define TQ_DEVICE_CHECK(cond, status) ((cond) ? true : ::tq::device_check_failed(status))
+#else
+#define TQ_DEVICE_CHECK(cond, status) (true)
+#endif
+#endif
+
 struct MatrixLimbs {
   __nv_bfloat16* hi;
   __nv_bfloat16* lo;

@@ -444,7 +444,7 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
             for (int q = 0; q < BITS; ++q)
               if (w0 + q < row_words) out_row[w0 + q] = words[q];
           }
-          if (MODE == 1 && row_ok) {
+          if (MODE == 1 && row_ok && TQ_DEVICE_CHECK(row < a.Mpad, a.status)) {
             uint4* d1 = reinterpret_cast<uint4*>(a.E1 + row * a.ldE + col0);
             uint4* d2 = reinterpret_cast<uint4*>(a.E2 + row * a.ldE + col0);
 #pragma unroll
@@ -464,7 +464,8 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
         if (CTAS == 2) mbar_arrive_leader(&tempty[acc]);
         else mbar_arrive(&tempty[acc]);
       }
-      if (MODE == 1 && row_ok) a.gpart[(int64_t)(EPS * tn + half) * a.Mpad + row] = gsum;
+      if (MODE == 1 && row_ok && TQ_DEVICE_CHECK(row < a.Mpad && tn < a.tiles_n, a.status))
+        a.gpart[(int64_t)(EPS * tn + half) * a.Mpad + row] = gsum;
       // pad words past the last tile's columns (rows whose stride exceeds the tiles' coverage)
       if (a.nibble && tn == a.tiles_n - 1 && half == EPS - 1 && row_ok) {
         if (MODE == 1) {   // words of the combined row that no group of 32 coordinates owns

@@ -531,7 +531,7 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
         const float est = __fmul_rn(nu, fmaf(gm, sv, av));
         if (row_ok && ql < a.nq_pass) {
           if (MODE == 0) {
-            a.scores[(int64_t)ql * a.lds + row] = est;
+            if (TQ_DEVICE_CHECK(row >= 0 && row < a.n && row < a.lds, a.status)) a.scores[(int64_t)ql * a.lds + row] = est;
           } else if (est >= __ldg(a.tau + ql)) {
             const int slot = atomicAdd(a.count + ql, 1);
             if (slot < a.cap) {

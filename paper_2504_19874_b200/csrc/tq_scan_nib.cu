@@ -419,7 +419,7 @@ scan_nib_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
       const float est = __fmul_rn(nu, fmaf(__fmul_rn(a.coef, gamma), sv, av));
       if (row < row_end && ql < a.nq_pass) {
         if (MODE == 0) {
-          a.scores[(int64_t)ql * a.lds + row] = est;
+          if (TQ_DEVICE_CHECK(row >= 0 && row < a.n && row < a.lds, a.status)) a.scores[(int64_t)ql * a.lds + row] = est;
         } else if (est >= __ldg(a.tau + ql)) {
           const int slot = atomicAdd(a.count + ql, 1);
           if (slot < a.cap) {

@@ -727,7 +727,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
           const float est = __fmul_rn(nu, fmaf(gm, sv, av));
           if (row_ok && ql < a.nqp) {
             if (MODE == 0) {
-              a.scores[(int64_t)ql * a.lds + row] = est;
+              if (TQ_DEVICE_CHECK(row >= 0 && row < a.n && row < a.lds, a.status)) a.scores[(int64_t)ql * a.lds + row] = est;
             } else if (est >= taus[ql]) {
               const int ls = atomicAdd(&lcnt[ql], 1);
               if (ls < LBUF) {
