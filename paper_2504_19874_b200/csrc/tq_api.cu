@@ -102,7 +102,7 @@ constexpr int64_t kDenseRowsMin = 4096;
 constexpr int kGroupQueries = tscan::kQueriesPerPass * tscan::kPassesPerGroup;
 
 // The two engines behind the bit-plane scan: register-fed integer MMA (2 or 4 queries per pass) for few
-// queries, tcgen05 (32 queries per pass) from 7 queries on (measured at d = 1536, b = 4, n = 10^6: a short
+// queries, tcgen05 (32 queries per pass, 64 in calls of more than 32 queries) from 7 queries on (measured at d = 1536, b = 4, n = 10^6: a short
 // tcgen05 pass 0.69 ms, register-fed passes 0.24 ms for 1-2 queries and 0.37 ms for 3-4, so 4 + 3 queries
 // already cost more).
 struct ScanEngine {
@@ -124,7 +124,7 @@ ScanEngine pick_engine(const tq_plan* plan, int nq) {
   const int tc_from = !e.nib ? 7 : nscan::queries_per_pass(plan, 8) == 8 ? 15 : 5;
   e.tc = nq >= tc_from && tscan::available(plan);
   e.nib = e.nib && !e.tc;
-  e.qpp = e.tc ? tscan::kQueriesPerPass : e.nib ? nscan::queries_per_pass(plan, nq) : mscan::queries_per_pass(plan, nq);
+  e.qpp = e.tc ? tscan::queries_per_pass(nq) : e.nib ? nscan::queries_per_pass(plan, nq) : mscan::queries_per_pass(plan, nq);
   e.dense_rows_pref = e.tc ? (1 << 18) : (1 << 20);
   e.ws_bytes = e.tc ? tscan::workspace_bytes(plan) : e.nib ? nscan::workspace_bytes(plan) : mscan::workspace_bytes(plan);
   return e;
@@ -153,7 +153,7 @@ int engine_run(const ScanEngine& e, int q0, int nqp, int64_t n, const uint8_t* i
 
 size_t ms_score_fixed(const tq_plan* plan, int nq) { return qcat_bytes(plan, nq) + align_up(pick_engine(plan, nq).ws_bytes, 256); }
 size_t ms_topk_fixed(const tq_plan* plan, int nq) {
-  return ms_score_fixed(plan, nq) + 512 /* tau, count, overflow */ + (size_t)pick_engine(plan, nq).qpp * kCandCap * 8;
+  return ms_score_fixed(plan, nq) + 1024 /* tau, count, overflow */ + (size_t)pick_engine(plan, nq).qpp * kCandCap * 8;
 }
 
 template <typename T>
@@ -890,10 +890,10 @@ static int topk_ms(const tq_plan* plan, const float* Qcat, int nq, int64_t n, co
   const ScanEngine eng = pick_engine(plan, nq);
   void* msw = ws;
   char* p = ws + align_up(eng.ws_bytes, 256);
-  float* tau = reinterpret_cast<float*>(p);          // [qpp] (qpp <= 32: 128 bytes)
-  int* count = reinterpret_cast<int*>(p + 128);      // [qpp], then the overflow flag
+  float* tau = reinterpret_cast<float*>(p);          // [qpp] (qpp <= 64: 256 bytes)
+  int* count = reinterpret_cast<int*>(p + 256);      // [qpp], then the overflow flag
   int* overflow = count + eng.qpp;
-  p += 512;
+  p += 1024;
   float* cand_s = reinterpret_cast<float*>(p);
   int* cand_i = reinterpret_cast<int*>(p + (size_t)eng.qpp * kCandCap * 4);
   p += (size_t)eng.qpp * kCandCap * 8;

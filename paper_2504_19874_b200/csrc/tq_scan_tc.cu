@@ -37,6 +37,7 @@
 #include <atomic>
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 
 #include "tq_nib_common.cuh"
 #include "tq_quantize_tc.h"
@@ -773,6 +774,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
 }
 
 // at least 120 KB so that a second CTA can never share the SM (the kernel allocates all of TMEM)
+#include "tq_scan_tcw.cuh"
+
 constexpr size_t kSmemUsed = B_STAGES * BTILE_BYTES + P_STAGES * PTILE_BYTES + 1024 + 512 + kQueriesPerPass * (sizeof(QConst) + sizeof(float) + sizeof(int) + LBUF * sizeof(uint2));
 constexpr size_t kSmemBytes = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;
 
@@ -795,6 +798,37 @@ cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& ms, const CUtenso
   return cudaGetLastError();
 }
 
+template <int BM, int MODE, bool NIB = false>
+cudaError_t launch_wide_t(const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
+                          const ScanArgs& args, cudaStream_t st) {
+  auto kern = scan_tcw_kernel<BM, MODE, NIB>;
+  static std::atomic<unsigned long long> attr_devices{0};
+  int attr_dev = 0;
+  if (cudaGetDevice(&attr_dev) != cudaSuccess) return cudaErrorInvalidDevice;
+  if (attr_dev >= 64 || !((attr_devices.load(std::memory_order_relaxed) >> attr_dev) & 1ull)) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWideSmemBytes);
+    if (e != cudaSuccess) return e;
+    if (attr_dev < 64) attr_devices.fetch_or(1ull << attr_dev, std::memory_order_relaxed);
+  }
+  const int grid = (int)std::min<int64_t>((args.n + TILE - 1) / TILE, tc::sm_count());
+  kern<<<grid, NTHREADS, kWideSmemBytes, st>>>(ma, ms, pa, ps, args);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+template <int MODE>
+cudaError_t launch_wide(int bm, const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
+                        const ScanArgs& args, cudaStream_t st) {
+  if (args.g.nib) return launch_wide_t<3, MODE, true>(ma, ms, pa, ps, args, st);
+  switch (bm) {
+    case 0: return launch_wide_t<0, MODE>(ma, ms, pa, ps, args, st);
+    case 1: return launch_wide_t<1, MODE>(ma, ms, pa, ps, args, st);
+    case 2: return launch_wide_t<2, MODE>(ma, ms, pa, ps, args, st);
+    case 3: return launch_wide_t<3, MODE>(ma, ms, pa, ps, args, st);
+    default: return launch_wide_t<4, MODE>(ma, ms, pa, ps, args, st);
+  }
+}
+
 template <int MODE>
 cudaError_t launch_bm(int bm, const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
                       const ScanArgs& args, cudaStream_t st) {
@@ -815,6 +849,15 @@ size_t b_bytes(const Geo& g, int part) {
 }  // namespace
 
 bool available(const tq_plan* plan) { return plan->ms.ok != 0; }
+
+// The wide form can be switched off (TQ_SCAN_WIDE=0) to compare the two kernels on one machine.
+int queries_per_pass(int nq) {
+  static const bool wide = [] {
+    const char* e = std::getenv("TQ_SCAN_WIDE");
+    return e == nullptr || e[0] != '0';
+  }();
+  return wide && nq > kQueriesPerPass ? W_QPP : kQueriesPerPass;
+}
 
 size_t workspace_bytes(const tq_plan* plan) {
   if (!available(plan)) return 0;
@@ -879,13 +922,19 @@ int run_pass(const tq_plan* plan, int pass, int nqp, int64_t n, const uint8_t* i
   const QConst* qc = static_cast<const QConst*>(workspace);
   const uint8_t* Ba = static_cast<const uint8_t*>(workspace) + kConstBytes;
   const uint8_t* Bs = Ba + b_bytes(g, 0);
+  // more than 32 queries: the wide kernel takes the B rows of this pass and the next as one box of 192 rows and one
+  // 128-vector tile at a time
+  const bool wide = nqp > kQueriesPerPass;
+  TQ_REQUIRE(nqp <= (wide ? W_QPP : kQueriesPerPass) && (!wide || (pass % 2 == 0 && pass + 2 <= kPassesPerGroup)), TQ_ERR_INVALID_ARG,
+             "%s: pass %d of %d queries", who, pass, nqp);
+  const uint32_t brows = wide ? W_NCOL : NCOL, prows = wide ? TILE : 2 * TILE;
   CUtensorMap ma, ms;
   const uint64_t rows = (uint64_t)kPassesPerGroup * NCOL;
   if (g.kba > 0)
-    TQ_REQUIRE(tc::make_byte_map(&ma, Ba, rows, (uint64_t)g.kba * KB_BYTES, (uint64_t)g.kba * KB_BYTES, KB_BYTES, NCOL, 128),
+    TQ_REQUIRE(tc::make_byte_map(&ma, Ba, rows, (uint64_t)g.kba * KB_BYTES, (uint64_t)g.kba * KB_BYTES, KB_BYTES, brows, 128),
                TQ_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (B, MSE part)", who);
   if (g.kbs > 0)
-    TQ_REQUIRE(tc::make_byte_map(&ms, Bs, rows, (uint64_t)g.kbs * KB_BYTES, (uint64_t)g.kbs * KB_BYTES, KB_BYTES, NCOL, 128),
+    TQ_REQUIRE(tc::make_byte_map(&ms, Bs, rows, (uint64_t)g.kbs * KB_BYTES, (uint64_t)g.kbs * KB_BYTES, KB_BYTES, brows, 128),
                TQ_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (B, QJL part)", who);
   if (g.kba == 0) ma = ms;
   if (g.kbs == 0) ms = ma;
@@ -893,15 +942,15 @@ int run_pass(const tq_plan* plan, int pass, int nqp, int64_t n, const uint8_t* i
   CUtensorMap pa, ps;
   const int gb = g.nib ? 64 : group_bytes(g.bm);
   if (g.nib) {
-    TQ_REQUIRE(tc::make_byte_map(&pa, idx, (uint64_t)n, plan->idx_row_bytes, plan->idx_row_bytes, 64, 2 * TILE, 64) &&
-                   tc::make_byte_map(&ps, qjl, (uint64_t)n, plan->qjl_row_bytes, plan->qjl_row_bytes, 64, 2 * TILE, 64),
+    TQ_REQUIRE(tc::make_byte_map(&pa, idx, (uint64_t)n, plan->idx_row_bytes, plan->idx_row_bytes, 64, prows, 64) &&
+                   tc::make_byte_map(&ps, qjl, (uint64_t)n, plan->qjl_row_bytes, plan->qjl_row_bytes, 64, prows, 64),
                TQ_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (code rows)", who);
   } else if (g.kba > 0)
-    TQ_REQUIRE(tc::make_byte_map(&pa, idx, (uint64_t)n, plan->idx_row_bytes, plan->idx_row_bytes, gb, 2 * TILE,
+    TQ_REQUIRE(tc::make_byte_map(&pa, idx, (uint64_t)n, plan->idx_row_bytes, plan->idx_row_bytes, gb, prows,
                                  gb == 64 ? 64 : gb == 32 ? 32 : 0),
                TQ_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (idx rows)", who);
   if (!g.nib && g.kbs > 0)
-    TQ_REQUIRE(tc::make_byte_map(&ps, qjl, (uint64_t)n, plan->qjl_row_bytes, plan->qjl_row_bytes, 64, 2 * TILE, 64), TQ_ERR_CUDA,
+    TQ_REQUIRE(tc::make_byte_map(&ps, qjl, (uint64_t)n, plan->qjl_row_bytes, plan->qjl_row_bytes, 64, prows, 64), TQ_ERR_CUDA,
                "%s: cuTensorMapEncodeTiled failed (qjl rows)", who);
   if (!g.nib && g.kba == 0) pa = ps;
   if (!g.nib && g.kbs == 0) ps = pa;
@@ -929,7 +978,8 @@ int run_pass(const tq_plan* plan, int pass, int nqp, int64_t n, const uint8_t* i
   a.cap = filter ? filter->cap : 0;
   a.run_if = run_if;
   a.status = plan->d_status;
-  TQ_CHECK_CUDA(filter ? launch_bm<1>(g.bm, ma, ms, pa, ps, a, st) : launch_bm<0>(g.bm, ma, ms, pa, ps, a, st), who);
+  if (wide) TQ_CHECK_CUDA(filter ? launch_wide<1>(g.bm, ma, ms, pa, ps, a, st) : launch_wide<0>(g.bm, ma, ms, pa, ps, a, st), who);
+  else TQ_CHECK_CUDA(filter ? launch_bm<1>(g.bm, ma, ms, pa, ps, a, st) : launch_bm<0>(g.bm, ma, ms, pa, ps, a, st), who);
   return TQ_OK;
 }
 
