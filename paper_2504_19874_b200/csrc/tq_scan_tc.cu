@@ -34,6 +34,9 @@
 // barrier (one commit per issuer).  Ring positions and phases are masks and shifts of 32-bit counters: the
 // single-lane roles run dependent instruction chains, where 64-bit division costs real time.  All waits
 // are bounded.
+//
+// Calls of more than 32 queries run the wide form of this kernel (tq_scan_tcw.cuh: 64 queries per pass, one tile
+// per iteration, four A slots, N = 192); this one serves 7..32 queries and the last, short pass of a longer call.
 #include <atomic>
 #include <algorithm>
 #include <cmath>
@@ -363,6 +366,16 @@ __device__ __forceinline__ void umma_i8_ts(uint32_t tmem_d, uint32_t tmem_a, uin
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The same over a CTA pair (M = 256: the leader's thread issues for both CTAs, each CTA holds its own rows of A and D in
+// TMEM and half of B's rows in shared memory).
+__device__ __forceinline__ void umma_i8_ts_pair(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
@@ -798,10 +811,10 @@ cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& ms, const CUtenso
   return cudaGetLastError();
 }
 
-template <int BM, int MODE, bool NIB = false>
-cudaError_t launch_wide_t(const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
+template <int BM, int MODE, bool NIB, int CTAS>
+cudaError_t launch_wide_c(const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
                           const ScanArgs& args, cudaStream_t st) {
-  auto kern = scan_tcw_kernel<BM, MODE, NIB>;
+  auto kern = scan_tcw_kernel<BM, MODE, NIB, CTAS>;
   static std::atomic<unsigned long long> attr_devices{0};
   int attr_dev = 0;
   if (cudaGetDevice(&attr_dev) != cudaSuccess) return cudaErrorInvalidDevice;
@@ -810,22 +823,46 @@ cudaError_t launch_wide_t(const CUtensorMap& ma, const CUtensorMap& ms, const CU
     if (e != cudaSuccess) return e;
     if (attr_dev < 64) attr_devices.fetch_or(1ull << attr_dev, std::memory_order_relaxed);
   }
-  const int grid = (int)std::min<int64_t>((args.n + TILE - 1) / TILE, tc::sm_count());
-  kern<<<grid, NTHREADS, kWideSmemBytes, st>>>(ma, ms, pa, ps, args);
   count_launches(1);
-  return cudaGetLastError();
+  const int64_t ntiles = (args.n + TILE - 1) / TILE;
+  if (CTAS == 1) {
+    kern<<<(int)std::min<int64_t>(ntiles, tc::sm_count()), NTHREADS, kWideSmemBytes, st>>>(ma, ms, pa, ps, args);
+    return cudaGetLastError();
+  }
+  const int units = (int)std::min<int64_t>((ntiles + CTAS - 1) / CTAS, tc::sm_count() / CTAS);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(units * CTAS));
+  cfg.blockDim = dim3(NTHREADS);
+  cfg.dynamicSmemBytes = kWideSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTAS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ma, ms, pa, ps, args);
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+// pairs = true: ma / ms are the B maps with boxes of half the rows
+template <int BM, int MODE, bool NIB = false>
+cudaError_t launch_wide_t(bool pairs, const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
+                          const ScanArgs& args, cudaStream_t st) {
+  return pairs ? launch_wide_c<BM, MODE, NIB, 2>(ma, ms, pa, ps, args, st) : launch_wide_c<BM, MODE, NIB, 1>(ma, ms, pa, ps, args, st);
 }
 
 template <int MODE>
-cudaError_t launch_wide(int bm, const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
+cudaError_t launch_wide(int bm, bool pairs, const CUtensorMap& ma, const CUtensorMap& ms, const CUtensorMap& pa, const CUtensorMap& ps,
                         const ScanArgs& args, cudaStream_t st) {
-  if (args.g.nib) return launch_wide_t<3, MODE, true>(ma, ms, pa, ps, args, st);
+  if (args.g.nib) return launch_wide_t<3, MODE, true>(pairs, ma, ms, pa, ps, args, st);
   switch (bm) {
-    case 0: return launch_wide_t<0, MODE>(ma, ms, pa, ps, args, st);
-    case 1: return launch_wide_t<1, MODE>(ma, ms, pa, ps, args, st);
-    case 2: return launch_wide_t<2, MODE>(ma, ms, pa, ps, args, st);
-    case 3: return launch_wide_t<3, MODE>(ma, ms, pa, ps, args, st);
-    default: return launch_wide_t<4, MODE>(ma, ms, pa, ps, args, st);
+    case 0: return launch_wide_t<0, MODE>(pairs, ma, ms, pa, ps, args, st);
+    case 1: return launch_wide_t<1, MODE>(pairs, ma, ms, pa, ps, args, st);
+    case 2: return launch_wide_t<2, MODE>(pairs, ma, ms, pa, ps, args, st);
+    case 3: return launch_wide_t<3, MODE>(pairs, ma, ms, pa, ps, args, st);
+    default: return launch_wide_t<4, MODE>(pairs, ma, ms, pa, ps, args, st);
   }
 }
 
@@ -927,7 +964,15 @@ int run_pass(const tq_plan* plan, int pass, int nqp, int64_t n, const uint8_t* i
   const bool wide = nqp > kQueriesPerPass;
   TQ_REQUIRE(nqp <= (wide ? W_QPP : kQueriesPerPass) && (!wide || (pass % 2 == 0 && pass + 2 <= kPassesPerGroup)), TQ_ERR_INVALID_ARG,
              "%s: pass %d of %d queries", who, pass, nqp);
-  const uint32_t brows = wide ? W_NCOL : NCOL, prows = wide ? TILE : 2 * TILE;
+  // The wide kernel also runs on CTA pairs (TQ_SCAN_PAIRS=1: M = 256, each CTA loads half of a B box's rows).  Off by
+  // default: the B boxes come from L2 and halving that traffic did not shorten a pass (measured 365 against 358 us per
+  // 32 queries at d = 1536, n = 10^6).
+  static const bool pairs_on = [] {
+    const char* e = std::getenv("TQ_SCAN_PAIRS");
+    return e != nullptr && e[0] == '1';
+  }();
+  const bool pairs = wide && pairs_on && n > TILE;
+  const uint32_t brows = wide ? (pairs ? W_NCOL / 2 : W_NCOL) : NCOL, prows = wide ? TILE : 2 * TILE;
   CUtensorMap ma, ms;
   const uint64_t rows = (uint64_t)kPassesPerGroup * NCOL;
   if (g.kba > 0)
@@ -978,7 +1023,7 @@ int run_pass(const tq_plan* plan, int pass, int nqp, int64_t n, const uint8_t* i
   a.cap = filter ? filter->cap : 0;
   a.run_if = run_if;
   a.status = plan->d_status;
-  if (wide) TQ_CHECK_CUDA(filter ? launch_wide<1>(g.bm, ma, ms, pa, ps, a, st) : launch_wide<0>(g.bm, ma, ms, pa, ps, a, st), who);
+  if (wide) TQ_CHECK_CUDA(filter ? launch_wide<1>(g.bm, pairs, ma, ms, pa, ps, a, st) : launch_wide<0>(g.bm, pairs, ma, ms, pa, ps, a, st), who);
   else TQ_CHECK_CUDA(filter ? launch_bm<1>(g.bm, ma, ms, pa, ps, a, st) : launch_bm<0>(g.bm, ma, ms, pa, ps, a, st), who);
   return TQ_OK;
 }

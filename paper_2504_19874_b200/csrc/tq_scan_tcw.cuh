@@ -22,9 +22,12 @@
 //
 // CTA (one per SM, persistent over tiles), 352 threads as in scan_tc_kernel:
 //   warp 0       TMA producer: per k-block one [192 rows x 128 B] box of B (6 stages); per row group the tile's packed
-//                rows ([128 rows x 32..64 B], 4 stages)
+//                rows ([128 rows x 32..64 B], 4 stages), requested as far ahead as their ring allows
 //   warps 1..2   MMA issuers, k-blocks in turn
 //   warps 3..10  transform + epilogue: set = (warp - 3) / 4, lane quadrant = warp % 4, thread = vector row
+// CTAS = 2 (an option of the launcher): two CTAs of a cluster run in lockstep on their own tiles and share every B
+// box -- each loads half of its rows (no multicast), the leader's issuers run the MMAs with M = 256 (cta_group::2),
+// the commits reach both CTAs' barriers.  It halves the B traffic from L2 and did not shorten a pass.
 // All waits are bounded.
 #pragma once
 
@@ -82,11 +85,14 @@ __device__ __forceinline__ RowGroup row_group(const Geo& g, int gi) {
   return rg;
 }
 
-template <int BM, int MODE, bool NIB>
+template <int BM, int MODE, bool NIB, int CTAS>
 __global__ void __launch_bounds__(NTHREADS, 1)
 scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__ CUtensorMap tmBs,
                 const __grid_constant__ CUtensorMap tmPa, const __grid_constant__ CUtensorMap tmPs, ScanArgs a) {
   if (a.run_if != nullptr && *a.run_if == 0) return;
+  const int rank = CTAS == 2 ? (int)tc::cluster_ctarank() : 0;
+  // a unit = one CTA or one pair of CTAs; in round i unit u's CTA `rank` takes tile (u + i nunits) CTAS + rank
+  const int64_t unit = blockIdx.x / CTAS, nunits = gridDim.x / CTAS;
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -110,10 +116,10 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nkb_total = a.g.kba + a.g.kbs;
   const int ngroups = NIB ? a.g.nblk : ((a.g.kba + 3) >> 2) + ((a.g.kbs + 3) >> 2);
-  const int64_t ntiles = (a.n + TILE - 1) / TILE;
+  const int64_t ntiles = (a.n + TILE - 1) / TILE, nrounds = (ntiles + CTAS - 1) / CTAS;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < W_SLOTS; ++s) tc::mbar_init(&afull[s], 4);
+    for (int s = 0; s < W_SLOTS; ++s) tc::mbar_init(&afull[s], 4 * CTAS);   // the leader's: the owning set of both CTAs
     for (int s = 0; s < W_BSTAGES; ++s) {
       tc::mbar_init(&bfull[s], 1);
       tc::mbar_init(&kdone[s], 1);
@@ -123,7 +129,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
       tc::mbar_init(&pempty[s], 4);
     }
     tc::mbar_init(dfull, N_ISSUERS);
-    tc::mbar_init(dfree, 8);
+    tc::mbar_init(dfree, 8 * CTAS);
     *abort_flag = 0;
     tc::fence_barrier_init();
     if (a.g.kba > 0) tc::tma_prefetch_desc(&tmBa);
@@ -138,9 +144,13 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
     taus[threadIdx.x] = (MODE == 1 && (int)threadIdx.x < a.nqp) ? a.tau[threadIdx.x] : 0.f;
     lcnt[threadIdx.x] = 0;
   }
-  if (warp == 1) tc::tmem_alloc(tmem_slot, TMEM_COLS);
+  if (warp == 1) {
+    if (CTAS == 2) tc::tmem_alloc_pair(tmem_slot, TMEM_COLS);
+    else tc::tmem_alloc(tmem_slot, TMEM_COLS);
+  }
   tc::tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) tc::cluster_sync();   // the partner's barriers exist before anything arrives on them
+  else __syncthreads();
   tc::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -148,22 +158,47 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
       int bst = 0;
-      uint32_t bph = 0, kc = 0, gc = 0;   // k-blocks and row groups issued so far by this CTA
+      uint32_t bph = 0, kc = 0, gc = 0;   // k-blocks and row groups reached so far by this CTA
       bool ok = true;
-      for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+      // The packed rows run ahead of the B boxes as far as their own ring allows: a row group's bytes are wanted by its
+      // set as soon as the set has stored its previous group, several k-blocks before the MMAs free a B stage for it.
+      int64_t prnd = unit;
+      int pgi = 0;
+      uint32_t pgc = 0;                   // row groups whose packed rows have been requested
+      auto load_rows = [&]() {
+        const RowGroup rg = row_group<BM, NIB>(a.g, pgi);
+        const uint32_t pst = pgc & (W_PSTAGES - 1);
+        tc::mbar_arrive_expect_tx(&pfull[pst], (uint32_t)(TILE * rg.bytes));
+        tc::tma_load_2d(pring + pst * W_PTILE, rg.from_qjl ? &tmPs : &tmPa, &pfull[pst], rg.x, (int)((prnd * CTAS + rank) * TILE));
+        ++pgc;
+        if (++pgi == ngroups) {
+          pgi = 0;
+          prnd += nunits;
+        }
+      };
+      for (int64_t rnd = unit; rnd < nrounds && ok; rnd += nunits) {   // a tile past the last one (odd count) reads zeros
         for (int gi = 0; gi < ngroups && ok; ++gi, ++gc) {
           const RowGroup rg = row_group<BM, NIB>(a.g, gi);
-          const uint32_t pst = gc & (W_PSTAGES - 1), pph = (gc / W_PSTAGES) & 1u;
-          if (!(ok = tc::mbar_wait(&pempty[pst], pph ^ 1u, abort_flag, a.status))) break;
-          tc::mbar_arrive_expect_tx(&pfull[pst], (uint32_t)(TILE * rg.bytes));
-          tc::tma_load_2d(pring + pst * W_PTILE, rg.from_qjl ? &tmPs : &tmPa, &pfull[pst], rg.x, (int)(tile * TILE));
+          while (pgc <= gc) {   // this group's rows at the latest now
+            if (!(ok = tc::mbar_wait(&pempty[pgc & (W_PSTAGES - 1)], ((pgc / W_PSTAGES) & 1u) ^ 1u, abort_flag, a.status))) break;
+            load_rows();
+          }
+          if (!ok) break;
           for (int j = 0; j < rg.cnt; ++j, ++kc) {
+            // one more row group ahead when its stage is free (a test, not a wait)
+            if (prnd < nrounds && tc::mbar_test_wait(&pempty[pgc & (W_PSTAGES - 1)], ((pgc / W_PSTAGES) & 1u) ^ 1u)) load_rows();
             const int f = rg.f0 + j;
             const int kb = rg.part_s ? f - a.g.kba : f;
             // B stage kc % W_BSTAGES was last read by the MMAs of k-block kc - W_BSTAGES
             if (kc >= W_BSTAGES && !(ok = tc::mbar_wait(&kdone[bst], bph ^ 1u, abort_flag, a.status))) break;
-            tc::mbar_arrive_expect_tx(&bfull[bst], W_BTILE);
-            tc::tma_load_2d(bring + bst * W_BTILE, rg.part_s ? &tmBs : &tmBa, &bfull[bst], kb * KB_BYTES, a.pass * NCOL);
+            if (CTAS == 2) {   // each CTA loads half of the box's rows; the bytes of both are counted on the leader's barrier
+              if (rank == 0) tc::mbar_arrive_expect_tx(&bfull[bst], W_BTILE);
+              tc::tma_load_2d_pair(bring + bst * W_BTILE, rg.part_s ? &tmBs : &tmBa, &bfull[bst], kb * KB_BYTES,
+                                   a.pass * NCOL + rank * (W_NCOL / 2));
+            } else {
+              tc::mbar_arrive_expect_tx(&bfull[bst], W_BTILE);
+              tc::tma_load_2d(bring + bst * W_BTILE, rg.part_s ? &tmBs : &tmBa, &bfull[bst], kb * KB_BYTES, a.pass * NCOL);
+            }
             if (++bst == W_BSTAGES) {
               bst = 0;
               bph ^= 1u;
@@ -178,15 +213,15 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
     __syncwarp();
   } else if (warp <= N_ISSUERS) {
     // ---------------------------------------------------------------- MMA issuers
-    if (lane == 0) {
-      constexpr uint32_t idesc = idesc_i8(TILE, W_NCOL);
+    if (lane == 0 && rank == 0) {   // the leader's threads issue for both CTAs of a pair (M = 256)
+      constexpr uint32_t idesc = idesc_i8(TILE * CTAS, W_NCOL);
       const int me = warp - 1;
       bool ok = true;
       uint32_t kc = 0, it = 0;
       int turn = 0;
       const uint64_t bdesc0 = tc::smem_desc_sw128(tc::smem_u32(bring));
-      for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
-        // both sets have read the previous tile's accumulators and zeroed them
+      for (int64_t rnd = unit; rnd < nrounds && ok; rnd += nunits, ++it) {
+        // both sets (of both CTAs) have read the previous tile's accumulators and zeroed them
         if (!(ok = tc::mbar_wait(dfree, it & 1u, abort_flag, a.status))) break;
         for (int f = 0; f < nkb_total; ++f, ++kc) {
           const bool mine = turn == me;
@@ -198,16 +233,23 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
           tc::tc_fence_after();
           const int kind = NIB ? f % 3 : 0;   // nibble layout: h bytes (signed A), l bytes, sign bits (second accumulator)
           const bool part_s = NIB ? kind == 2 : f >= a.g.kba;
-          const uint32_t idesc_f = (NIB && kind == 0) ? idesc_i8(TILE, W_NCOL, true) : idesc;
+          const uint32_t idesc_f = (NIB && kind == 0) ? idesc_i8(TILE * CTAS, W_NCOL, true) : idesc;
           const uint64_t bdesc = bdesc0 + (uint64_t)(bst * (W_BTILE >> 4));
           const uint32_t a_tmem = tmem_base + (uint32_t)(W_ACOL0 + slot * 32);
           const uint32_t d_tmem = tmem_base + (uint32_t)(part_s ? W_NCOL : 0);
 #pragma unroll
-          for (int step = 0; step < 4; ++step)   // 32 K-bytes per MMA: 8 TMEM columns of A, +32 bytes inside B's swizzled row
-            umma_i8_ts(d_tmem, a_tmem + 8 * step, bdesc + 2 * step, idesc_f, 1u);
-          tc::umma_commit(&kdone[bst]);   // A slot and B stage reusable once these MMAs have read them
+          for (int step = 0; step < 4; ++step) {   // 32 K-bytes per MMA: 8 TMEM columns of A, +32 bytes inside B's swizzled row
+            if (CTAS == 2) umma_i8_ts_pair(d_tmem, a_tmem + 8 * step, bdesc + 2 * step, idesc_f, 1u);
+            else umma_i8_ts(d_tmem, a_tmem + 8 * step, bdesc + 2 * step, idesc_f, 1u);
+          }
+          // A slot and B stage (of both CTAs) reusable once these MMAs have read them
+          if (CTAS == 2) tc::umma_commit_pair(&kdone[bst]);
+          else tc::umma_commit(&kdone[bst]);
         }
-        if (ok) tc::umma_commit(dfull);   // all MMAs this thread issued for the tile
+        if (ok) {   // all MMAs this thread issued for the tile
+          if (CTAS == 2) tc::umma_commit_pair(dfull);
+          else tc::umma_commit(dfull);
+        }
       }
     }
     __syncwarp();
@@ -228,13 +270,14 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
       const int64_t rw = tl * TILE + r;
       return (rw < a.n && (a.g.kbs > 0 || NIB)) ? a.coef * __ldg(a.gamma + rw) : 0.f;
     };
-    float nu_next = load_nu(blockIdx.x), gm_next = load_gm(blockIdx.x);
-    for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
+    float nu_next = load_nu(unit * CTAS + rank), gm_next = load_gm(unit * CTAS + rank);
+    for (int64_t rnd = unit; rnd < nrounds && ok; rnd += nunits, ++it) {
+      const int64_t tile = rnd * CTAS + rank;
       const int64_t row = tile * TILE + r;
       const bool row_ok = row < a.n;
       const float nu = nu_next, gm = gm_next;
-      nu_next = load_nu(tile + gridDim.x);
-      gm_next = load_gm(tile + gridDim.x);
+      nu_next = load_nu(tile + nunits * CTAS);
+      gm_next = load_gm(tile + nunits * CTAS);
 
       // this thread's columns of both accumulators start from zero (its own epilogue of the previous tile has read them)
 #pragma unroll
@@ -245,7 +288,10 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
       tc::tmem_st_wait();
       tc::tc_fence_before();
       __syncwarp();
-      if (lane == 0) tc::mbar_arrive(dfree);
+      if (lane == 0) {
+        if (CTAS == 2) tc::mbar_arrive_leader(dfree);
+        else tc::mbar_arrive(dfree);
+      }
 
       const uint32_t kt0 = it * (uint32_t)nkb_total;   // this tile's first k-block in the CTA's count
       // stores k-block kt's 32 A registers of this row into slot kt % W_SLOTS and announces it
@@ -260,7 +306,10 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
         tc::tmem_st_wait();
         tc::tc_fence_before();
         __syncwarp();
-        if (lane == 0) tc::mbar_arrive(&afull[slot]);
+        if (lane == 0) {
+          if (CTAS == 2) tc::mbar_arrive_leader(&afull[slot]);
+          else tc::mbar_arrive(&afull[slot]);
+        }
         return true;
       };
       // expands one k-block's words of the bit streams into the row's 128 bytes of A
@@ -421,10 +470,12 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
   }
 
   tc::tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) tc::cluster_sync();   // neither CTA leaves while the partner may still arrive on its barriers
+  else __syncthreads();
   if (warp == 1) {
     tc::tc_fence_after();
-    tc::tmem_dealloc(tmem_base, TMEM_COLS);
+    if (CTAS == 2) tc::tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    else tc::tmem_dealloc(tmem_base, TMEM_COLS);
   }
   if (MODE == 1 && warp > N_ISSUERS) {   // the eight transform warps append eight queries' collected pairs each
     for (int ql = (warp - 1 - N_ISSUERS) * 8; ql < (warp - N_ISSUERS) * 8; ++ql) {

@@ -153,3 +153,53 @@ def test_topk_adversarial_order_descending_scores():
     ts, ti = su.topk(Q, n, *codes, k)
     want = np.lexsort((np.arange(n), -sc[0].cpu().numpy().astype(np.float64)))[:k]
     assert np.array_equal(ti[0].cpu().numpy(), want)
+
+
+_KERNEL_FORM_CHILD = r"""
+import sys
+import torch
+sys.path.insert(0, sys.argv[1])
+import paper_2504_19874_b200 as tq
+from tests import parity as P
+blob = torch.load(sys.argv[2])
+for case in blob["cases"]:
+    su = P.Setup(case["d"], case["bits"], case["mode"], layout=case["layout"])
+    codes = tuple(None if t is None else t.to("cuda:0") for t in case["codes"])
+    Q = case["Q"].to("cuda:0")
+    n = case["n"]
+    sc = su.score(Q, n, *codes)
+    assert torch.equal(sc.cpu(), case["scores"]), "dense scores differ"
+    ts, ti = su.topk(Q, n, *codes, case["k"])
+    assert torch.equal(ts.cpu(), case["top_scores"]) and torch.equal(ti.cpu(), case["top_ids"]), "top-k differs"
+print("kernel form ok")
+"""
+
+
+@pytest.mark.parametrize("env", [{"TQ_SCAN_WIDE": "0"}, {"TQ_SCAN_PAIRS": "1"}])
+def test_other_forms_of_the_many_query_kernel_give_the_same_estimates(env, tmp_path):
+    """Calls of more than 32 queries run the wide tcgen05 kernel (64 queries per pass, one CTA per tile).  TQ_SCAN_WIDE=0
+    keeps the 32-query kernel and TQ_SCAN_PAIRS=1 runs the wide kernel on CTA pairs (both read once per process): the
+    same integers, so dense estimates and top-k must be bit-identical.  Sizes: an odd number of 128-vector tiles with a
+    ragged tail, 70 queries (a full pass and a short one), and one thresholded top-k (n >= 65,536)."""
+    import os
+    import subprocess
+    import sys
+    cases = []
+    for d, bits, mode, layout, n, k in ((1536, 4, tq.TQ_PROD, tq.TQ_LAYOUT_NIBBLE, 1300, 20), (264, 4, tq.TQ_PROD, None, 1300, 20),
+                                        (520, 3, tq.TQ_MSE, None, 1300, 20), (200, 3, tq.TQ_PROD, None, 66000, 10)):
+        su = P.Setup(d, bits, mode, layout=layout)
+        X, Q = _data(d, n, 70, 7 * d + bits)
+        codes = su.quantize(X)
+        sc = su.score(Q, n, *codes)
+        if n <= 2000:
+            P.check_scores(su, sc, Q, *codes)
+        ts, ti = su.topk(Q, n, *codes, k)
+        cases.append({"d": d, "bits": bits, "mode": mode, "layout": layout, "n": n, "k": k, "Q": Q.cpu(),
+                      "codes": tuple(None if t is None else t.cpu() for t in codes), "scores": sc.cpu(),
+                      "top_scores": ts.cpu(), "top_ids": ti.cpu()})
+    blob = tmp_path / "scan_forms.pt"
+    torch.save({"cases": cases}, blob)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", _KERNEL_FORM_CHILD, root, str(blob)], env=dict(os.environ, **env),
+                       capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0 and "kernel form ok" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
