@@ -292,9 +292,93 @@ __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __rest
   }
 }
 
+// Many queries: the same sums in the same order (a lane adds its products over ascending columns 4 lane + 128 i in
+// fp32, the 32 partial sums are added in fp64 by the same butterfly), so a query's rotated form does not depend on
+// which kernel formed it -- but a warp holds eight matrix rows against the eight staged queries, and a CTA 64 rows:
+// the queries are read once per 64 output columns instead of once per 8, and 64 FMAs follow every pair of loads.
+constexpr int kRmRows = 8, kRmChunk = 256, kRmRowsPerBlock = 8 * kRmRows;
+constexpr int kRotManyFrom = 64;   // queries from which the blocked kernel is used (d a multiple of 4)
+
+template <typename T>
+__global__ void __launch_bounds__(256) rotate_many_kernel(const float* __restrict__ Rot, int nrows, int d,
+                                                          const T* __restrict__ Q, int64_t ldq, int nq,
+                                                          float* __restrict__ Qcat, int64_t ldo) {
+  __shared__ __align__(16) float qs[kRotQ][kRmChunk];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int j0 = blockIdx.x * kRmRowsPerBlock + warp * kRmRows;
+  const int q_begin = blockIdx.y * kRotQPerBlock, q_end = min(nq, q_begin + kRotQPerBlock);
+  for (int q0 = q_begin; q0 < q_end; q0 += kRotQ) {
+    float acc[kRmRows][kRotQ];
+#pragma unroll
+    for (int rr = 0; rr < kRmRows; ++rr)
+#pragma unroll
+      for (int qq = 0; qq < kRotQ; ++qq) acc[rr][qq] = 0.f;
+    const int nact = min(kRotQ, q_end - q0);
+    for (int c0 = 0; c0 < d; c0 += kRmChunk) {
+      const int len = min(kRmChunk, d - c0);
+      float4 r[kRmRows][kRmChunk / 128];
+#pragma unroll
+      for (int rr = 0; rr < kRmRows; ++rr) {
+        const float4* row4 = reinterpret_cast<const float4*>(Rot + (size_t)min(j0 + rr, nrows - 1) * d + c0);
+#pragma unroll
+        for (int i = 0; i < kRmChunk / 128; ++i) {
+          const int c4 = lane + 32 * i;
+          r[rr][i] = (4 * c4 < len) ? __ldg(row4 + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+      __syncthreads();
+      for (int e = threadIdx.x; e < nact * (kRmChunk / 4); e += blockDim.x) {
+        const int qq = e / (kRmChunk / 4), c = 4 * (e % (kRmChunk / 4));
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        if (c < len) {
+          const T* src = Q + (int64_t)(q0 + qq) * ldq + c0 + c;
+#pragma unroll
+          for (int t = 0; t < 4; ++t)
+            if (c + t < len) v[t] = scan::to_f32<T>(src[t]);
+        }
+        *reinterpret_cast<float4*>(&qs[qq][c]) = make_float4(v[0], v[1], v[2], v[3]);
+      }
+      __syncthreads();
+#pragma unroll
+      for (int i = 0; i < kRmChunk / 128; ++i) {
+        const int c4 = lane + 32 * i;
+        if (4 * c4 < len) {
+#pragma unroll
+          for (int qq = 0; qq < kRotQ; ++qq) {
+            if (qq < nact) {
+              const float4 v = *reinterpret_cast<const float4*>(&qs[qq][4 * c4]);
+#pragma unroll
+              for (int rr = 0; rr < kRmRows; ++rr)
+                acc[rr][qq] = fmaf(r[rr][i].x, v.x, fmaf(r[rr][i].y, v.y, fmaf(r[rr][i].z, v.z, fmaf(r[rr][i].w, v.w, acc[rr][qq]))));
+            }
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int rr = 0; rr < kRmRows; ++rr) {
+#pragma unroll
+      for (int qq = 0; qq < kRotQ; ++qq) {
+        if (qq >= nact) break;
+        double v = (double)acc[rr][qq];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0 && j0 + rr < nrows) Qcat[(int64_t)(q0 + qq) * ldo + j0 + rr] = (float)v;
+      }
+    }
+  }
+}
+
 template <typename T>
 cudaError_t launch_rotate_queries(const tq_plan* plan, const T* Q, int64_t ldq, int nq, float* Qcat, cudaStream_t st) {
   const int ncols = plan->ncat * plan->dpad;
+  if (nq >= kRotManyFrom && (plan->d & 3) == 0) {
+    const dim3 grid((unsigned)((ncols + kRmRowsPerBlock - 1) / kRmRowsPerBlock), (unsigned)((nq + kRotQPerBlock - 1) / kRotQPerBlock));
+    rotate_many_kernel<T><<<grid, 256, 0, st>>>(plan->dRotCat, ncols, plan->d, Q, ldq, nq, Qcat, ncols);
+    count_launches(1);
+    return cudaGetLastError();
+  }
   constexpr int smem = kRotQ * kRotChunk * (int)sizeof(float);
   // function attributes are per device: remember the devices this launcher has prepared
   static std::atomic<unsigned long long> attr_devices{0};   // written by any thread that launches
@@ -316,8 +400,8 @@ cudaError_t prepare_queries(const tq_plan* plan, const void* Q, int q_dtype, int
                             cudaStream_t st) {
   const int ncols = plan->ncat * plan->dpad;
   (void)ncols;
-  // One kernel for every query count, so that a query's rotated form (and hence its estimates) does not
-  // depend on how many other queries came with it.
+  // Both kernels add the same products in the same order, so that a query's rotated form (and hence its
+  // estimates) does not depend on how many other queries came with it.
   if (q_dtype == TQ_F32) return launch_rotate_queries(plan, static_cast<const float*>(Q), ldq, nq, Qcat, st);
   return launch_rotate_queries(plan, static_cast<const __nv_bfloat16*>(Q), ldq, nq, Qcat, st);
 }
