@@ -294,16 +294,18 @@ __global__ void __launch_bounds__(256) rotate_queries_kernel(const float* __rest
 
 // Many queries: the same sums in the same order (a lane adds its products over ascending columns 4 lane + 128 i in
 // fp32, the 32 partial sums are added in fp64 by the same butterfly), so a query's rotated form does not depend on
-// which kernel formed it -- but a warp holds eight matrix rows against the eight staged queries, and a CTA 64 rows:
-// the queries are read once per 64 output columns instead of once per 8, and 64 FMAs follow every pair of loads.
-constexpr int kRmRows = 8, kRmChunk = 256, kRmRowsPerBlock = 8 * kRmRows;
+// which kernel formed it -- but a warp holds eight matrix rows against the eight staged queries (64 FMAs per pair of
+// 16-byte loads), a CTA of four warps 32 rows, and the queries are read once per 32 output columns instead of once
+// per 8.  Three CTAs per SM hide each other's staging.
+constexpr int kRmRows = 8, kRmWarps = 4, kRmRowsPerBlock = kRmWarps * kRmRows;
 constexpr int kRotManyFrom = 64;   // queries from which the blocked kernel is used (d a multiple of 4)
 
 template <typename T>
-__global__ void __launch_bounds__(256) rotate_many_kernel(const float* __restrict__ Rot, int nrows, int d,
-                                                          const T* __restrict__ Q, int64_t ldq, int nq,
-                                                          float* __restrict__ Qcat, int64_t ldo) {
-  __shared__ __align__(16) float qs[kRotQ][kRmChunk];
+__global__ void __launch_bounds__(32 * kRmWarps) rotate_many_kernel(const float* __restrict__ Rot, int nrows, int d,
+                                                                    const T* __restrict__ Q, int64_t ldq, int nq,
+                                                                    float* __restrict__ Qcat, int64_t ldo) {
+  extern __shared__ __align__(16) float qs_raw[];
+  float (*qs)[kRotChunk] = reinterpret_cast<float (*)[kRotChunk]>(qs_raw);
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int j0 = blockIdx.x * kRmRowsPerBlock + warp * kRmRows;
@@ -315,57 +317,63 @@ __global__ void __launch_bounds__(256) rotate_many_kernel(const float* __restric
 #pragma unroll
       for (int qq = 0; qq < kRotQ; ++qq) acc[rr][qq] = 0.f;
     const int nact = min(kRotQ, q_end - q0);
-    for (int c0 = 0; c0 < d; c0 += kRmChunk) {
-      const int len = min(kRmChunk, d - c0);
-      float4 r[kRmRows][kRmChunk / 128];
-#pragma unroll
-      for (int rr = 0; rr < kRmRows; ++rr) {
-        const float4* row4 = reinterpret_cast<const float4*>(Rot + (size_t)min(j0 + rr, nrows - 1) * d + c0);
-#pragma unroll
-        for (int i = 0; i < kRmChunk / 128; ++i) {
-          const int c4 = lane + 32 * i;
-          r[rr][i] = (4 * c4 < len) ? __ldg(row4 + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-      }
+    for (int c0 = 0; c0 < d; c0 += kRotChunk) {
+      const int len = min(kRotChunk, d - c0);
       __syncthreads();
-      for (int e = threadIdx.x; e < nact * (kRmChunk / 4); e += blockDim.x) {
-        const int qq = e / (kRmChunk / 4), c = 4 * (e % (kRmChunk / 4));
-        float v[4] = {0.f, 0.f, 0.f, 0.f};
-        if (c < len) {
-          const T* src = Q + (int64_t)(q0 + qq) * ldq + c0 + c;
+      for (int e = threadIdx.x; e < nact * (kRotChunk / 4); e += blockDim.x) {
+        const int qq = e / (kRotChunk / 4), c = 4 * (e % (kRotChunk / 4));
+        if (c >= len) continue;   // columns past the chunk's end are not read below
+        const T* src = Q + (int64_t)(q0 + qq) * ldq + c0 + c;
+        float v[4];
 #pragma unroll
-          for (int t = 0; t < 4; ++t)
-            if (c + t < len) v[t] = scan::to_f32<T>(src[t]);
-        }
+        for (int t = 0; t < 4; ++t) v[t] = scan::to_f32<T>(src[t]);   // d is a multiple of 4: whole groups of four
         *reinterpret_cast<float4*>(&qs[qq][c]) = make_float4(v[0], v[1], v[2], v[3]);
       }
       __syncthreads();
-#pragma unroll
-      for (int i = 0; i < kRmChunk / 128; ++i) {
+#pragma unroll 2
+      for (int i = 0; i < kRotChunk / 128; ++i) {
         const int c4 = lane + 32 * i;
-        if (4 * c4 < len) {
+        if (4 * c4 >= len) break;
+        float4 r[kRmRows];
 #pragma unroll
-          for (int qq = 0; qq < kRotQ; ++qq) {
-            if (qq < nact) {
-              const float4 v = *reinterpret_cast<const float4*>(&qs[qq][4 * c4]);
+        for (int rr = 0; rr < kRmRows; ++rr)
+          r[rr] = __ldg(reinterpret_cast<const float4*>(Rot + (size_t)min(j0 + rr, nrows - 1) * d + c0) + c4);
 #pragma unroll
-              for (int rr = 0; rr < kRmRows; ++rr)
-                acc[rr][qq] = fmaf(r[rr][i].x, v.x, fmaf(r[rr][i].y, v.y, fmaf(r[rr][i].z, v.z, fmaf(r[rr][i].w, v.w, acc[rr][qq]))));
-            }
+        for (int qq = 0; qq < kRotQ; ++qq) {
+          if (qq < nact) {
+            const float4 v = *reinterpret_cast<const float4*>(&qs[qq][4 * c4]);
+#pragma unroll
+            for (int rr = 0; rr < kRmRows; ++rr)
+              acc[rr][qq] = fmaf(r[rr].x, v.x, fmaf(r[rr].y, v.y, fmaf(r[rr].z, v.z, fmaf(r[rr].w, v.w, acc[rr][qq]))));
           }
         }
       }
     }
+    // The 32 partial sums of each of the warp's 64 outputs are added in fp64 along the tree of the xor butterfly
+    // (lanes l and l ^ 16, then ^ 8, 4, 2, 1: every lane of the butterfly ends with the same bits, additions being
+    // commutative), but transposed: at each level a lane keeps half of its values and hands the other half to its
+    // partner, so that 62 fp64 additions per lane do what 320 would; lane l ends with outputs 2 l and 2 l + 1.
+    static_assert(kRmRows * kRotQ == 64, "the transposed reduction is written for 64 outputs per warp");
+    const bool b4 = (lane & 16) != 0, b3 = (lane & 8) != 0, b2 = (lane & 4) != 0, b1 = (lane & 2) != 0, b0 = (lane & 1) != 0;
+    double w1[32], w2[16], w3[8], w4[4], w5[2];
 #pragma unroll
-    for (int rr = 0; rr < kRmRows; ++rr) {
+    for (int k = 0; k < 32; ++k) {
+      const float lo = acc[k / kRotQ][k % kRotQ], hi = acc[(k + 32) / kRotQ][k % kRotQ];
+      const float got = __shfl_xor_sync(0xffffffffu, b4 ? lo : hi, 16);
+      w1[k] = (double)(b4 ? hi : lo) + (double)got;
+    }
 #pragma unroll
-      for (int qq = 0; qq < kRotQ; ++qq) {
-        if (qq >= nact) break;
-        double v = (double)acc[rr][qq];
+    for (int k = 0; k < 16; ++k) w2[k] = (b3 ? w1[k + 16] : w1[k]) + __shfl_xor_sync(0xffffffffu, b3 ? w1[k] : w1[k + 16], 8);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0 && j0 + rr < nrows) Qcat[(int64_t)(q0 + qq) * ldo + j0 + rr] = (float)v;
-      }
+    for (int k = 0; k < 8; ++k) w3[k] = (b2 ? w2[k + 8] : w2[k]) + __shfl_xor_sync(0xffffffffu, b2 ? w2[k] : w2[k + 8], 4);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) w4[k] = (b1 ? w3[k + 4] : w3[k]) + __shfl_xor_sync(0xffffffffu, b1 ? w3[k] : w3[k + 4], 2);
+#pragma unroll
+    for (int k = 0; k < 2; ++k) w5[k] = (b0 ? w4[k + 2] : w4[k]) + __shfl_xor_sync(0xffffffffu, b0 ? w4[k] : w4[k + 2], 1);
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int idx = 2 * lane + k, rr = idx / kRotQ, qq = idx % kRotQ;
+      if (qq < nact && j0 + rr < nrows) Qcat[(int64_t)(q0 + qq) * ldo + j0 + rr] = (float)w5[k];
     }
   }
 }
@@ -373,12 +381,6 @@ __global__ void __launch_bounds__(256) rotate_many_kernel(const float* __restric
 template <typename T>
 cudaError_t launch_rotate_queries(const tq_plan* plan, const T* Q, int64_t ldq, int nq, float* Qcat, cudaStream_t st) {
   const int ncols = plan->ncat * plan->dpad;
-  if (nq >= kRotManyFrom && (plan->d & 3) == 0) {
-    const dim3 grid((unsigned)((ncols + kRmRowsPerBlock - 1) / kRmRowsPerBlock), (unsigned)((nq + kRotQPerBlock - 1) / kRotQPerBlock));
-    rotate_many_kernel<T><<<grid, 256, 0, st>>>(plan->dRotCat, ncols, plan->d, Q, ldq, nq, Qcat, ncols);
-    count_launches(1);
-    return cudaGetLastError();
-  }
   constexpr int smem = kRotQ * kRotChunk * (int)sizeof(float);
   // function attributes are per device: remember the devices this launcher has prepared
   static std::atomic<unsigned long long> attr_devices{0};   // written by any thread that launches
@@ -388,6 +390,18 @@ cudaError_t launch_rotate_queries(const tq_plan* plan, const T* Q, int64_t ldq, 
     cudaError_t e = cudaFuncSetAttribute(rotate_queries_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     if (attr_dev < 64) attr_devices.fetch_or(1ull << attr_dev, std::memory_order_relaxed);
+  }
+  if (nq >= kRotManyFrom && (plan->d & 3) == 0) {
+    static std::atomic<unsigned long long> many_devices{0};
+    if (attr_dev >= 64 || !((many_devices.load(std::memory_order_relaxed) >> attr_dev) & 1ull)) {
+      cudaError_t e = cudaFuncSetAttribute(rotate_many_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      if (e != cudaSuccess) return e;
+      if (attr_dev < 64) many_devices.fetch_or(1ull << attr_dev, std::memory_order_relaxed);
+    }
+    const dim3 grid((unsigned)((ncols + kRmRowsPerBlock - 1) / kRmRowsPerBlock), (unsigned)((nq + kRotQPerBlock - 1) / kRotQPerBlock));
+    rotate_many_kernel<T><<<grid, 32 * kRmWarps, smem, st>>>(plan->dRotCat, ncols, plan->d, Q, ldq, nq, Qcat, ncols);
+    count_launches(1);
+    return cudaGetLastError();
   }
   const dim3 grid((unsigned)((ncols + 7) / 8), (unsigned)((nq + kRotQPerBlock - 1) / kRotQPerBlock));
   rotate_queries_kernel<T><<<grid, 256, smem, st>>>(plan->dRotCat, ncols, plan->d, Q, ldq, nq, Qcat, ncols);
