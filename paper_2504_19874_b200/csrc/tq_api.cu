@@ -125,7 +125,7 @@ ScanEngine pick_engine(const tq_plan* plan, int nq) {
   e.tc = nq >= tc_from && tscan::available(plan);
   e.nib = e.nib && !e.tc;
   e.qpp = e.tc ? tscan::queries_per_pass(nq) : e.nib ? nscan::queries_per_pass(plan, nq) : mscan::queries_per_pass(plan, nq);
-  e.dense_rows_pref = e.tc ? (1 << 18) : (1 << 20);
+  e.dense_rows_pref = 1 << 20;   // n = 10^6: the guarded rescue is one scan + one selection launch per pass
   e.ws_bytes = e.tc ? tscan::workspace_bytes(plan) : e.nib ? nscan::workspace_bytes(plan) : mscan::workspace_bytes(plan);
   return e;
 }

@@ -270,16 +270,9 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
       const int64_t rw = tl * TILE + r;
       return (rw < a.n && (a.g.kbs > 0 || NIB)) ? a.coef * __ldg(a.gamma + rw) : 0.f;
     };
-    float nu_next = load_nu(unit * CTAS + rank), gm_next = load_gm(unit * CTAS + rank);
-    for (int64_t rnd = unit; rnd < nrounds && ok; rnd += nunits, ++it) {
-      const int64_t tile = rnd * CTAS + rank;
-      const int64_t row = tile * TILE + r;
-      const bool row_ok = row < a.n;
-      const float nu = nu_next, gm = gm_next;
-      nu_next = load_nu(tile + nunits * CTAS);
-      gm_next = load_gm(tile + nunits * CTAS);
-
-      // this thread's columns of both accumulators start from zero (its own epilogue of the previous tile has read them)
+    // zeroes this thread's columns of both accumulators and tells the issuers (before the first tile, and in every
+    // epilogue as soon as the columns have been read into registers)
+    auto release_accumulators = [&]() {
 #pragma unroll
       for (int c = 0; c < NCOL; c += 16) {
         tc::tmem_fill16(lane_addr + (uint32_t)(NCOL * set + c), 0u);
@@ -292,6 +285,16 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
         if (CTAS == 2) tc::mbar_arrive_leader(dfree);
         else tc::mbar_arrive(dfree);
       }
+    };
+    release_accumulators();
+    float nu_next = load_nu(unit * CTAS + rank), gm_next = load_gm(unit * CTAS + rank);
+    for (int64_t rnd = unit; rnd < nrounds && ok; rnd += nunits, ++it) {
+      const int64_t tile = rnd * CTAS + rank;
+      const int64_t row = tile * TILE + r;
+      const bool row_ok = row < a.n;
+      const float nu = nu_next, gm = gm_next;
+      nu_next = load_nu(tile + nunits * CTAS);
+      gm_next = load_gm(tile + nunits * CTAS);
 
       const uint32_t kt0 = it * (uint32_t)nkb_total;   // this tile's first k-block in the CTA's count
       // stores k-block kt's 32 A registers of this row into slot kt % W_SLOTS and announces it
@@ -421,9 +424,11 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
       if (!(ok = tc::mbar_wait(dfull, it & 1u, abort_flag, a.status))) break;
       tc::tc_fence_after();
       const uint32_t taddr = lane_addr + (uint32_t)(NCOL * set);
+      // halves of 16 queries; a short last pass: columns of absent queries are not read
+      const int nh = min(2, max(0, (a.nqp - 32 * set + 15) >> 4));
+      if (nh == 0) release_accumulators();
 #pragma unroll 1
-      for (int h = 0; h < 2; ++h) {   // 16 queries per half: digit l of query 32 set + 16 h + qq sits in column 96 set + 32 l + 16 h + qq
-        if (32 * set + h * 16 >= a.nqp) break;   // a short last pass: columns of absent queries are not read
+      for (int h = 0; h < nh; ++h) {   // digit l of query 32 set + 16 h + qq sits in column 96 set + 32 l + 16 h + qq
         uint32_t va[LIMBS][16], vs[LIMBS][16];
 #pragma unroll
         for (int l = 0; l < LIMBS; ++l) {
@@ -431,6 +436,8 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
           if (a.g.kbs > 0 || NIB) tc::tmem_ld16(taddr + W_NCOL + l * 32 + h * 16, vs[l]);
         }
         tc::tmem_ld_wait();
+        // the last columns are in registers: the next tile's MMAs may start while their estimates are formed
+        if (h == nh - 1) release_accumulators();
 #pragma unroll
         for (int qq = 0; qq < 16; ++qq) {
           const int ql = 32 * set + h * 16 + qq;
