@@ -203,3 +203,58 @@ def test_other_forms_of_the_many_query_kernel_give_the_same_estimates(env, tmp_p
     r = subprocess.run([sys.executable, "-c", _KERNEL_FORM_CHILD, root, str(blob)], env=dict(os.environ, **env),
                        capture_output=True, text=True, timeout=900)
     assert r.returncode == 0 and "kernel form ok" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+@pytest.mark.parametrize("nq", [33, 48, 49, 64, 65, 97])
+@pytest.mark.parametrize("n", [1, 127, 129, 1153])
+def test_wide_many_query_kernel_query_counts_and_ragged_tiles(nq, n):
+    """More than 32 queries take the 64-query kernel: one query in the second half of a pass (33), a half-filled and a
+    just-over-half second set (48, 49), a full pass (64), a full pass plus a 32-query-kernel pass of one (65) and 64 + 33
+    (97); a single row, one ragged tile, one tile plus one row, and an odd number of tiles with a ragged tail.  Every
+    query's row must equal what the few-query engine gives for it alone, and everything must match the oracle."""
+    d = 264
+    su = P.Setup(d, 4, tq.TQ_PROD)
+    X, Q = _data(d, n, nq, 13 * nq + n)
+    codes = su.quantize(X)
+    sc = su.score(Q, n, *codes)
+    P.check_scores(su, sc, Q, *codes)
+    for q in (0, 31, 32, nq - 1):
+        one = su.score(Q[q:q + 1].contiguous(), n, *codes)
+        assert torch.equal(one[0], sc[q])
+    k = min(n, 9)
+    ts, ti = su.topk(Q, n, *codes, k)
+    for q in (0, 32, nq - 1):
+        vals, order = torch.sort(sc[q], descending=True, stable=True)
+        assert torch.equal(ti[q].long(), order[:k]) and torch.equal(ts[q], vals[:k])
+
+
+def test_wide_kernel_topk_overflow_rescue_and_adversarial_order():
+    """The two hard top-k flows with 40 queries (the 64-query kernel in filter mode).  All vectors identical: every
+    score ties, each CTA's shared-memory list and then the global candidate list overflow, and the guarded rescue pass
+    must return the k smallest ids.  Best vectors last: the pilot threshold is weak and the filter admits many pairs."""
+    d = 128
+    su = P.Setup(d, 2, tq.TQ_MSE)
+    n, k, nq = 66000, 50, 40
+    row = torch.randn((1, d), generator=torch.Generator().manual_seed(3))
+    X = row.expand(n, d).contiguous().to(DEV)
+    Q = torch.randn((nq, d), generator=torch.Generator().manual_seed(4)).to(DEV)
+    codes = su.quantize(X)
+    ts, ti = su.topk(Q, n, *codes, k)
+    assert torch.equal(ti, torch.arange(k, dtype=torch.int32, device=DEV).expand(nq, k))
+    sc = su.score(Q, n, *codes)
+    assert torch.equal(ts, sc[:, :k])
+
+    cfg = wl.CONFIGS["c2"]
+    su = P.Setup(cfg.d, 3, tq.TQ_PROD, cfg.pi_seed, cfg.s_seed)
+    n, k = 66049, 64
+    X = wl.database(cfg, n, device=DEV)
+    Q = wl.queries(cfg, nq, device=DEV)
+    order = torch.argsort(X @ Q[:8].mean(dim=0))     # ascending inner product with the first queries' mean
+    X = X[order].contiguous()
+    codes = su.quantize(X)
+    sc = su.score(Q, n, *codes)
+    ts, ti = su.topk(Q, n, *codes, k)
+    for q in (0, 7, 33, nq - 1):
+        want = np.lexsort((np.arange(n), -sc[q].cpu().numpy().astype(np.float64)))[:k]
+        assert np.array_equal(ti[q].cpu().numpy(), want)
+        assert torch.equal(ts[q], sc[q][torch.from_numpy(want).to(DEV)])
