@@ -61,6 +61,12 @@ def test_c4_d1536_prod_b4_one_million_nibble_layout():
     _check_full("c4", 4, tq.TQ_PROD, 1_000_000, 8, 100, layout=tq.TQ_LAYOUT_NIBBLE)
 
 
+def test_c4_d1536_prod_b4_one_million_nibble_layout_many_queries():
+    """96 queries: a full pass of the 64-query tcgen05 kernel and a pass of the 32-query kernel, dense and thresholded,
+    in the launch configuration of the benchmark's many-query leg."""
+    _check_full("c4", 4, tq.TQ_PROD, 1_000_000, 96, 100, layout=tq.TQ_LAYOUT_NIBBLE)
+
+
 def test_c4_d1536_mse_b2_one_million():
     _check_full("c4", 2, tq.TQ_MSE, 1_000_000, 8, 100)
 
