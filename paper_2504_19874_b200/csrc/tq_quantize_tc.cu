@@ -92,55 +92,113 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-// One warp per row: nu = ||x|| (optional), u = x / nu, u = hi + lo in bf16.  Rows warp, warp + nwarps, ...
-template <typename T, bool NORMALIZE>
-__device__ __forceinline__ void split_rows(const T* __restrict__ X, int64_t ldx, int64_t n, int d, int dpad,
-                                           __nv_bfloat16* __restrict__ L1, __nv_bfloat16* __restrict__ L2,
-                                           float* __restrict__ norms, int64_t warp, int64_t nwarps, int lane) {
-  // fp32 rows, 16-byte aligned: segments of 2048 elements held in registers (16 x 16 bytes per lane, all loads in
-  // flight at once); a row of one segment is read once, longer rows a second time (from L2) after the norm is known
-  if constexpr (sizeof(T) == 4) {
-    if ((d & 3) == 0 && (ldx & 3) == 0 && (reinterpret_cast<uintptr_t>(X) & 15) == 0 && dpad == d) {
-      const int nseg = (d + 2047) / 2048;
-      for (int64_t r = warp; r < n; r += nwarps) {
-        const float4* row4 = reinterpret_cast<const float4*>(X + r * ldx);
-        float4 v[16];
-        auto load_seg = [&](int seg) {
+// fp32 rows, 16-byte aligned, of at most 2048 NV / 16 elements per segment: a segment is held in registers (NV x 16
+// bytes per lane, all loads in flight at once); a row of one segment is read once, longer rows a second time (from L2)
+// after the norm is known.  NV follows d, so that short rows do not pay for sixteen mostly empty rounds (at d = 200 the
+// kernel was bound by the issue of predicated-off instructions, 2.6 TB/s).  The sums are those of NV = 16: the rounds
+// left out added fma(0, 0, s) = s.
+template <bool NORMALIZE, int NV>
+__device__ __forceinline__ void split_rows_vec(const float* __restrict__ X, int64_t ldx, int64_t n, int d, int dpad,
+                                               __nv_bfloat16* __restrict__ L1, __nv_bfloat16* __restrict__ L2,
+                                               float* __restrict__ norms, int64_t warp, int64_t nwarps, int lane) {
+  const int nseg = (d + 128 * NV - 1) / (128 * NV);
+  if (NV < 16) {
+    // short rows (one segment): 16 / NV rows of a warp are in flight at once -- a single row of 800 bytes per warp
+    // does not keep enough bytes in flight to fill the memory pipe
+    constexpr int RB = 16 / NV;
+    for (int64_t r0 = warp * RB; r0 < n; r0 += nwarps * RB) {
+      float4 v[RB][NV];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int c = seg * 512 + lane + 32 * i;
-            v[i] = (4 * c < d) ? __ldg(row4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
-          }
-        };
+      for (int k = 0; k < RB; ++k) {
+        const float4* row4 = reinterpret_cast<const float4*>(X + min(r0 + k, n - 1) * ldx);
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+          const int c = lane + 32 * i;
+          v[k][i] = (4 * c < d) ? __ldg(row4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < RB; ++k) {
+        const int64_t r = r0 + k;
+        if (r >= n) break;
         float inv = 1.f;
-        load_seg(0);
         if (NORMALIZE) {
           float s = 0.f;
-          for (int seg = 0; seg < nseg; ++seg) {
-            if (seg > 0) load_seg(seg);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) s = fmaf(v[i].x, v[i].x, fmaf(v[i].y, v[i].y, fmaf(v[i].z, v[i].z, fmaf(v[i].w, v[i].w, s))));
-          }
+          for (int i = 0; i < NV; ++i)
+            s = fmaf(v[k][i].x, v[k][i].x, fmaf(v[k][i].y, v[k][i].y, fmaf(v[k][i].z, v[k][i].z, fmaf(v[k][i].w, v[k][i].w, s))));
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
           const float nu = sqrtf(s);
           inv = (nu > 0.f) ? 1.f / nu : 0.f;
           if (lane == 0 && norms != nullptr) norms[r] = nu;
         }
-        for (int seg = 0; seg < nseg; ++seg) {
-          if (nseg > 1 && (seg > 0 || NORMALIZE)) load_seg(seg);   // registers hold the last segment read
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int c = seg * 512 + lane + 32 * i;
-            if (4 * c >= d) continue;
-            const float u0 = v[i].x * inv, u1 = v[i].y * inv, u2 = v[i].z * inv, u3 = v[i].w * inv;
-            const float h0 = __bfloat162float(__float2bfloat16_rn(u0)), h1 = __bfloat162float(__float2bfloat16_rn(u1));
-            const float h2 = __bfloat162float(__float2bfloat16_rn(u2)), h3 = __bfloat162float(__float2bfloat16_rn(u3));
-            *reinterpret_cast<uint2*>(L1 + r * dpad + 4 * c) = make_uint2(pack_bf16x2(h0, h1), pack_bf16x2(h2, h3));
-            *reinterpret_cast<uint2*>(L2 + r * dpad + 4 * c) = make_uint2(pack_bf16x2(u0 - h0, u1 - h1), pack_bf16x2(u2 - h2, u3 - h3));
-          }
+        for (int i = 0; i < NV; ++i) {
+          const int c = lane + 32 * i;
+          if (4 * c >= d) continue;
+          const float u0 = v[k][i].x * inv, u1 = v[k][i].y * inv, u2 = v[k][i].z * inv, u3 = v[k][i].w * inv;
+          const float h0 = __bfloat162float(__float2bfloat16_rn(u0)), h1 = __bfloat162float(__float2bfloat16_rn(u1));
+          const float h2 = __bfloat162float(__float2bfloat16_rn(u2)), h3 = __bfloat162float(__float2bfloat16_rn(u3));
+          *reinterpret_cast<uint2*>(L1 + r * dpad + 4 * c) = make_uint2(pack_bf16x2(h0, h1), pack_bf16x2(h2, h3));
+          *reinterpret_cast<uint2*>(L2 + r * dpad + 4 * c) = make_uint2(pack_bf16x2(u0 - h0, u1 - h1), pack_bf16x2(u2 - h2, u3 - h3));
         }
       }
+    }
+    return;
+  }
+  for (int64_t r = warp; r < n; r += nwarps) {
+    const float4* row4 = reinterpret_cast<const float4*>(X + r * ldx);
+    float4 v[NV];
+    auto load_seg = [&](int seg) {
+#pragma unroll
+      for (int i = 0; i < NV; ++i) {
+        const int c = seg * 32 * NV + lane + 32 * i;
+        v[i] = (4 * c < d) ? __ldg(row4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    };
+    float inv = 1.f;
+    load_seg(0);
+    if (NORMALIZE) {
+      float s = 0.f;
+      for (int seg = 0; seg < nseg; ++seg) {
+        if (seg > 0) load_seg(seg);
+#pragma unroll
+        for (int i = 0; i < NV; ++i) s = fmaf(v[i].x, v[i].x, fmaf(v[i].y, v[i].y, fmaf(v[i].z, v[i].z, fmaf(v[i].w, v[i].w, s))));
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      const float nu = sqrtf(s);
+      inv = (nu > 0.f) ? 1.f / nu : 0.f;
+      if (lane == 0 && norms != nullptr) norms[r] = nu;
+    }
+    for (int seg = 0; seg < nseg; ++seg) {
+      if (nseg > 1 && (seg > 0 || NORMALIZE)) load_seg(seg);   // registers hold the last segment read
+#pragma unroll
+      for (int i = 0; i < NV; ++i) {
+        const int c = seg * 32 * NV + lane + 32 * i;
+        if (4 * c >= d) continue;
+        const float u0 = v[i].x * inv, u1 = v[i].y * inv, u2 = v[i].z * inv, u3 = v[i].w * inv;
+        const float h0 = __bfloat162float(__float2bfloat16_rn(u0)), h1 = __bfloat162float(__float2bfloat16_rn(u1));
+        const float h2 = __bfloat162float(__float2bfloat16_rn(u2)), h3 = __bfloat162float(__float2bfloat16_rn(u3));
+        *reinterpret_cast<uint2*>(L1 + r * dpad + 4 * c) = make_uint2(pack_bf16x2(h0, h1), pack_bf16x2(h2, h3));
+        *reinterpret_cast<uint2*>(L2 + r * dpad + 4 * c) = make_uint2(pack_bf16x2(u0 - h0, u1 - h1), pack_bf16x2(u2 - h2, u3 - h3));
+      }
+    }
+  }
+}
+
+// One warp per row: nu = ||x|| (optional), u = x / nu, u = hi + lo in bf16.  Rows warp, warp + nwarps, ...
+template <typename T, bool NORMALIZE>
+__device__ __forceinline__ void split_rows(const T* __restrict__ X, int64_t ldx, int64_t n, int d, int dpad,
+                                           __nv_bfloat16* __restrict__ L1, __nv_bfloat16* __restrict__ L2,
+                                           float* __restrict__ norms, int64_t warp, int64_t nwarps, int lane) {
+  if constexpr (sizeof(T) == 4) {
+    if ((d & 3) == 0 && (ldx & 3) == 0 && (reinterpret_cast<uintptr_t>(X) & 15) == 0 && dpad == d) {
+      if (d <= 256) split_rows_vec<NORMALIZE, 2>(X, ldx, n, d, dpad, L1, L2, norms, warp, nwarps, lane);
+      else if (d <= 512) split_rows_vec<NORMALIZE, 4>(X, ldx, n, d, dpad, L1, L2, norms, warp, nwarps, lane);
+      else if (d <= 1024) split_rows_vec<NORMALIZE, 8>(X, ldx, n, d, dpad, L1, L2, norms, warp, nwarps, lane);
+      else split_rows_vec<NORMALIZE, 16>(X, ldx, n, d, dpad, L1, L2, norms, warp, nwarps, lane);
       return;
     }
   }
