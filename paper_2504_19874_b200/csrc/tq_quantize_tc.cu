@@ -40,7 +40,7 @@ struct Cfg {
   static constexpr int kStageBytes = 2 * BM * BK * 2 + 2 * kBRows * BK * 2; // A hi/lo + B hi/lo
   static constexpr int kStages = CTAS == 2 ? 3 : ((BN == 256) ? 2 : (BN == 128 ? 3 : 4));
   static constexpr int kTmemCols = 2 * BN;                                  // two accumulators
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers, centroids*/;
 };
 
 struct GemmArgs {
@@ -268,6 +268,10 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
   uint64_t* tempty = tfull + 2;             // [2]        epilogue -> MMA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  // the centroids in shared memory: indexed by the code they are one wavefront per load, where the same index into
+  // the kernel's constant arguments is replayed once per distinct code of the warp
+  float* cs = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(bars) + 128);   // [16]
+  if (MODE == 1 && threadIdx.x < 16) cs[threadIdx.x] = a.cb.c[threadIdx.x];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = (a.K + BK - 1) / BK;
@@ -478,7 +482,7 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
                 }
               }
               if (MODE == 1) {
-                const float e = (col_ok && !zero_row) ? (y - a.cb.c[code]) : 0.f;
+                const float e = (col_ok && !zero_row) ? (y - cs[code]) : 0.f;
                 gsum = fmaf(e, e, gsum);
                 ehi[q] = __bfloat162float(__float2bfloat16_rn(e));
                 elo[q] = e - ehi[q];
