@@ -826,13 +826,13 @@ cudaError_t launch_wide_c(const CUtensorMap& ma, const CUtensorMap& ms, const CU
   count_launches(1);
   const int64_t ntiles = (args.n + TILE - 1) / TILE;
   if (CTAS == 1) {
-    kern<<<(int)std::min<int64_t>(ntiles, tc::sm_count()), NTHREADS, kWideSmemBytes, st>>>(ma, ms, pa, ps, args);
+    kern<<<(int)std::min<int64_t>(ntiles, tc::sm_count()), W_NTHREADS, kWideSmemBytes, st>>>(ma, ms, pa, ps, args);
     return cudaGetLastError();
   }
   const int units = (int)std::min<int64_t>((ntiles + CTAS - 1) / CTAS, tc::sm_count() / CTAS);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(units * CTAS));
-  cfg.blockDim = dim3(NTHREADS);
+  cfg.blockDim = dim3(W_NTHREADS);
   cfg.dynamicSmemBytes = kWideSmemBytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];

@@ -34,11 +34,15 @@
 constexpr int W_QPP = 2 * kQueriesPerPass;      // 64 queries per pass
 constexpr int W_NCOL = 2 * NCOL;                // 192 MMA columns
 constexpr int W_SLOTS = 4;                      // k-blocks of A resident in TMEM
-constexpr int W_BSTAGES = 6;                    // ring of B boxes
+constexpr int W_BSTAGES = 6;                    // ring of B boxes (a CTA of a pair holds half of each: 12 stages in the same bytes)
 constexpr int W_BTILE = W_NCOL * KB_BYTES;      // 24 KB
 constexpr int W_PSTAGES = 4;                    // ring of packed-row groups
 constexpr int W_PTILE = TILE * 64;              // 8 KB: 128 rows x at most 64 bytes
 constexpr int W_ACOL0 = 2 * W_NCOL;             // first TMEM column of the A slots
+constexpr int W_ISSUERS = 3;                    // MMA-issuing warps: a thread that has committed a k-block's MMAs does not get to its
+                                                // next k-block before they have completed (~1000 cycles per k-block and thread),
+                                                // so two threads feed 4 MMAs of ~97 cycles every ~500 cycles, three every ~333
+constexpr int W_NTHREADS = 32 * (1 + W_ISSUERS + 8);
 constexpr int W_LBUF = 64;                      // candidates per query a CTA collects before it appends them
 static_assert(W_ACOL0 + W_SLOTS * 32 <= TMEM_COLS, "TMEM columns");
 static_assert((W_SLOTS & (W_SLOTS - 1)) == 0 && (W_PSTAGES & (W_PSTAGES - 1)) == 0, "ring sizes used as masks");
@@ -86,10 +90,14 @@ __device__ __forceinline__ RowGroup row_group(const Geo& g, int gi) {
 }
 
 template <int BM, int MODE, bool NIB, int CTAS>
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __launch_bounds__(W_NTHREADS, 1)
 scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__ CUtensorMap tmBs,
                 const __grid_constant__ CUtensorMap tmPa, const __grid_constant__ CUtensorMap tmPs, ScanArgs a) {
   if (a.run_if != nullptr && *a.run_if == 0) return;
+  // B ring of this CTA: a CTA of a pair holds half of every box, so the same shared memory gives twice the stages --
+  // the boxes arrive ~2500 cycles after they are requested (all SMs read the same lines of L2 at about the same time),
+  // and the number of boxes in flight, not the bytes, sets the rate at which they arrive
+  constexpr int BST = W_BSTAGES * CTAS, BTILE = W_BTILE / CTAS;
   const int rank = CTAS == 2 ? (int)tc::cluster_ctarank() : 0;
   // a unit = one CTA or one pair of CTAs; in round i unit u's CTA `rank` takes tile (u + i nunits) CTAS + rank
   const int64_t unit = blockIdx.x / CTAS, nunits = gridDim.x / CTAS;
@@ -100,9 +108,9 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
   unsigned char* pring = smem + W_BSTAGES * W_BTILE;
   uint64_t* bars = reinterpret_cast<uint64_t*>(pring + W_PSTAGES * W_PTILE);
   uint64_t* afull = bars;                           // [W_SLOTS]    the owning set's four warps -> MMA
-  uint64_t* bfull = afull + W_SLOTS;                // [W_BSTAGES]  TMA -> MMA
-  uint64_t* kdone = bfull + W_BSTAGES;              // [W_BSTAGES]  MMAs of a k-block complete: its B stage and A slot are free
-  uint64_t* pfull = kdone + W_BSTAGES;              // [W_PSTAGES]  TMA (packed rows) -> the owning set
+  uint64_t* bfull = afull + W_SLOTS;                // [BST]  TMA -> MMA
+  uint64_t* kdone = bfull + BST;                    // [BST]  MMAs of a k-block complete: its B stage and A slot are free
+  uint64_t* pfull = kdone + BST;              // [W_PSTAGES]  TMA (packed rows) -> the owning set
   uint64_t* pempty = pfull + W_PSTAGES;             // [W_PSTAGES]  the owning set -> TMA producer
   uint64_t* dfull = pempty + W_PSTAGES;             // accumulators complete -> epilogue
   uint64_t* dfree = dfull + 1;                      // accumulators read and zeroed -> MMA
@@ -120,7 +128,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < W_SLOTS; ++s) tc::mbar_init(&afull[s], 4 * CTAS);   // the leader's: the owning set of both CTAs
-    for (int s = 0; s < W_BSTAGES; ++s) {
+    for (int s = 0; s < BST; ++s) {
       tc::mbar_init(&bfull[s], 1);
       tc::mbar_init(&kdone[s], 1);
     }
@@ -128,7 +136,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
       tc::mbar_init(&pfull[s], 1);
       tc::mbar_init(&pempty[s], 4);
     }
-    tc::mbar_init(dfull, N_ISSUERS);
+    tc::mbar_init(dfull, W_ISSUERS);
     tc::mbar_init(dfree, 8 * CTAS);
     *abort_flag = 0;
     tc::fence_barrier_init();
@@ -189,17 +197,17 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
             if (prnd < nrounds && tc::mbar_test_wait(&pempty[pgc & (W_PSTAGES - 1)], ((pgc / W_PSTAGES) & 1u) ^ 1u)) load_rows();
             const int f = rg.f0 + j;
             const int kb = rg.part_s ? f - a.g.kba : f;
-            // B stage kc % W_BSTAGES was last read by the MMAs of k-block kc - W_BSTAGES
-            if (kc >= W_BSTAGES && !(ok = tc::mbar_wait(&kdone[bst], bph ^ 1u, abort_flag, a.status))) break;
+            // B stage kc % BST was last read by the MMAs of k-block kc - BST
+            if (kc >= BST && !(ok = tc::mbar_wait(&kdone[bst], bph ^ 1u, abort_flag, a.status))) break;
             if (CTAS == 2) {   // each CTA loads half of the box's rows; the bytes of both are counted on the leader's barrier
               if (rank == 0) tc::mbar_arrive_expect_tx(&bfull[bst], W_BTILE);
-              tc::tma_load_2d_pair(bring + bst * W_BTILE, rg.part_s ? &tmBs : &tmBa, &bfull[bst], kb * KB_BYTES,
+              tc::tma_load_2d_pair(bring + bst * BTILE, rg.part_s ? &tmBs : &tmBa, &bfull[bst], kb * KB_BYTES,
                                    a.pass * NCOL + rank * (W_NCOL / 2));
             } else {
               tc::mbar_arrive_expect_tx(&bfull[bst], W_BTILE);
-              tc::tma_load_2d(bring + bst * W_BTILE, rg.part_s ? &tmBs : &tmBa, &bfull[bst], kb * KB_BYTES, a.pass * NCOL);
+              tc::tma_load_2d(bring + bst * BTILE, rg.part_s ? &tmBs : &tmBa, &bfull[bst], kb * KB_BYTES, a.pass * NCOL);
             }
-            if (++bst == W_BSTAGES) {
+            if (++bst == BST) {
               bst = 0;
               bph ^= 1u;
             }
@@ -211,7 +219,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
       }
     }
     __syncwarp();
-  } else if (warp <= N_ISSUERS) {
+  } else if (warp <= W_ISSUERS) {
     // ---------------------------------------------------------------- MMA issuers
     if (lane == 0 && rank == 0) {   // the leader's threads issue for both CTAs of a pair (M = 256)
       constexpr uint32_t idesc = idesc_i8(TILE * CTAS, W_NCOL);
@@ -225,16 +233,16 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
         if (!(ok = tc::mbar_wait(dfree, it & 1u, abort_flag, a.status))) break;
         for (int f = 0; f < nkb_total; ++f, ++kc) {
           const bool mine = turn == me;
-          if (++turn == N_ISSUERS) turn = 0;
+          if (++turn == W_ISSUERS) turn = 0;
           if (!mine) continue;
-          const uint32_t bst = kc % W_BSTAGES, slot = kc & (W_SLOTS - 1);
-          if (!(ok = tc::mbar_wait(&bfull[bst], (kc / W_BSTAGES) & 1u, abort_flag, a.status))) break;
+          const uint32_t bst = kc % BST, slot = kc & (W_SLOTS - 1);
+          if (!(ok = tc::mbar_wait(&bfull[bst], (kc / BST) & 1u, abort_flag, a.status))) break;
           if (!(ok = tc::mbar_wait(&afull[slot], (kc / W_SLOTS) & 1u, abort_flag, a.status))) break;
           tc::tc_fence_after();
           const int kind = NIB ? f % 3 : 0;   // nibble layout: h bytes (signed A), l bytes, sign bits (second accumulator)
           const bool part_s = NIB ? kind == 2 : f >= a.g.kba;
           const uint32_t idesc_f = (NIB && kind == 0) ? idesc_i8(TILE * CTAS, W_NCOL, true) : idesc;
-          const uint64_t bdesc = bdesc0 + (uint64_t)(bst * (W_BTILE >> 4));
+          const uint64_t bdesc = bdesc0 + (uint64_t)(bst * (BTILE >> 4));
           const uint32_t a_tmem = tmem_base + (uint32_t)(W_ACOL0 + slot * 32);
           const uint32_t d_tmem = tmem_base + (uint32_t)(part_s ? W_NCOL : 0);
 #pragma unroll
@@ -255,7 +263,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
     __syncwarp();
   } else {
     // ---------------------------------------------------------------- transform + epilogue (thread = vector row)
-    const int e = warp - 1 - N_ISSUERS;
+    const int e = warp - 1 - W_ISSUERS;
     const int set = e >> 2;                 // takes the row groups gi % 2 == set and the queries [32 set, 32 set + 32)
     const int quad = warp & 3;              // TMEM lane group this warp may access
     const int r = quad * 32 + lane;         // row inside the tile
@@ -302,7 +310,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
         const uint32_t slot = kt & (W_SLOTS - 1);
         if (kt >= W_SLOTS) {   // the slot was last read by the MMAs of k-block kt - W_SLOTS
           const uint32_t kp = kt - W_SLOTS;
-          if (!tc::mbar_wait(&kdone[kp % W_BSTAGES], (kp / W_BSTAGES) & 1u, abort_flag, a.status)) return false;
+          if (!tc::mbar_wait(&kdone[kp % BST], (kp / BST) & 1u, abort_flag, a.status)) return false;
         }
         tc::tc_fence_after();
         tc::tmem_st32(lane_addr + (uint32_t)(W_ACOL0 + slot * 32), v);
@@ -484,8 +492,8 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
     if (CTAS == 2) tc::tmem_dealloc_pair(tmem_base, TMEM_COLS);
     else tc::tmem_dealloc(tmem_base, TMEM_COLS);
   }
-  if (MODE == 1 && warp > N_ISSUERS) {   // the eight transform warps append eight queries' collected pairs each
-    for (int ql = (warp - 1 - N_ISSUERS) * 8; ql < (warp - N_ISSUERS) * 8; ++ql) {
+  if (MODE == 1 && warp > W_ISSUERS) {   // the eight transform warps append eight queries' collected pairs each
+    for (int ql = (warp - 1 - W_ISSUERS) * 8; ql < (warp - W_ISSUERS) * 8; ++ql) {
       const int m = min(lcnt[ql], W_LBUF);
       if (m == 0 || ql >= a.nqp) continue;
       int base = 0;
