@@ -964,12 +964,12 @@ int run_pass(const tq_plan* plan, int pass, int nqp, int64_t n, const uint8_t* i
   const bool wide = nqp > kQueriesPerPass;
   TQ_REQUIRE(nqp <= (wide ? W_QPP : kQueriesPerPass) && (!wide || (pass % 2 == 0 && pass + 2 <= kPassesPerGroup)), TQ_ERR_INVALID_ARG,
              "%s: pass %d of %d queries", who, pass, nqp);
-  // The wide kernel also runs on CTA pairs (TQ_SCAN_PAIRS=1: M = 256, each CTA loads half of a B box's rows).  Off by
-  // default: the B boxes come from L2 and halving that traffic did not shorten a pass (measured 365 against 358 us per
-  // 32 queries at d = 1536, n = 10^6).
+  // The wide kernel runs on CTA pairs wherever there is more than one tile (M = 256, each CTA loads half of a B box's
+  // rows into one of twelve half-size stages: measured 316 against 339 us per 32 queries at d = 1536, n = 10^6).
+  // TQ_SCAN_PAIRS=0 keeps single CTAs, to compare the two on one machine.
   static const bool pairs_on = [] {
     const char* e = std::getenv("TQ_SCAN_PAIRS");
-    return e != nullptr && e[0] == '1';
+    return e == nullptr || e[0] != '0';
   }();
   const bool pairs = wide && pairs_on && n > TILE;
   const uint32_t brows = wide ? (pairs ? W_NCOL / 2 : W_NCOL) : NCOL, prows = wide ? TILE : 2 * TILE;

@@ -17,17 +17,20 @@
 //     groups of four k-blocks of the bit streams) in turn, so that two warps work on every lane quadrant's chain;
 //     a set's threads read back and emit 32 of the 64 queries each;
 //   - a k-block is 4 MMAs of N = 192 instead of 8 of N = 96 (an MMA of N = 96 costs as much as one of N = 128).
-// The accumulators are single-buffered: the issuers wait (dfree) until both sets have read and zeroed their
-// columns of the previous tile.
+// The accumulators are single-buffered: the issuers wait (dfree) until both sets have read their columns of the
+// previous tile into registers and zeroed them.
 //
-// CTA (one per SM, persistent over tiles), 352 threads as in scan_tc_kernel:
+// CTA (one per SM, persistent over tiles), 384 threads:
 //   warp 0       TMA producer: per k-block one [192 rows x 128 B] box of B (6 stages); per row group the tile's packed
 //                rows ([128 rows x 32..64 B], 4 stages), requested as far ahead as their ring allows
-//   warps 1..2   MMA issuers, k-blocks in turn
-//   warps 3..10  transform + epilogue: set = (warp - 3) / 4, lane quadrant = warp % 4, thread = vector row
-// CTAS = 2 (an option of the launcher): two CTAs of a cluster run in lockstep on their own tiles and share every B
-// box -- each loads half of its rows (no multicast), the leader's issuers run the MMAs with M = 256 (cta_group::2),
-// the commits reach both CTAs' barriers.  It halves the B traffic from L2 and did not shorten a pass.
+//   warps 1..3   MMA issuers, k-blocks in turn.  A thread issues an MMA every ~82 cycles and does not get to its next
+//                k-block before the MMAs it committed have completed (~1000 cycles per k-block and thread): two
+//                threads fed 4 MMAs of ~97 cycles every ~500 cycles, three keep the pipe busy between epilogues.
+//   warps 4..11  transform + epilogue: set = (warp - 4) / 4, lane quadrant = warp % 4, thread = vector row
+// CTAS = 2 (the default where there is more than one tile): two CTAs of a cluster run in lockstep on their own tiles
+// and share every B box -- each loads half of its rows (no multicast) into one of twelve half-size stages, the
+// leader's issuers run the MMAs with M = 256 (cta_group::2), the commits reach both CTAs' barriers.  Halving the B
+// traffic from L2 alone gave nothing; the deeper ring in the same bytes and the third issuer together 7 %.
 // All waits are bounded.
 #pragma once
 
@@ -98,6 +101,14 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
   // the boxes arrive ~2500 cycles after they are requested (all SMs read the same lines of L2 at about the same time),
   // and the number of boxes in flight, not the bytes, sets the rate at which they arrive
   constexpr int BST = W_BSTAGES * CTAS, BTILE = W_BTILE / CTAS;
+  // The completion barriers of the k-blocks form a ring of their own, kdone[k % KD].  Several threads issue, so the
+  // k-blocks complete out of order, and a waiter must never find that its barrier has completed twice since the
+  // k-block it waits for (the parity would look unchanged): the producer waits for k - BST before it loads k, the
+  // transform warps for k - W_SLOTS before they store k, and the next k-block on either's barrier, k - BST + KD resp.
+  // k - W_SLOTS + KD, cannot complete before k itself is loaded resp. k + W_SLOTS stored when KD >= BST and
+  // KD >= 2 W_SLOTS.  (With kdone[k % 6] and three issuers k + 2 could complete before k was stored.)
+  constexpr int KD = CTAS == 2 ? 16 : 8;
+  static_assert(KD >= BST && KD >= 2 * W_SLOTS && (KD & (KD - 1)) == 0, "ring of completion barriers");
   const int rank = CTAS == 2 ? (int)tc::cluster_ctarank() : 0;
   // a unit = one CTA or one pair of CTAs; in round i unit u's CTA `rank` takes tile (u + i nunits) CTAS + rank
   const int64_t unit = blockIdx.x / CTAS, nunits = gridDim.x / CTAS;
@@ -109,8 +120,8 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
   uint64_t* bars = reinterpret_cast<uint64_t*>(pring + W_PSTAGES * W_PTILE);
   uint64_t* afull = bars;                           // [W_SLOTS]    the owning set's four warps -> MMA
   uint64_t* bfull = afull + W_SLOTS;                // [BST]  TMA -> MMA
-  uint64_t* kdone = bfull + BST;                    // [BST]  MMAs of a k-block complete: its B stage and A slot are free
-  uint64_t* pfull = kdone + BST;              // [W_PSTAGES]  TMA (packed rows) -> the owning set
+  uint64_t* kdone = bfull + BST;                    // [KD]   MMAs of k-block k complete (kdone[k % KD]): its B stage and A slot are free
+  uint64_t* pfull = kdone + KD;              // [W_PSTAGES]  TMA (packed rows) -> the owning set
   uint64_t* pempty = pfull + W_PSTAGES;             // [W_PSTAGES]  the owning set -> TMA producer
   uint64_t* dfull = pempty + W_PSTAGES;             // accumulators complete -> epilogue
   uint64_t* dfree = dfull + 1;                      // accumulators read and zeroed -> MMA
@@ -128,10 +139,8 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < W_SLOTS; ++s) tc::mbar_init(&afull[s], 4 * CTAS);   // the leader's: the owning set of both CTAs
-    for (int s = 0; s < BST; ++s) {
-      tc::mbar_init(&bfull[s], 1);
-      tc::mbar_init(&kdone[s], 1);
-    }
+    for (int s = 0; s < BST; ++s) tc::mbar_init(&bfull[s], 1);
+    for (int s = 0; s < KD; ++s) tc::mbar_init(&kdone[s], 1);
     for (int s = 0; s < W_PSTAGES; ++s) {
       tc::mbar_init(&pfull[s], 1);
       tc::mbar_init(&pempty[s], 4);
@@ -166,7 +175,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
       int bst = 0;
-      uint32_t bph = 0, kc = 0, gc = 0;   // k-blocks and row groups reached so far by this CTA
+      uint32_t kc = 0, gc = 0;   // k-blocks and row groups reached so far by this CTA
       bool ok = true;
       // The packed rows run ahead of the B boxes as far as their own ring allows: a row group's bytes are wanted by its
       // set as soon as the set has stored its previous group, several k-blocks before the MMAs free a B stage for it.
@@ -198,7 +207,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
             const int f = rg.f0 + j;
             const int kb = rg.part_s ? f - a.g.kba : f;
             // B stage kc % BST was last read by the MMAs of k-block kc - BST
-            if (kc >= BST && !(ok = tc::mbar_wait(&kdone[bst], bph ^ 1u, abort_flag, a.status))) break;
+            if (kc >= BST && !(ok = tc::mbar_wait(&kdone[(kc - BST) & (KD - 1)], ((kc - BST) / KD) & 1u, abort_flag, a.status))) break;
             if (CTAS == 2) {   // each CTA loads half of the box's rows; the bytes of both are counted on the leader's barrier
               if (rank == 0) tc::mbar_arrive_expect_tx(&bfull[bst], W_BTILE);
               tc::tma_load_2d_pair(bring + bst * BTILE, rg.part_s ? &tmBs : &tmBa, &bfull[bst], kb * KB_BYTES,
@@ -207,10 +216,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
               tc::mbar_arrive_expect_tx(&bfull[bst], W_BTILE);
               tc::tma_load_2d(bring + bst * BTILE, rg.part_s ? &tmBs : &tmBa, &bfull[bst], kb * KB_BYTES, a.pass * NCOL);
             }
-            if (++bst == BST) {
-              bst = 0;
-              bph ^= 1u;
-            }
+            if (++bst == BST) bst = 0;
           }
         }
       }
@@ -251,8 +257,8 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
             else umma_i8_ts(d_tmem, a_tmem + 8 * step, bdesc + 2 * step, idesc_f, 1u);
           }
           // A slot and B stage (of both CTAs) reusable once these MMAs have read them
-          if (CTAS == 2) tc::umma_commit_pair(&kdone[bst]);
-          else tc::umma_commit(&kdone[bst]);
+          if (CTAS == 2) tc::umma_commit_pair(&kdone[kc & (KD - 1)]);
+          else tc::umma_commit(&kdone[kc & (KD - 1)]);
         }
         if (ok) {   // all MMAs this thread issued for the tile
           if (CTAS == 2) tc::umma_commit_pair(dfull);
@@ -310,7 +316,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
         const uint32_t slot = kt & (W_SLOTS - 1);
         if (kt >= W_SLOTS) {   // the slot was last read by the MMAs of k-block kt - W_SLOTS
           const uint32_t kp = kt - W_SLOTS;
-          if (!tc::mbar_wait(&kdone[kp % BST], (kp / BST) & 1u, abort_flag, a.status)) return false;
+          if (!tc::mbar_wait(&kdone[kp & (KD - 1)], (kp / KD) & 1u, abort_flag, a.status)) return false;
         }
         tc::tc_fence_after();
         tc::tmem_st32(lane_addr + (uint32_t)(W_ACOL0 + slot * 32), v);

@@ -175,10 +175,10 @@ print("kernel form ok")
 """
 
 
-@pytest.mark.parametrize("env", [{"TQ_SCAN_WIDE": "0"}, {"TQ_SCAN_PAIRS": "1"}])
+@pytest.mark.parametrize("env", [{"TQ_SCAN_WIDE": "0"}, {"TQ_SCAN_PAIRS": "0"}])
 def test_other_forms_of_the_many_query_kernel_give_the_same_estimates(env, tmp_path):
-    """Calls of more than 32 queries run the wide tcgen05 kernel (64 queries per pass, one CTA per tile).  TQ_SCAN_WIDE=0
-    keeps the 32-query kernel and TQ_SCAN_PAIRS=1 runs the wide kernel on CTA pairs (both read once per process): the
+    """Calls of more than 32 queries run the wide tcgen05 kernel (64 queries per pass) on CTA pairs.  TQ_SCAN_WIDE=0
+    keeps the 32-query kernel and TQ_SCAN_PAIRS=0 runs the wide kernel on single CTAs (both read once per process): the
     same integers, so dense estimates and top-k must be bit-identical.  Sizes: an odd number of 128-vector tiles with a
     ragged tail, 70 queries (a full pass and a short one), and one thresholded top-k (n >= 65,536)."""
     import os
