@@ -108,6 +108,13 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
   // k - W_SLOTS + KD, cannot complete before k itself is loaded resp. k + W_SLOTS stored when KD >= BST and
   // KD >= 2 W_SLOTS.  (With kdone[k % 6] and three issuers k + 2 could complete before k was stored.)
   constexpr int KD = CTAS == 2 ? 16 : 8;
+  // A parity wait also passes when its barrier is two completions behind, so whoever waits for a completion must
+  // itself have seen the one before it.  The "A stored" barriers therefore form a ring of lcm(issuers, slots) = 12:
+  // the thread that issues k-block k waited on afull[k % 12] for k - 12 (with afull[k % 4] the completion before k's
+  // is k - 4's, another thread's, and k - 4 may not be stored yet when the other set is ahead).  The B rings (6 and
+  // 12 stages) are multiples of the issuer count for the same reason.
+  constexpr int AF = 12;
+  static_assert(AF % W_ISSUERS == 0 && AF % W_SLOTS == 0 && BST % W_ISSUERS == 0, "a waiter has seen the completion before the one it waits for");
   static_assert(KD >= BST && KD >= 2 * W_SLOTS && (KD & (KD - 1)) == 0, "ring of completion barriers");
   const int rank = CTAS == 2 ? (int)tc::cluster_ctarank() : 0;
   // a unit = one CTA or one pair of CTAs; in round i unit u's CTA `rank` takes tile (u + i nunits) CTAS + rank
@@ -118,8 +125,8 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
   unsigned char* bring = smem;
   unsigned char* pring = smem + W_BSTAGES * W_BTILE;
   uint64_t* bars = reinterpret_cast<uint64_t*>(pring + W_PSTAGES * W_PTILE);
-  uint64_t* afull = bars;                           // [W_SLOTS]    the owning set's four warps -> MMA
-  uint64_t* bfull = afull + W_SLOTS;                // [BST]  TMA -> MMA
+  uint64_t* afull = bars;                           // [AF]   k-block k stored by the owning set's four warps (afull[k % AF]) -> MMA
+  uint64_t* bfull = afull + AF;                // [BST]  TMA -> MMA
   uint64_t* kdone = bfull + BST;                    // [KD]   MMAs of k-block k complete (kdone[k % KD]): its B stage and A slot are free
   uint64_t* pfull = kdone + KD;              // [W_PSTAGES]  TMA (packed rows) -> the owning set
   uint64_t* pempty = pfull + W_PSTAGES;             // [W_PSTAGES]  the owning set -> TMA producer
@@ -138,7 +145,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
   const int64_t ntiles = (a.n + TILE - 1) / TILE, nrounds = (ntiles + CTAS - 1) / CTAS;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < W_SLOTS; ++s) tc::mbar_init(&afull[s], 4 * CTAS);   // the leader's: the owning set of both CTAs
+    for (int s = 0; s < AF; ++s) tc::mbar_init(&afull[s], 4 * CTAS);   // the leader's: the owning set of both CTAs
     for (int s = 0; s < BST; ++s) tc::mbar_init(&bfull[s], 1);
     for (int s = 0; s < KD; ++s) tc::mbar_init(&kdone[s], 1);
     for (int s = 0; s < W_PSTAGES; ++s) {
@@ -243,7 +250,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
           if (!mine) continue;
           const uint32_t bst = kc % BST, slot = kc & (W_SLOTS - 1);
           if (!(ok = tc::mbar_wait(&bfull[bst], (kc / BST) & 1u, abort_flag, a.status))) break;
-          if (!(ok = tc::mbar_wait(&afull[slot], (kc / W_SLOTS) & 1u, abort_flag, a.status))) break;
+          if (!(ok = tc::mbar_wait(&afull[kc % AF], (kc / AF) & 1u, abort_flag, a.status))) break;
           tc::tc_fence_after();
           const int kind = NIB ? f % 3 : 0;   // nibble layout: h bytes (signed A), l bytes, sign bits (second accumulator)
           const bool part_s = NIB ? kind == 2 : f >= a.g.kba;
@@ -324,8 +331,8 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
         tc::tc_fence_before();
         __syncwarp();
         if (lane == 0) {
-          if (CTAS == 2) tc::mbar_arrive_leader(&afull[slot]);
-          else tc::mbar_arrive(&afull[slot]);
+          if (CTAS == 2) tc::mbar_arrive_leader(&afull[kt % AF]);
+          else tc::mbar_arrive(&afull[kt % AF]);
         }
         return true;
       };
