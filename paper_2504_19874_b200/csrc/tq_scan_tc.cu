@@ -65,6 +65,11 @@ constexpr int PTILE_BYTES = 2 * TILE * 64;           // 16 KB: 256 rows x at mos
 constexpr int D_COLS = 2 * NCOL;                     // accumulator columns per tile (MSE part, QJL part)
 constexpr int A_COL0 = 2 * D_COLS;                   // first TMEM column of the A slots
 constexpr int N_ISSUERS = 2;             // MMA-issuing warps (a tcgen05.commit stalls its thread; a second issuer hides it)
+// The barrier rings count on this number: a parity wait also passes when its barrier is two completions behind, so the
+// thread that waits for k-block k must itself have waited for the completion before it on the same barrier -- A_SLOTS
+// and B_STAGES are multiples of N_ISSUERS.  (Three issuers with rings of 6 / 9 / 16 barriers, as in the 64-query
+// kernel, were measured here: 464 against 471 us per pass; this kernel is bound by its transform warps.)
+static_assert(A_SLOTS % N_ISSUERS == 0 && B_STAGES % N_ISSUERS == 0, "a waiter has seen the completion before the one it waits for");
 constexpr int NTHREADS = 32 * (1 + N_ISSUERS + 8);
 constexpr int TMEM_COLS = 512;
 constexpr int LBUF = 128;              // candidates per query a CTA collects in shared memory before it appends them
