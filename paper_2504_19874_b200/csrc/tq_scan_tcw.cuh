@@ -26,7 +26,8 @@
 //   warps 1..3   MMA issuers, k-blocks in turn.  A thread issues an MMA every ~82 cycles and does not get to its next
 //                k-block before the MMAs it committed have completed (~1000 cycles per k-block and thread): two
 //                threads fed 4 MMAs of ~97 cycles every ~500 cycles, three keep the pipe busy between epilogues.
-//   warps 4..11  transform + epilogue: set = (warp - 4) / 4, lane quadrant = warp % 4, thread = vector row
+//   warps 4..11  transform + epilogue: set = (warp - 4) / 4, lane quadrant = warp % 4, thread = vector row; a set takes
+//                every second row group of the CTA's running count
 // CTAS = 2 (the default where there is more than one tile): two CTAs of a cluster run in lockstep on their own tiles
 // and share every B box -- each loads half of its rows (no multicast) into one of twelve half-size stages, the
 // leader's issuers run the MMAs with M = 256 (cta_group::2), the commits reach both CTAs' barriers.  Halving the B
@@ -365,7 +366,10 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
         return store_a(v, kt0 + (uint32_t)f);
       };
 
-      for (int gi = set; gi < ngroups && ok; gi += 2) {
+      // the sets take the row groups in turn by the CTA's running count of groups (not by the group's number inside the
+      // tile, which changes sides from tile to tile when a tile has an odd number of groups): a set then meets a
+      // packed-row stage every second time it is used, always after it has itself waited for the use before
+      for (int gi = (set + (int)((it * (uint32_t)ngroups) & 1u)) & 1; gi < ngroups && ok; gi += 2) {
         const RowGroup rg = row_group<BM, NIB>(a.g, gi);
         const uint32_t gc = it * (uint32_t)ngroups + (uint32_t)gi;
         const uint32_t pst = gc & (W_PSTAGES - 1), pph = (gc / W_PSTAGES) & 1u;
