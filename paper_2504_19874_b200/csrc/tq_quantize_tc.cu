@@ -40,7 +40,8 @@ struct Cfg {
   static constexpr int kStageBytes = 2 * BM * BK * 2 + 2 * kBRows * BK * 2; // A hi/lo + B hi/lo
   static constexpr int kStages = CTAS == 2 ? 3 : ((BN == 256) ? 2 : (BN == 128 ? 3 : 4));
   static constexpr int kTmemCols = 2 * BN;                                  // two accumulators
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers, centroids*/;
+  static constexpr int kStoreBytes = 4 * EPS * 2048;   // MODE 1: one [32 rows x 64 B] box per epilogue warp, staged for a TMA store
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers, centroids*/ + kStoreBytes;
 };
 
 struct GemmArgs {
@@ -52,6 +53,8 @@ struct GemmArgs {
   size_t out_rb;
   __nv_bfloat16* E1;     // MODE 1: residual limbs, pitch ldE
   __nv_bfloat16* E2;
+  const CUtensorMap* store_e1;   // host pointers to the TMA store maps of E1 / E2 (box 32 rows x 32 columns, 64-byte swizzle);
+  const CUtensorMap* store_e2;   // the launcher passes them on as kernel arguments
   int64_t ldE;
   float* gpart;          // MODE 1: [EPS * tiles_n][Mpad] partial sums of e^2 (one per epilogue warp's columns)
   int64_t Mpad;
@@ -255,7 +258,8 @@ __global__ void __launch_bounds__(256) split_rows_kernel(const T* __restrict__ X
 template <int BN, int MODE, int BITS, int CTAS>
 __global__ void __launch_bounds__(NTHREADS, 1)
 quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2,
-                     const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmArgs a) {
+                     const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
+                     const __grid_constant__ CUtensorMap tmE1, const __grid_constant__ CUtensorMap tmE2, GemmArgs a) {
   using C = Cfg<BN, CTAS>;
   const int rank = CTAS == 2 ? (int)cluster_ctarank() : 0;   // CTA of the pair; rank 0 issues the MMAs
   const int64_t unit = blockIdx.x / CTAS, nunits = gridDim.x / CTAS;   // a unit = one CTA or one pair
@@ -271,6 +275,7 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
   // the centroids in shared memory: indexed by the code they are one wavefront per load, where the same index into
   // the kernel's constant arguments is replayed once per distinct code of the warp
   float* cs = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(bars) + 128);   // [16]
+  unsigned char* stg = reinterpret_cast<unsigned char*>(bars) + 512;                    // [4 EPS][2048], 512-byte aligned
   if (MODE == 1 && threadIdx.x < 16) cs[threadIdx.x] = a.cb.c[threadIdx.x];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -506,14 +511,31 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
             for (int q = 0; q < BITS; ++q)
               if (w0 + q < row_words) out_row[w0 + q] = words[q];
           }
-          if (MODE == 1 && row_ok && TQ_DEVICE_CHECK(row < a.Mpad, a.status)) {
-            uint4* d1 = reinterpret_cast<uint4*>(a.E1 + row * a.ldE + col0);
-            uint4* d2 = reinterpret_cast<uint4*>(a.E2 + row * a.ldE + col0);
+          if (MODE == 1) {
+            // The warp's 32 rows x 32 columns of each residual limb go out as one TMA store: a row per thread, staged in
+            // shared memory in the 64-byte swizzle (16-byte piece q of row r at q ^ ((r >> 1) & 3): four wavefronts per
+            // instruction, the minimum for 512 bytes).  Stores straight from the registers were 16 bytes per lane at the
+            // matrix's row stride, 32 lines per instruction, and cost a tenth of the whole quantiser.  Rows past M and
+            // columns past N hold zeros or scratch inside the buffer's padding; the map clips columns past ldE.
+            unsigned char* buf = stg + (warp - 2) * 2048;
+            const int64_t row0 = row - lane;
+            {   // (the map is Mpad rows high: a tile that overhangs the buffer is clipped by the store itself)
+              const uint32_t sw = (uint32_t)((lane >> 1) & 3);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              if (col0 + q * 8 + 8 <= a.ldE) {
-                d1[q] = make_uint4(e1[4 * q], e1[4 * q + 1], e1[4 * q + 2], e1[4 * q + 3]);
-                d2[q] = make_uint4(e2[4 * q], e2[4 * q + 1], e2[4 * q + 2], e2[4 * q + 3]);
+              for (int limb = 0; limb < 2; ++limb) {
+                if (lane == 0) tma_store_wait_read();   // the previous box has left the buffer
+                __syncwarp();
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  const uint32_t* e = limb == 0 ? e1 : e2;
+                  *reinterpret_cast<uint4*>(buf + lane * 64 + ((q ^ sw) << 4)) = make_uint4(e[4 * q], e[4 * q + 1], e[4 * q + 2], e[4 * q + 3]);
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                  tma_store_2d(limb == 0 ? &tmE1 : &tmE2, buf, col0, (int)row0);
+                  tma_store_commit();
+                }
               }
             }
           }
@@ -543,6 +565,10 @@ quantize_gemm_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_cons
           for (size_t w = covered; w < row_words; ++w) out_row[w] = 0u;
         }
       }
+    }
+    if (MODE == 1) {   // the residual stores of this warp have completed before the CTA gives up its shared memory
+      if (lane == 0) tma_store_wait_all();
+      __syncwarp();
     }
   }
 
@@ -598,6 +624,19 @@ bool make_map(CUtensorMap* map, const __nv_bfloat16* base, int64_t rows, int col
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// bf16 matrix [rows, cols] with row pitch `pitch` elements, for TMA stores of [32 rows x 32 columns] boxes staged in
+// shared memory in the 64-byte swizzle.
+bool make_store_map(CUtensorMap* map, __nv_bfloat16* base, int64_t rows, int64_t cols, int64_t pitch) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)pitch * 2};
+  const cuuint32_t box[2] = {32, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 // Byte matrix [rows, row_bytes] with row pitch `pitch` bytes; box = box_bytes x box_rows; `swizzle` = 0 (plain
@@ -650,8 +689,11 @@ cudaError_t launch_gemm_t(const CUtensorMap& a1, const CUtensorMap& a2, const CU
   const int64_t tiles = (int64_t)args.tiles_m * args.tiles_n;   // tiles_m counts rows of BM * CTAS
   const int units = (int)std::min<int64_t>(tiles, sm_count() / CTAS);
   count_launches(1);
+  // the store maps of the residual limbs (MODE 1); any valid map otherwise
+  const CUtensorMap& e1 = args.store_e1 ? *args.store_e1 : a1;
+  const CUtensorMap& e2 = args.store_e2 ? *args.store_e2 : a2;
   if (CTAS == 1) {
-    kern<<<units, NTHREADS, C::kSmemBytes, st>>>(a1, a2, b1, b2, args);
+    kern<<<units, NTHREADS, C::kSmemBytes, st>>>(a1, a2, b1, b2, e1, e2, args);
     return cudaGetLastError();
   }
   cudaLaunchConfig_t cfg = {};
@@ -666,7 +708,7 @@ cudaError_t launch_gemm_t(const CUtensorMap& a1, const CUtensorMap& a2, const CU
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, a1, a2, b1, b2, args);
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, a1, a2, b1, b2, e1, e2, args);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
@@ -833,6 +875,14 @@ int quantize(const tq_plan* plan, const void* X, int x_dtype, int64_t n, int64_t
     g.E1 = EL1;
     g.E2 = EL2;
     g.ldE = dpad;
+    CUtensorMap sE1, sE2;
+    g.store_e1 = g.store_e2 = nullptr;
+    if (prod) {
+      TQ_REQUIRE(make_store_map(&sE1, EL1, R, dpad, dpad) && make_store_map(&sE2, EL2, R, dpad, dpad), TQ_ERR_CUDA,
+                 "%s: cuTensorMapEncodeTiled failed (residual stores)", who);
+      g.store_e1 = &sE1;
+      g.store_e2 = &sE2;
+    }
     g.gpart = gpart;
     g.Mpad = R;
     g.nu = nu_out;
