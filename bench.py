@@ -549,9 +549,9 @@ def run_b200(args):
 
 
 # DRAM bytes of the dominant kernels from ncu captures (one launch each; see the summaries under profiles/)
-# rotate launch (692.5 MB read + 671.4 MB written) + project launch (690.4 + 72.1 MB) of the CTA-pair GEMM, from ncu;
+# rotate launch (680.8 MB read + 650.5 MB written) + project launch (690.2 + 71.4 MB) of the CTA-pair GEMM, from ncu;
 # + the split_rows launch of the block (reads 98,304 x 6144 B, writes two bf16 limbs of the same size: 604 + 604 MB)
-QUANTIZE_TRAFFIC_PER_98304_ROWS = (692.5e6 + 671.4e6) + (690.4e6 + 72.1e6) + 2 * 604.0e6
+QUANTIZE_TRAFFIC_PER_98304_ROWS = (680.8e6 + 650.5e6) + (690.2e6 + 71.4e6) + 2 * 604.0e6
 SCAN_TRAFFIC_PER_VECTOR = (205.9e6 + 5.0e6) / 262144
 
 
