@@ -334,9 +334,13 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
         for (int r = 0; r < a.R; ++r) {
           if (!(ok = tc::mbar_wait(&empty[stage], phase ^ 1u, abort_flag, a.status))) break;
           unsigned char* sb = stage_base + (size_t)stage * STAGE_BYTES;
-          tc::mbar_arrive_expect_tx(&full[stage], STAGE_BYTES);
+          // 64-byte blocks wholly beyond the row (short rows: d well below a multiple of 512) are not copied at all;
+          // the consumers skip their k-steps
+          const int nvalid = (BM == 3) ? BM : max(0, min(BM, (a.idx_rb - r * 64 * BM + 63) / 64));
+          tc::mbar_arrive_expect_tx(&full[stage], (uint32_t)((nvalid + (PROD ? 1 : 0)) * VT * 64));
 #pragma unroll
-          for (int u = 0; u < BM; ++u) tc::tma_load_2d(sb + u * VT * 64, &tmIdx, &full[stage], r * 64 * BM + u * 64, y);
+          for (int u = 0; u < BM; ++u)
+            if (u < nvalid) tc::tma_load_2d(sb + u * VT * 64, &tmIdx, &full[stage], r * 64 * BM + u * 64, y);
           if (PROD) tc::tma_load_2d(sb + BM * VT * 64, &tmQjl, &full[stage], r * 64, y);
           if (++stage == a.stages) {
             stage = 0;
@@ -358,6 +362,20 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
   int stage = 0;
   uint32_t phase = 0;
   bool ok = true;
+  // Per-row scalars of the epilogue (nu, coef * gamma), requested one tile ahead: with short rows (d = 200: one
+  // pipeline step per tile) a request made at the top of its own tile is still in flight when the epilogue needs it.
+  float nu_next[MT], gm_next[MT];
+  auto request_scalars = [&](int64_t tile) {
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+      const int64_t row = tile * VT + cw * (MT * 16) + m * 16 + g + ((t4 & 1) ? 8 : 0);
+      const bool in = row < a.n;   // (also false for a tile past the last)
+      nu_next[m] = (in && a.norms != nullptr) ? __ldg(a.norms + row) : 1.f;
+      gm_next[m] = (PROD && in) ? __ldg(a.gamma + row) : 0.f;   // multiplied by coef where it is used: no wait here
+    }
+  };
+  constexpr bool AHEAD = (NT == 1);   // with two column tiles the longer tile hides the request and the registers cost more
+  if (AHEAD) request_scalars(blockIdx.x);
   for (int64_t tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x) {
     int accA[MT][NT][2][4], accS[MT][NT][2][4];
 #pragma unroll
@@ -369,14 +387,14 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
 #pragma unroll
           for (int i = 0; i < 4; ++i) accA[m][nt][e][i] = accS[m][nt][e][i] = 0;
 
-    // per-row scalars of the epilogue, requested now so that their latency hides behind the tile
     float nu_pre[MT], gm_pre[MT];
+    if (!AHEAD) request_scalars(tile);
 #pragma unroll
     for (int m = 0; m < MT; ++m) {
-      const int64_t row = tile * VT + cw * (MT * 16) + m * 16 + g + ((t4 & 1) ? 8 : 0);
-      nu_pre[m] = (row < a.n && a.norms != nullptr) ? __ldg(a.norms + row) : 1.f;
-      gm_pre[m] = (PROD && row < a.n) ? a.coef * __ldg(a.gamma + row) : 0.f;
+      nu_pre[m] = nu_next[m];
+      gm_pre[m] = gm_next[m];
     }
+    if (AHEAD) request_scalars(tile + gridDim.x);
 
     for (int r = 0; r < a.R; ++r) {
       if (!(ok = tc::mbar_wait(&full[stage], phase, abort_flag, a.status))) break;
@@ -399,6 +417,7 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
               blk = u;
               off = t4 * 16;
             }
+            // (a block that the producer left out holds stale bytes: its k-steps are skipped below)
             const uint4 v = *reinterpret_cast<const uint4*>(sb + blk * VT * 64 + row * 64 + off);
             w[m][h][4 * u] = v.x; w[m][h][4 * u + 1] = v.y; w[m][h][4 * u + 2] = v.z; w[m][h][4 * u + 3] = v.w;
           }
@@ -445,7 +464,7 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
       for (int nt = 0; nt < NT; ++nt) Bb[nt] = reinterpret_cast<const uint4*>(Bs + ((size_t)(nt * a.R + r) * KS) * 32) + lane;
 
       // 64-byte blocks of this range that hold row bytes at all (short rows: d well below a multiple of 512);
-      // the others are zero fill, whose k-steps add nothing
+      // the others were not copied (they would be zero fill), and their k-steps, which would add nothing, are skipped
       const int nvalid = (BM == 3) ? BM : max(0, min(BM, (a.idx_rb - r * 64 * BM + 63) / 64));
 #pragma unroll
       for (int p = 0; p < WA / 2; ++p) {
@@ -508,7 +527,7 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap tmIdx, const __grid_constant
       const int64_t row0 = tile * VT + cw * (MT * 16) + m * 16;
       const int64_t row = row0 + g + ((t4 & 1) ? 8 : 0);
       const bool row_ok = row < a.n;
-      const float nu = nu_pre[m], gm = gm_pre[m];
+      const float nu = nu_pre[m], gm = PROD ? a.coef * gm_pre[m] : 0.f;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
         auto combine = [&](const int (&acc)[2][4]) -> float {
