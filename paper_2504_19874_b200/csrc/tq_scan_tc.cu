@@ -558,7 +558,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
     };
     auto load_gm = [&](int64_t pr) -> float {
       const int64_t rw = pr * (2 * TILE) + t * TILE + r;
-      return (pr < a.npairs && rw < a.n && (a.g.kbs > 0 || NIB)) ? a.coef * __ldg(a.gamma + rw) : 0.f;
+      return (pr < a.npairs && rw < a.n && (a.g.kbs > 0 || NIB)) ? __ldg(a.gamma + rw) : 0.f;   // times coef where it is used, so that nothing waits for the load here
     };
     float nu_next = load_nu(blockIdx.x), gm_next = load_gm(blockIdx.x);
     for (int64_t pair = blockIdx.x; pair < a.npairs && ok; pair += gridDim.x, ++it) {
@@ -743,7 +743,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant__
             const long long T = ((long long)(int)vs[2][qq] * 256 + (int)vs[1][qq]) * 256 + (int)vs[0][qq];
             sv = fmaf((float)T, c.ss, c.cs);
           }
-          const float est = __fmul_rn(nu, fmaf(gm, sv, av));
+          const float est = __fmul_rn(nu, fmaf(__fmul_rn(a.coef, gm), sv, av));
           if (row_ok && ql < a.nqp) {
             if (MODE == 0) {
               if (TQ_DEVICE_CHECK(row >= 0 && row < a.n && row < a.lds, a.status)) a.scores[(int64_t)ql * a.lds + row] = est;

@@ -290,7 +290,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
     };
     auto load_gm = [&](int64_t tl) -> float {
       const int64_t rw = tl * TILE + r;
-      return (rw < a.n && (a.g.kbs > 0 || NIB)) ? a.coef * __ldg(a.gamma + rw) : 0.f;
+      return (rw < a.n && (a.g.kbs > 0 || NIB)) ? __ldg(a.gamma + rw) : 0.f;   // times coef where it is used, so that nothing waits for the load here
     };
     // zeroes this thread's columns of both accumulators and tells the issuers (before the first tile, and in every
     // epilogue as soon as the columns have been read into registers)
@@ -478,7 +478,7 @@ scan_tcw_kernel(const __grid_constant__ CUtensorMap tmBa, const __grid_constant_
             const long long T = ((long long)(int)vs[2][qq] * 256 + (int)vs[1][qq]) * 256 + (int)vs[0][qq];
             sv = fmaf((float)T, c.ss, c.cs);
           }
-          const float est = __fmul_rn(nu, fmaf(gm, sv, av));
+          const float est = __fmul_rn(nu, fmaf(__fmul_rn(a.coef, gm), sv, av));
           if (row_ok) {
             if (MODE == 0) {
               if (TQ_DEVICE_CHECK(row >= 0 && row < a.n && row < a.lds, a.status)) a.scores[(int64_t)ql * a.lds + row] = est;
