@@ -392,7 +392,8 @@ __global__ void __launch_bounds__(NT) partial_kernel(Args a) {
 // call) is fetched into shared memory before the wait for the kernel ahead, and the threads are many enough that
 // every load of a step is in flight at once.
 constexpr int MERGE_NT = 512;
-__global__ void __launch_bounds__(MERGE_NT) merge_kernel(Args a, float* __restrict__ out, int64_t ldo) {
+constexpr int MERGE_PF = 2;    // partial sums a merge thread requests ahead (more would take the registers that let the CTA start beside the partial kernel)
+__global__ void __launch_bounds__(MERGE_NT, 2) merge_kernel(Args a, float* __restrict__ out, int64_t ldo) {
   extern __shared__ __align__(16) float pis[];   // [d][d] Pi_V
   __shared__ float4 wsl[MERGE_NT];
   __shared__ float4 yp[MERGE_NT];
@@ -413,10 +414,27 @@ __global__ void __launch_bounds__(MERGE_NT) merge_kernel(Args a, float* __restri
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");   // the slices' partial results come from the kernel before
   const float4* ml4 = reinterpret_cast<const float4*>(a.part_ml + (size_t)h * a.nslices * 2 * MAXQ);   // [slice][max, sum]
+  // Everything this thread needs from the partial kernel for the first MERGE_NT slices is requested at once -- its
+  // slice's maximum and sum, and the first MERGE_PF partial sums of its coordinate -- so that the reductions below
+  // run while the loads are in flight, instead of one round trip to L2 per phase.  Sums and their order are unchanged.
+  const int nph = MERGE_NT / d, c = tid % d, ph = tid / d;   // thread = (coordinate c of the group, slice phase ph)
+  const float4* acc4 = reinterpret_cast<const float4*>(a.part_acc) + (size_t)h * a.nslices * ncoord + gi * d + c;
+  const int ns_first = min(MERGE_NT, a.nslices);
+  float4 m_own = make_float4(-FLT_MAX, -FLT_MAX, -FLT_MAX, -FLT_MAX), l_own = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (tid < ns_first) {
+    m_own = ml4[2 * tid];
+    l_own = ml4[2 * tid + 1];
+  }
+  float4 vpre[MERGE_PF];
+#pragma unroll
+  for (int i = 0; i < MERGE_PF; ++i) {
+    const int s = ph + i * nph;
+    vpre[i] = (ph < nph && s < ns_first) ? acc4[(size_t)s * ncoord] : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
   {   // global maximum and sum per query
     float M[MAXQ] = {-FLT_MAX, -FLT_MAX, -FLT_MAX, -FLT_MAX};
     for (int s = tid; s < a.nslices; s += MERGE_NT) {
-      const float4 m = ml4[2 * s];
+      const float4 m = (s == tid) ? m_own : ml4[2 * s];
       M[0] = fmaxf(M[0], m.x); M[1] = fmaxf(M[1], m.y); M[2] = fmaxf(M[2], m.z); M[3] = fmaxf(M[3], m.w);
     }
 #pragma unroll
@@ -433,7 +451,7 @@ __global__ void __launch_bounds__(MERGE_NT) merge_kernel(Args a, float* __restri
     }
     double L[MAXQ] = {0.0, 0.0, 0.0, 0.0};
     for (int s = tid; s < a.nslices; s += MERGE_NT) {
-      const float4 m = ml4[2 * s], l = ml4[2 * s + 1];
+      const float4 m = (s == tid) ? m_own : ml4[2 * s], l = (s == tid) ? l_own : ml4[2 * s + 1];
       L[0] += (double)l.x * (double)expf(m.x - M[0]); L[1] += (double)l.y * (double)expf(m.y - M[1]);
       L[2] += (double)l.z * (double)expf(m.z - M[2]); L[3] += (double)l.w * (double)expf(m.w - M[3]);
     }
@@ -454,21 +472,28 @@ __global__ void __launch_bounds__(MERGE_NT) merge_kernel(Args a, float* __restri
   }
   const float4 Mv = make_float4(stat[0][0], stat[0][1], stat[0][2], stat[0][3]);
   const float4 inv = make_float4(stat[1][0], stat[1][1], stat[1][2], stat[1][3]);
-  // thread = (coordinate c of the group, slice phase ph)
-  const int nph = MERGE_NT / d, c = tid % d, ph = tid / d;
-  const float4* acc4 = reinterpret_cast<const float4*>(a.part_acc) + (size_t)h * a.nslices * ncoord + gi * d + c;
   float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int s0 = 0; s0 < a.nslices; s0 += MERGE_NT) {
     const int ns = min(MERGE_NT, a.nslices - s0);
     __syncthreads();
     if (tid < ns) {
-      const float4 m = ml4[2 * (s0 + tid)];
+      const float4 m = (s0 == 0) ? m_own : ml4[2 * (s0 + tid)];
       wsl[tid] = make_float4(expf(m.x - Mv.x) * inv.x, expf(m.y - Mv.y) * inv.y, expf(m.z - Mv.z) * inv.z, expf(m.w - Mv.w) * inv.w);
     }
     __syncthreads();
     if (ph < nph) {
+      int s = ph;
+      if (s0 == 0) {   // the partial sums already in registers
+#pragma unroll
+        for (int i = 0; i < MERGE_PF; ++i, s += nph) {
+          if (s < ns) {
+            const float4 v = vpre[i], w = wsl[s];
+            y.x = fmaf(w.x, v.x, y.x); y.y = fmaf(w.y, v.y, y.y); y.z = fmaf(w.z, v.z, y.z); y.w = fmaf(w.w, v.w, y.w);
+          }
+        }
+      }
 #pragma unroll 8
-      for (int s = ph; s < ns; s += nph) {
+      for (; s < ns; s += nph) {
         const float4 v = acc4[(size_t)(s0 + s) * ncoord], w = wsl[s];
         y.x = fmaf(w.x, v.x, y.x); y.y = fmaf(w.y, v.y, y.y); y.z = fmaf(w.z, v.z, y.z); y.w = fmaf(w.w, v.w, y.w);
       }
