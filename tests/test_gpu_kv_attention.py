@@ -189,7 +189,8 @@ def test_fused_decode_full_shape_against_the_separate_calls(groups):
     assert float(err_o.max()) <= S5_TOL, float(err_o.max())
 
 
-@pytest.mark.parametrize("heads,T,qpk", [(2, 2500, 3), (1, 1024, 1), (3, 77, 4)])
+# (1, 140000, 2): 547 slices of 256 tokens, more than the merge kernel's 512 threads take in one round
+@pytest.mark.parametrize("heads,T,qpk", [(2, 2500, 3), (1, 1024, 1), (3, 77, 4), (1, 140000, 2)])
 def test_fused_decode_against_the_oracle(groups, heads, T, qpk):
     gK, gV = groups
     K, V, Q = wl.kv_cache(heads=heads, tokens=T, q_per_kv=qpk, seed=5 + T, device=DEV)
